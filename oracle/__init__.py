@@ -1,0 +1,135 @@
+"""CPU oracle for EAGLE tree verification (test infrastructure, never on the product path).
+
+Thin ctypes loader around ``eagle_oracle.c`` (plain C, fp64).  Only ``tests/``, the smoke check and
+``bench.py``'s CPU-baseline legs may import this package; the CUDA library and its Python binding
+share no code with it and never import it.
+
+The arithmetic lives in the C file; the functions here only marshal numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "eagle_oracle.c"
+_LIB = _HERE / "liboracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile the oracle with gcc (-O2, OpenMP, no fast-math) into ``oracle/liboracle.so``."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".so.tmp{os.getpid()}")
+        cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+               "-o", str(tmp), str(_SRC), "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(str(_LIB))
+        i32, dbl, vp = ctypes.c_int, ctypes.c_double, ctypes.c_void_p
+        lib.oracle_tree_ancestors.argtypes = [vp, vp, i32, i32, vp, vp]
+        lib.oracle_tree_ancestors.restype = i32
+        lib.oracle_tree_verify_attn.argtypes = [i32, i32, i32, i32, i32, i32, vp, dbl, vp, vp, vp, vp, vp, vp]
+        lib.oracle_tree_verify_attn.restype = i32
+        lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 13
+        lib.oracle_tree_accept.restype = i32
+        lib.oracle_num_threads.restype = i32
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _as(a, dtype):
+    if a is None:
+        return None
+    if hasattr(a, "detach"):  # torch CPU tensor
+        import torch
+        if a.dtype == torch.bfloat16:
+            a = a.contiguous().view(torch.int16)
+        a = a.detach().cpu().numpy()
+    a = np.ascontiguousarray(a)
+    if dtype == np.uint16 and a.dtype == np.int16:
+        a = a.view(np.uint16)
+    if a.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {a.dtype}")
+    return a
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def tree_ancestors(tree_parent, tree_sizes=None):
+    """Ancestor-or-self bit sets (uint64) and depths (int32) by walking parent links."""
+    par = _as(tree_parent, np.int32)
+    B, T = par.shape
+    ts = _as(tree_sizes, np.int32)
+    anc = np.zeros((B, T), np.uint64)
+    depth = np.zeros((B, T), np.int32)
+    rc = _load().oracle_tree_ancestors(_ptr(par), _ptr(ts), B, T, _ptr(anc), _ptr(depth))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_ancestors failed: {rc}")
+    return anc, depth
+
+
+def tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, tree_sizes=None, sm_scale: float = 0.0):
+    """fp64 tree-masked attention.  q/k/v are bf16 (torch tensors, or their uint16 bit patterns).
+
+    q [B, T_max, Hq, D]; k_cache, v_cache [B, Hkv, S_cap, D]; returns float64 [B, T_max, Hq, D].
+    """
+    qa, ka, va = _as(q, np.uint16), _as(k_cache, np.uint16), _as(v_cache, np.uint16)
+    B, T, Hq, D = qa.shape
+    Hkv, S = ka.shape[1], ka.shape[2]
+    assert ka.shape == va.shape == (B, Hkv, S, D)
+    sl, par, ts = _as(seq_lens, np.int32), _as(tree_parent, np.int32), _as(tree_sizes, np.int32)
+    assert par.shape == (B, T)
+    out = np.zeros((B, T, Hq, D), np.float64)
+    rc = _load().oracle_tree_verify_attn(B, Hq, Hkv, D, T, S, _ptr(ts), float(sm_scale), _ptr(qa), _ptr(ka),
+                                         _ptr(va), _ptr(sl), _ptr(par), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_verify_attn failed: {rc}")
+    return out
+
+
+def tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, tree_sizes=None, greedy=None,
+                path_cap: int | None = None):
+    """Acceptance walk (Algorithm 1 at every node, or the greedy rule).  Returns a dict of numpy arrays:
+    accepted_path [B, path_cap], bonus_token [B], accept_len [B], min_margin [B], n_sweeps [B],
+    n_zero_mass [B]."""
+    tp = _as(target_probs, np.float32)
+    B, T1, V = tp.shape
+    T = T1 - 1
+    dp = _as(draft_probs, np.float32)
+    tok, par = _as(draft_tokens, np.int32), _as(tree_parent, np.int32)
+    un = _as(uniforms, np.float32)
+    ts, gr = _as(tree_sizes, np.int32), _as(greedy, np.uint8)
+    assert tok.shape == par.shape == (B, T)
+    if dp is not None:
+        assert dp.shape == (B, T, V)
+    if un is not None:
+        assert un.shape == (B, T + 1)
+    cap = T if path_cap is None else path_cap
+    res = dict(accepted_path=np.full((B, cap), -1, np.int32), bonus_token=np.full((B,), -1, np.int32),
+               accept_len=np.zeros((B,), np.int32), min_margin=np.zeros((B,), np.float64),
+               n_sweeps=np.zeros((B,), np.int32), n_zero_mass=np.zeros((B,), np.int32))
+    rc = _load().oracle_tree_accept(B, T, V, cap, _ptr(ts), _ptr(gr), _ptr(tp), _ptr(dp), _ptr(tok), _ptr(par),
+                                    _ptr(un), _ptr(res["accepted_path"]), _ptr(res["bonus_token"]),
+                                    _ptr(res["accept_len"]), _ptr(res["min_margin"]), _ptr(res["n_sweeps"]),
+                                    _ptr(res["n_zero_mass"]))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_accept failed: {rc}")
+    return res

@@ -1,0 +1,330 @@
+/*
+ * CPU oracle for the tree-verification step of EAGLE speculative decoding.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the CUDA library is
+ * checked against.  It shares no code with the CUDA path, and nothing in the product path may
+ * call it.  Everything is fp64 and written as the definition / the algorithm's steps, with no
+ * blocking, fusion or reordering.  OpenMP only distributes independent (sequence, head) units.
+ *
+ * What each function follows:
+ *   oracle_tree_ancestors    - "tree attention" (Sec. 3.1, Sec. 3.3, App. A.1): a draft token sees the
+ *                              tokens on its own root path.  The set is found by walking parent links.
+ *   oracle_tree_verify_attn  - Sec. 3.3 / App. A.1: one target forward pass scores every tree token;
+ *                              for one attention layer that is softmax attention over the committed
+ *                              prefix plus the node's ancestors and itself (plain definition).
+ *   oracle_tree_accept       - Algorithm 1 (multi-round speculative sampling, App. A.2) applied
+ *                              recursively at every node from the root (Sec. 3.3); the greedy setting
+ *                              (Preliminaries) is the same rule with a one-hot target distribution.
+ *
+ * Readings taken where the paper is silent or garbled are listed next to the code that uses them.
+ * Pins: see tests/test_oracle_*.py.  The sibling order, the lowest-index tie-break of argmax and the
+ * assignment of uniforms to decisions are conventions of this library, not fixed by the paper:
+ * "parity unpinned" for those three conventions (they are pinned only by this file's own statement).
+ */
+#include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG (-1)
+#define ORACLE_ERR_TREE (-2)
+#define ORACLE_ERR_NOMEM (-3)
+
+static double bf16_to_f64(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+static int tree_size_of(const int32_t* tree_sizes, int b, int max_tree) {
+  return tree_sizes ? tree_sizes[b] : max_tree;
+}
+
+/* A parent array is valid when -1 <= parent[i] < i (topological order; -1 = child of the context). */
+static int tree_valid(const int32_t* parent, int n) {
+  for (int i = 0; i < n; ++i)
+    if (parent[i] < -1 || parent[i] >= i) return 0;
+  return 1;
+}
+
+/*
+ * Ancestor-or-self set of every node, as a bit set, and the node's depth (top-level nodes have
+ * depth 1).  Found by following parent links up to the context; no recurrence over earlier results.
+ * parent: int32 [batch, max_tree]; tree_sizes: int32 [batch] or NULL; anc: uint64 [batch, max_tree];
+ * depth: int32 [batch, max_tree].  Entries of nodes >= tree size are set to 0.
+ */
+int oracle_tree_ancestors(const int32_t* parent, const int32_t* tree_sizes, int batch, int max_tree,
+                          uint64_t* anc, int32_t* depth) {
+  if (!parent || !anc || batch < 0 || max_tree < 0 || max_tree > 64) return ORACLE_ERR_ARG;
+  for (int b = 0; b < batch; ++b) {
+    const int n = tree_size_of(tree_sizes, b, max_tree);
+    if (n < 0 || n > max_tree) return ORACLE_ERR_ARG;
+    const int32_t* par = parent + (size_t)b * max_tree;
+    if (!tree_valid(par, n)) return ORACLE_ERR_TREE;
+    for (int i = 0; i < max_tree; ++i) {
+      uint64_t set = 0;
+      int d = 0;
+      if (i < n) {
+        for (int c = i; c >= 0; c = par[c]) {
+          set |= (uint64_t)1 << c;
+          ++d;
+        }
+      }
+      anc[(size_t)b * max_tree + i] = set;
+      if (depth) depth[(size_t)b * max_tree + i] = d;
+    }
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Tree-masked attention of one layer, by definition.
+ *
+ *   q        bf16 bits [batch, max_tree, num_q_heads, head_dim]
+ *   k_cache  bf16 bits [batch, num_kv_heads, kv_capacity, head_dim]   (v_cache alike)
+ *   seq_lens int32 [batch]   committed prefix length L_b; tree node m's key/value sit at slot L_b + m
+ *   out      fp64  [batch, max_tree, num_q_heads, head_dim]; rows of nodes >= tree size are 0
+ *
+ * Node i of sequence b, query head h (KV head h / G, G = num_q_heads / num_kv_heads) sees slot j iff
+ * j < L_b, or j = L_b + m with m on the path from i up to the context (i itself included).
+ * s_j = sm_scale * <q, k_j>;  out = sum_j softmax(s)_j v_j.   Slots that are not visible are never
+ * read, so they may hold anything (NaN included).
+ */
+int oracle_tree_verify_attn(int batch, int num_q_heads, int num_kv_heads, int head_dim, int max_tree,
+                            int kv_capacity, const int32_t* tree_sizes, double sm_scale,
+                            const uint16_t* q, const uint16_t* k_cache, const uint16_t* v_cache,
+                            const int32_t* seq_lens, const int32_t* tree_parent, double* out) {
+  if (batch < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || head_dim <= 0 || max_tree < 0 ||
+      max_tree > 64 || num_q_heads % num_kv_heads != 0 || !seq_lens || !tree_parent || !out)
+    return ORACLE_ERR_ARG;
+  const int G = num_q_heads / num_kv_heads;
+  const int D = head_dim;
+  if (sm_scale == 0.0) sm_scale = 1.0 / sqrt((double)D);
+  for (int b = 0; b < batch; ++b) {
+    const int n = tree_size_of(tree_sizes, b, max_tree);
+    if (n < 0 || n > max_tree || seq_lens[b] < 0 || seq_lens[b] + n > kv_capacity) return ORACLE_ERR_ARG;
+    if (!tree_valid(tree_parent + (size_t)b * max_tree, n)) return ORACLE_ERR_TREE;
+  }
+  memset(out, 0, sizeof(double) * (size_t)batch * max_tree * num_q_heads * D);
+  int failed = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+  for (int b = 0; b < batch; ++b) {
+    for (int h = 0; h < num_q_heads; ++h) {
+      const int n = tree_size_of(tree_sizes, b, max_tree);
+      const int L = seq_lens[b];
+      const int g = h / G;
+      const int32_t* par = tree_parent + (size_t)b * max_tree;
+      const uint16_t* kb = k_cache + ((size_t)b * num_kv_heads + g) * (size_t)kv_capacity * D;
+      const uint16_t* vb = v_cache + ((size_t)b * num_kv_heads + g) * (size_t)kv_capacity * D;
+      int* slots = (int*)malloc(sizeof(int) * (size_t)(L + max_tree + 1));
+      double* s = (double*)malloc(sizeof(double) * (size_t)(L + max_tree + 1));
+      if (!slots || !s) {
+        failed = 1;
+        free(slots);
+        free(s);
+        continue;
+      }
+      for (int i = 0; i < n; ++i) {
+        const uint16_t* qi = q + (((size_t)b * max_tree + i) * num_q_heads + h) * D;
+        double* oi = out + (((size_t)b * max_tree + i) * num_q_heads + h) * D;
+        /* visible slots: the whole prefix, then the root path of node i */
+        int cnt = 0;
+        for (int j = 0; j < L; ++j) slots[cnt++] = j;
+        for (int c = i; c >= 0; c = par[c]) slots[cnt++] = L + c;
+        double smax = -INFINITY;
+        for (int t = 0; t < cnt; ++t) {
+          const uint16_t* kj = kb + (size_t)slots[t] * D;
+          double acc = 0.0;
+          for (int d = 0; d < D; ++d) acc += bf16_to_f64(qi[d]) * bf16_to_f64(kj[d]);
+          s[t] = sm_scale * acc;
+          if (s[t] > smax) smax = s[t];
+        }
+        double denom = 0.0;
+        for (int t = 0; t < cnt; ++t) {
+          s[t] = exp(s[t] - smax);
+          denom += s[t];
+        }
+        for (int d = 0; d < D; ++d) {
+          double acc = 0.0;
+          for (int t = 0; t < cnt; ++t) acc += s[t] * bf16_to_f64(vb[(size_t)slots[t] * D + d]);
+          oi[d] = acc / denom;
+        }
+      }
+      free(slots);
+      free(s);
+    }
+  }
+  return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
+}
+
+/*
+ * Acceptance along the tree.
+ *
+ *   target_probs fp32 [batch, max_tree + 1, vocab]  row 0: distribution after the committed context;
+ *                                                    row i + 1: distribution after tree node i
+ *   draft_probs  fp32 [batch, max_tree, vocab]       row i: the distribution node i's token was drawn from
+ *   draft_tokens int32 [batch, max_tree]
+ *   tree_parent  int32 [batch, max_tree]
+ *   uniforms     fp32 [batch, max_tree + 1]          entry i: the r of node i's accept test;
+ *                                                    entry max_tree: the final draw
+ *   greedy       uint8 [batch] or NULL               1: temperature-0 rule for that sequence
+ *   accepted_path int32 [batch, path_cap] (-1 padded), bonus_token int32 [batch], accept_len int32 [batch]
+ *   min_margin   fp64 [batch] or NULL: smallest distance to a decision boundary met on the walk
+ *                (accept test: |r - p(t)/p^(t)|; final draw: distance of u to the nearer edge of the
+ *                chosen cell of the normalised CDF; greedy: gap between the two largest probabilities)
+ *   n_sweeps     int32 [batch] or NULL: vocabulary-wide passes the walk needed (rejections + final draw,
+ *                or one argmax per visited node)
+ *   n_zero_mass  int32 [batch] or NULL: rejections whose residual had zero mass (distribution kept)
+ *
+ * Walk (Sec. 3.3: Algorithm 1 applied at every node, starting from the root):
+ *   cur = context.  p = target row of cur (used as given, each node starts from its own row).
+ *   Candidates = children of cur, ascending node index (Algorithm 1's i = 1..k).
+ *   Stochastic (Algorithm 1): for each candidate i with token t: r = uniforms[i]; accept iff
+ *   r < p(t)/p^_i(t), evaluated as r * p^_i(t) < p(t) so that p^_i(t) = 0 needs no division;
+ *   on rejection p <- norm(max(0, p - p^_i)) over the whole vocabulary (the Preliminaries' vector
+ *   form of the update; Algorithm 1 prints it with scalar arguments); zero residual mass keeps p.
+ *   After the candidates are exhausted (k = 0 at a leaf included) draw x ~ p by inverse CDF in
+ *   ascending token id with u = uniforms[max_tree]: smallest x with cumsum(x) > u * total.
+ *   Greedy: a = argmax p (lowest id on ties); move to the lowest-index child whose token is a,
+ *   else emit a.  Exactly one extra token is emitted per call.
+ */
+int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const int32_t* tree_sizes,
+                       const uint8_t* greedy, const float* target_probs, const float* draft_probs,
+                       const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                       int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
+                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass) {
+  if (batch < 0 || max_tree < 0 || max_tree > 64 || vocab <= 0 || path_cap < 0 || !target_probs ||
+      !tree_parent || !draft_tokens || !accepted_path || !bonus_token)
+    return ORACLE_ERR_ARG;
+  for (int b = 0; b < batch; ++b) {
+    const int n = tree_size_of(tree_sizes, b, max_tree);
+    if (n < 0 || n > max_tree) return ORACLE_ERR_ARG;
+    if (!tree_valid(tree_parent + (size_t)b * max_tree, n)) return ORACLE_ERR_TREE;
+    for (int i = 0; i < n; ++i) {
+      const int t = draft_tokens[(size_t)b * max_tree + i];
+      if (t < 0 || t >= vocab) return ORACLE_ERR_ARG;
+    }
+    const int is_greedy = greedy ? greedy[b] != 0 : 0;
+    if (!is_greedy && (!draft_probs || !uniforms)) return ORACLE_ERR_ARG;
+  }
+  int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int b = 0; b < batch; ++b) {
+    const int n = tree_size_of(tree_sizes, b, max_tree);
+    const int is_greedy = greedy ? greedy[b] != 0 : 0;
+    const int32_t* par = tree_parent + (size_t)b * max_tree;
+    const int32_t* tok = draft_tokens + (size_t)b * max_tree;
+    int32_t* path = accepted_path + (size_t)b * path_cap;
+    for (int j = 0; j < path_cap; ++j) path[j] = -1;
+    double* p = (double*)malloc(sizeof(double) * (size_t)vocab);
+    if (!p) {
+      failed = 1;
+      continue;
+    }
+    int cur = -1, len = 0, sweeps = 0, zero_mass = 0, bonus = -1;
+    double margin = INFINITY;
+    for (;;) {
+      const float* prow = target_probs + ((size_t)b * (max_tree + 1) + (size_t)(cur + 1)) * vocab;
+      for (int v = 0; v < vocab; ++v) p[v] = (double)prow[v];
+      int next = -1;
+      if (is_greedy) {
+        int a = 0;
+        for (int v = 1; v < vocab; ++v)
+          if (p[v] > p[a]) a = v;
+        double second = -INFINITY;
+        for (int v = 0; v < vocab; ++v)
+          if (v != a && p[v] > second) second = p[v];
+        if (vocab > 1 && p[a] - second < margin) margin = p[a] - second;
+        ++sweeps;
+        for (int i = 0; i < n && next < 0; ++i)
+          if (par[i] == cur && tok[i] == a) next = i;
+        if (next < 0) bonus = a;
+      } else {
+        for (int i = 0; i < n && next < 0; ++i) {
+          if (par[i] != cur) continue;
+          const float* qrow = draft_probs + ((size_t)b * max_tree + i) * vocab;
+          const int t = tok[i];
+          const double r = (double)uniforms[(size_t)b * (max_tree + 1) + i];
+          const double pt = p[t], qt = (double)qrow[t];
+          if (qt > 0.0) {
+            const double m = fabs(r - pt / qt);
+            if (m < margin) margin = m;
+          }
+          if (r * qt < pt) {
+            next = i;
+          } else {
+            double Z = 0.0;
+            for (int v = 0; v < vocab; ++v) {
+              const double d = p[v] - (double)qrow[v];
+              Z += d > 0.0 ? d : 0.0;
+            }
+            ++sweeps;
+            if (Z > 0.0) {
+              for (int v = 0; v < vocab; ++v) {
+                const double d = p[v] - (double)qrow[v];
+                p[v] = (d > 0.0 ? d : 0.0) / Z;
+              }
+            } else {
+              ++zero_mass;
+            }
+          }
+        }
+        if (next < 0) {
+          const double u = (double)uniforms[(size_t)b * (max_tree + 1) + max_tree];
+          double total = 0.0;
+          for (int v = 0; v < vocab; ++v) total += p[v];
+          const double thr = u * total;
+          double c = 0.0, c_prev = 0.0;
+          int x = -1, last_pos = -1;
+          for (int v = 0; v < vocab; ++v) {
+            if (p[v] > 0.0) last_pos = v;
+            c_prev = c;
+            c += p[v];
+            if (c > thr) {
+              x = v;
+              break;
+            }
+          }
+          if (x < 0) {
+            x = last_pos >= 0 ? last_pos : vocab - 1;
+          } else if (total > 0.0) {
+            const double lo = (thr - c_prev) / total, hi = (c - thr) / total;
+            const double m = lo < hi ? lo : hi;
+            if (m < margin) margin = m;
+          }
+          ++sweeps;
+          bonus = x;
+        }
+      }
+      if (next < 0) break;
+      if (len < path_cap) path[len] = next;
+      ++len;
+      cur = next;
+    }
+    bonus_token[b] = bonus;
+    if (accept_len) accept_len[b] = len;
+    if (min_margin) min_margin[b] = margin;
+    if (n_sweeps) n_sweeps[b] = sweeps;
+    if (n_zero_mass) n_zero_mass[b] = zero_mass;
+    free(p);
+  }
+  return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
+}
+
+/* Threads the OpenMP loops above use (reported next to the oracle's timing). */
+int oracle_num_threads(void) {
+  int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+  {
+#pragma omp single
+    n = omp_get_num_threads();
+  }
+#endif
+  return n;
+}
