@@ -1,0 +1,320 @@
+#!/usr/bin/env python
+"""Benchmark of the tree-verification step (tree attention + acceptance) on B200.
+
+One *step* = ``eagle_tree_verify_attn`` (planner, split-KV attention, combine) followed by
+``eagle_tree_accept`` for one batch of synthetic input, on one stream.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+* ``value``: whole-job verify-steps/s with the inputs resident in HBM (device-timed with CUDA events, max
+  over ranks).  With N > 1 every rank runs its own batch (no data-path collective: the path shards by
+  sequence), so per-GPU work is fixed ("weak").
+* ``e2e``: the same step driven from pinned HOST buffers: every step copies its inputs host->device, runs
+  the two C-ABI calls and reads the results back.
+* ``roofline``: the split-KV attention kernel alone, timed live with CUDA events around that kernel inside
+  the timed region, against the measured HBM copy bandwidth.
+* ``cpu_baseline``: the fp64 oracle, as it stands, on a bounded sample of the same workload.
+* ``--impl reference``: the oracle arm (CPU); rank 0 only.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import torch
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+from paper_2401_15077_b200 import workloads as W  # noqa: E402
+
+METRIC = "tree_verify_steps_per_s"
+UNIT = "steps/s"
+HBM_FALLBACK_GBS = 6650.0
+L2_BYTES = 126 * 2 ** 20
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
+# profiles/ (bytes per launch on the named workload); None until a capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_hbm_peak():
+    f = ROOT / "MEASURED_PEAKS.json"
+    try:
+        return float(json.loads(f.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback (profiling recipe, 6.65 TB/s)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax = float(r[1])
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def host_inputs(cfg, salt, rho):
+    attn = W.make_attn_inputs(cfg, salt=salt)
+    acc = W.make_accept_inputs(cfg, salt=salt, rho=rho, trees=(attn.tree_sizes, attn.tree_parent))
+    return attn, acc
+
+
+def oracle_step_sample(attn, acc, budget_s, max_seqs=None):
+    """Runs the oracle sequence by sequence (attention + acceptance) until ``budget_s`` is spent.
+    Returns (sequences done, seconds)."""
+    import oracle
+    oracle.build()
+    B = attn.cfg.batch
+    done, t0 = 0, time.perf_counter()
+    for b in range(B if max_seqs is None else min(B, max_seqs)):
+        s = slice(b, b + 1)
+        end = int(attn.seq_lens[b] + attn.tree_sizes[b])
+        oracle.tree_verify_attn(attn.q[s], attn.k_cache[s, :, :end].contiguous(), attn.v_cache[s, :, :end].contiguous(),
+                                attn.seq_lens[s], attn.tree_parent[s], attn.tree_sizes[s])
+        oracle.tree_accept(acc.target_probs[s], acc.draft_probs[s], acc.draft_tokens[s], acc.tree_parent[s],
+                           acc.uniforms[s], tree_sizes=acc.tree_sizes[s], greedy=acc.greedy[s])
+        done += 1
+        if time.perf_counter() - t0 > budget_s:
+            break
+    return done, time.perf_counter() - t0, oracle.num_threads()
+
+
+def run_reference(args, cfg, rank, world):
+    if rank != 0:
+        return
+    attn, acc = host_inputs(cfg, 0, args.rho)
+    per_step = max(1, min(cfg.batch, args.ref_seqs))
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        oracle_step_sample(attn, acc, 1e9, per_step)
+    t0 = time.perf_counter()
+    cores = 1
+    for _ in range(args.steps):
+        _, _, cores = oracle_step_sample(attn, acc, 1e9, per_step)
+    dt = time.perf_counter() - t0
+    value = args.steps * (per_step / cfg.batch) / dt
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "batch": cfg.batch, "rho": args.rho},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"each step runs the first {per_step} of {cfg.batch} sequences (attention + acceptance); "
+                                       "value scaled to whole batches"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="serving_mix", choices=list(W.CONFIGS))
+    ap.add_argument("--rho", type=float, default=0.9, help="target/draft logit correlation of the synthetic acceptance inputs")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
+    ap.add_argument("--ref-seqs", type=int, default=1, help="sequences per step of the reference arm")
+    ap.add_argument("--num-splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    cfg = W.CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+
+    import torch.distributed as dist
+    from paper_2401_15077_b200 import binding as E, build
+    if rank == 0 or world == 1:
+        build.build()
+    E.load()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    attn, acc = host_inputs(cfg, rank, args.rho)
+    alg_bytes, alg_flops = attn.algorithmic_bytes(), attn.algorithmic_flops()
+
+    # ---- device-resident input sets; rotate over R sets so that consecutive steps never hit a warm L2
+    step_bytes = sum(t.numel() * t.element_size() for t in (attn.k_cache, attn.v_cache))
+    touched = alg_bytes
+    R = 1 if touched > 2 * L2_BYTES else int(min(48, -(-(1 << 30) // max(touched, 1))))
+    host = dict(q=attn.q, k=attn.k_cache, v=attn.v_cache, sl=attn.seq_lens, par=attn.tree_parent, ts=attn.tree_sizes,
+                tp=acc.target_probs, dp=acc.draft_probs, tok=acc.draft_tokens, un=acc.uniforms, gr=acc.greedy)
+    sets = [{k: v.to(dev) for k, v in host.items()} for _ in range(R)]
+    B, T = cfg.batch, cfg.max_tree
+    out = torch.empty_like(sets[0]["q"])
+    ws = E.alloc_workspace(sets[0]["q"], sets[0]["k"], args.num_splits)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    path = torch.empty((B, T), dtype=torch.int32, device=dev)
+    bonus = torch.empty((B,), dtype=torch.int32, device=dev)
+    alen = torch.empty((B,), dtype=torch.int32, device=dev)
+
+    def step(s, events=None):
+        E.eagle_tree_verify_attn(s["q"], s["k"], s["v"], s["sl"], s["par"], out, tree_sizes=s["ts"], workspace=ws,
+                                 status=status, num_splits=args.num_splits, events=events)
+        E.eagle_tree_accept(s["tp"], s["dp"], s["tok"], s["par"], s["un"], path, bonus, tree_sizes=s["ts"], greedy=s["gr"],
+                            accept_len=alen, status=status)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(sets[i % R])
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, E.status_string(int(status.item()))
+
+    K = args.steps
+    ev_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in ev_pairs:   # create the underlying CUDA events before handing their handles to the library
+        a.record()
+        b.record()
+    ev_acc = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = E.launch_count()
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    start.record()
+    for i in range(K):
+        step(sets[(args.warmup + i) % R], ev_pairs[i])
+    stop.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = E.launch_count() - launches0
+    elapsed_ms = start.elapsed_time(stop)
+    attn_ms = statistics.mean(a.elapsed_time(b) for a, b in ev_pairs)
+    assert int(status.item()) == 0
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    elapsed_ms = float(t.item())
+    value = world * K / (elapsed_ms * 1e-3)
+
+    # ---- acceptance alone (reported, not part of the headline)
+    for i in range(min(K, 10)):
+        s = sets[i % R]
+        ev_acc[i][0].record()
+        E.eagle_tree_accept(s["tp"], s["dp"], s["tok"], s["par"], s["un"], path, bonus, tree_sizes=s["ts"], greedy=s["gr"],
+                            accept_len=alen, status=status)
+        ev_acc[i][1].record()
+    torch.cuda.synchronize()
+    accept_ms = statistics.mean(ev_acc[i][0].elapsed_time(ev_acc[i][1]) for i in range(min(K, 10)))
+    mean_tokens = float(alen.float().mean().item()) + 1.0
+
+    # ---- end to end from pinned host buffers
+    pinned = {k: v.pin_memory() for k, v in host.items()}
+    dset = sets[0]
+    h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    h_path, h_bonus = torch.empty(path.shape, dtype=path.dtype).pin_memory(), torch.empty(bonus.shape, dtype=bonus.dtype).pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values())
+    d2h = sum(v.numel() * v.element_size() for v in (h_out, h_path, h_bonus))
+
+    def e2e_step():
+        for k2, v in pinned.items():
+            dset[k2].copy_(v, non_blocking=True)
+        step(dset)
+        h_out.copy_(out, non_blocking=True)
+        h_path.copy_(path, non_blocking=True)
+        h_bonus.copy_(bonus, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * args.e2e_steps / (float(te.item()) * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_hbm_peak()
+    achieved = alg_bytes / (attn_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": B, "num_q_heads": cfg.num_q_heads, "num_kv_heads": cfg.num_kv_heads,
+                   "head_dim": cfg.head_dim, "prefix": list(cfg.prefix), "tree": list(cfg.tree), "vocab": cfg.vocab,
+                   "greedy": cfg.greedy, "rho": args.rho, "parallelism": f"replicas x{world}",
+                   "l2": (f"rotating over {R} input sets" if R > 1 else "inputs larger than L2 (single set)")},
+        "clocks": clocks, "gpu_launches": launches,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps},
+        "roofline": {"bound": "hbm", "kernel": "split-KV tree attention", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                     "algorithmic_bytes": alg_bytes, "ms_per_launch": attn_ms,
+                     "tflops": alg_flops / (attn_ms * 1e-3) / 1e12},
+        "breakdown": {"attn_kernel_ms": attn_ms, "accept_ms": accept_ms, "tokens_per_step": mean_tokens,
+                      "sequence_steps_per_s": value * B},
+    }
+    if not args.no_cpu_baseline:
+        done, secs, cores = oracle_step_sample(attn, acc, args.cpu_budget)
+        line["cpu_baseline"] = {"value": (done / B) / secs, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"first {done} of {B} sequences of the same batch (attention + acceptance), "
+                                          f"{secs:.1f} s; value scaled to whole batches"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

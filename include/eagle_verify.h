@@ -1,0 +1,162 @@
+/*
+ * eagle_verify.h - C ABI of the B200 (sm_100a) tree-verification library for EAGLE speculative decoding.
+ *
+ * The verification phase (Sec. 3.3, App. A.1 and A.2 of the EAGLE paper) scores every token of a
+ * tree-structured draft in one target forward pass with tree attention, then walks the tree applying
+ * multi-round speculative sampling (Algorithm 1) at every node.  This library implements, for one
+ * attention layer and for the acceptance walk, exactly those two operations:
+ *
+ *   eagle_tree_verify_attn  tree-masked attention of the T draft-tree tokens against the committed
+ *                           KV prefix plus the tree's own keys (a node sees the prefix, its ancestors
+ *                           and itself)
+ *   eagle_tree_accept       acceptance along the tree: greedy, or Algorithm 1 at every node
+ *
+ * Conventions shared by every call
+ *   - Every pointer marked "device" is a device pointer owned by the caller; the library keeps none of
+ *     them after the call returns, allocates no memory and never synchronises: work is enqueued on
+ *     `stream` and the call returns.  Pointers marked "host" are ordinary host pointers.
+ *   - Return value: EAGLE_OK, or a negative EAGLE_ERR_* when the host-side check of the arguments fails
+ *     (nothing is launched) or a launch fails.  Problems only the device can see (a parent entry out of
+ *     range, a prefix that does not fit the cache, a wait that ran out) are written to `*status`
+ *     (device int32, first error wins, 0 = none); the affected sequence's rows are zeroed (attention)
+ *     or its outputs set to "nothing accepted, bonus -1" (acceptance).  No trap is ever raised.
+ *   - Tree: node i of sequence b has parent tree_parent[b, i] in [-1, i-1]; -1 means "child of the
+ *     committed context".  At most 64 nodes per tree.  Entries at i >= tree size are ignored.
+ */
+#ifndef EAGLE_VERIFY_H_
+#define EAGLE_VERIFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque CUDA handles: a cudaStream_t / cudaEvent_t passed as a pointer-sized value. */
+typedef void* eagle_stream_t;
+typedef void* eagle_event_t;
+
+enum {
+  EAGLE_OK = 0,
+  EAGLE_ERR_NULL = -1,       /* a required pointer is NULL */
+  EAGLE_ERR_SHAPE = -2,      /* batch / heads / head_dim / max_tree / vocab out of the supported range */
+  EAGLE_ERR_WORKSPACE = -3,  /* workspace missing, misaligned (256 B) or too small */
+  EAGLE_ERR_LAUNCH = -4,     /* CUDA reported an error when launching */
+  EAGLE_ERR_TREE = -5,       /* device-detected: parent entry outside [-1, i-1], or tree size out of range */
+  EAGLE_ERR_SEQ = -6,        /* device-detected: seq_lens[b] < 0 or seq_lens[b] + tree size > kv_capacity */
+  EAGLE_ERR_TOKEN = -7,      /* device-detected: draft token outside [0, vocab) */
+  EAGLE_ERR_TIMEOUT = -8,    /* device-detected: a bounded wait inside a kernel ran out */
+  EAGLE_ERR_DEVICE = -9      /* the GPU is not an sm_100 device, or it lacks a required limit */
+};
+
+#define EAGLE_MAX_TREE 64
+
+/*
+ * Descriptor of one attention call.  Plain data, read during the call only.
+ */
+typedef struct eagle_attn_desc {
+  int32_t batch;               /* B >= 0 */
+  int32_t num_q_heads;         /* Hq; Hq % Hkv == 0, group size G = Hq / Hkv <= 16 */
+  int32_t num_kv_heads;        /* Hkv */
+  int32_t head_dim;            /* D: 64 or 128 */
+  int32_t max_tree;            /* T_max <= 64: row stride of tree_parent, q and out */
+  int32_t kv_capacity;         /* S_cap: slots per (sequence, KV head) of k_cache / v_cache */
+  const int32_t* tree_sizes;   /* device int32 [B], or NULL: every tree has T_max nodes */
+  float sm_scale;              /* softmax scale; 0 means 1/sqrt(D) */
+  int32_t num_splits;          /* KV splits per sequence; 0 lets the device-side planner choose */
+  void* workspace;             /* device, 256-byte aligned, >= eagle_tree_verify_attn_workspace() bytes */
+  size_t workspace_bytes;
+  int32_t* status;             /* device int32 or NULL */
+  eagle_event_t ev_attn_begin; /* optional: recorded on `stream` right before / after the split-KV   */
+  eagle_event_t ev_attn_end;   /* attention kernel (the dominant kernel), for timing it alone; or NULL */
+} eagle_attn_desc;
+
+/* Bytes of scratch one call with this descriptor needs (host function, no CUDA work).
+ * Depends on batch, heads, head_dim and max_tree only.  Returns 0 if the shape is unsupported. */
+size_t eagle_tree_verify_attn_workspace(const eagle_attn_desc* desc);
+
+/*
+ * Tree-masked attention of one layer (tree attention of the verification pass: Sec. 3.3, App. A.1).
+ *
+ *   q        device bf16 [B, T_max, Hq, D]        queries of the tree tokens (already position-encoded)
+ *   k_cache  device bf16 [B, Hkv, S_cap, D]       keys; slots [0, L_b) hold the committed prefix, slot
+ *   v_cache  device bf16 [B, Hkv, S_cap, D]       L_b + m holds tree node m; later slots are never used
+ *                                                 in the result, whatever they contain (NaN included)
+ *   seq_lens device int32 [B]                     L_b, the committed prefix length (tree not included)
+ *   tree_parent device int32 [B, T_max]
+ *   out      device bf16 [B, T_max, Hq, D]        out[b,i,h,:] = sum_j softmax_j(scale * q[b,i,h]·k[b,h/G,j]) v[b,h/G,j]
+ *                                                 over j < L_b and j = L_b + m, m an ancestor of i or i itself;
+ *                                                 rows of nodes i >= tree size are written as zeros
+ *
+ * Arithmetic: bf16 inputs, fp32 scores / softmax / accumulation, bf16 output (round to nearest even).
+ * k_cache and v_cache must be 16-byte aligned.  Launches, in order on `stream`: the planner (tree masks +
+ * work list), the split-KV attention kernel, the combine kernel.  The workspace must not be shared by
+ * calls that can overlap on the GPU.
+ */
+int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                           const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream);
+
+/*
+ * Descriptor of one acceptance call.
+ */
+typedef struct eagle_accept_desc {
+  int32_t batch;               /* B >= 0 */
+  int32_t max_tree;            /* T_max <= 64: row stride of the per-node arrays */
+  int32_t vocab;               /* V >= 1 */
+  int32_t path_cap;            /* entries per row of accepted_path; >= the deepest tree (T_max is always enough) */
+  const int32_t* tree_sizes;   /* device int32 [B] or NULL */
+  const uint8_t* greedy;       /* device uint8 [B] or NULL (= every sequence stochastic); 1: temperature-0 rule */
+  int32_t* accept_len;         /* device int32 [B] or NULL: number of accepted nodes */
+  int32_t* status;             /* device int32 or NULL */
+} eagle_accept_desc;
+
+/*
+ * Acceptance along the draft tree: Algorithm 1 (multi-round speculative sampling, App. A.2) applied at
+ * every node starting from the committed context (Sec. 3.3), or the greedy rule (Preliminaries).
+ *
+ *   target_probs device fp32 [B, T_max+1, V]   row 0: target distribution after the context;
+ *                                              row i+1: target distribution after tree node i
+ *   draft_probs  device fp32 [B, T_max, V]     row i: the distribution node i's token was drawn from
+ *                                              (may be NULL when every sequence is greedy)
+ *   draft_tokens device int32 [B, T_max]
+ *   tree_parent  device int32 [B, T_max]
+ *   uniforms     device fp32 [B, T_max+1]      entry i: the uniform of node i's accept test; entry T_max:
+ *                                              the uniform of the final draw (may be NULL when all greedy)
+ *   accepted_path device int32 [B, path_cap]   accepted node indices from the top of the tree down, then -1
+ *   bonus_token  device int32 [B]              the one extra token every step emits
+ *
+ * Per sequence: cur = context.  The children of cur, in ascending index, are Algorithm 1's candidates
+ * against p = target row of cur: candidate i with token t is accepted iff r_i * p^_i(t) < p(t) (that is
+ * r_i < p(t)/p^_i(t)); on rejection p <- norm(max(0, p - p^_i)) over the vocabulary (kept if its mass is
+ * zero).  An accepted child becomes cur and starts again from its own target row.  When no child is
+ * accepted (a leaf included) the bonus token is drawn from p by inverse CDF in ascending token id: the
+ * smallest x with sum_{v<=x} p(v) > u * sum_v p(v).  Greedy sequences move to the lowest-index child whose
+ * token equals argmax p (lowest id on ties), else emit that argmax.  Rows are used as given (not
+ * renormalised).  Scalars and sums are fp64, so decisions agree with an fp64 reference except within
+ * rounding of a boundary.
+ */
+int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, const float* draft_probs,
+                      const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                      int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream);
+
+/*
+ * Tree-mask builder alone (the mask "tree attention" implies: Sec. 3.1, Sec. 3.3): for every node the bit set
+ * of its ancestors and itself, and its depth (top-level nodes: 1).
+ *   tree_parent device int32 [B, T_max]; tree_sizes device int32 [B] or NULL;
+ *   anc_mask device uint64 [B, T_max]; depth device uint8 [B, T_max] or NULL; status device int32 or NULL.
+ * Entries of nodes >= tree size, and of sequences with an invalid tree, are 0.
+ */
+int eagle_tree_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int32_t batch, int32_t max_tree,
+                          uint64_t* anc_mask, uint8_t* depth, int32_t* status, eagle_stream_t stream);
+
+/* Human-readable name of a return / status code (host function; never NULL). */
+const char* eagle_status_string(int code);
+
+/* Number of kernels this library has launched in this process so far (host counter, for accounting). */
+uint64_t eagle_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EAGLE_VERIFY_H_ */

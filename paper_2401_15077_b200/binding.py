@@ -1,0 +1,182 @@
+"""ctypes binding of ``libeagle_verify.so``: argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory and streams are torch's), checks dtypes and
+shapes, fills the C descriptor and calls the C ABI declared in ``include/eagle_verify.h`` on the
+current CUDA stream.  All arithmetic happens in the library's kernels.  There is no fallback: if the
+shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libeagle_verify.so"
+EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_tree_accept",
+           "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count"]
+_lib = None
+
+
+class EagleError(RuntimeError):
+    pass
+
+
+class AttnDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("max_tree", ctypes.c_int32), ("kv_capacity", ctypes.c_int32),
+                ("tree_sizes", ctypes.c_void_p), ("sm_scale", ctypes.c_float), ("num_splits", ctypes.c_int32),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+                ("ev_attn_begin", ctypes.c_void_p), ("ev_attn_end", ctypes.c_void_p)]
+
+
+class AcceptDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("max_tree", ctypes.c_int32), ("vocab", ctypes.c_int32),
+                ("path_cap", ctypes.c_int32), ("tree_sizes", ctypes.c_void_p), ("greedy", ctypes.c_void_p),
+                ("accept_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+def load():
+    """Loads the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise EagleError(f"{LIB_PATH} is missing: build it with `python -m paper_2401_15077_b200.build` "
+                             "(there is no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        vp, i32 = ctypes.c_void_p, ctypes.c_int32
+        lib.eagle_tree_verify_attn_workspace.argtypes = [ctypes.POINTER(AttnDesc)]
+        lib.eagle_tree_verify_attn_workspace.restype = ctypes.c_size_t
+        lib.eagle_tree_verify_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.eagle_tree_verify_attn.restype = ctypes.c_int
+        lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.eagle_tree_accept.restype = ctypes.c_int
+        lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+        lib.eagle_tree_build_mask.restype = ctypes.c_int
+        lib.eagle_status_string.argtypes = [ctypes.c_int]
+        lib.eagle_status_string.restype = ctypes.c_char_p
+        lib.eagle_launch_count.restype = ctypes.c_uint64
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load().eagle_status_string(int(code)).decode()
+
+
+def launch_count() -> int:
+    return int(load().eagle_launch_count())
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise EagleError(f"{what} failed: {rc} ({status_string(rc)})")
+
+
+def _dev(t, dtype, name, allow_none=False):
+    if t is None:
+        if allow_none:
+            return None
+        raise EagleError(f"{name} is required")
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise EagleError(f"{name} must be a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _attn_desc(q, k_cache, tree_sizes, sm_scale, num_splits, workspace, status, events):
+    B, T, Hq, D = q.shape
+    Hkv, S = k_cache.shape[1], k_cache.shape[2]
+    d = AttnDesc(B, Hq, Hkv, D, T, S, _dev(tree_sizes, torch.int32, "tree_sizes", True), float(sm_scale),
+                 int(num_splits), None, 0, _dev(status, torch.int32, "status", True), None, None)
+    if workspace is not None:
+        d.workspace = workspace.data_ptr()
+        d.workspace_bytes = workspace.numel() * workspace.element_size()
+    if events is not None:
+        d.ev_attn_begin, d.ev_attn_end = events[0].cuda_event, events[1].cuda_event
+    return d
+
+
+def eagle_tree_verify_attn_workspace(batch, num_q_heads, num_kv_heads, head_dim, max_tree, num_splits=0) -> int:
+    d = AttnDesc(batch, num_q_heads, num_kv_heads, head_dim, max_tree, 0, None, 0.0, num_splits, None, 0, None, None, None)
+    n = load().eagle_tree_verify_attn_workspace(ctypes.byref(d))
+    if n == 0:
+        raise EagleError("unsupported attention shape")
+    return int(n)
+
+
+def alloc_workspace(q, k_cache, num_splits=0) -> torch.Tensor:
+    """Device scratch for ``eagle_tree_verify_attn`` (uint8, 256-byte aligned by the torch allocator)."""
+    B, T, Hq, D = q.shape
+    n = eagle_tree_verify_attn_workspace(B, Hq, k_cache.shape[1], D, T, num_splits)
+    return torch.empty(n, dtype=torch.uint8, device=q.device)
+
+
+def eagle_tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, out=None, *, tree_sizes=None, sm_scale=0.0,
+                           num_splits=0, workspace=None, status=None, events=None):
+    """Tree-masked attention.  q [B,T,Hq,D] bf16; k_cache/v_cache [B,Hkv,S,D] bf16; seq_lens [B] int32;
+    tree_parent [B,T] int32; returns out [B,T,Hq,D] bf16.  ``events``: optional pair of recorded-capable
+    torch.cuda.Event(enable_timing=True) placed around the attention kernel alone."""
+    lib = load()
+    if q.dim() != 4 or k_cache.dim() != 4 or k_cache.shape != v_cache.shape:
+        raise EagleError("bad tensor ranks / shapes")
+    B, T, Hq, D = q.shape
+    if k_cache.shape[0] != B or k_cache.shape[3] != D or tuple(tree_parent.shape) != (B, T) or tuple(seq_lens.shape) != (B,):
+        raise EagleError("inconsistent shapes")
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = alloc_workspace(q, k_cache, num_splits)
+    d = _attn_desc(q, k_cache, tree_sizes, sm_scale, num_splits, workspace, status, events)
+    rc = lib.eagle_tree_verify_attn(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
+                                    _dev(v_cache, torch.bfloat16, "v_cache"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                    _dev(tree_parent, torch.int32, "tree_parent"), _dev(out, torch.bfloat16, "out"), _stream())
+    _check(rc, "eagle_tree_verify_attn")
+    return out
+
+
+def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, accepted_path=None,
+                      bonus_token=None, *, tree_sizes=None, greedy=None, accept_len=None, status=None, path_cap=None):
+    """Acceptance walk.  target_probs [B,T+1,V] fp32; draft_probs [B,T,V] fp32; draft_tokens/tree_parent [B,T]
+    int32; uniforms [B,T+1] fp32.  Returns (accepted_path [B,path_cap] int32, bonus_token [B] int32)."""
+    lib = load()
+    B, T1, V = target_probs.shape
+    T = T1 - 1
+    dev = target_probs.device
+    cap = T if path_cap is None else int(path_cap)
+    if accepted_path is None:
+        accepted_path = torch.empty((B, cap), dtype=torch.int32, device=dev)
+    if bonus_token is None:
+        bonus_token = torch.empty((B,), dtype=torch.int32, device=dev)
+    if tuple(draft_tokens.shape) != (B, T) or tuple(tree_parent.shape) != (B, T) or tuple(accepted_path.shape) != (B, cap):
+        raise EagleError("inconsistent shapes")
+    if draft_probs is not None and tuple(draft_probs.shape) != (B, T, V):
+        raise EagleError("draft_probs must be [B, T, V]")
+    if uniforms is not None and tuple(uniforms.shape) != (B, T + 1):
+        raise EagleError("uniforms must be [B, T+1]")
+    d = AcceptDesc(B, T, V, cap, _dev(tree_sizes, torch.int32, "tree_sizes", True), _dev(greedy, torch.uint8, "greedy", True),
+                   _dev(accept_len, torch.int32, "accept_len", True), _dev(status, torch.int32, "status", True))
+    rc = lib.eagle_tree_accept(ctypes.byref(d), _dev(target_probs, torch.float32, "target_probs"),
+                               _dev(draft_probs, torch.float32, "draft_probs", True),
+                               _dev(draft_tokens, torch.int32, "draft_tokens"), _dev(tree_parent, torch.int32, "tree_parent"),
+                               _dev(uniforms, torch.float32, "uniforms", True), _dev(accepted_path, torch.int32, "accepted_path"),
+                               _dev(bonus_token, torch.int32, "bonus_token"), _stream())
+    _check(rc, "eagle_tree_accept")
+    return accepted_path, bonus_token
+
+
+def eagle_tree_build_mask(tree_parent, tree_sizes=None, status=None, with_depth=True):
+    """Ancestor-or-self bit masks (int64 tensor holding the uint64 bit pattern) and depths (uint8)."""
+    lib = load()
+    B, T = tree_parent.shape
+    anc = torch.empty((B, T), dtype=torch.int64, device=tree_parent.device)
+    depth = torch.empty((B, T), dtype=torch.uint8, device=tree_parent.device) if with_depth else None
+    rc = lib.eagle_tree_build_mask(_dev(tree_parent, torch.int32, "tree_parent"), _dev(tree_sizes, torch.int32, "tree_sizes", True),
+                                   B, T, anc.data_ptr(), None if depth is None else depth.data_ptr(),
+                                   _dev(status, torch.int32, "status", True), _stream())
+    _check(rc, "eagle_tree_build_mask")
+    return anc, depth

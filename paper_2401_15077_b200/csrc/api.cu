@@ -1,0 +1,205 @@
+// C ABI of the tree-verification library: argument checks, workspace carving and kernel launches.
+// Nothing here allocates or synchronises; every launch goes to the caller's stream.
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace eagle {
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+
+struct DeviceInfo {
+  bool ready = false;
+  int sm_count = 0;
+  int cc_major = 0;
+  bool mma_prepared[2] = {false, false};
+};
+constexpr int kMaxDevices = 64;
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
+
+// Per-device facts, queried once.  Returns nullptr if the current device is unusable.
+DeviceInfo* device_info(int* err) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    *err = EAGLE_ERR_DEVICE;
+    return nullptr;
+  }
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  DeviceInfo& d = g_dev[dev];
+  if (!d.ready) {
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || d.sm_count <= 0) {
+      *err = EAGLE_ERR_DEVICE;
+      return nullptr;
+    }
+    d.ready = true;
+  }
+  if (d.cc_major != 10) {
+    *err = EAGLE_ERR_DEVICE;
+    return nullptr;
+  }
+  return &d;
+}
+
+}  // namespace
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+}  // namespace eagle
+
+using namespace eagle;
+
+extern "C" {
+
+size_t eagle_tree_verify_attn_workspace(const eagle_attn_desc* desc) {
+  if (!desc) return 0;
+  Workspace w;
+  if (!carve_workspace(*desc, nullptr, &w)) return 0;
+  return w.bytes;
+}
+
+int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                           const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const eagle_attn_desc& d = *desc;
+  Workspace w;
+  if (d.kv_capacity < 0 || !carve_workspace(d, d.workspace, &w)) return EAGLE_ERR_SHAPE;
+  if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
+  if (!q || !k_cache || !v_cache || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
+  if (!d.workspace || (reinterpret_cast<uintptr_t>(d.workspace) & 255) || d.workspace_bytes < w.bytes) return EAGLE_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(k_cache) & 15) || (reinterpret_cast<uintptr_t>(v_cache) & 15) ||
+      (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+    return EAGLE_ERR_SHAPE;
+  int err = 0;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int di = d.head_dim == 128 ? 1 : 0;
+  if (!dev->mma_prepared[di]) {
+    if (attn_mma_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
+    dev->mma_prepared[di] = true;
+  }
+  const int G = d.num_q_heads / d.num_kv_heads;
+  const int num_ctas = dev->sm_count * attn_mma_ctas_per_sm(d.head_dim);
+
+  PlanParams pp;
+  pp.seq_lens = seq_lens;
+  pp.tree_sizes = d.tree_sizes;
+  pp.tree_parent = tree_parent;
+  pp.B = d.batch;
+  pp.Hkv = d.num_kv_heads;
+  pp.G = G;
+  pp.T_max = d.max_tree;
+  pp.S_cap = d.kv_capacity;
+  pp.tile_keys = attn_mma_tile_keys();
+  pp.num_ctas = num_ctas;
+  pp.forced_splits = d.num_splits;
+  pp.min_chunk_tiles = 256 / pp.tile_keys > 0 ? 256 / pp.tile_keys : 1;
+  pp.item_cap = w.item_cap;
+  pp.slot_cap = w.slot_cap;
+  pp.hdr = w.hdr;
+  pp.seq = w.seq;
+  pp.anc = w.anc;
+  pp.items = w.items;
+  pp.status = d.status;
+  if (launch_plan(pp, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+
+  AttnParams ap;
+  ap.q = static_cast<const __nv_bfloat16*>(q);
+  ap.k = static_cast<const __nv_bfloat16*>(k_cache);
+  ap.v = static_cast<const __nv_bfloat16*>(v_cache);
+  ap.out = static_cast<__nv_bfloat16*>(out);
+  ap.B = d.batch;
+  ap.Hq = d.num_q_heads;
+  ap.Hkv = d.num_kv_heads;
+  ap.G = G;
+  ap.D = d.head_dim;
+  ap.T_max = d.max_tree;
+  ap.S_cap = d.kv_capacity;
+  const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
+  ap.scale_log2 = scale * 1.4426950408889634f;
+  ap.hdr = w.hdr;
+  ap.seq = w.seq;
+  ap.anc = w.anc;
+  ap.items = w.items;
+  ap.part_ml = w.part_ml;
+  ap.part_o = w.part_o;
+  ap.status = d.status;
+  if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_attn_mma(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, nullptr, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
+
+int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, const float* draft_probs,
+                      const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                      int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const eagle_accept_desc& d = *desc;
+  if (d.batch < 0 || d.max_tree < 0 || d.max_tree > kMaxTree || d.vocab < 1 || d.path_cap < 0) return EAGLE_ERR_SHAPE;
+  if (d.batch == 0) return EAGLE_OK;
+  if (!target_probs || !draft_tokens || !tree_parent || !accepted_path || !bonus_token) return EAGLE_ERR_NULL;
+  // stochastic sequences need the draft rows and the uniforms; only an all-greedy call may omit them
+  if ((!draft_probs || !uniforms) && !d.greedy) return EAGLE_ERR_NULL;
+  int err = 0;
+  if (!device_info(&err)) return err;
+  AcceptParams ap;
+  ap.target = target_probs;
+  ap.draft = draft_probs;
+  ap.tokens = draft_tokens;
+  ap.parent = tree_parent;
+  ap.uniforms = uniforms;
+  ap.tree_sizes = d.tree_sizes;
+  ap.greedy = d.greedy;
+  ap.path = accepted_path;
+  ap.bonus = bonus_token;
+  ap.accept_len = d.accept_len;
+  ap.status = d.status;
+  ap.B = d.batch;
+  ap.T = d.max_tree;
+  ap.V = d.vocab;
+  ap.path_cap = d.path_cap;
+  if (launch_accept(ap, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
+
+int eagle_tree_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int32_t batch, int32_t max_tree,
+                          uint64_t* anc_mask, uint8_t* depth, int32_t* status, eagle_stream_t stream_) {
+  if (batch < 0 || max_tree < 0 || max_tree > kMaxTree) return EAGLE_ERR_SHAPE;
+  if (batch == 0 || max_tree == 0) return EAGLE_OK;
+  if (!tree_parent || !anc_mask) return EAGLE_ERR_NULL;
+  int err = 0;
+  if (!device_info(&err)) return err;
+  if (launch_build_mask(tree_parent, tree_sizes, batch, max_tree, anc_mask, depth, status,
+                        static_cast<cudaStream_t>(stream_)) != cudaSuccess)
+    return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
+
+const char* eagle_status_string(int code) {
+  switch (code) {
+    case EAGLE_OK: return "ok";
+    case EAGLE_ERR_NULL: return "a required pointer is NULL";
+    case EAGLE_ERR_SHAPE: return "unsupported shape or misaligned tensor";
+    case EAGLE_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case EAGLE_ERR_LAUNCH: return "CUDA launch failed";
+    case EAGLE_ERR_TREE: return "invalid tree (parent outside [-1, i-1] or tree size out of range)";
+    case EAGLE_ERR_SEQ: return "invalid sequence length (negative, or prefix + tree exceeds kv_capacity)";
+    case EAGLE_ERR_TOKEN: return "draft token outside the vocabulary";
+    case EAGLE_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case EAGLE_ERR_DEVICE: return "no usable sm_100 device is current";
+    default: return "unknown status";
+  }
+}
+
+uint64_t eagle_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

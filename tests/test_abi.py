@@ -1,0 +1,80 @@
+"""The C-ABI library builds, loads without a GPU, exports what include/eagle_verify.h declares, and its
+host-side argument checks answer before anything is launched."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2401_15077_b200 import build, binding
+    build.build()
+    return binding.load()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2401_15077_b200 import binding
+    header = (ROOT / "include" / "eagle_verify.h").read_text()
+    declared = set(re.findall(r"\b(eagle_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_status_strings(lib):
+    from paper_2401_15077_b200 import binding
+    assert binding.status_string(0) == "ok"
+    seen = {binding.status_string(c) for c in range(-9, 1)}
+    assert len(seen) == 10 and "unknown status" not in seen
+    assert binding.status_string(-1234) == "unknown status"
+
+
+def test_workspace_query_and_shape_checks(lib):
+    from paper_2401_15077_b200 import binding
+    n = binding.eagle_tree_verify_attn_workspace(4, 64, 8, 128, 60)
+    assert n > 0 and n % 256 == 0
+    # forced splits need (units * splits) partial slots
+    assert binding.eagle_tree_verify_attn_workspace(4, 64, 8, 128, 60, num_splits=4) > 0
+    assert binding.eagle_tree_verify_attn_workspace(1, 8, 8, 64, 8, num_splits=1) < n
+    for bad in [dict(head_dim=96), dict(num_q_heads=12, num_kv_heads=8), dict(max_tree=65), dict(num_q_heads=64, num_kv_heads=2)]:
+        kw = dict(batch=1, num_q_heads=8, num_kv_heads=8, head_dim=64, max_tree=8)
+        kw.update(bad)
+        with pytest.raises(binding.EagleError):
+            binding.eagle_tree_verify_attn_workspace(**kw)
+
+
+def test_host_checks_return_before_any_launch(lib):
+    from paper_2401_15077_b200 import binding
+    before = binding.launch_count()
+    assert lib.eagle_tree_verify_attn(None, None, None, None, None, None, None, None) == -1
+    d = binding.AttnDesc(1, 8, 8, 64, 8, 300, None, 0.0, 0, None, 0, None, None, None)
+    # null tensors
+    assert lib.eagle_tree_verify_attn(ctypes.byref(d), None, None, None, None, None, None, None) == -1
+    # batch 0 is a no-op
+    d0 = binding.AttnDesc(0, 8, 8, 64, 8, 300, None, 0.0, 0, None, 0, None, None, None)
+    assert lib.eagle_tree_verify_attn(ctypes.byref(d0), None, None, None, None, None, None, None) == 0
+    # non-null tensors but no workspace
+    fake = ctypes.c_void_p(4096)
+    assert lib.eagle_tree_verify_attn(ctypes.byref(d), fake, fake, fake, fake, fake, fake, None) == -3
+    dbad = binding.AttnDesc(1, 8, 8, 80, 8, 300, None, 0.0, 0, None, 0, None, None, None)
+    assert lib.eagle_tree_verify_attn(ctypes.byref(dbad), fake, fake, fake, fake, fake, fake, None) == -2
+    a = binding.AcceptDesc(1, 65, 10, 8, None, None, None, None)
+    assert lib.eagle_tree_accept(ctypes.byref(a), fake, fake, fake, fake, fake, fake, fake, None) == -2
+    a = binding.AcceptDesc(1, 8, 10, 8, None, None, None, None)
+    assert lib.eagle_tree_accept(ctypes.byref(a), None, fake, fake, fake, fake, fake, fake, None) == -1
+    assert lib.eagle_tree_accept(ctypes.byref(a), fake, None, fake, fake, fake, fake, fake, None) == -1
+    assert lib.eagle_tree_build_mask(None, None, 1, 8, None, None, None, None) == -1
+    assert lib.eagle_tree_build_mask(fake, None, 1, 99, fake, None, None, None) == -2
+    assert binding.launch_count() == before
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    from paper_2401_15077_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", tmp_path / "nope.so")
+    with pytest.raises(binding.EagleError):
+        binding.load()

@@ -1,0 +1,137 @@
+"""Parity of the CUDA acceptance kernel (through the C ABI) with the oracle's walk.  Needs a B200.
+
+Greedy sequences must agree exactly.  Stochastic sequences must agree exactly given the same uniforms,
+except where the oracle itself reports that a decision on its walk came within 1e-5 of its boundary;
+such sequences are counted, and the count is asserted to stay small.
+"""
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+from paper_2401_15077_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+MARGIN = 1e-5
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2401_15077_b200 import build, binding
+    build.build()
+    binding.load()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _gpu_accept(E, inp, greedy_flags=True, path_cap=None, draft=True):
+    d = torch.device("cuda:0")
+    B = inp.target_probs.shape[0]
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    alen = torch.full((B,), -7, dtype=torch.int32, device=d)
+    path, bonus = E.eagle_tree_accept(inp.target_probs.to(d), inp.draft_probs.to(d) if draft else None,
+                                      inp.draft_tokens.to(d), inp.tree_parent.to(d),
+                                      inp.uniforms.to(d) if draft else None, tree_sizes=inp.tree_sizes.to(d),
+                                      greedy=inp.greedy.to(d) if greedy_flags else None, accept_len=alen,
+                                      status=status, path_cap=path_cap)
+    torch.cuda.synchronize()
+    return path.cpu().numpy(), bonus.cpu().numpy(), alen.cpu().numpy(), int(status.item())
+
+
+def _compare(inp, ref, path, bonus, alen):
+    """Returns the number of tolerated (near-boundary) mismatches; asserts on any other."""
+    same = (path == ref["accepted_path"]).all(axis=1) & (bonus == ref["bonus_token"]) & (alen == ref["accept_len"])
+    tolerated = 0
+    for b in np.nonzero(~same)[0]:
+        assert not inp.greedy[b], f"greedy sequence {b} differs"
+        assert ref["min_margin"][b] < MARGIN, (b, ref["min_margin"][b], path[b], ref["accepted_path"][b], bonus[b], ref["bonus_token"][b])
+        tolerated += 1
+    return tolerated
+
+
+CASES = [
+    ("tiny", W.CONFIGS["tiny"], dict(rho=0.9), "none"),
+    ("tiny_greedy", W.CONFIGS["tiny"], dict(rho=0.9, greedy="all"), "all"),
+    ("tiny_rho0", W.CONFIGS["tiny"], dict(rho=0.0), "none"),
+    ("7b_t1", W.CONFIGS["7b_mha"], dict(rho=0.9), "none"),
+    ("7b_t0", W.CONFIGS["7b_mha"], dict(rho=0.9, greedy="all"), "all"),
+    ("70b", W.CONFIGS["70b_gqa"], dict(rho=0.9), "none"),
+    ("70b_rho0", W.CONFIGS["70b_gqa"], dict(rho=0.0), "none"),
+    ("mix_small", W.scaled(W.CONFIGS["serving_mix"], batch=12), dict(rho=0.9), "half"),
+    ("odd_vocab_batch", W.scaled(W.CONFIGS["tiny"], batch=300, tree=(0, 20), vocab=4099), dict(rho=0.7, greedy="half"), "half"),
+    ("small_vocab_batch", W.scaled(W.CONFIGS["tiny"], batch=2000, tree=(0, 14), vocab=37), dict(rho=0.5, greedy="half"), "half"),
+]
+
+
+@pytest.mark.parametrize("name,cfg,kw,mode", CASES, ids=[c[0] for c in CASES])
+def test_accept_matches_oracle(E, oracle, name, cfg, kw, mode):
+    tolerated_total, seqs = 0, 0
+    for salt in range(3 if cfg.batch * cfg.vocab < 4_000_000 else 1):
+        inp = W.make_accept_inputs(cfg, salt=salt, **kw)
+        ref = oracle.tree_accept(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
+                                 tree_sizes=inp.tree_sizes, greedy=inp.greedy)
+        path, bonus, alen, status = _gpu_accept(E, inp)
+        assert status == 0
+        tolerated_total += _compare(inp, ref, path, bonus, alen)
+        seqs += cfg.batch
+    # near-boundary disagreements are possible in principle, but fp64 sums make them very rare
+    assert tolerated_total <= max(1, seqs // 100), tolerated_total
+
+
+def test_all_greedy_without_draft_rows(E, oracle):
+    cfg = W.scaled(W.CONFIGS["7b_mha"], batch=3)
+    inp = W.make_accept_inputs(cfg, salt=9, greedy="all")
+    ref = oracle.tree_accept(inp.target_probs, None, inp.draft_tokens, inp.tree_parent, None, tree_sizes=inp.tree_sizes,
+                             greedy=inp.greedy)
+    path, bonus, alen, status = _gpu_accept(E, inp, draft=False)
+    assert status == 0
+    assert _compare(inp, ref, path, bonus, alen) == 0
+    assert ref["accept_len"].max() >= 1
+
+
+def test_path_cap_and_full_width_tree(E, oracle):
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=40, tree=(64, 64), max_depth=64, vocab=50)
+    inp = W.make_accept_inputs(cfg, salt=1, rho=0.95)
+    ref = oracle.tree_accept(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
+                             tree_sizes=inp.tree_sizes, path_cap=70)
+    path, bonus, alen, status = _gpu_accept(E, inp, greedy_flags=False, path_cap=70)
+    assert status == 0 and path.shape == (40, 70)
+    assert _compare(inp, ref, path, bonus, alen) <= 1
+
+
+def test_invalid_inputs_are_reported(E):
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=4, vocab=64)
+    inp = W.make_accept_inputs(cfg, salt=2)
+    inp.draft_tokens[1, 0] = 64        # outside the vocabulary
+    inp.tree_parent[2, 3] = 5          # parent after child
+    path, bonus, alen, status = _gpu_accept(E, inp)
+    assert status in (-5, -7)
+    assert bonus[1] == -1 and bonus[2] == -1 and alen[1] == 0 and alen[2] == 0
+    assert (path[1] == -1).all() and (path[2] == -1).all()
+    assert bonus[0] >= 0 and bonus[3] >= 0
+
+
+def test_output_distribution_on_gpu_chi_square(E):
+    """The kernel itself preserves the target distribution (Sec. 3.3): 16-token vocabulary, 3 children of the
+    context, tokens re-drawn per trial, one batched call of 1e5 trees."""
+    V, n = 16, 100_000
+    rng = np.random.default_rng(99)
+    p_root = rng.dirichlet(np.ones(V)).astype(np.float32)
+    q_root = rng.dirichlet(np.ones(V)).astype(np.float32)
+    T = 3
+    cdf = np.cumsum(q_root.astype(np.float64) / q_root.astype(np.float64).sum())
+    tokens = np.searchsorted(cdf, rng.random((n, T)), side="right").clip(0, V - 1).astype(np.int32)
+    target = np.broadcast_to(p_root, (n, T + 1, V)).copy()
+    draft = np.broadcast_to(q_root, (n, T, V)).copy()
+    parent = np.full((n, T), -1, np.int32)
+    un = rng.random((n, T + 1), dtype=np.float32)
+    d = torch.device("cuda:0")
+    alen = torch.zeros(n, dtype=torch.int32, device=d)
+    path, bonus = E.eagle_tree_accept(torch.from_numpy(target).to(d), torch.from_numpy(draft).to(d),
+                                      torch.from_numpy(tokens).to(d), torch.from_numpy(parent).to(d),
+                                      torch.from_numpy(un).to(d), accept_len=alen)
+    torch.cuda.synchronize()
+    path, bonus, alen = path.cpu().numpy(), bonus.cpu().numpy(), alen.cpu().numpy()
+    first = np.where(alen > 0, tokens[np.arange(n), np.maximum(path[:, 0], 0)], bonus)
+    pr = p_root.astype(np.float64) / p_root.astype(np.float64).sum()
+    assert stats.chisquare(np.bincount(first, minlength=V), pr * n).pvalue > 1e-3

@@ -1,0 +1,176 @@
+"""Parity of the CUDA tree attention (through the C ABI) with the fp64 oracle.  Needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2401_15077_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3   # unit-variance bf16 inputs: bounds on |gpu - oracle|
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2401_15077_b200 import build, binding
+    build.build()
+    binding.load()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _to_dev(inp):
+    d = torch.device("cuda:0")
+    return dict(q=inp.q.to(d), k=inp.k_cache.to(d), v=inp.v_cache.to(d), sl=inp.seq_lens.to(d),
+                par=inp.tree_parent.to(d), ts=inp.tree_sizes.to(d))
+
+
+def _run(E, inp, num_splits=0, use_sizes=True, sm_scale=0.0):
+    t = _to_dev(inp)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    out = torch.full_like(t["q"], float("nan"))
+    E.eagle_tree_verify_attn(t["q"], t["k"], t["v"], t["sl"], t["par"], out, tree_sizes=t["ts"] if use_sizes else None,
+                             num_splits=num_splits, status=status, sm_scale=sm_scale)
+    torch.cuda.synchronize()
+    return out.cpu(), int(status.item())
+
+
+def _check(out, ref, sizes):
+    got = out.double().numpy()
+    assert np.isfinite(got).all()
+    err = np.abs(got - ref)
+    rows = np.zeros(ref.shape[:2], bool)
+    for b, n in enumerate(sizes):
+        rows[b, :int(n)] = True
+        assert np.all(got[b, int(n):] == 0.0), "rows past the tree size must be zero"
+    if rows.any():
+        assert err[rows].max() <= MAX_ABS, err[rows].max()
+        assert err[rows].mean() <= MEAN_ABS, err[rows].mean()
+    return float(err.max())
+
+
+CASES = {
+    "tiny": W.CONFIGS["tiny"],
+    "7b_mha": W.CONFIGS["7b_mha"],
+    "70b_gqa_b2": W.scaled(W.CONFIGS["70b_gqa"], batch=2),
+    "mixtral_gqa_small": W.scaled(W.CONFIGS["mixtral_gqa"], batch=2, prefix=(1500, 3000)),
+    "serving_mix_small": W.scaled(W.CONFIGS["serving_mix"], batch=6, prefix=(100, 1500)),
+    "d64_gqa_ragged": W.scaled(W.CONFIGS["tiny"], batch=5, num_q_heads=16, num_kv_heads=4, prefix=(0, 700), tree=(1, 33)),
+    "big_group_full_tree": W.scaled(W.CONFIGS["70b_gqa"], batch=2, num_q_heads=32, num_kv_heads=2, prefix=(130, 400),
+                                    tree=(64, 64), max_depth=64, child_cap=0),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_attention_matches_oracle(E, oracle, name):
+    cfg = CASES[name]
+    inp = W.make_attn_inputs(cfg, capacity_pad=37)
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    out, status = _run(E, inp)
+    assert status == 0
+    _check(out, ref, inp.tree_sizes)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7, 64])
+def test_forced_splits_agree(E, oracle, splits):
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=3, prefix=(60, 900), tree=(5, 40))
+    inp = W.make_attn_inputs(cfg, salt=2)
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    out, status = _run(E, inp, num_splits=splits)
+    assert status == 0
+    _check(out, ref, inp.tree_sizes)
+    again, _ = _run(E, inp, num_splits=splits)
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16)), "same call twice must be bit-identical"
+
+
+def test_chain_tree_no_sizes_custom_scale(E, oracle):
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=2, prefix=(0, 90), tree=(9, 9))
+    inp = W.make_attn_inputs(cfg, salt=4, poison=True)
+    inp.tree_parent[:] = torch.arange(-1, 8, dtype=torch.int32)
+    assert int(inp.seq_lens.min()) >= 0
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, None, sm_scale=0.21)
+    out, status = _run(E, inp, use_sizes=False, sm_scale=0.21)
+    assert status == 0
+    _check(out, ref, [9, 9])
+
+
+def test_empty_prefix_empty_tree_and_single_node(E, oracle):
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=4, prefix=(0, 0), tree=(1, 6))
+    inp = W.make_attn_inputs(cfg, salt=5)
+    inp.tree_sizes[1] = 0
+    inp.tree_sizes[2] = 1
+    inp.seq_lens[3] = 70
+    # regenerate the cache of sequence 3 so that its longer prefix is filled
+    g = torch.Generator().manual_seed(5)
+    cap = 70 + cfg.max_tree
+    k = torch.full((4, cfg.num_kv_heads, cap, cfg.head_dim), float("nan"), dtype=torch.bfloat16)
+    v = k.clone()
+    k[:, :, :inp.kv_capacity] = inp.k_cache
+    v[:, :, :inp.kv_capacity] = inp.v_cache
+    k[3] = torch.randn(k[3].shape, generator=g).to(torch.bfloat16)
+    v[3] = torch.randn(v[3].shape, generator=g).to(torch.bfloat16)
+    inp.k_cache, inp.v_cache = k, v
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    out, status = _run(E, inp)
+    assert status == 0
+    _check(out, ref, inp.tree_sizes)
+
+
+def test_invalid_inputs_are_reported_not_trapped(E, oracle):
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=3, prefix=(20, 50), tree=(4, 8))
+    inp = W.make_attn_inputs(cfg, salt=6)
+    good_ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    bad = W.make_attn_inputs(cfg, salt=6)
+    bad.tree_parent[1, 2] = 2          # parent must be < node index
+    out, status = _run(E, bad)
+    assert status == -5
+    got = out.double().numpy()
+    assert np.all(got[1] == 0.0)       # the invalid sequence is zeroed
+    for b in (0, 2):                   # the others are still right
+        n = int(inp.tree_sizes[b])
+        assert np.abs(got[b, :n] - good_ref[b, :n]).max() <= MAX_ABS
+    bad2 = W.make_attn_inputs(cfg, salt=6)
+    bad2.seq_lens[0] = bad2.kv_capacity   # prefix + tree does not fit the cache
+    out, status = _run(E, bad2)
+    assert status == -6 and np.all(out.double().numpy()[0] == 0.0)
+
+
+def test_mask_builder_matches_oracle(E, oracle):
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=50, tree=(0, 64), max_depth=64)
+    sizes, parent = W.make_trees(cfg, salt=7)
+    anc_ref, depth_ref = oracle.tree_ancestors(parent.numpy(), sizes.numpy())
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    anc, depth = E.eagle_tree_build_mask(parent.cuda(), sizes.cuda(), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(anc.cpu().numpy().view(np.uint64), anc_ref)
+    assert np.array_equal(depth.cpu().numpy().astype(np.int32), depth_ref)
+
+
+@pytest.mark.parametrize("name", ["mixtral_gqa", "serving_mix"])
+def test_full_size_sampled_rows(E, oracle, name):
+    """Full BASELINE sizes in the bench's launch configuration; the oracle checks sampled (sequence, KV head)
+    units, and cheap properties are checked everywhere."""
+    cfg = W.CONFIGS[name]
+    inp = W.make_attn_inputs(cfg)
+    out, status = _run(E, inp)
+    assert status == 0
+    got = out.double().numpy()
+    assert np.isfinite(got).all()
+    for b in range(cfg.batch):
+        assert np.all(got[b, int(inp.tree_sizes[b]):] == 0.0)
+    G = cfg.num_q_heads // cfg.num_kv_heads
+    rng = np.random.default_rng(0)
+    lens = inp.seq_lens.numpy()
+    picks = {(int(np.argmax(lens)), 0), (int(np.argmin(lens)), cfg.num_kv_heads - 1)}
+    while len(picks) < 4:
+        picks.add((int(rng.integers(cfg.batch)), int(rng.integers(cfg.num_kv_heads))))
+    for b, g in sorted(picks):
+        n = int(inp.tree_sizes[b])
+        end = int(lens[b]) + n
+        ref = oracle.tree_verify_attn(inp.q[b:b + 1, :, g * G:(g + 1) * G].contiguous(),
+                                      inp.k_cache[b:b + 1, g:g + 1, :end].contiguous(),
+                                      inp.v_cache[b:b + 1, g:g + 1, :end].contiguous(),
+                                      inp.seq_lens[b:b + 1], inp.tree_parent[b:b + 1], inp.tree_sizes[b:b + 1])
+        err = np.abs(got[b, :n, g * G:(g + 1) * G] - ref[0, :n])
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (b, g, err.max(), err.mean())
