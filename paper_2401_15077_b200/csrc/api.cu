@@ -19,6 +19,7 @@ struct DeviceInfo {
   int sm_count = 0;
   int cc_major = 0;
   bool mma_prepared[2] = {false, false};
+  bool tc_prepared[2] = {false, false};
 };
 constexpr int kMaxDevices = 64;
 DeviceInfo g_dev[kMaxDevices];
@@ -82,12 +83,18 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   if (!dev) return err;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int di = d.head_dim == 128 ? 1 : 0;
-  if (!dev->mma_prepared[di]) {
+  const char* impl_env = std::getenv("EAGLE_ATTN_IMPL");
+  const bool use_tc = impl_env && std::strcmp(impl_env, "tc") == 0;
+  if (use_tc && !dev->tc_prepared[di]) {
+    if (attn_tc_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
+    dev->tc_prepared[di] = true;
+  }
+  if (!use_tc && !dev->mma_prepared[di]) {
     if (attn_mma_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
     dev->mma_prepared[di] = true;
   }
   const int G = d.num_q_heads / d.num_kv_heads;
-  const int num_ctas = dev->sm_count * attn_mma_ctas_per_sm(d.head_dim);
+  const int num_ctas = use_tc ? dev->sm_count : dev->sm_count * attn_mma_ctas_per_sm(d.head_dim);
 
   PlanParams pp;
   pp.seq_lens = seq_lens;
@@ -98,7 +105,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.G = G;
   pp.T_max = d.max_tree;
   pp.S_cap = d.kv_capacity;
-  pp.tile_keys = attn_mma_tile_keys();
+  pp.tile_keys = use_tc ? attn_tc_tile_keys() : attn_mma_tile_keys();
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
   pp.min_chunk_tiles = 256 / pp.tile_keys > 0 ? 256 / pp.tile_keys : 1;
@@ -133,7 +140,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.part_o = w.part_o;
   ap.status = d.status;
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_attn_mma(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if ((use_tc ? launch_attn_tc(ap, num_ctas, stream) : launch_attn_mma(ap, num_ctas, stream)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_combine(ap, nullptr, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;

@@ -138,6 +138,9 @@ cudaError_t launch_attn_mma(const AttnParams& p, int num_ctas, cudaStream_t stre
 int attn_mma_tile_keys();
 int attn_mma_ctas_per_sm(int head_dim);
 cudaError_t attn_mma_prepare(int head_dim);
+cudaError_t launch_attn_tc(const AttnParams& p, int num_ctas, cudaStream_t stream);
+int attn_tc_tile_keys();
+cudaError_t attn_tc_prepare(int head_dim);
 cudaError_t launch_combine(const AttnParams& p, const int32_t* tree_sizes_unused, cudaStream_t stream);
 
 cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream);
