@@ -159,9 +159,12 @@ def main():
     ap.add_argument("--ref-seqs", type=int, default=1, help="sequences per step of the reference arm")
     ap.add_argument("--num-splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling captures on a smaller case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     cfg = W.CONFIGS[args.workload]
+    if args.batch > 0:
+        cfg = W.scaled(cfg, batch=args.batch)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -1,53 +1,93 @@
 // Acceptance along the draft tree: Algorithm 1 (multi-round speculative sampling, App. A.2) applied at every
 // node from the committed context down (Sec. 3.3), or the greedy rule (Preliminaries).
 //
-// One team of threads walks one tree: a warp when the vocabulary is small (many trees per launch), a whole
-// CTA otherwise.  Every thread of the team carries the same walk state; the vocabulary-wide steps (residual
-// mass after a rejection, the final inverse-CDF draw, the greedy argmax) are spread over the team and reduced
-// with warp shuffles (plus one shared-memory hop for a CTA team).  All sums and scalars are fp64.
+// One team of threads walks one tree; every thread of the team carries the same walk state, and the
+// vocabulary-wide steps (residual mass after a rejection, the final inverse-CDF draw, the greedy argmax) are
+// spread over the team.  A team is
+//   - one warp when the vocabulary is small (many trees per CTA), or
+//   - a thread-block cluster of 1, 2, 4 or 8 CTAs of 512 threads (fewer trees -> wider teams, so that one
+//     tree's 128 KB rows are pulled by several SMs at once); partial results cross CTAs through
+//     distributed shared memory and a cluster barrier.
+// Thread g of a team owns the contiguous token range [g*chunk, (g+1)*chunk) in every sweep, so prefix sums in
+// token order need one scan of per-thread sums.  All sums and scalars are fp64; reductions combine partials
+// in a fixed order, so a call is reproducible bit for bit.
 //
-// After m rejections at a node the residual distribution is not stored: an element is recomputed from the
-// target row, the m rejected candidates' draft rows and their m normalisers,
-//   x <- p(v);  for each rejected candidate j in order:  x <- max(0, x - p^_j(v)) / Z_j,
-// which is exactly the sequence of updates Algorithm 1 performs (rows are L2-resident after their first use).
+// After m rejections at a node the residual is not stored but recomputed, unnormalised, from the target row,
+// the rejected candidates' draft rows and m scalars:  u_0 = p, W_0 = 1,
+//   u_k(v) = max(0, u_{k-1}(v) - W_{k-1} * p^_k(v)),   W_k = sum_v u_k(v),
+// so that Algorithm 1's normalised residual is u_m / W_m, its accept test r < p(t)/p^(t) reads
+// r * p^(t) * W_m < u_m(t), and the final draw (scale-free) is taken from u_m.  No division is needed.
 #include "common.cuh"
 
 namespace eagle {
 
 namespace {
 
-constexpr int kCtaTeam = 512;
+constexpr int kCtaThreads = 512;
 constexpr int kWarpTeamsPerCta = 8;
+constexpr int kMaxCluster = 8;
 
-template <int NT>
-struct TeamScratch {
-  double d[NT / 32 > 0 ? NT / 32 : 1];
-  unsigned long long u[NT / 32 > 0 ? NT / 32 : 1];
-};
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void dsmem_store_u64(const void* local_smem, uint32_t cta, unsigned long long v) {
+  const uint32_t a = static_cast<uint32_t>(__cvta_generic_to_shared(local_smem));
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(cta));
+  asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(ra), "l"(v) : "memory");
+}
 
-template <int NT>
+// NT threads per CTA (32: a warp is the team), CL CTAs per team.
+template <int NT, int CL>
 struct Team {
-  int rank;
-  TeamScratch<NT>* sc;
+  static constexpr int kWarps = NT / 32;
+  struct Scratch {
+    unsigned long long warp[kWarps > 0 ? kWarps : 1];
+    unsigned long long xch[2][kMaxCluster];   // all-gather slots, double buffered
+  };
+  Scratch* sc;
+  int tid;        // thread within the CTA (or lane, for a warp team)
+  int cta;        // CTA rank within the cluster
+  int phase;      // which xch buffer the next cross-CTA exchange uses
 
-  __device__ __forceinline__ void sync() const {
+  __device__ __forceinline__ int rank() const { return cta * NT + tid; }
+  static constexpr int kSize = NT * CL;
+
+  __device__ __forceinline__ void sync_cta() const {
     if (NT == 32) __syncwarp();
     else __syncthreads();
   }
-  // Sum over the team; every thread gets the same value, combined in a fixed order.
-  __device__ double sum(double v) const {
+  // every CTA publishes one 64-bit word to all CTAs; afterwards xch[buf][c] holds CTA c's word everywhere
+  __device__ __forceinline__ int exchange(unsigned long long mine) {
+    const int buf = phase;
+    phase ^= 1;
+    if (tid < CL) dsmem_store_u64(&sc->xch[buf][cta], static_cast<uint32_t>(tid), mine);
+    cluster_sync_all();
+    return buf;
+  }
+  __device__ double sum(double v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     if (NT == 32) return v;
     __syncthreads();
-    if ((rank & 31) == 0) sc->d[rank >> 5] = v;
+    if ((tid & 31) == 0) sc->warp[tid >> 5] = __double_as_longlong(v);
     __syncthreads();
     double t = 0.0;
 #pragma unroll
-    for (int w = 0; w < NT / 32; ++w) t += sc->d[w];
-    return t;
+    for (int w = 0; w < kWarps; ++w) t += __longlong_as_double(sc->warp[w]);
+    if (CL == 1) return t;
+    const int buf = exchange(__double_as_longlong(t));
+    double a = 0.0;
+#pragma unroll
+    for (int c = 0; c < CL; ++c) a += __longlong_as_double(sc->xch[buf][c]);
+    return a;
   }
-  __device__ unsigned long long max_u64(unsigned long long v) const {
+  __device__ unsigned long long max_u64(unsigned long long v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       const unsigned long long x = __shfl_xor_sync(0xffffffffu, v, o);
@@ -55,38 +95,55 @@ struct Team {
     }
     if (NT == 32) return v;
     __syncthreads();
-    if ((rank & 31) == 0) sc->u[rank >> 5] = v;
+    if ((tid & 31) == 0) sc->warp[tid >> 5] = v;
     __syncthreads();
     unsigned long long t = 0ull;
 #pragma unroll
-    for (int w = 0; w < NT / 32; ++w) t = sc->u[w] > t ? sc->u[w] : t;
-    return t;
+    for (int w = 0; w < kWarps; ++w) t = sc->warp[w] > t ? sc->warp[w] : t;
+    if (CL == 1) return t;
+    const int buf = exchange(t);
+    unsigned long long a = 0ull;
+#pragma unroll
+    for (int c = 0; c < CL; ++c) a = sc->xch[buf][c] > a ? sc->xch[buf][c] : a;
+    return a;
   }
-  // Exclusive prefix of v in rank order, and the team total.
-  __device__ double exclusive_scan(double v, double* total) const {
+  // exclusive prefix of v in team-rank order, and the team total
+  __device__ double exclusive_scan(double v, double* total) {
     double inc = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const double x = __shfl_up_sync(0xffffffffu, inc, o);
-      if ((rank & 31) >= o) inc += x;
-    }
-    double before = 0.0;
-    if (NT == 32) {
-      *total = __shfl_sync(0xffffffffu, inc, 31);
-    } else {
-      __syncthreads();
-      if ((rank & 31) == 31) sc->d[rank >> 5] = inc;
-      __syncthreads();
-      double t = 0.0;
-#pragma unroll
-      for (int w = 0; w < NT / 32; ++w) {
-        if (w == (rank >> 5)) before = t;
-        t += sc->d[w];
-      }
-      *total = t;
+      if ((tid & 31) >= o) inc += x;
     }
     const double prev = __shfl_up_sync(0xffffffffu, inc, 1);
-    return before + ((rank & 31) ? prev : 0.0);
+    double before = (tid & 31) ? prev : 0.0;
+    if (NT == 32) {
+      *total = __shfl_sync(0xffffffffu, inc, 31);
+      return before;
+    }
+    __syncthreads();
+    if ((tid & 31) == 31) sc->warp[tid >> 5] = __double_as_longlong(inc);
+    __syncthreads();
+    double t = 0.0, warp_before = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+      if (w == (tid >> 5)) warp_before = t;
+      t += __longlong_as_double(sc->warp[w]);
+    }
+    before = warp_before + before;
+    if (CL == 1) {
+      *total = t;
+      return before;
+    }
+    const int buf = exchange(__double_as_longlong(t));
+    double a = 0.0, cta_before = 0.0;
+#pragma unroll
+    for (int c = 0; c < CL; ++c) {
+      if (c == cta) cta_before = a;
+      a += __longlong_as_double(sc->xch[buf][c]);
+    }
+    *total = a;
+    return cta_before + before;
   }
 };
 
@@ -95,41 +152,57 @@ __device__ __forceinline__ unsigned int ordered_bits(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-struct Chain {
+// The residual after the rejections recorded so far, evaluated on the fly.
+struct Residual {
   const float* target_row;
   const float* draft_base;  // draft rows of this sequence
   const int* rej;           // rejected candidates at the current node, in order
-  const double* Z;          // their normalisers
-  int n_rej;
+  const double* scale;      // scale[k] = W_k, the mass of the residual before rejection k+1 (W_0 = 1)
+  int m;                    // rejections recorded
   int V;
-  // residual probability of token v after the rejections recorded so far
+
   __device__ __forceinline__ double at(int v) const {
-    double x = static_cast<double>(target_row[v]);
-    for (int j = 0; j < n_rej; ++j) {
-      const double d = x - static_cast<double>(draft_base[static_cast<size_t>(rej[j]) * V + v]);
-      x = (d > 0.0 ? d : 0.0) / Z[j];
-    }
+    double x = static_cast<double>(__ldg(target_row + v));
+    for (int k = 0; k < m; ++k)
+      x = fmax(0.0, fma(-scale[k], static_cast<double>(__ldg(draft_base + static_cast<size_t>(rej[k]) * V + v)), x));
     return x;
+  }
+  // four consecutive tokens starting at v (v % 4 == 0, rows 16-byte aligned)
+  __device__ __forceinline__ void at4(int v, double (&x)[4]) const {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(target_row + v));
+    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+    for (int k = 0; k < m; ++k) {
+      const float4 q = __ldg(reinterpret_cast<const float4*>(draft_base + static_cast<size_t>(rej[k]) * V + v));
+      const double w = -scale[k];
+      x[0] = fmax(0.0, fma(w, static_cast<double>(q.x), x[0]));
+      x[1] = fmax(0.0, fma(w, static_cast<double>(q.y), x[1]));
+      x[2] = fmax(0.0, fma(w, static_cast<double>(q.z), x[2]));
+      x[3] = fmax(0.0, fma(w, static_cast<double>(q.w), x[3]));
+    }
   }
 };
 
-template <int NT>
+struct TreeSmem {
+  int par[kMaxTree], tok[kMaxTree], rej[kMaxTree];
+  double scale[kMaxTree];
+};
+
+template <int NT, int CL>
 __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_kernel(AcceptParams p) {
+  using TeamT = Team<NT, CL>;
   constexpr int TEAMS = NT == 32 ? kWarpTeamsPerCta : 1;
-  __shared__ TeamScratch<NT> s_scratch[TEAMS];
-  __shared__ int s_par[TEAMS][kMaxTree], s_tok[TEAMS][kMaxTree], s_rej[TEAMS][kMaxTree];
-  __shared__ double s_Z[TEAMS][kMaxTree];
+  __shared__ typename TeamT::Scratch s_scratch[TEAMS];
+  __shared__ TreeSmem s_tree[TEAMS];
 
   const int team_id = NT == 32 ? (threadIdx.x >> 5) : 0;
-  const int b = NT == 32 ? blockIdx.x * TEAMS + team_id : blockIdx.x;
-  if (b >= p.B) return;   // a whole team leaves together (a warp, or the CTA)
-  Team<NT> team;
-  team.rank = NT == 32 ? (threadIdx.x & 31) : threadIdx.x;
+  TeamT team;
+  team.tid = NT == 32 ? (threadIdx.x & 31) : threadIdx.x;
+  team.cta = CL > 1 ? static_cast<int>(cluster_ctarank()) : 0;
+  team.phase = 0;
   team.sc = &s_scratch[team_id];
-  int* par = s_par[team_id];
-  int* tok = s_tok[team_id];
-  int* rej = s_rej[team_id];
-  double* Zs = s_Z[team_id];
+  const int b = NT == 32 ? blockIdx.x * TEAMS + team_id : static_cast<int>(blockIdx.x) / CL;
+  if (b >= p.B) return;   // a whole team leaves together (a warp; clusters are launched exactly)
+  TreeSmem& ts = s_tree[team_id];
 
   const int T = p.T, V = p.V;
   int n = p.tree_sizes ? p.tree_sizes[b] : T;
@@ -137,35 +210,42 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
   int bad = (n < 0 || n > T) ? EAGLE_ERR_TREE : 0;
   if (!bad && !is_greedy && (!p.draft || !p.uniforms)) bad = EAGLE_ERR_NULL;  // a stochastic walk needs both
   if (bad) n = 0;
-  for (int i = team.rank; i < n; i += NT) {
-    const int pi = p.parent[static_cast<size_t>(b) * T + i];
-    const int ti = p.tokens[static_cast<size_t>(b) * T + i];
-    par[i] = pi;
-    tok[i] = ti;
+  for (int i = team.tid; i < n; i += NT) {
+    ts.par[i] = p.parent[static_cast<size_t>(b) * T + i];
+    ts.tok[i] = p.tokens[static_cast<size_t>(b) * T + i];
   }
-  team.sync();
+  team.sync_cta();
   if (!bad) {
     // every thread checks every node, so the verdict is the same everywhere
     for (int i = 0; i < n; ++i) {
-      if (par[i] < -1 || par[i] >= i) bad = EAGLE_ERR_TREE;
-      else if (tok[i] < 0 || tok[i] >= V) bad = bad ? bad : EAGLE_ERR_TOKEN;
+      if (ts.par[i] < -1 || ts.par[i] >= i) bad = EAGLE_ERR_TREE;
+      else if (ts.tok[i] < 0 || ts.tok[i] >= V) bad = bad ? bad : EAGLE_ERR_TOKEN;
     }
   }
+  const bool writer = team.rank() == 0;
   int32_t* path = p.path + static_cast<size_t>(b) * p.path_cap;
-  for (int j = team.rank; j < p.path_cap; j += NT) path[j] = -1;
+  if (team.cta == 0)
+    for (int j = team.tid; j < p.path_cap; j += NT) path[j] = -1;
   if (bad) {
-    if (team.rank == 0) {
+    if (writer) {
       report_status(p.status, bad);
       p.bonus[b] = -1;
       if (p.accept_len) p.accept_len[b] = 0;
     }
-    return;
+    return;   // uniform over the team: nobody is left waiting at a cluster barrier
   }
-  team.sync();   // the -1 fill is ordered before the path entries written below (same team)
+  team.sync_cta();   // the -1 fill is ordered before the path entries written below (same CTA)
 
   const float* target_b = p.target + static_cast<size_t>(b) * (T + 1) * V;
   const float* draft_b = p.draft ? p.draft + static_cast<size_t>(b) * T * V : nullptr;
   const float* uni_b = p.uniforms ? p.uniforms + static_cast<size_t>(b) * (T + 1) : nullptr;
+
+  // token range of this thread; vector loads need V % 4 == 0 (then every row starts 16-byte aligned)
+  const bool vec = (V & 3) == 0 && (reinterpret_cast<uintptr_t>(p.target) & 15) == 0 &&
+                   (p.draft == nullptr || (reinterpret_cast<uintptr_t>(p.draft) & 15) == 0);
+  int chunk = (V + TeamT::kSize - 1) / TeamT::kSize;
+  chunk = (chunk + 3) & ~3;
+  const int v0 = min(team.rank() * chunk, V), v1 = min(v0 + chunk, V);
 
   int cur = -1, len = 0, bonus = -1;
   for (;;) {
@@ -174,113 +254,188 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
     if (is_greedy) {
       // argmax, lowest token id on ties: key = (ordered value, ~id)
       unsigned long long best = 0ull;
-      for (int v = team.rank; v < V; v += NT) {
-        const unsigned long long key = (static_cast<unsigned long long>(ordered_bits(prow[v])) << 32) |
-                                       static_cast<unsigned int>(~static_cast<unsigned int>(v));
+      auto consider = [&](float f, int v) {
+        const unsigned long long key = (static_cast<unsigned long long>(ordered_bits(f)) << 32) | static_cast<unsigned int>(~static_cast<unsigned int>(v));
         best = key > best ? key : best;
+      };
+      if (vec) {
+#pragma unroll 4
+        for (int v = v0; v < v1; v += 4) {
+          const float4 t = __ldg(reinterpret_cast<const float4*>(prow + v));
+          consider(t.x, v); consider(t.y, v + 1); consider(t.z, v + 2); consider(t.w, v + 3);
+        }
+      } else {
+        for (int v = v0; v < v1; ++v) consider(__ldg(prow + v), v);
       }
       best = team.max_u64(best);
       const int a = static_cast<int>(~static_cast<unsigned int>(best & 0xffffffffull));
       for (int i = 0; i < n && next < 0; ++i)
-        if (par[i] == cur && tok[i] == a) next = i;
+        if (ts.par[i] == cur && ts.tok[i] == a) next = i;
       if (next < 0) bonus = a;
     } else {
-      Chain ch{prow, draft_b, rej, Zs, 0, V};
+      Residual res{prow, draft_b, ts.rej, ts.scale, 0, V};
+      double W = 1.0;   // mass of the current residual
       for (int i = 0; i < n && next < 0; ++i) {
-        if (par[i] != cur) continue;
+        if (ts.par[i] != cur) continue;
         const float* qrow = draft_b + static_cast<size_t>(i) * V;
-        const int t = tok[i];
+        const int t = ts.tok[i];
         const double r = static_cast<double>(uni_b[i]);
-        const double pt = ch.at(t), qt = static_cast<double>(qrow[t]);
-        if (r * qt < pt) {
+        const double ut = res.at(t), qt = static_cast<double>(__ldg(qrow + t));
+        if (r * qt * W < ut) {
           next = i;
         } else {
-          // mass of max(0, p - p^_i) over the vocabulary
+          // mass of max(0, u - W * p^_i) over the vocabulary
           double z = 0.0;
-          for (int v = team.rank; v < V; v += NT) {
-            const double d = ch.at(v) - static_cast<double>(qrow[v]);
-            z += d > 0.0 ? d : 0.0;
+          if (vec) {
+#pragma unroll 4
+            for (int v = v0; v < v1; v += 4) {
+              double x[4];
+              res.at4(v, x);
+              const float4 q = __ldg(reinterpret_cast<const float4*>(qrow + v));
+              z += fmax(0.0, fma(-W, static_cast<double>(q.x), x[0]));
+              z += fmax(0.0, fma(-W, static_cast<double>(q.y), x[1]));
+              z += fmax(0.0, fma(-W, static_cast<double>(q.z), x[2]));
+              z += fmax(0.0, fma(-W, static_cast<double>(q.w), x[3]));
+            }
+          } else {
+            for (int v = v0; v < v1; ++v) z += fmax(0.0, fma(-W, static_cast<double>(__ldg(qrow + v)), res.at(v)));
           }
           z = team.sum(z);
           if (z > 0.0) {           // zero residual mass: the distribution is kept as it is
-            team.sync();           // nobody still reads the list with the old length
-            if (team.rank == 0) {
-              rej[ch.n_rej] = i;
-              Zs[ch.n_rej] = z;
+            // entry res.m is not read by anyone yet (readers stop at res.m), so it can be written in place
+            if (team.tid == 0) {
+              ts.rej[res.m] = i;
+              ts.scale[res.m] = W;
             }
-            team.sync();
-            ch.n_rej += 1;
+            team.sync_cta();
+            res.m += 1;
+            W = z;
           }
         }
       }
       if (next < 0) {
-        // inverse CDF in ascending token id: contiguous chunk per thread, scan of chunk sums, rescan of one chunk
+        // final draw by inverse CDF over the residual, ascending token id: per-thread sums of contiguous
+        // ranges, one scan, then the owning thread walks its own range
         const double u = static_cast<double>(uni_b[T]);
-        const int chunk = (V + NT - 1) / NT;
-        const int v0 = team.rank * chunk < V ? team.rank * chunk : V;
-        const int v1 = v0 + chunk < V ? v0 + chunk : V;
         double s = 0.0;
         int last_pos = -1;
-        for (int v = v0; v < v1; ++v) {
-          const double x = ch.at(v);
-          if (x > 0.0) last_pos = v;
-          s += x;
+        if (vec) {
+#pragma unroll 4
+          for (int v = v0; v < v1; v += 4) {
+            double x[4];
+            res.at4(v, x);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              s += x[e];
+              if (x[e] > 0.0) last_pos = v + e;
+            }
+          }
+        } else {
+          for (int v = v0; v < v1; ++v) {
+            const double x = res.at(v);
+            s += x;
+            if (x > 0.0) last_pos = v;
+          }
         }
         double total;
         const double before = team.exclusive_scan(s, &total);
         const double thr = u * total;
         const bool mine = before + s > thr;
-        // first thread (lowest rank) whose inclusive prefix passes the threshold; else the last positive token
-        const unsigned long long key_owner = mine ? (0x100000000ull | static_cast<unsigned int>(~static_cast<unsigned int>(team.rank))) : 0ull;
-        const unsigned long long key_last = static_cast<unsigned long long>(static_cast<unsigned int>(last_pos + 1));
-        const unsigned long long w_owner = team.max_u64(key_owner);
-        int x_found = -1;
-        if (w_owner) {
-          const int owner = static_cast<int>(~static_cast<unsigned int>(w_owner & 0xffffffffull));
-          unsigned long long key_x = 0ull;
-          if (team.rank == owner) {
-            double c = 0.0;
-            for (int v = v0; v < v1; ++v) {
-              c += ch.at(v);
+        // the first thread (lowest rank) whose inclusive prefix passes the threshold finds the token inside its
+        // range by repeating exactly the additions that produced s
+        unsigned long long key = 0ull;
+        if (mine) {
+          int x_found = v1 - 1;
+          double c = 0.0;
+          bool found = false;
+          if (vec) {
+            for (int v = v0; v < v1 && !found; v += 4) {
+              double x[4];
+              res.at4(v, x);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                c += x[e];
+                if (!found && before + c > thr) {
+                  x_found = v + e;
+                  found = true;
+                }
+              }
+            }
+          } else {
+            for (int v = v0; v < v1 && !found; ++v) {
+              c += res.at(v);
               if (before + c > thr) {
-                key_x = static_cast<unsigned long long>(v) + 1ull;
-                break;
+                x_found = v;
+                found = true;
               }
             }
           }
-          x_found = static_cast<int>(team.max_u64(key_x)) - 1;
+          // rank in the high half (inverted: lowest rank wins the max), token in the low half
+          key = (static_cast<unsigned long long>(0x7fffffffu - static_cast<unsigned int>(team.rank())) << 32) |
+                static_cast<unsigned int>(x_found + 1);
         }
-        if (x_found < 0) {
-          const int lp = static_cast<int>(team.max_u64(key_last)) - 1;
-          x_found = lp >= 0 ? lp : V - 1;
+        const unsigned long long win = team.max_u64(key);
+        if (win) {
+          bonus = static_cast<int>(win & 0xffffffffull) - 1;
+        } else {
+          // rounding left u * total at or above every prefix: take the last token with positive mass
+          const int lp = static_cast<int>(team.max_u64(static_cast<unsigned long long>(static_cast<unsigned int>(last_pos + 1)))) - 1;
+          bonus = lp >= 0 ? lp : V - 1;
         }
-        bonus = x_found;
       }
     }
     if (next < 0) break;
-    if (team.rank == 0 && len < p.path_cap) path[len] = next;
+    if (writer && len < p.path_cap) path[len] = next;
     ++len;
     cur = next;
-    team.sync();   // the rejected-candidate list of the finished node is dead before the next node reuses it
+    team.sync_cta();   // the rejected-candidate list of the finished node is dead before the next node reuses it
   }
-  if (team.rank == 0) {
+  if (writer) {
     p.bonus[b] = bonus;
     if (p.accept_len) p.accept_len[b] = len;
   }
 }
 
+template <int CL>
+cudaError_t launch_cluster(const AcceptParams& p, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(p.B) * CL, 1, 1);
+  cfg.blockDim = dim3(kCtaThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CL;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, accept_kernel<kCtaThreads, CL>, p);
+}
+
 }  // namespace
 
-cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
+// Team width: a warp per tree for small vocabularies; otherwise CTAs of 512 threads, clustered so that
+// about one SM's worth of trees still spreads over the whole GPU.
+cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream) {
   if (p.B == 0) return cudaSuccess;
+  cudaError_t e;
   if (p.V <= 4096) {
     const unsigned blocks = static_cast<unsigned>((p.B + kWarpTeamsPerCta - 1) / kWarpTeamsPerCta);
-    accept_kernel<32><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
+    accept_kernel<32, 1><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
+    e = cudaGetLastError();
   } else {
-    accept_kernel<kCtaTeam><<<static_cast<unsigned>(p.B), kCtaTeam, 0, stream>>>(p);
+    const long long per_tree = sm_count / p.B;   // SMs available per tree
+    if (per_tree >= 8) e = launch_cluster<8>(p, stream);
+    else if (per_tree >= 4) e = launch_cluster<4>(p, stream);
+    else if (per_tree >= 2) e = launch_cluster<2>(p, stream);
+    else {
+      accept_kernel<kCtaThreads, 1><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
+      e = cudaGetLastError();
+    }
   }
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace eagle

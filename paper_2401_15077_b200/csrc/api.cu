@@ -157,7 +157,8 @@ int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, 
   // stochastic sequences need the draft rows and the uniforms; only an all-greedy call may omit them
   if ((!draft_probs || !uniforms) && !d.greedy) return EAGLE_ERR_NULL;
   int err = 0;
-  if (!device_info(&err)) return err;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
   AcceptParams ap;
   ap.target = target_probs;
   ap.draft = draft_probs;
@@ -174,7 +175,7 @@ int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, 
   ap.T = d.max_tree;
   ap.V = d.vocab;
   ap.path_cap = d.path_cap;
-  if (launch_accept(ap, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_accept(ap, dev->sm_count, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 

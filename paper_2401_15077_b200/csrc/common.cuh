@@ -143,7 +143,7 @@ int attn_tc_tile_keys();
 cudaError_t attn_tc_prepare(int head_dim);
 cudaError_t launch_combine(const AttnParams& p, const int32_t* tree_sizes_unused, cudaStream_t stream);
 
-cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream);
+cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
 void count_launch();
 
