@@ -63,7 +63,7 @@ typedef struct eagle_attn_desc {
   int32_t max_tree;            /* T_max <= 64: row stride of tree_parent, q and out */
   int32_t kv_capacity;         /* S_cap: slots per (sequence, KV head) of k_cache / v_cache */
   const int32_t* tree_sizes;   /* device int32 [B], or NULL: every tree has T_max nodes */
-  float sm_scale;              /* softmax scale; 0 means 1/sqrt(D) */
+  float sm_scale;              /* softmax scale, > 0; 0 means 1/sqrt(D); negative or NaN is EAGLE_ERR_SHAPE */
   int32_t num_splits;          /* KV splits per sequence; 0 lets the device-side planner choose */
   void* workspace;             /* device, 256-byte aligned, >= eagle_tree_verify_attn_workspace() bytes */
   size_t workspace_bytes;

@@ -20,6 +20,7 @@ struct DeviceInfo {
   int cc_major = 0;
   bool mma_prepared[2] = {false, false};
   bool tc_prepared[2] = {false, false};
+  bool tc2_prepared[2] = {false, false};
 };
 constexpr int kMaxDevices = 64;
 DeviceInfo g_dev[kMaxDevices];
@@ -71,7 +72,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   if (!desc) return EAGLE_ERR_NULL;
   const eagle_attn_desc& d = *desc;
   Workspace w;
-  if (d.kv_capacity < 0 || !carve_workspace(d, d.workspace, &w)) return EAGLE_ERR_SHAPE;
+  if (d.kv_capacity < 0 || !(d.sm_scale >= 0.f) || !carve_workspace(d, d.workspace, &w)) return EAGLE_ERR_SHAPE;
   if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
   if (!q || !k_cache || !v_cache || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
   if (!d.workspace || (reinterpret_cast<uintptr_t>(d.workspace) & 255) || d.workspace_bytes < w.bytes) return EAGLE_ERR_WORKSPACE;
@@ -84,8 +85,13 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int di = d.head_dim == 128 ? 1 : 0;
   const char* impl_env = std::getenv("EAGLE_ATTN_IMPL");
-  const bool use_tc = impl_env && std::strcmp(impl_env, "tc") == 0;
-  if (use_tc && !dev->tc_prepared[di]) {
+  const bool use_tc2 = impl_env && std::strcmp(impl_env, "tc2") == 0;
+  const bool use_tc = use_tc2 || (impl_env && std::strcmp(impl_env, "tc") == 0);
+  if (use_tc2 && !dev->tc2_prepared[di]) {
+    if (attn_tc2_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
+    dev->tc2_prepared[di] = true;
+  }
+  if (use_tc && !use_tc2 && !dev->tc_prepared[di]) {
     if (attn_tc_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
     dev->tc_prepared[di] = true;
   }
@@ -109,6 +115,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
   pp.min_chunk_tiles = 256 / pp.tile_keys > 0 ? 256 / pp.tile_keys : 1;
+  pp.pair = use_tc2 ? 1 : 0;
   pp.item_cap = w.item_cap;
   pp.slot_cap = w.slot_cap;
   pp.hdr = w.hdr;
@@ -132,6 +139,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.S_cap = d.kv_capacity;
   const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
   ap.scale_log2 = scale * 1.4426950408889634f;
+  ap.pair = use_tc2 ? 1 : 0;
   ap.hdr = w.hdr;
   ap.seq = w.seq;
   ap.anc = w.anc;
@@ -140,7 +148,9 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.part_o = w.part_o;
   ap.status = d.status;
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if ((use_tc ? launch_attn_tc(ap, num_ctas, stream) : launch_attn_mma(ap, num_ctas, stream)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  const cudaError_t le = use_tc2 ? launch_attn_tc2(ap, num_ctas, stream)
+                                 : (use_tc ? launch_attn_tc(ap, num_ctas, stream) : launch_attn_mma(ap, num_ctas, stream));
+  if (le != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_combine(ap, nullptr, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;

@@ -29,10 +29,20 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
   if (sp.splits <= 1) return;
   const int g = h / p.G, R = i * p.G + h % p.G;
   const int mt = R / kBlockM, r = R % kBlockM;
-  const size_t slot0 = static_cast<size_t>(sp.slot_base) + (static_cast<size_t>(g) * sp.mtiles + mt) * sp.splits;
+  // unpaired plans: one slot per (KV head, query tile, split); paired plans: two slots per (KV head, pair, split),
+  // the second used only when the pair really holds two query tiles
+  size_t slot0, stride;
+  if (p.pair) {
+    const int units = (sp.mtiles + 1) / 2;
+    slot0 = static_cast<size_t>(sp.slot_base) + 2 * (static_cast<size_t>(g) * units + mt / 2) * sp.splits + (mt & 1);
+    stride = 2;
+  } else {
+    slot0 = static_cast<size_t>(sp.slot_base) + (static_cast<size_t>(g) * sp.mtiles + mt) * sp.splits;
+    stride = 1;
+  }
   float m_star = -INFINITY;
   for (int s = 0; s < sp.splits; ++s) {
-    const float2 ml = p.part_ml[(slot0 + s) * kBlockM + r];
+    const float2 ml = p.part_ml[(slot0 + s * stride) * kBlockM + r];
     if (ml.y > 0.f) m_star = fmaxf(m_star, ml.x);
   }
   float acc[E];
@@ -40,11 +50,11 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
   for (int e = 0; e < E; ++e) acc[e] = 0.f;
   float l_star = 0.f;
   for (int s = 0; s < sp.splits; ++s) {
-    const float2 ml = p.part_ml[(slot0 + s) * kBlockM + r];
+    const float2 ml = p.part_ml[(slot0 + s * stride) * kBlockM + r];
     if (!(ml.y > 0.f)) continue;   // a split in which this row saw no key
     const float w = exp2f(ml.x - m_star);
     l_star += ml.y * w;
-    const float* po = p.part_o + ((slot0 + s) * kBlockM + r) * D + lane * E;
+    const float* po = p.part_o + ((slot0 + s * stride) * kBlockM + r) * D + lane * E;
     if (E == 4) {
       const float4 v = *reinterpret_cast<const float4*>(po);
       acc[0] += v.x * w; acc[1] += v.y * w; acc[2 % E] += v.z * w; acc[3 % E] += v.w * w;

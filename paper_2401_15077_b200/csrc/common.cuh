@@ -17,8 +17,9 @@ constexpr int kSlotBudgetAuto = 2048; // partial slots the planner may use when 
 struct WorkItem {
   int32_t b, g, mt;
   int32_t tile_begin, tile_end;  // KV tiles [begin, end) of `tile_keys` keys each
-  int32_t slot;                  // partial slot, or -1: the only split, write the output directly
-  int32_t pad0, pad1;
+  int32_t slot;                  // first partial slot, or -1: the only split, write the output directly
+  int32_t mode;                  // paired planning only: 0 = one query tile (mt), 1 = two query tiles (mt, mt+1)
+  int32_t pad1;
 };
 
 struct SeqPlan {
@@ -27,8 +28,9 @@ struct SeqPlan {
   int32_t n;           // tree size used (0 when the sequence is invalid or empty)
   int32_t L;           // committed prefix length
   int32_t slot_base;   // first partial slot (splits > 1), else -1
-  int32_t mtiles;      // 128-row tiles per KV head
-  int32_t pad0, pad1;
+  int32_t mtiles;      // 128-row query tiles per KV head
+  int32_t ntiles;      // KV tiles covering prefix + tree
+  int32_t key;         // KV tiles per work item (sort key of the planner)
 };
 
 struct PlanHeader {
@@ -60,7 +62,8 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   if (d.num_splits < 0 || d.num_splits > 1024) return false;
   const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
   const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? mtiles : 1);
-  const long long slots = d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : kSlotBudgetAuto);
+  // two slots per item leave room for plans that pair query tiles (one slot per query tile of the pair)
+  const long long slots = 2 * (d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : kSlotBudgetAuto));
   const long long items = units + slots;
   if (items > (1ll << 30)) return false;
   char* p = static_cast<char*>(base);
@@ -85,6 +88,7 @@ struct AttnParams {
   __nv_bfloat16* out;
   int32_t B, Hq, Hkv, G, D, T_max, S_cap;
   float scale_log2;      // sm_scale * log2(e)
+  int32_t pair;          // 1: items cover pairs of query tiles and own two consecutive partial slots
   PlanHeader* hdr;
   const SeqPlan* seq;
   const uint64_t* anc;
@@ -103,6 +107,7 @@ struct PlanParams {
   int32_t num_ctas;        // CTAs of the persistent attention kernel
   int32_t forced_splits;   // 0: choose
   int32_t min_chunk_tiles;
+  int32_t pair;            // 1: one item per pair of query tiles, two partial slots per item
   int32_t item_cap, slot_cap;
   PlanHeader* hdr;
   SeqPlan* seq;
@@ -141,6 +146,9 @@ cudaError_t attn_mma_prepare(int head_dim);
 cudaError_t launch_attn_tc(const AttnParams& p, int num_ctas, cudaStream_t stream);
 int attn_tc_tile_keys();
 cudaError_t attn_tc_prepare(int head_dim);
+cudaError_t launch_attn_tc2(const AttnParams& p, int num_ctas, cudaStream_t stream);
+int attn_tc2_tile_keys();
+cudaError_t attn_tc2_prepare(int head_dim);
 cudaError_t launch_combine(const AttnParams& p, const int32_t* tree_sizes_unused, cudaStream_t stream);
 
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);

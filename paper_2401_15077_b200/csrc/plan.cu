@@ -35,6 +35,9 @@ __device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc,
   return true;
 }
 
+// work units per KV head: query tiles, or pairs of them
+__device__ __forceinline__ int units_of(int mtiles, int pair) { return pair ? (mtiles + 1) / 2 : mtiles; }
+
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
   __shared__ long long s_red[32];
   __shared__ int s_chunk;
@@ -64,10 +67,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
     sp.item_base = 0;
     sp.splits = 1;
     sp.slot_base = -1;
-    sp.pad0 = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;  // KV tiles (kept in pad0 while planning)
-    sp.pad1 = 0;
+    sp.ntiles = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;
+    sp.key = 0;
     p.seq[b] = sp;
-    work += static_cast<long long>(p.Hkv) * sp.mtiles * sp.pad0;
+    work += static_cast<long long>(p.Hkv) * units_of(sp.mtiles, p.pair) * sp.ntiles;
   }
   const long long total_work = block_sum(work, s_red);
 
@@ -87,8 +90,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
       long long slots = 0;
       for (int b = tid; b < p.B; b += kPlanThreads) {
         const SeqPlan sp = p.seq[b];
-        const int splits = (sp.pad0 + chunk - 1) / chunk;
-        if (splits > 1) slots += static_cast<long long>(p.Hkv) * sp.mtiles * splits;
+        const int splits = (sp.ntiles + chunk - 1) / chunk;
+        if (splits > 1) slots += static_cast<long long>(p.Hkv) * units_of(sp.mtiles, p.pair) * splits * (p.pair ? 2 : 1);
       }
       const long long total_slots = block_sum(slots, s_red);
       if (total_slots <= p.slot_cap) break;
@@ -103,11 +106,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
   for (int b = tid; b < p.B; b += kPlanThreads) {
     SeqPlan sp = p.seq[b];
     int splits;
-    if (p.forced_splits > 0) splits = sp.pad0 < p.forced_splits ? sp.pad0 : p.forced_splits;
-    else splits = (sp.pad0 + chunk - 1) / chunk;
+    if (p.forced_splits > 0) splits = sp.ntiles < p.forced_splits ? sp.ntiles : p.forced_splits;
+    else splits = (sp.ntiles + chunk - 1) / chunk;
     if (splits < 1) splits = 1;
     sp.splits = splits;
-    sp.pad1 = (sp.pad0 + splits - 1) / splits;   // tiles per item: the sort key
+    sp.key = (sp.ntiles + splits - 1) / splits;   // tiles per item: the sort key
     p.seq[b] = sp;
   }
   __syncthreads();
@@ -119,32 +122,34 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
     long long item_base = 0, slot_base = 0;
     for (int o = 0; o < p.B; ++o) {
       // read only the planning fields: item_base / slot_base of other records are being written
-      const int o_key = p.seq[o].pad1, o_splits = p.seq[o].splits, o_mtiles = p.seq[o].mtiles;
-      const bool before = o_key > me.pad1 || (o_key == me.pad1 && o < b);
+      const int o_key = p.seq[o].key, o_splits = p.seq[o].splits, o_mtiles = p.seq[o].mtiles;
+      const bool before = o_key > me.key || (o_key == me.key && o < b);
       if (before) {
-        const long long cnt = static_cast<long long>(p.Hkv) * o_mtiles * o_splits;
+        const long long cnt = static_cast<long long>(p.Hkv) * units_of(o_mtiles, p.pair) * o_splits;
         item_base += cnt;
-        if (o_splits > 1) slot_base += cnt;
+        if (o_splits > 1) slot_base += cnt * (p.pair ? 2 : 1);
       }
     }
-    const long long cnt = static_cast<long long>(p.Hkv) * me.mtiles * me.splits;
+    const int units = units_of(me.mtiles, p.pair), per_item = p.pair ? 2 : 1;
+    const long long cnt = static_cast<long long>(p.Hkv) * units * me.splits;
     my_items += cnt;
-    const bool fits = item_base + cnt <= p.item_cap && (me.splits == 1 || slot_base + cnt <= p.slot_cap);
+    const bool fits = item_base + cnt <= p.item_cap && (me.splits == 1 || slot_base + cnt * per_item <= p.slot_cap);
     // cannot happen with a workspace of the advertised size; refuse rather than overrun
     if (!fits && cnt > 0) report_status(p.status, EAGLE_ERR_WORKSPACE);
     if (fits) {
       int idx = static_cast<int>(item_base);
       for (int g = 0; g < p.Hkv; ++g)
-        for (int mt = 0; mt < me.mtiles; ++mt)
+        for (int mu = 0; mu < units; ++mu)
           for (int s = 0; s < me.splits; ++s, ++idx) {
             WorkItem it;
             it.b = b;
             it.g = g;
-            it.mt = mt;
-            it.tile_begin = static_cast<int>(static_cast<long long>(me.pad0) * s / me.splits);
-            it.tile_end = static_cast<int>(static_cast<long long>(me.pad0) * (s + 1) / me.splits);
-            it.slot = me.splits > 1 ? static_cast<int>(slot_base) + (idx - static_cast<int>(item_base)) : -1;
-            it.pad0 = it.pad1 = 0;
+            it.mt = p.pair ? 2 * mu : mu;
+            it.mode = (p.pair && 2 * mu + 1 < me.mtiles) ? 1 : 0;
+            it.tile_begin = static_cast<int>(static_cast<long long>(me.ntiles) * s / me.splits);
+            it.tile_end = static_cast<int>(static_cast<long long>(me.ntiles) * (s + 1) / me.splits);
+            it.slot = me.splits > 1 ? static_cast<int>(slot_base) + (idx - static_cast<int>(item_base)) * per_item : -1;
+            it.pad1 = 0;
             p.items[idx] = it;
           }
     }
