@@ -115,7 +115,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
   pp.min_chunk_tiles = 256 / pp.tile_keys > 0 ? 256 / pp.tile_keys : 1;
-  pp.pair = use_tc2 ? 1 : 0;
+  pp.pair = 0;
   pp.item_cap = w.item_cap;
   pp.slot_cap = w.slot_cap;
   pp.hdr = w.hdr;
@@ -139,7 +139,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.S_cap = d.kv_capacity;
   const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
   ap.scale_log2 = scale * 1.4426950408889634f;
-  ap.pair = use_tc2 ? 1 : 0;
+  ap.pair = 0;
   ap.hdr = w.hdr;
   ap.seq = w.seq;
   ap.anc = w.anc;

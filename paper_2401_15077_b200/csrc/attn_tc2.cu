@@ -1,21 +1,18 @@
-// Split-KV tree attention for sm_100a, two softmax warpgroups per CTA.
+// Split-KV tree attention for sm_100a: TMA-staged KV tiles, tcgen05 MMAs, accumulators in TMEM.
 //
-// TMA stages 128-key K and V tiles (128-byte swizzled boxes) through one ring of five 32 KB shared-memory
-// slots; tcgen05 MMAs compute S = Q K^T and O += P V with accumulators in TMEM; one persistent CTA per SM
-// walks a static slice of the planner's work list.  An item covers a range of KV tiles of one (sequence,
-// KV head) for either
-//   mode 1: two 128-row query tiles (rows = tree node * G + head-in-group): warpgroup w owns query tile w;
-//           every K / V tile in shared memory feeds both, so the cache is read once for 256 query rows; or
-//   mode 0: one query tile: warpgroup 0 takes the even KV tiles of the range, warpgroup 1 the odd ones,
-//           each with its own running max / sum / accumulator; the two are merged in the epilogue.
-// Either way each warpgroup runs the chain  QK -> softmax -> PV  on its own TMEM columns (S_w, with P_w
-// written over the first half of S_w; O_w), and the tensor pipe interleaves the two chains, so one
-// warpgroup's exponentials overlap the other's MMAs.
-// Warp roles: warps 0-3 and 4-7 softmax warpgroups (thread r <-> query row r <-> TMEM lane r), warp 8 TMA
-// producer, warp 9 MMA issuer.  Softmax is fp32 in the log2 domain; the tree mask is applied in registers
-// only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are zeroed in
-// shared memory before the MMA reads them.  The accumulator is rescaled only when the running max grows by
-// more than 2^8.  Every wait is bounded (mbarrier try_wait + timer); on expiry the CTA raises
+// One persistent CTA per SM walks a static slice of the planner's work list.  An item is one 128-row query
+// tile (row = tree node * G + head-in-group) of one (sequence, KV head) over a range of 128-key KV tiles;
+// step s of the item handles KV tile s:
+//     S[s&1] = Q K^T   ->   softmax   ->   P[s&1] (packed bf16)   ->   O += P V.
+// S and P are double buffered in TMEM (S0 S1 | O | P0 P1 = 512 columns), so the score MMA of step s+1 and the
+// PV MMA of step s-1 run while the softmax warps work on step s.
+// Warp roles: warps 0-7 softmax (thread pair (r, r+128) shares query row r = TMEM lane r, 64 score columns
+// each; the pair agrees on the row max through shared memory), warp 8 TMA producer (K and V tiles through a
+// ring of six 32 KB slots, 128-byte swizzled boxes), warp 9 issues the QK MMAs and warp 10 the PV MMAs (each
+// waits only on what its own MMA needs).  Softmax is fp32 in the log2 domain; the tree mask is applied in
+// registers only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are
+// zeroed in shared memory before the MMA reads them.  The accumulator is rescaled only when the running max
+// grows by more than 2^8.  Every wait is bounded (mbarrier try_wait + timer); on expiry the CTA raises
 // EAGLE_ERR_TIMEOUT, all roles leave their loops, TMEM is released and the kernel returns.
 #include <cuda.h>
 
@@ -26,12 +23,13 @@ namespace eagle {
 namespace {
 
 constexpr int kTileN = 128;          // keys per KV tile
-constexpr int kSlots = 5;            // ring slots; tile g uses slot (2g) % 5 for K and (2g+1) % 5 for V
-constexpr int kThreads = 320;
-constexpr int kWgThreads = 128;
+constexpr int kSlots = 6;            // ring slots; tile g uses slot (2g) % 6 for K and (2g+1) % 6 for V
+constexpr int kThreads = 352;
+constexpr int kSoftmaxThreads = 256;
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;        // S_w at w*128; P_w (packed bf16, 64 columns) overwrites its first half
-constexpr uint32_t kColO = 256;      // O_w at 256 + w*128
+constexpr uint32_t kColS = 0;        // S[b] at b*128
+constexpr uint32_t kColO = 256;
+constexpr uint32_t kColP = 384;      // P[b] (packed bf16: 64 columns) at 384 + b*64
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -61,8 +59,18 @@ __device__ __forceinline__ unsigned long long global_timer() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false if the CTA has been aborted or the time limit passed (and raises the abort flag).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_test_wait(bar, parity)) return true;     // non-blocking probe: the phase is often complete already
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer();
   for (uint32_t spins = 1;; ++spins) {
@@ -90,20 +98,6 @@ __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sy
 
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t* r) {
@@ -144,18 +138,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
-//   K-major operand (Q, K): rows of 128 bytes (64 bf16 along the contraction), LBO unused.
-//   MN-major operand (V):   rows of 128 bytes (64 bf16 along N), `lbo_bytes` between 64-wide N chunks.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr >> 4) & 0x3fffu);
-  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fffu) << 16;
-  d |= static_cast<uint64_t>((1024u >> 4) & 0x3fffu) << 32;   // stride between 8-row groups
-  d |= 1ull << 46;                                            // descriptor version of sm_100
-  d |= 2ull << 61;                                            // SWIZZLE_128B
-  return d;
-}
 // kind::f16 instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(N >> 3) << 17) |
@@ -163,16 +145,100 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
 }
 
 
+#ifdef EAGLE_TRACE
+// Debug builds only: CTA 0 logs (tag, clock) pairs per role; read back with eagle_debug_trace().
+__device__ unsigned long long g_trace[4][1024];
+__device__ int g_trace_n[4];
+#define TRACE(role, tag)                                                                          \
+  do {                                                                                            \
+    if (blockIdx.x == 0 && trace_n < 1024) {                                                      \
+      g_trace[role][trace_n] = (static_cast<unsigned long long>(tag) << 48) | (static_cast<unsigned long long>(clock64()) & 0xffffffffffffull); \
+      g_trace_n[role] = ++trace_n;                                                                \
+    }                                                                                             \
+  } while (0)
+#else
+#define TRACE(role, tag) do { } while (0)
+#endif
+
+// Descriptor halves.  The low word holds the start address (>>4) and the leading-dimension offset, so stepping along
+// the contraction is a 32-bit add on the low word; the high word (8-row-group stride, version, swizzle) is constant.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) { return ((addr >> 4) & 0x3fffu) | ((lbo_bytes >> 4) << 16); }
+// One asm block per 128-key tile: the MMAs of a tile are issued back to back by one thread, so the instruction
+// stream between them is kept to the descriptor adds (the tensor pipe finishes a 128x128x16 MMA in about 64 cycles).
+// S[128 x 128] = Q[128 x D] K^T: D/16 MMAs; low descriptor words step 32 bytes per k step, 16 KB per 64-column slab.
+template <int D>
+__device__ __forceinline__ void issue_qk_tile(uint32_t d_tmem, uint32_t q_lo, uint32_t k_lo, uint32_t idesc) {
+  if constexpr (D == 128) {
+    asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+      "add.u32 ta, %1, 0;\n\tadd.u32 tb, %2, 0;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 0, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 1024;\n\tadd.u32 tb, %2, 1024;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 1026;\n\tadd.u32 tb, %2, 1026;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 1028;\n\tadd.u32 tb, %2, 1028;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 1030;\n\tadd.u32 tb, %2, 1030;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "}"
+      ::"r"(d_tmem), "r"(q_lo), "r"(k_lo), "r"(idesc), "r"(kDescHi) : "memory");
+  } else {
+    asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+      "add.u32 ta, %1, 0;\n\tadd.u32 tb, %2, 0;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 0, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\tmov.b64 da, {ta, %4};\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+      "}"
+      ::"r"(d_tmem), "r"(q_lo), "r"(k_lo), "r"(idesc), "r"(kDescHi) : "memory");
+  }
+}
+// O[128 x D] (+)= P[128 x 128] V[128 x D]: 8 MMAs; P steps 8 TMEM columns, V steps 16 keys (2 KB) per k step.
+__device__ __forceinline__ void issue_pv_tile(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_lo, uint32_t idesc, uint32_t acc0) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t.reg .b32 ta, tb;\n\t"
+      "add.u32 ta, %1, 0;\n\tadd.u32 tb, %2, 0;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 8;\n\tadd.u32 tb, %2, 128;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 16;\n\tadd.u32 tb, %2, 256;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 24;\n\tadd.u32 tb, %2, 384;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 32;\n\tadd.u32 tb, %2, 512;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 40;\n\tadd.u32 tb, %2, 640;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 48;\n\tadd.u32 tb, %2, 768;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "add.u32 ta, %1, 56;\n\tadd.u32 tb, %2, 896;\n\tmov.b64 db, {tb, %4};\n\t"
+      "setp.ne.b32 p, 1, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p;\n\t"
+      "}"
+      ::"r"(o_tmem), "r"(p_tmem), "r"(v_lo), "r"(idesc), "r"(kDescHi), "r"(acc0) : "memory");
+}
+
 template <int D>
 struct Smem2 {
   static constexpr int kSlabs = D / 64;                     // 64 bf16 = one 128-byte swizzled row
   static constexpr int kSlabBytes = kTileN * 128;            // 128 rows x 128 bytes
   static constexpr int kTileBytes = kSlabs * kSlabBytes;     // one Q / K / V tile
-  static constexpr int kQ = 0;                               // two query tiles
-  static constexpr int kRing = 2 * kTileBytes;
-  static constexpr int kMl = kRing + kSlots * kTileBytes;    // float2 [2][128]: (max, sum) exchange of mode 0
-  static constexpr int kBar = kMl + 2 * kBlockM * 8;
-  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 4;
+  static constexpr int kQ = 0;
+  static constexpr int kRing = kTileBytes;
+  static constexpr int kXch = kRing + kSlots * kTileBytes;   // float [2 parities][2 halves][128 rows]: row-max exchange
+  static constexpr int kBar = kXch + 2 * 2 * kBlockM * 4;
+  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 3 + 4;
   static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag
   static constexpr int kBytes = kMisc + 16;
 };
@@ -180,7 +246,8 @@ struct Smem2 {
 struct Bars2 {
   uint32_t full[kSlots], empty[kSlots];
   uint32_t s_full[2], p_full[2], o_done[2];
-  uint32_t q_full, q_empty, o_free, ml_full;
+  uint32_t q_full, q_empty, o_free;
+  uint32_t pair[4];   // one per TMEM lane quarter: the two softmax warps that share its rows
 };
 
 __device__ __forceinline__ int item_index(int row, int cta, int grid) {
@@ -210,7 +277,7 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
     B.q_full = b; b += 8;
     B.q_empty = b; b += 8;
     B.o_free = b; b += 8;
-    B.ml_full = b;
+    for (int i = 0; i < 4; ++i) { B.pair[i] = b; b += 8; }
   }
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + S::kMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + S::kMisc + 4);
@@ -222,13 +289,13 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(B.s_full[i], 1);
-      mbar_init(B.p_full[i], kWgThreads);
+      mbar_init(B.p_full[i], kSoftmaxThreads);
       mbar_init(B.o_done[i], 1);
     }
-    mbar_init(B.q_full, 2 * kWgThreads);
+    mbar_init(B.q_full, kSoftmaxThreads);
     mbar_init(B.q_empty, 1);
-    mbar_init(B.o_free, 2 * kWgThreads);
-    mbar_init(B.ml_full, 2 * kWgThreads);
+    mbar_init(B.o_free, kSoftmaxThreads);
+    for (int i = 0; i < 4; ++i) mbar_init(B.pair[i], 64);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -243,6 +310,9 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
 
   const int n_items = p.hdr->n_items;
   const int grid = gridDim.x, cta = blockIdx.x;
+#ifdef EAGLE_TRACE
+  int trace_n = 0;
+#endif
 
   if (warp == 8) {
     // =========================================================================== TMA producer
@@ -254,12 +324,14 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
         if (idx >= n_items) break;
         const WorkItem it = p.items[idx];
         const int z = it.b * p.Hkv + it.g;
+        TRACE(0, 1);
         for (int tile = it.tile_begin; tile < it.tile_end && ok; ++tile, ++g) {
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t n = 2 * g + kv, slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
             ok = mbar_wait(B.empty[slot], par, s_abort);
             if (!ok) break;
+            TRACE(0, ((2 + kv) << 10) | (g & 1023u));
             mbar_expect_tx(B.full[slot], S::kTileBytes);
 #pragma unroll
             for (int s = 0; s < S::kSlabs; ++s)
@@ -270,181 +342,189 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
       }
     }
   } else if (warp == 9) {
-    // =========================================================================== MMA issuer
+    // =========================================================================== QK issuer
+    // Ring item n = 2*tile (+1 for V) lives in slot n % 6 with phase parity (n / 6) & 1.  Positions are kept as
+    // running counters (no divisions on the threads that keep the tensor pipe fed).
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(kBlockM, kTileN, false);
-      constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, true);
-      uint32_t g_base = 0, item_count = 0;
-      uint32_t cw[2] = {0u, 0u};       // steps issued per warpgroup stream (phase counters of s_full / p_full / o_done)
+      uint32_t ks = 0, kp = 0;       // slot / parity of the K tile of the next QK
+      uint32_t gq = 0;               // steps issued so far (all items)
+      uint32_t item_count = 0;
+      const uint32_t q_lo = desc_lo(sbase + S::kQ, 16), ring_lo_k = desc_lo(sbase + S::kRing, 16);
+      constexpr uint32_t kTileStep = S::kTileBytes >> 4;
       bool ok = true;
       for (int row = 0; ok; ++row) {
         const int idx = item_index(row, cta, grid);
         if (idx >= n_items) break;
         const WorkItem it = p.items[idx];
-        const int nt = it.tile_end - it.tile_begin, mode = it.mode;
-        const int steps[2] = {mode ? nt : (nt + 1) / 2, mode ? nt : nt / 2};
-        int qk_left = steps[0] + steps[1];
-        bool first_pv = true;
+        const int steps = it.tile_end - it.tile_begin;
+        TRACE(1, 1);
         ok = mbar_wait(B.q_full, item_count & 1u, s_abort);
         if (!ok) break;
-        tc_fence_after();
-        auto issue_qk = [&](int w, int k) -> bool {
-          const uint32_t g = g_base + (mode ? k : 2 * k + w);
-          const uint32_t n = 2 * g, slot = n % kSlots, par = (n / kSlots) & 1u;
-          if (!mbar_wait(B.full[slot], par, s_abort)) return false;
+        TRACE(1, 2);
+        for (int s = 0; s < steps && ok; ++s, ++gq) {
+          // S[gq & 1] is free once the softmax warps have read the scores of step gq - 2
+          if (gq >= 2) {
+            ok = mbar_wait(B.p_full[gq & 1u], ((gq - 2) >> 1) & 1u, s_abort);
+            if (!ok) break;
+          }
+          ok = mbar_wait(B.full[ks], kp, s_abort);
+          if (!ok) break;
+          TRACE(1, (10 << 10) | (gq & 1023u));
           tc_fence_after();
-          const uint32_t d_tmem = tmem + kColS + w * kTileN;
-          const uint32_t q_addr = sbase + S::kQ + (mode ? w : 0) * S::kTileBytes;
-          const uint32_t k_addr = sbase + S::kRing + slot * S::kTileBytes;
-#pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint32_t off = (kk / 4) * S::kSlabBytes + (kk % 4) * 32;
-            umma_ss(d_tmem, smem_desc(q_addr + off, 16), smem_desc(k_addr + off, 16), idesc_qk, kk > 0 ? 1u : 0u);
-          }
-          tc_commit(B.s_full[w]);
-          if (!mode || w == 1) tc_commit(B.empty[slot]);   // last reader of this K tile
-          if (--qk_left == 0) tc_commit(B.q_empty);         // every QK of this item has been issued
-          return true;
-        };
-        auto issue_pv = [&](int w, int k) -> bool {
-          const uint32_t g = g_base + (mode ? k : 2 * k + w);
-          const uint32_t n = 2 * g + 1, slot = n % kSlots, par = (n / kSlots) & 1u;
-          if (!mbar_wait(B.p_full[w], cw[w] & 1u, s_abort)) return false;
-          if (!mbar_wait(B.full[slot], par, s_abort)) return false;
-          if (first_pv && item_count > 0) {
-            if (!mbar_wait(B.o_free, (item_count - 1) & 1u, s_abort)) return false;   // previous epilogue has read O
-          }
-          first_pv = false;
-          tc_fence_after();
-          const uint32_t a_tmem = tmem + kColS + w * kTileN;
-          const uint32_t v_addr = sbase + S::kRing + slot * S::kTileBytes;
-#pragma unroll
-          for (int kk = 0; kk < kTileN / 16; ++kk)
-            umma_ts(tmem + kColO + w * kTileN, a_tmem + kk * 8, smem_desc(v_addr + kk * 2048, S::kSlabBytes), idesc_pv,
-                    (k > 0 || kk > 0) ? 1u : 0u);
-          tc_commit(B.o_done[w]);
-          if (!mode || w == 1) tc_commit(B.empty[slot]);   // last reader of this V tile
-          ++cw[w];
-          return true;
-        };
-        ok = issue_qk(0, 0);
-        if (ok && steps[1] > 0) ok = issue_qk(1, 0);
-        for (int k = 0; k < steps[0] && ok; ++k) {
-#pragma unroll
-          for (int w = 0; w < 2; ++w) {
-            if (!ok || k >= steps[w]) continue;
-            ok = issue_pv(w, k);
-            if (ok && k + 1 < steps[w]) ok = issue_qk(w, k + 1);
-          }
+          issue_qk_tile<D>(tmem + kColS + (gq & 1u) * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
+          tc_commit(B.s_full[gq & 1u]);
+          tc_commit(B.empty[ks]);
+          ks += 2;
+          if (ks >= kSlots) { ks -= kSlots; kp ^= 1u; }
+          if (s == steps - 1) tc_commit(B.q_empty);          // every QK of this item has been issued
+          TRACE(1, (11 << 10) | (gq & 1023u));
         }
-        g_base += nt;
+        ++item_count;
+      }
+    }
+  } else if (warp == 10) {
+    // =========================================================================== PV issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, true);
+      uint32_t vs = 1, vp = 0;       // slot / parity of the V tile of the next PV
+      uint32_t gp = 0;               // steps issued so far (all items)
+      uint32_t item_count = 0;
+      const uint32_t ring_lo_v = desc_lo(sbase + S::kRing, S::kSlabBytes);
+      constexpr uint32_t kTileStep = S::kTileBytes >> 4;
+      bool ok = true;
+      for (int row = 0; ok; ++row) {
+        const int idx = item_index(row, cta, grid);
+        if (idx >= n_items) break;
+        const WorkItem it = p.items[idx];
+        const int steps = it.tile_end - it.tile_begin;
+        for (int s = 0; s < steps && ok; ++s, ++gp) {
+          ok = mbar_wait(B.p_full[gp & 1u], (gp >> 1) & 1u, s_abort);
+          if (!ok) break;
+          TRACE(3, (20 << 10) | (gp & 1023u));
+          ok = mbar_wait(B.full[vs], vp, s_abort);
+          if (!ok) break;
+          if (s == 0 && item_count > 0) {
+            ok = mbar_wait(B.o_free, (item_count - 1) & 1u, s_abort);   // previous epilogue has read O
+            if (!ok) break;
+          }
+          TRACE(3, (30 << 10) | (gp & 1023u));
+          tc_fence_after();
+          issue_pv_tile(tmem + kColO, tmem + kColP + (gp & 1u) * (kTileN / 2), ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
+          tc_commit(B.o_done[gp & 1u]);
+          tc_commit(B.empty[vs]);
+          vs += 2;
+          if (vs >= kSlots) { vs -= kSlots; vp ^= 1u; }
+          TRACE(3, (31 << 10) | (gp & 1023u));
+        }
         ++item_count;
       }
     }
   } else {
-    // =========================================================================== softmax warpgroups + epilogue
-    const int w = warp >> 2;                              // warpgroup = stream
-    const int r = tid & (kWgThreads - 1);                 // query row of this thread within its tile == TMEM lane
+    // =========================================================================== softmax + epilogue (warps 0-7)
+    const int h = warp >> 2;                              // which 64-column half of the score row this thread owns
+    const int r = tid & (kBlockM - 1);                    // query row within the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    uint32_t g_base = 0, item_count = 0, cws = 0, mode0_count = 0;
+    const uint32_t pair_bar = B.pair[warp & 3];   // barrier shared with the partner warp (bounded waits, like all others)
+    uint32_t pair_phase = 0;
+    auto pair_sync = [&]() -> bool {
+      mbar_arrive(pair_bar);
+      const bool k = mbar_wait_warp(pair_bar, pair_phase & 1u, s_abort);
+      ++pair_phase;
+      return k;
+    };
+    float* xch = reinterpret_cast<float*>(smem + S::kXch);
+    uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps done so far
     bool ok = true;
     for (int row = 0; ok; ++row) {
       const int idx = item_index(row, cta, grid);
       if (idx >= n_items) break;
       const WorkItem it = p.items[idx];
       const SeqPlan sp = p.seq[it.b];
-      const int L = sp.L, n = sp.n, G = p.G, mode = it.mode;
-      const int m_valid = n * G;
-      const int R = (it.mt + (mode ? w : 0)) * kBlockM + r;
+      const int L = sp.L, n = sp.n, G = p.G;
+      const int m_valid = n * G, kv_end = L + n;
+      const int steps = it.tile_end - it.tile_begin;
+      const int R = it.mt * kBlockM + r;
       const bool row_valid = R < m_valid;
       const int node = row_valid ? R / G : 0, hh = row_valid ? R % G : 0;
       const uint64_t anc = row_valid ? p.anc[static_cast<size_t>(it.b) * p.T_max + node] : 0ull;
-      const int kv_end = L + n;
-      const int nt = it.tile_end - it.tile_begin;
-      const int steps = mode ? nt : (w == 0 ? (nt + 1) / 2 : nt / 2);
 
-      // ---- stage Q: mode 1: this warpgroup's own tile, whole rows; mode 0: the shared tile, 64-column slab per warpgroup
+      // ---- stage Q: thread (h, r) writes the h-th 64-column slab of row r (D = 64: h = 0 only)
+      if (tid == 0) TRACE(2, 1);
       ok = mbar_wait_warp(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
       if (!ok) break;
-      {
-        const uint4* src = reinterpret_cast<const uint4*>(p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D);
-        unsigned char* qdst = smem + S::kQ + (mode ? w : 0) * S::kTileBytes;
-        if (mode || D == 64) {
-          if (mode || w == 0) {
+      if (tid == 0) TRACE(2, 2);
+      if (h < S::kSlabs) {
+        const uint4* src = reinterpret_cast<const uint4*>(
+            p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * 64);
+        unsigned char* qdst = smem + S::kQ + h * S::kSlabBytes + r * 128;
 #pragma unroll
-            for (int c = 0; c < D / 8; ++c) {
-              const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-              *reinterpret_cast<uint4*>(qdst + (c / 8) * S::kSlabBytes + r * 128 + (((c % 8) ^ (r & 7)) << 4)) = v;
-            }
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 v = row_valid ? __ldg(src + w * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(qdst + w * S::kSlabBytes + r * 128 + ((c ^ (r & 7)) << 4)) = v;
-          }
+        for (int c = 0; c < 8; ++c) {
+          const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(qdst + ((c ^ (r & 7)) << 4)) = v;
         }
       }
       fence_proxy_async();
       mbar_arrive(B.q_full);
+      if (tid == 0) TRACE(2, 3);
 
       float m_ref = -INFINITY;   // reference max (scaled, log2 domain) of every exponential taken so far
-      float l_sum = 0.f;
-      for (int k = 0; k < steps && ok; ++k, ++cws) {
-        const uint32_t g = g_base + (mode ? k : 2 * k + w);
-        ok = mbar_wait_warp(B.s_full[w], cws & 1u, s_abort);
+      float l_sum = 0.f;         // this thread's half of the row sum
+      for (int s = 0; s < steps && ok; ++s) {
+        const uint32_t gs = sg + s, buf = gs & 1u;
+        ok = mbar_wait_warp(B.s_full[buf], (gs >> 1) & 1u, s_abort);
         if (!ok) break;
+        if (tid == 0) TRACE(2, (10 << 10) | (gs & 1023u));
         tc_fence_after();
-        const int key0 = (it.tile_begin + static_cast<int>(g - g_base)) * kTileN;
-        const bool tail = key0 + kTileN > L;   // the tile reaches past the committed prefix: tree mask + cache tail
-        const uint32_t s_addr = tmem + lane_addr + kColS + w * kTileN;
         uint32_t raw[64];
-        // 64 score columns starting at column h*64, masked on tail tiles (two passes over TMEM keep registers low)
-        auto load_half = [&](int h) {
-          tmem_ld32(s_addr + h * 64, raw);
-          tmem_ld32(s_addr + h * 64 + 32, raw + 32);
-          tc_wait_ld();
-          if (tail) {
+        tmem_ld32(tmem + lane_addr + kColS + buf * kTileN + h * 64, raw);
+        tmem_ld32(tmem + lane_addr + kColS + buf * kTileN + h * 64 + 32, raw + 32);
+        tc_wait_ld();
+        const int key0 = (it.tile_begin + s) * kTileN;
+        if (key0 + kTileN > L) {          // the tile reaches past the committed prefix: tree mask + cache tail
 #pragma unroll
-            for (int e = 0; e < 64; ++e) {
-              const int mrel = key0 + h * 64 + e - L;
-              const bool vis = mrel < 0 || (mrel < n && ((anc >> mrel) & 1ull));
-              raw[e] = vis ? raw[e] : 0xff800000u;   // -inf
-            }
-          }
-        };
-        // ---- pass 1: row max
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          load_half(h);
-#pragma unroll
-          for (int e = 0; e < 64; e += 4) {
-            mx[0] = fmaxf(mx[0], __uint_as_float(raw[e]));
-            mx[1] = fmaxf(mx[1], __uint_as_float(raw[e + 1]));
-            mx[2] = fmaxf(mx[2], __uint_as_float(raw[e + 2]));
-            mx[3] = fmaxf(mx[3], __uint_as_float(raw[e + 3]));
+          for (int e = 0; e < 64; ++e) {
+            const int mrel = key0 + h * 64 + e - L;
+            const bool vis = mrel < 0 || (mrel < n && ((anc >> mrel) & 1ull));
+            raw[e] = vis ? raw[e] : 0xff800000u;   // -inf
           }
         }
-        const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // scale > 0
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int e = 0; e < 64; e += 4) {
+          mx[0] = fmaxf(mx[0], __uint_as_float(raw[e]));
+          mx[1] = fmaxf(mx[1], __uint_as_float(raw[e + 1]));
+          mx[2] = fmaxf(mx[2], __uint_as_float(raw[e + 2]));
+          mx[3] = fmaxf(mx[3], __uint_as_float(raw[e + 3]));
+        }
+        const float half_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        // agree on the row max with the partner thread (other half of the row, same lane, warp +-4)
+        xch[(buf * 2 + h) * kBlockM + r] = half_max;
+        if (tid == 0) TRACE(2, (12 << 10) | (gs & 1023u));
+        ok = pair_sync();
+        if (!ok) break;
+        if (tid == 0) TRACE(2, (13 << 10) | (gs & 1023u));
+        const float tmax = fmaxf(half_max, xch[(buf * 2 + (h ^ 1)) * kBlockM + r]) * p.scale_log2;   // scale > 0
 
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
-          const uint32_t nv = 2 * g + 1, slot = nv % kSlots, par = (nv / kSlots) & 1u;
+          const uint32_t nv = 2 * (g_base + s) + 1, slot = nv % kSlots, par = (nv / kSlots) & 1u;
           ok = mbar_wait_warp(B.full[slot], par, s_abort);
           if (!ok) break;
-          if (key0 + r >= kv_end) {
+          if (key0 + r >= kv_end && h < S::kSlabs) {
 #pragma unroll
-            for (int sl = 0; sl < S::kSlabs; ++sl)
-#pragma unroll
-              for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(smem + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+            for (int c = 0; c < 8; ++c)
+              *reinterpret_cast<uint4*>(smem + S::kRing + slot * S::kTileBytes + h * S::kSlabBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
           fence_proxy_async();
         }
 
-        // lazy rescale: move the reference only when the row max outgrows it by more than the threshold.
-        // (PV of the previous step of this stream has completed: the QK that produced this S was issued after it.)
+        // P[buf] was last read by the PV of step gs - 2 (this wait also keeps every thread within one phase of o_done)
+        if (gs >= 2) {
+          ok = mbar_wait_warp(B.o_done[buf], ((gs - 2) >> 1) & 1u, s_abort);
+          if (!ok) break;
+        }
+        // lazy rescale: move the reference only when the row max outgrows it by more than the threshold
         const bool grow = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         float factor = 1.f;
         if (grow) {
@@ -452,58 +532,69 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
           m_ref = tmax;
           l_sum *= factor;
         }
-        if (k > 0 && __any_sync(0xffffffffu, grow)) {
+        if (s > 0 && __any_sync(0xffffffffu, grow)) {
+          // the previous step accumulated into O and may still be running
+          ok = mbar_wait_warp(B.o_done[buf ^ 1u], ((gs - 1) >> 1) & 1u, s_abort);
+          if (!ok) break;
+          tc_fence_after();
+          constexpr int HC = D / 2;           // this thread's half of the accumulator columns
           uint32_t o[32];
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            tmem_ld32(tmem + lane_addr + kColO + w * kTileN + c * 32, o);
+          for (int c = 0; c < HC / 32; ++c) {
+            const uint32_t o_addr = tmem + lane_addr + kColO + h * HC + c * 32;
+            tmem_ld32(o_addr, o);
             tc_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-            tmem_st32(tmem + lane_addr + kColO + w * kTileN + c * 32, o);
+            tmem_st32(o_addr, o);
           }
           tc_wait_st();
         }
-        // ---- pass 2: exponentials; packed bf16 P goes over score columns that have already been read
         const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          load_half(h);
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(raw[2 * e]), p.scale_log2, neg_base));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 1]), p.scale_log2, neg_base));
-            const float p2 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 2]), p.scale_log2, neg_base));
-            const float p3 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 3]), p.scale_log2, neg_base));
-            ls[0] += p0; ls[1] += p1; ls[2] += p2; ls[3] += p3;
-            raw[e] = pack_bf16(p0, p1);          // packed P overwrites entries already consumed
-            raw[e + 1] = pack_bf16(p2, p3);
-          }
-          tmem_st32(s_addr + h * 32, raw);
+        for (int e = 0; e < 32; e += 2) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(raw[2 * e]), p.scale_log2, neg_base));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 1]), p.scale_log2, neg_base));
+          const float p2 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 2]), p.scale_log2, neg_base));
+          const float p3 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 3]), p.scale_log2, neg_base));
+          ls[0] += p0; ls[1] += p1; ls[2] += p2; ls[3] += p3;
+          raw[e] = pack_bf16(p0, p1);          // packed P overwrites entries already consumed
+          raw[e + 1] = pack_bf16(p2, p3);
         }
         l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        if (tid == 0) TRACE(2, (14 << 10) | (gs & 1023u));
+        tmem_st32(tmem + lane_addr + kColP + buf * (kTileN / 2) + h * 32, raw);   // this thread's 64 P values
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(B.p_full[w]);
+        mbar_arrive(B.p_full[buf]);
+        if (tid == 0) TRACE(2, (11 << 10) | (gs & 1023u));
       }
       if (!ok) break;
 
-      // ---- epilogue
-      if (steps > 0) {
-        ok = mbar_wait_warp(B.o_done[w], (cws - 1) & 1u, s_abort);
+      // ---- epilogue: wait for the last PV (they complete in order), add the two halves of the row sum,
+      // then each thread writes its half of the columns of its row
+      {
+        const uint32_t gl = sg + steps - 1;
+        ok = mbar_wait_warp(B.o_done[gl & 1u], (gl >> 1) & 1u, s_abort);
         if (!ok) break;
+        if (tid == 0) TRACE(2, 20);
         tc_fence_after();
-      }
-      if (mode) {
-        // two query tiles: each warpgroup owns its rows outright
-        const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-        __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D;
-        float* part_row = it.slot >= 0 ? p.part_o + (static_cast<size_t>(it.slot + w) * kBlockM + r) * D : nullptr;
+        float* lx = xch;   // reuse the exchange area: [h][row]; every max exchange of this item is over
+        ok = pair_sync();
+        if (!ok) break;
+        lx[h * kBlockM + r] = l_sum;
+        ok = pair_sync();
+        if (!ok) break;
+        constexpr int HC = D / 2;
+        const float l_row = l_sum + lx[(h ^ 1) * kBlockM + r];
+        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+        __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * HC;
+        float* part_row = it.slot >= 0 ? p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D + h * HC : nullptr;
         uint32_t o[32];
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          tmem_ld32(tmem + lane_addr + kColO + w * kTileN + c * 32, o);
+        for (int c = 0; c < HC / 32; ++c) {
+          tmem_ld32(tmem + lane_addr + kColO + h * HC + c * 32, o);
           tc_wait_ld();
           if (row_valid) {
             if (it.slot < 0) {
@@ -523,62 +614,15 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
             }
           }
         }
-        if (row_valid && it.slot >= 0) p.part_ml[static_cast<size_t>(it.slot + w) * kBlockM + r] = make_float2(m_ref, l_sum);
-      } else {
-        // one query tile split over even / odd KV tiles: merge the two streams; warpgroup w writes half the columns
-        float2* ml = reinterpret_cast<float2*>(smem + S::kMl);
-        ml[w * kBlockM + r] = make_float2(m_ref, l_sum);
-        mbar_arrive(B.ml_full);
-        ok = mbar_wait_warp(B.ml_full, mode0_count & 1u, s_abort);
-        ++mode0_count;
+        if (row_valid && it.slot >= 0 && h == 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_ref, l_row);
+        ok = pair_sync();   // the partner has read the exchanged sum
         if (!ok) break;
-        tc_fence_after();
-        const float2 mine = make_float2(m_ref, l_sum), other = ml[(w ^ 1) * kBlockM + r];
-        const float2 a = w == 0 ? mine : other, bq = w == 0 ? other : mine;      // stream 0, stream 1
-        const float m_star = fmaxf(a.y > 0.f ? a.x : -INFINITY, bq.y > 0.f ? bq.x : -INFINITY);
-        const float wa = a.y > 0.f ? fast_exp2(a.x - m_star) : 0.f, wb = bq.y > 0.f ? fast_exp2(bq.x - m_star) : 0.f;
-        const float l_star = a.y * wa + bq.y * wb;
-        const float inv = l_star > 0.f ? 1.f / l_star : 0.f;
-        const float fa = it.slot < 0 ? wa * inv : wa, fb = it.slot < 0 ? wb * inv : wb;
-        constexpr int HALF = D / 2;
-        __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + w * HALF;
-        float* part_row = it.slot >= 0 ? p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D + w * HALF : nullptr;
-        uint32_t oa[32], ob[32];
-#pragma unroll
-        for (int c = 0; c < HALF / 32; ++c) {
-          tmem_ld32(tmem + lane_addr + kColO + w * HALF + c * 32, oa);
-          tmem_ld32(tmem + lane_addr + kColO + kTileN + w * HALF + c * 32, ob);
-          tc_wait_ld();
-          float v[32];
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            const float xa = wa > 0.f ? __uint_as_float(oa[e]) * fa : 0.f;   // a stream without keys left its columns untouched
-            const float xb = wb > 0.f ? __uint_as_float(ob[e]) * fb : 0.f;
-            v[e] = xa + xb;
-          }
-          if (row_valid) {
-            if (it.slot < 0) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                uint4 u;
-                u.x = pack_bf16(v[e + 0], v[e + 1]);
-                u.y = pack_bf16(v[e + 2], v[e + 3]);
-                u.z = pack_bf16(v[e + 4], v[e + 5]);
-                u.w = pack_bf16(v[e + 6], v[e + 7]);
-                *reinterpret_cast<uint4*>(out_row + c * 32 + e) = u;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<float4*>(part_row + c * 32 + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
-            }
-          }
-        }
-        if (row_valid && it.slot >= 0 && w == 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_star, l_star);
       }
       tc_fence_before();
       mbar_arrive(B.o_free);
-      g_base += nt;
+      if (tid == 0) TRACE(2, 21);
+      g_base += steps;
+      sg += steps;
       ++item_count;
     }
   }
@@ -622,6 +666,19 @@ bool make_kv_map(CUtensorMap* map, const void* base, int D, int S_cap, long long
 }
 
 }  // namespace
+
+#ifdef EAGLE_TRACE
+}  // namespace eagle
+extern "C" int eagle_debug_trace(unsigned long long* dst, int* counts) {
+  int zero[4] = {0, 0, 0, 0};
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(dst, eagle::g_trace, sizeof(unsigned long long) * 4 * 1024);
+  cudaMemcpyFromSymbol(counts, eagle::g_trace_n, sizeof(int) * 4);
+  cudaMemcpyToSymbol(eagle::g_trace_n, zero, sizeof(zero));
+  return 0;
+}
+namespace eagle {
+#endif
 
 int attn_tc2_tile_keys() { return kTileN; }
 
