@@ -18,9 +18,7 @@ struct DeviceInfo {
   bool ready = false;
   int sm_count = 0;
   int cc_major = 0;
-  bool mma_prepared[2] = {false, false};
-  bool tc_prepared[2] = {false, false};
-  bool tc2_prepared[2] = {false, false};
+  bool attn_prepared[2] = {false, false};
 };
 constexpr int kMaxDevices = 64;
 DeviceInfo g_dev[kMaxDevices];
@@ -84,23 +82,12 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   if (!dev) return err;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int di = d.head_dim == 128 ? 1 : 0;
-  const char* impl_env = std::getenv("EAGLE_ATTN_IMPL");
-  const bool use_tc2 = impl_env && std::strcmp(impl_env, "tc2") == 0;
-  const bool use_tc = use_tc2 || (impl_env && std::strcmp(impl_env, "tc") == 0);
-  if (use_tc2 && !dev->tc2_prepared[di]) {
-    if (attn_tc2_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
-    dev->tc2_prepared[di] = true;
-  }
-  if (use_tc && !use_tc2 && !dev->tc_prepared[di]) {
-    if (attn_tc_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
-    dev->tc_prepared[di] = true;
-  }
-  if (!use_tc && !dev->mma_prepared[di]) {
-    if (attn_mma_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
-    dev->mma_prepared[di] = true;
+  if (!dev->attn_prepared[di]) {
+    if (attn_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
+    dev->attn_prepared[di] = true;
   }
   const int G = d.num_q_heads / d.num_kv_heads;
-  const int num_ctas = use_tc ? dev->sm_count : dev->sm_count * attn_mma_ctas_per_sm(d.head_dim);
+  const int num_ctas = dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas;   // one persistent CTA per SM
 
   PlanParams pp;
   pp.seq_lens = seq_lens;
@@ -111,16 +98,19 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.G = G;
   pp.T_max = d.max_tree;
   pp.S_cap = d.kv_capacity;
-  pp.tile_keys = use_tc ? attn_tc_tile_keys() : attn_mma_tile_keys();
+  pp.tile_keys = attn_tile_keys();
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
-  pp.min_chunk_tiles = 256 / pp.tile_keys > 0 ? 256 / pp.tile_keys : 1;
-  pp.pair = 0;
+  pp.snap_tiles = 2;
+  pp.item_overhead_tiles = 4;
+  pp.unit_cap = w.unit_cap;
   pp.item_cap = w.item_cap;
   pp.slot_cap = w.slot_cap;
   pp.hdr = w.hdr;
   pp.seq = w.seq;
   pp.anc = w.anc;
+  pp.units = w.units;
+  pp.cta_first = w.cta_first;
   pp.items = w.items;
   pp.status = d.status;
   if (launch_plan(pp, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
@@ -139,20 +129,19 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.S_cap = d.kv_capacity;
   const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
   ap.scale_log2 = scale * 1.4426950408889634f;
-  ap.pair = 0;
   ap.hdr = w.hdr;
   ap.seq = w.seq;
   ap.anc = w.anc;
+  ap.units = w.units;
+  ap.cta_first = w.cta_first;
   ap.items = w.items;
   ap.part_ml = w.part_ml;
   ap.part_o = w.part_o;
   ap.status = d.status;
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  const cudaError_t le = use_tc2 ? launch_attn_tc2(ap, num_ctas, stream)
-                                 : (use_tc ? launch_attn_tc(ap, num_ctas, stream) : launch_attn_mma(ap, num_ctas, stream));
-  if (le != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_combine(ap, nullptr, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 

@@ -1,15 +1,19 @@
 // Split-KV tree attention for sm_100a: TMA-staged KV tiles, tcgen05 MMAs, accumulators in TMEM.
 //
-// One persistent CTA per SM walks a static slice of the planner's work list.  An item is one 128-row query
-// tile (row = tree node * G + head-in-group) of one (sequence, KV head) over a range of 128-key KV tiles;
+// One persistent CTA per SM walks its share of the planner's work list (equal numbers of KV tiles per CTA).  An
+// item is one 128-row query tile (row = tree node * G + head-in-group) of one (sequence, KV head) over a range of
+// 128-key KV tiles;
 // step s of the item handles KV tile s:
 //     S[s&1] = Q K^T   ->   softmax   ->   P[s&1] (packed bf16)   ->   O += P V.
 // S and P are double buffered in TMEM (S0 S1 | O | P0 P1 = 512 columns), so the score MMA of step s+1 and the
 // PV MMA of step s-1 run while the softmax warps work on step s.
 // Warp roles: warps 0-7 softmax (thread pair (r, r+128) shares query row r = TMEM lane r, 64 score columns
 // each; the pair agrees on the row max through shared memory), warp 8 TMA producer (K and V tiles through a
-// ring of six 32 KB slots, 128-byte swizzled boxes), warp 9 issues the QK MMAs and warp 10 the PV MMAs (each
-// waits only on what its own MMA needs).  Softmax is fp32 in the log2 domain; the tree mask is applied in
+// ring of five 32 KB slots, and the query tile of the NEXT item into the other half of a double-buffered Q
+// area; 128-byte swizzled boxes), warp 9 issues the QK MMAs and warp 10 the PV MMAs (each waits only on what
+// its own MMA needs).  Items overlap at their seams: the score MMA of the next item's first tile is issued
+// while the current item finishes, and the softmax warps take that first step before they write the finished
+// item's output, so the accumulator drain and the pipeline fill hide behind each other.  Softmax is fp32 in the log2 domain; the tree mask is applied in
 // registers only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are
 // zeroed in shared memory before the MMA reads them.  The accumulator is rescaled only when the running max
 // grows by more than 2^8.  Every wait is bounded (mbarrier try_wait + timer); on expiry the CTA raises
@@ -23,7 +27,7 @@ namespace eagle {
 namespace {
 
 constexpr int kTileN = 128;          // keys per KV tile
-constexpr int kSlots = 6;            // ring slots; tile g uses slot (2g) % 6 for K and (2g+1) % 6 for V
+constexpr int kSlots = 5;            // ring slots; tile g uses slot (2g) % 5 for K and (2g+1) % 5 for V
 constexpr int kThreads = 352;
 constexpr int kSoftmaxThreads = 256;
 constexpr uint32_t kTmemCols = 512;
@@ -127,6 +131,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -149,6 +159,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
 // Debug builds only: CTA 0 logs (tag, clock) pairs per role; read back with eagle_debug_trace().
 __device__ unsigned long long g_trace[4][1024];
 __device__ int g_trace_n[4];
+__device__ long long g_cta_stat[1024][4];   // per CTA: cycles, items, tiles, tail tiles
 #define TRACE(role, tag)                                                                          \
   do {                                                                                            \
     if (blockIdx.x == 0 && trace_n < 1024) {                                                      \
@@ -230,34 +241,31 @@ __device__ __forceinline__ void issue_pv_tile(uint32_t o_tmem, uint32_t p_tmem, 
 }
 
 template <int D>
-struct Smem2 {
+struct Smem {
   static constexpr int kSlabs = D / 64;                     // 64 bf16 = one 128-byte swizzled row
   static constexpr int kSlabBytes = kTileN * 128;            // 128 rows x 128 bytes
   static constexpr int kTileBytes = kSlabs * kSlabBytes;     // one Q / K / V tile
-  static constexpr int kQ = 0;
-  static constexpr int kRing = kTileBytes;
+  static constexpr int kQ = 0;                               // two query tiles (double buffer)
+  static constexpr int kRing = 2 * kTileBytes;
   static constexpr int kXch = kRing + kSlots * kTileBytes;   // float [2 parities][2 halves][128 rows]: row-max exchange
   static constexpr int kBar = kXch + 2 * 2 * kBlockM * 4;
-  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 3 + 4;
+  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 5 + 4;
   static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag
   static constexpr int kBytes = kMisc + 16;
 };
 
-struct Bars2 {
+struct Bars {
   uint32_t full[kSlots], empty[kSlots];
   uint32_t s_full[2], p_full[2], o_done[2];
-  uint32_t q_full, q_empty, o_free;
+  uint32_t q_full[2], q_empty[2], o_free;
   uint32_t pair[4];   // one per TMEM lane quarter: the two softmax warps that share its rows
 };
 
-__device__ __forceinline__ int item_index(int row, int cta, int grid) {
-  return row * grid + ((row & 1) ? (grid - 1 - cta) : cta);
-}
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
-  using S = Smem2<D>;
+attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+            const __grid_constant__ CUtensorMap map_q) {
+  using S = Smem<D>;
   extern __shared__ __align__(1024) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -266,7 +274,7 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
     return;
   }
 
-  Bars2 B;
+  Bars B;
   {
     uint32_t b = sbase + S::kBar;
     for (int i = 0; i < kSlots; ++i) { B.full[i] = b; b += 8; }
@@ -274,8 +282,8 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
     for (int i = 0; i < 2; ++i) { B.s_full[i] = b; b += 8; }
     for (int i = 0; i < 2; ++i) { B.p_full[i] = b; b += 8; }
     for (int i = 0; i < 2; ++i) { B.o_done[i] = b; b += 8; }
-    B.q_full = b; b += 8;
-    B.q_empty = b; b += 8;
+    for (int i = 0; i < 2; ++i) { B.q_full[i] = b; b += 8; }
+    for (int i = 0; i < 2; ++i) { B.q_empty[i] = b; b += 8; }
     B.o_free = b; b += 8;
     for (int i = 0; i < 4; ++i) { B.pair[i] = b; b += 8; }
   }
@@ -292,8 +300,10 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
       mbar_init(B.p_full[i], kSoftmaxThreads);
       mbar_init(B.o_done[i], 1);
     }
-    mbar_init(B.q_full, kSoftmaxThreads);
-    mbar_init(B.q_empty, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(B.q_full[i], p.q_tma ? 1 : kSoftmaxThreads);   // one TMA transaction, or every softmax thread's rows
+      mbar_init(B.q_empty[i], 1);
+    }
     mbar_init(B.o_free, kSoftmaxThreads);
     for (int i = 0; i < 4; ++i) mbar_init(B.pair[i], 64);
     *s_abort = 0;
@@ -308,23 +318,34 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  const int n_items = p.hdr->n_items;
-  const int grid = gridDim.x, cta = blockIdx.x;
+  // this CTA's share of the work line: items [item_lo, item_hi)
+  const int item_lo = p.cta_first[blockIdx.x], item_hi = p.cta_first[blockIdx.x + 1];
 #ifdef EAGLE_TRACE
   int trace_n = 0;
+  const long long trace_t0 = clock64();
 #endif
 
   if (warp == 8) {
     // =========================================================================== TMA producer
     if (lane == 0) {
       uint32_t g = 0;   // KV tiles issued by this CTA so far
+      uint32_t item_count = 0;
       bool ok = true;
-      for (int row = 0; ok; ++row) {
-        const int idx = item_index(row, cta, grid);
-        if (idx >= n_items) break;
+      for (int idx = item_lo; idx < item_hi && ok; ++idx, ++item_count) {
         const WorkItem it = p.items[idx];
         const int z = it.b * p.Hkv + it.g;
         TRACE(0, 1);
+        if (p.q_tma) {
+          // query tile: box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
+          const uint32_t qb = item_count & 1u;
+          ok = mbar_wait(B.q_empty[qb], ((item_count >> 1) & 1u) ^ 1u, s_abort);
+          if (!ok) break;
+          mbar_expect_tx(B.q_full[qb], S::kTileBytes);
+#pragma unroll
+          for (int s = 0; s < S::kSlabs; ++s)
+            tma_load_4d(sbase + S::kQ + qb * S::kTileBytes + s * S::kSlabBytes, &map_q, s * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b,
+                        B.q_full[qb]);
+        }
         for (int tile = it.tile_begin; tile < it.tile_end && ok; ++tile, ++g) {
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
@@ -350,18 +371,18 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
       uint32_t ks = 0, kp = 0;       // slot / parity of the K tile of the next QK
       uint32_t gq = 0;               // steps issued so far (all items)
       uint32_t item_count = 0;
-      const uint32_t q_lo = desc_lo(sbase + S::kQ, 16), ring_lo_k = desc_lo(sbase + S::kRing, 16);
+      const uint32_t q_lo0 = desc_lo(sbase + S::kQ, 16), ring_lo_k = desc_lo(sbase + S::kRing, 16);
       constexpr uint32_t kTileStep = S::kTileBytes >> 4;
       bool ok = true;
-      for (int row = 0; ok; ++row) {
-        const int idx = item_index(row, cta, grid);
-        if (idx >= n_items) break;
+      for (int idx = item_lo; idx < item_hi && ok; ++idx) {
         const WorkItem it = p.items[idx];
         const int steps = it.tile_end - it.tile_begin;
         TRACE(1, 1);
-        ok = mbar_wait(B.q_full, item_count & 1u, s_abort);
+        const uint32_t qb = item_count & 1u;
+        ok = mbar_wait(B.q_full[qb], (item_count >> 1) & 1u, s_abort);
         if (!ok) break;
         TRACE(1, 2);
+        const uint32_t q_lo = q_lo0 + qb * kTileStep;
         for (int s = 0; s < steps && ok; ++s, ++gq) {
           // S[gq & 1] is free once the softmax warps have read the scores of step gq - 2
           if (gq >= 2) {
@@ -377,7 +398,7 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
           tc_commit(B.empty[ks]);
           ks += 2;
           if (ks >= kSlots) { ks -= kSlots; kp ^= 1u; }
-          if (s == steps - 1) tc_commit(B.q_empty);          // every QK of this item has been issued
+          if (s == steps - 1) tc_commit(B.q_empty[qb]);      // every QK of this item has been issued
           TRACE(1, (11 << 10) | (gq & 1023u));
         }
         ++item_count;
@@ -393,9 +414,7 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
       const uint32_t ring_lo_v = desc_lo(sbase + S::kRing, S::kSlabBytes);
       constexpr uint32_t kTileStep = S::kTileBytes >> 4;
       bool ok = true;
-      for (int row = 0; ok; ++row) {
-        const int idx = item_index(row, cta, grid);
-        if (idx >= n_items) break;
+      for (int idx = item_lo; idx < item_hi && ok; ++idx) {
         const WorkItem it = p.items[idx];
         const int steps = it.tile_end - it.tile_begin;
         for (int s = 0; s < steps && ok; ++s, ++gp) {
@@ -434,11 +453,65 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
       return k;
     };
     float* xch = reinterpret_cast<float*>(smem + S::kXch);
+    constexpr int HC = D / 2;                             // this thread's half of the accumulator columns
+
+    // What the epilogue of an item needs after its last softmax step.
+    struct Done {
+      bool live, row_valid;
+      int slot;
+      uint32_t last_step;      // global number of the item's last step
+      float m_ref, l_sum;
+      __nv_bfloat16* out_row;  // this thread's half of its output row
+    };
+    Done prev;
+    prev.live = false;
+    // Wait for the item's last PV (PVs complete in order), add the two halves of the row sum, then write this
+    // thread's half of the columns of its row: bf16 output, or the unnormalised fp32 partial of a cut unit.
+    auto epilogue = [&](const Done& d) -> bool {
+      if (!mbar_wait_warp(B.o_done[d.last_step & 1u], (d.last_step >> 1) & 1u, s_abort)) return false;
+      if (tid == 0) TRACE(2, 20);
+      tc_fence_after();
+      float* lx = xch;   // [half][row]; the surrounding pair syncs keep it apart from the row-max exchanges
+      if (!pair_sync()) return false;
+      lx[h * kBlockM + r] = d.l_sum;
+      if (!pair_sync()) return false;
+      const float l_row = d.l_sum + lx[(h ^ 1) * kBlockM + r];
+      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+      float* part_row = d.slot >= 0 ? p.part_o + (static_cast<size_t>(d.slot) * kBlockM + r) * D + h * HC : nullptr;
+      uint32_t o[32];
+#pragma unroll
+      for (int c = 0; c < HC / 32; ++c) {
+        tmem_ld32(tmem + lane_addr + kColO + h * HC + c * 32, o);
+        tc_wait_ld();
+        if (d.row_valid) {
+          if (d.slot < 0) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 8) {
+              uint4 v;
+              v.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
+              v.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+              v.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+              v.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
+              *reinterpret_cast<uint4*>(d.out_row + c * 32 + e) = v;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<uint4*>(part_row + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+          }
+        }
+      }
+      if (d.row_valid && d.slot >= 0 && h == 0) p.part_ml[static_cast<size_t>(d.slot) * kBlockM + r] = make_float2(d.m_ref, l_row);
+      if (!pair_sync()) return false;   // the partner has read the exchanged sum
+      tc_fence_before();
+      mbar_arrive(B.o_free);            // the next item's first PV may overwrite the accumulator
+      if (tid == 0) TRACE(2, 21);
+      return true;
+    };
+
     uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps done so far
     bool ok = true;
-    for (int row = 0; ok; ++row) {
-      const int idx = item_index(row, cta, grid);
-      if (idx >= n_items) break;
+    for (int idx = item_lo; idx < item_hi && ok; ++idx) {
       const WorkItem it = p.items[idx];
       const SeqPlan sp = p.seq[it.b];
       const int L = sp.L, n = sp.n, G = p.G;
@@ -449,23 +522,25 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
       const int node = row_valid ? R / G : 0, hh = row_valid ? R % G : 0;
       const uint64_t anc = row_valid ? p.anc[static_cast<size_t>(it.b) * p.T_max + node] : 0ull;
 
-      // ---- stage Q: thread (h, r) writes the h-th 64-column slab of row r (D = 64: h = 0 only)
-      if (tid == 0) TRACE(2, 1);
-      ok = mbar_wait_warp(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
-      if (!ok) break;
-      if (tid == 0) TRACE(2, 2);
-      if (h < S::kSlabs) {
-        const uint4* src = reinterpret_cast<const uint4*>(
-            p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * 64);
-        unsigned char* qdst = smem + S::kQ + h * S::kSlabBytes + r * 128;
+      if (!p.q_tma) {
+        // group sizes that do not divide 128: the softmax threads stage the query tile themselves;
+        // thread (h, r) writes the h-th 64-column slab of row r (D = 64: h = 0 only)
+        const uint32_t qb = item_count & 1u;
+        ok = mbar_wait_warp(B.q_empty[qb], ((item_count >> 1) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        if (h < S::kSlabs) {
+          const uint4* src = reinterpret_cast<const uint4*>(
+              p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * 64);
+          unsigned char* qdst = smem + S::kQ + qb * S::kTileBytes + h * S::kSlabBytes + r * 128;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-          *reinterpret_cast<uint4*>(qdst + ((c ^ (r & 7)) << 4)) = v;
+          for (int c = 0; c < 8; ++c) {
+            const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(qdst + ((c ^ (r & 7)) << 4)) = v;
+          }
         }
+        fence_proxy_async();
+        mbar_arrive(B.q_full[qb]);
       }
-      fence_proxy_async();
-      mbar_arrive(B.q_full);
       if (tid == 0) TRACE(2, 3);
 
       float m_ref = -INFINITY;   // reference max (scaled, log2 domain) of every exponential taken so far
@@ -482,11 +557,19 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
         tc_wait_ld();
         const int key0 = (it.tile_begin + s) * kTileN;
         if (key0 + kTileN > L) {          // the tile reaches past the committed prefix: tree mask + cache tail
+          // visibility of this thread's 64 keys as one 64-bit word: keys before L are all visible, key L + m is
+          // visible iff bit m of the node's ancestor mask is set (the mask has no bits at or above the tree size)
+          const int rel = key0 + h * 64 - L;          // tree index of this thread's first key (negative: still in the prefix)
+          uint64_t vis;
+          if (rel >= 64) vis = 0ull;
+          else if (rel >= 0) vis = anc >> rel;
+          else if (rel > -64) vis = (anc << (-rel)) | ((1ull << (-rel)) - 1ull);
+          else vis = ~0ull;
+          const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
 #pragma unroll
-          for (int e = 0; e < 64; ++e) {
-            const int mrel = key0 + h * 64 + e - L;
-            const bool vis = mrel < 0 || (mrel < n && ((anc >> mrel) & 1ull));
-            raw[e] = vis ? raw[e] : 0xff800000u;   // -inf
+          for (int e = 0; e < 32; ++e) {
+            raw[e] = (vlo >> e) & 1u ? raw[e] : 0xff800000u;            // -inf
+            raw[32 + e] = (vhi >> e) & 1u ? raw[32 + e] : 0xff800000u;
           }
         }
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -500,10 +583,8 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
         const float half_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         // agree on the row max with the partner thread (other half of the row, same lane, warp +-4)
         xch[(buf * 2 + h) * kBlockM + r] = half_max;
-        if (tid == 0) TRACE(2, (12 << 10) | (gs & 1023u));
         ok = pair_sync();
         if (!ok) break;
-        if (tid == 0) TRACE(2, (13 << 10) | (gs & 1023u));
         const float tmax = fmaxf(half_max, xch[(buf * 2 + (h ^ 1)) * kBlockM + r]) * p.scale_log2;   // scale > 0
 
         if (key0 + kTileN > kv_end) {
@@ -537,7 +618,6 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
           ok = mbar_wait_warp(B.o_done[buf ^ 1u], ((gs - 1) >> 1) & 1u, s_abort);
           if (!ok) break;
           tc_fence_after();
-          constexpr int HC = D / 2;           // this thread's half of the accumulator columns
           uint32_t o[32];
 #pragma unroll
           for (int c = 0; c < HC / 32; ++c) {
@@ -563,74 +643,54 @@ attn_tc2_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const _
           raw[e + 1] = pack_bf16(p2, p3);
         }
         l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-        if (tid == 0) TRACE(2, (14 << 10) | (gs & 1023u));
         tmem_st32(tmem + lane_addr + kColP + buf * (kTileN / 2) + h * 32, raw);   // this thread's 64 P values
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(B.p_full[buf]);
         if (tid == 0) TRACE(2, (11 << 10) | (gs & 1023u));
+
+        // the finished item's output is written after the first step of this one: its last PV has had time
+        // to complete, and this item's second score tile is being computed meanwhile
+        if (s == 0 && prev.live) {
+          ok = epilogue(prev);
+          prev.live = false;
+        }
       }
       if (!ok) break;
-
-      // ---- epilogue: wait for the last PV (they complete in order), add the two halves of the row sum,
-      // then each thread writes its half of the columns of its row
-      {
-        const uint32_t gl = sg + steps - 1;
-        ok = mbar_wait_warp(B.o_done[gl & 1u], (gl >> 1) & 1u, s_abort);
-        if (!ok) break;
-        if (tid == 0) TRACE(2, 20);
-        tc_fence_after();
-        float* lx = xch;   // reuse the exchange area: [h][row]; every max exchange of this item is over
-        ok = pair_sync();
-        if (!ok) break;
-        lx[h * kBlockM + r] = l_sum;
-        ok = pair_sync();
-        if (!ok) break;
-        constexpr int HC = D / 2;
-        const float l_row = l_sum + lx[(h ^ 1) * kBlockM + r];
-        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-        __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * HC;
-        float* part_row = it.slot >= 0 ? p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D + h * HC : nullptr;
-        uint32_t o[32];
-#pragma unroll
-        for (int c = 0; c < HC / 32; ++c) {
-          tmem_ld32(tmem + lane_addr + kColO + h * HC + c * 32, o);
-          tc_wait_ld();
-          if (row_valid) {
-            if (it.slot < 0) {
-#pragma unroll
-              for (int e = 0; e < 32; e += 8) {
-                uint4 v;
-                v.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
-                v.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-                v.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-                v.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-                *reinterpret_cast<uint4*>(out_row + c * 32 + e) = v;
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < 32; e += 4)
-                *reinterpret_cast<uint4*>(part_row + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
-            }
-          }
-        }
-        if (row_valid && it.slot >= 0 && h == 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_ref, l_row);
-        ok = pair_sync();   // the partner has read the exchanged sum
-        if (!ok) break;
-      }
-      tc_fence_before();
-      mbar_arrive(B.o_free);
-      if (tid == 0) TRACE(2, 21);
+      prev.live = true;
+      prev.row_valid = row_valid;
+      prev.slot = it.slot;
+      prev.last_step = sg + steps - 1;
+      prev.m_ref = m_ref;
+      prev.l_sum = l_sum;
+      prev.out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * HC;
       g_base += steps;
       sg += steps;
       ++item_count;
     }
+    if (ok && prev.live) ok = epilogue(prev);
   }
 
+#ifdef EAGLE_TRACE
+  if (tid == 0) {
+    long long tiles = 0, tails = 0;
+    for (int idx = item_lo; idx < item_hi; ++idx) {
+      const WorkItem it = p.items[idx];
+      tiles += it.tile_end - it.tile_begin;
+      tails += (it.tile_end * kTileN > p.seq[it.b].L) ? 1 : 0;
+    }
+    g_cta_stat[blockIdx.x][1] = item_hi - item_lo;
+    g_cta_stat[blockIdx.x][2] = tiles;
+    g_cta_stat[blockIdx.x][3] = tails;
+  }
+#endif
   // ---- teardown: everyone arrives here (normally or after an abort); release TMEM
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && *s_abort) report_status(p.status, EAGLE_ERR_TIMEOUT);
+#ifdef EAGLE_TRACE
+  if (tid == 0) g_cta_stat[blockIdx.x][0] = clock64() - trace_t0;
+#endif
   if (warp == 9) {
     __syncwarp();
     tc_fence_after();
@@ -665,10 +725,30 @@ bool make_kv_map(CUtensorMap* map, const void* base, int D, int S_cap, long long
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// q [B, T_max, Hq, D] bf16 viewed as (d, head, node, sequence); box = 64 x G x 128/G x 1: the 128 query rows of one
+// (sequence, KV head, query tile) in (node, head-in-group) order.  Needs 128 % G == 0.
+bool make_q_map(CUtensorMap* map, const void* base, int D, int Hq, int T_max, int B, int G) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(Hq), static_cast<cuuint64_t>(T_max),
+                              static_cast<cuuint64_t>(B)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(Hq) * D * 2,
+                                 static_cast<cuuint64_t>(T_max) * Hq * D * 2};
+  const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(G), static_cast<cuuint32_t>(kBlockM / G), 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 #ifdef EAGLE_TRACE
 }  // namespace eagle
+extern "C" int eagle_debug_cta_stat(long long* dst) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(dst, eagle::g_cta_stat, sizeof(long long) * 1024 * 4);
+  return 0;
+}
 extern "C" int eagle_debug_trace(unsigned long long* dst, int* counts) {
   int zero[4] = {0, 0, 0, 0};
   cudaDeviceSynchronize();
@@ -680,21 +760,28 @@ extern "C" int eagle_debug_trace(unsigned long long* dst, int* counts) {
 namespace eagle {
 #endif
 
-int attn_tc2_tile_keys() { return kTileN; }
+int attn_tile_keys() { return kTileN; }
 
-cudaError_t attn_tc2_prepare(int head_dim) {
+cudaError_t attn_prepare(int head_dim) {
   if (head_dim == 128)
-    return cudaFuncSetAttribute(attn_tc2_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem2<128>::kBytes);
-  return cudaFuncSetAttribute(attn_tc2_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem2<64>::kBytes);
+    return cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kBytes);
+  return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
 }
 
 // Returns cudaErrorInvalidValue when the tensor maps cannot be encoded.
-cudaError_t launch_attn_tc2(const AttnParams& p, int num_ctas, cudaStream_t stream) {
-  CUtensorMap mk, mv;
+cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t stream) {
+  AttnParams p = p_in;
+  CUtensorMap mk, mv, mq;
   const long long bh = static_cast<long long>(p.B) * p.Hkv;
   if (!make_kv_map(&mk, p.k, p.D, p.S_cap, bh) || !make_kv_map(&mv, p.v, p.D, p.S_cap, bh)) return cudaErrorInvalidValue;
-  if (p.D == 128) attn_tc2_kernel<128><<<num_ctas, kThreads, Smem2<128>::kBytes, stream>>>(p, mk, mv);
-  else attn_tc2_kernel<64><<<num_ctas, kThreads, Smem2<64>::kBytes, stream>>>(p, mk, mv);
+  p.q_tma = (kBlockM % p.G == 0) ? 1 : 0;
+  if (p.q_tma) {
+    if (!make_q_map(&mq, p.q, p.D, p.Hq, p.T_max, p.B, p.G)) return cudaErrorInvalidValue;
+  } else {
+    mq = mk;   // unused by the kernel
+  }
+  if (p.D == 128) attn_kernel<128><<<num_ctas, kThreads, Smem<128>::kBytes, stream>>>(p, mk, mv, mq);
+  else attn_kernel<64><<<num_ctas, kThreads, Smem<64>::kBytes, stream>>>(p, mk, mv, mq);
   count_launch();
   return cudaGetLastError();
 }

@@ -1,5 +1,5 @@
 // Merge of the split-KV partials: m* = max_s m_s, l* = sum_s l_s 2^(m_s - m*), O = sum_s O_s 2^(m_s - m*) / l*.
-// One warp per output row (sequence, node, query head).  Rows of sequences that were not split were already
+// One warp per output row (sequence, node, query head).  Rows of work units that stayed in one piece were already
 // written by the attention kernel and are skipped; rows of nodes past the tree size are written as zeros.
 #include "common.cuh"
 
@@ -26,35 +26,27 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
     else *reinterpret_cast<uint32_t*>(dst) = 0u;
     return;
   }
-  if (sp.splits <= 1) return;
   const int g = h / p.G, R = i * p.G + h % p.G;
   const int mt = R / kBlockM, r = R % kBlockM;
-  // unpaired plans: one slot per (KV head, query tile, split); paired plans: two slots per (KV head, pair, split),
-  // the second used only when the pair really holds two query tiles
-  size_t slot0, stride;
-  if (p.pair) {
-    const int units = (sp.mtiles + 1) / 2;
-    slot0 = static_cast<size_t>(sp.slot_base) + 2 * (static_cast<size_t>(g) * units + mt / 2) * sp.splits + (mt & 1);
-    stride = 2;
-  } else {
-    slot0 = static_cast<size_t>(sp.slot_base) + (static_cast<size_t>(g) * sp.mtiles + mt) * sp.splits;
-    stride = 1;
-  }
+  const UnitPlan up = p.units[sp.unit_base + g * sp.mtiles + mt];
+  if (up.n_pieces <= 1) return;   // written directly by the attention kernel
+  const size_t slot0 = static_cast<size_t>(up.slot_base);
+  const int splits = up.n_pieces;
   float m_star = -INFINITY;
-  for (int s = 0; s < sp.splits; ++s) {
-    const float2 ml = p.part_ml[(slot0 + s * stride) * kBlockM + r];
+  for (int s = 0; s < splits; ++s) {
+    const float2 ml = p.part_ml[(slot0 + s) * kBlockM + r];
     if (ml.y > 0.f) m_star = fmaxf(m_star, ml.x);
   }
   float acc[E];
 #pragma unroll
   for (int e = 0; e < E; ++e) acc[e] = 0.f;
   float l_star = 0.f;
-  for (int s = 0; s < sp.splits; ++s) {
-    const float2 ml = p.part_ml[(slot0 + s * stride) * kBlockM + r];
+  for (int s = 0; s < splits; ++s) {
+    const float2 ml = p.part_ml[(slot0 + s) * kBlockM + r];
     if (!(ml.y > 0.f)) continue;   // a split in which this row saw no key
     const float w = exp2f(ml.x - m_star);
     l_star += ml.y * w;
-    const float* po = p.part_o + ((slot0 + s * stride) * kBlockM + r) * D + lane * E;
+    const float* po = p.part_o + ((slot0 + s) * kBlockM + r) * D + lane * E;
     if (E == 4) {
       const float4 v = *reinterpret_cast<const float4*>(po);
       acc[0] += v.x * w; acc[1] += v.y * w; acc[2 % E] += v.z * w; acc[3 % E] += v.w * w;
@@ -75,7 +67,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
 
 }  // namespace
 
-cudaError_t launch_combine(const AttnParams& p, const int32_t*, cudaStream_t stream) {
+cudaError_t launch_combine(const AttnParams& p, cudaStream_t stream) {
   const long long rows = static_cast<long long>(p.B) * p.T_max * p.Hq;
   if (rows == 0) return cudaSuccess;
   const unsigned blocks = static_cast<unsigned>((rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32));

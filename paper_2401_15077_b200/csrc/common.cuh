@@ -9,36 +9,45 @@
 namespace eagle {
 
 constexpr int kMaxTree = EAGLE_MAX_TREE;
-constexpr int kBlockM = 128;          // query rows (tree node x head-in-group) per work item
+constexpr int kBlockM = 128;          // query rows (tree node x head-in-group) per work unit
 constexpr int kMaxGroup = 16;         // largest GQA group size supported
-constexpr int kSlotBudgetAuto = 2048; // partial slots the planner may use when it chooses the splits itself
+constexpr int kMaxPlanCtas = 256;     // upper bound on the CTAs of the persistent attention kernel (one per SM)
 
-// One unit of attention work: a 128-row query tile of one (sequence, KV head) over a range of KV tiles.
+// A work unit is one 128-row query tile of one (sequence, KV head); its work is the sequence's KV tiles.
+// Units are laid end to end in (sequence, KV head, query tile) order; every CTA of the attention kernel takes
+// an equal, contiguous share of that line.  A share boundary inside a unit cuts it into pieces (work items);
+// a unit in several pieces is merged by the combine kernel.
 struct WorkItem {
   int32_t b, g, mt;
   int32_t tile_begin, tile_end;  // KV tiles [begin, end) of `tile_keys` keys each
-  int32_t slot;                  // first partial slot, or -1: the only split, write the output directly
-  int32_t mode;                  // paired planning only: 0 = one query tile (mt), 1 = two query tiles (mt, mt+1)
-  int32_t pad1;
+  int32_t slot;                  // partial slot, or -1: the unit is in one piece, write the output directly
+  int32_t pad0, pad1;
 };
 
 struct SeqPlan {
-  int32_t item_base;   // first work item of this sequence
-  int32_t splits;      // KV splits of every (KV head, row tile) of this sequence
   int32_t n;           // tree size used (0 when the sequence is invalid or empty)
   int32_t L;           // committed prefix length
-  int32_t slot_base;   // first partial slot (splits > 1), else -1
   int32_t mtiles;      // 128-row query tiles per KV head
   int32_t ntiles;      // KV tiles covering prefix + tree
-  int32_t key;         // KV tiles per work item (sort key of the planner)
+  int32_t unit_base;   // index of this sequence's first unit; unit = unit_base + g * mtiles + mt
+  int32_t pad0;
+  long long start;     // position of the first unit on the work line (in KV tiles)
+};
+
+struct UnitPlan {
+  int32_t first_item;  // the unit's pieces are items first_item .. first_item + n_pieces - 1
+  int32_t n_pieces;
+  int32_t slot_base;   // first partial slot (n_pieces > 1), else -1
+  int32_t pad0;
 };
 
 struct PlanHeader {
   int32_t n_items;
-  int32_t next_item;   // work counter of the persistent attention kernel
-  int32_t chunk_tiles;
   int32_t n_slots;
-  int32_t pad[12];
+  int32_t n_units;
+  int32_t ctas_used;
+  long long total_tiles;
+  int32_t pad[10];
 };
 
 // Workspace carving (all offsets multiples of 256 bytes).
@@ -46,10 +55,12 @@ struct Workspace {
   PlanHeader* hdr;
   SeqPlan* seq;        // [B]
   uint64_t* anc;       // [B, T_max]
+  UnitPlan* units;     // [unit_cap]
+  int32_t* cta_first;  // [kMaxPlanCtas + 1]: CTA c owns items cta_first[c] .. cta_first[c+1] - 1
   WorkItem* items;     // [item_cap]
-  float2* part_ml;     // [slot_cap, 128]   (running max in the log2 domain, running sum)
+  float2* part_ml;     // [slot_cap, 128]   (reference max in the log2 domain, row sum)
   float* part_o;       // [slot_cap, 128, D] unnormalised partial outputs
-  int32_t item_cap, slot_cap;
+  int32_t unit_cap, item_cap, slot_cap;
   size_t bytes;
 };
 
@@ -62,9 +73,10 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   if (d.num_splits < 0 || d.num_splits > 1024) return false;
   const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
   const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? mtiles : 1);
-  // two slots per item leave room for plans that pair query tiles (one slot per query tile of the pair)
-  const long long slots = 2 * (d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : kSlotBudgetAuto));
-  const long long items = units + slots;
+  // chosen by the planner: every share boundary adds at most one piece, and a cut unit has at most
+  // (cuts + 1) <= 2 * cuts pieces; forced: every unit in num_splits pieces
+  const long long slots = d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : 2 * kMaxPlanCtas);
+  const long long items = d.num_splits > 1 ? units * d.num_splits : units + kMaxPlanCtas;
   if (items > (1ll << 30)) return false;
   char* p = static_cast<char*>(base);
   size_t off = 0;
@@ -72,9 +84,12 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   w->hdr = reinterpret_cast<PlanHeader*>(take(sizeof(PlanHeader)));
   w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * (size_t)(d.batch > 0 ? d.batch : 1)));
   w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * (size_t)(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
+  w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * (size_t)(units > 0 ? units : 1)));
+  w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
   w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * (size_t)(items > 0 ? items : 1)));
   w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * (size_t)slots * kBlockM));
   w->part_o = reinterpret_cast<float*>(take(sizeof(float) * (size_t)slots * kBlockM * d.head_dim));
+  w->unit_cap = static_cast<int32_t>(units);
   w->item_cap = static_cast<int32_t>(items);
   w->slot_cap = static_cast<int32_t>(slots);
   w->bytes = off;
@@ -88,10 +103,12 @@ struct AttnParams {
   __nv_bfloat16* out;
   int32_t B, Hq, Hkv, G, D, T_max, S_cap;
   float scale_log2;      // sm_scale * log2(e)
-  int32_t pair;          // 1: items cover pairs of query tiles and own two consecutive partial slots
-  PlanHeader* hdr;
+  int32_t q_tma;         // set by the launcher: query tiles are fetched with TMA (group size divides 128)
+  const PlanHeader* hdr;
   const SeqPlan* seq;
   const uint64_t* anc;
+  const UnitPlan* units;
+  const int32_t* cta_first;
   const WorkItem* items;
   float2* part_ml;
   float* part_o;
@@ -104,14 +121,16 @@ struct PlanParams {
   const int32_t* tree_parent;
   int32_t B, Hkv, G, T_max, S_cap;
   int32_t tile_keys;       // keys per KV tile of the attention kernel
-  int32_t num_ctas;        // CTAs of the persistent attention kernel
-  int32_t forced_splits;   // 0: choose
-  int32_t min_chunk_tiles;
-  int32_t pair;            // 1: one item per pair of query tiles, two partial slots per item
-  int32_t item_cap, slot_cap;
+  int32_t num_ctas;        // CTAs of the persistent attention kernel (<= kMaxPlanCtas)
+  int32_t forced_splits;   // 0: equal shares; s > 0: every unit in min(s, KV tiles) equal pieces
+  int32_t snap_tiles;      // a share boundary closer than this to a unit's edge moves to the edge
+  int32_t item_overhead_tiles;   // fixed cost of starting a unit, in KV-tile equivalents
+  int32_t unit_cap, item_cap, slot_cap;
   PlanHeader* hdr;
   SeqPlan* seq;
   uint64_t* anc;
+  UnitPlan* units;
+  int32_t* cta_first;
   WorkItem* items;
   int32_t* status;
 };
@@ -139,18 +158,10 @@ __device__ inline void report_status(int32_t* status, int code) {
 cudaError_t launch_plan(const PlanParams& p, cudaStream_t stream);
 cudaError_t launch_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int batch, int max_tree,
                               uint64_t* anc, uint8_t* depth, int32_t* status, cudaStream_t stream);
-cudaError_t launch_attn_mma(const AttnParams& p, int num_ctas, cudaStream_t stream);
-int attn_mma_tile_keys();
-int attn_mma_ctas_per_sm(int head_dim);
-cudaError_t attn_mma_prepare(int head_dim);
-cudaError_t launch_attn_tc(const AttnParams& p, int num_ctas, cudaStream_t stream);
-int attn_tc_tile_keys();
-cudaError_t attn_tc_prepare(int head_dim);
-cudaError_t launch_attn_tc2(const AttnParams& p, int num_ctas, cudaStream_t stream);
-int attn_tc2_tile_keys();
-cudaError_t attn_tc2_prepare(int head_dim);
-cudaError_t launch_combine(const AttnParams& p, const int32_t* tree_sizes_unused, cudaStream_t stream);
-
+cudaError_t launch_attn(const AttnParams& p, int num_ctas, cudaStream_t stream);
+int attn_tile_keys();
+cudaError_t attn_prepare(int head_dim);
+cudaError_t launch_combine(const AttnParams& p, cudaStream_t stream);
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
 void count_launch();

@@ -2,8 +2,14 @@
 //
 // The host never reads seq_lens or tree_sizes (they are device arrays and the call must not synchronise),
 // so one small CTA turns them into (1) the per-node ancestor-or-self bit masks that define tree attention
-// (Sec. 3.1 / 3.3: a draft token attends to the context and to its own root path) and (2) a list of work
-// items for the persistent split-KV attention kernel, longest first, sized so that every SM gets work.
+// (Sec. 3.1 / 3.3: a draft token attends to the context and to its own root path) and (2) the work split of
+// the persistent attention kernel: work units (sequence, KV head, 128-row query tile) are laid end to end,
+// each as long as its sequence's KV tiles, and every CTA gets an equal contiguous share of that line.  A
+// share boundary that falls inside a unit cuts it into pieces; boundaries closer than `snap_tiles` to a
+// unit's edge move to the edge, so no piece is shorter than that.  Each CTA therefore does the same number
+// of KV tiles (to within the snap) whatever the mix of sequence lengths and tree sizes.  Every unit also
+// carries a fixed cost of `item_overhead_tiles` tile-equivalents at its start (query staging, pipeline fill,
+// epilogue), so that a share made of many short units is not mistaken for an equally cheap one.
 #include "common.cuh"
 
 namespace eagle {
@@ -12,16 +18,39 @@ namespace {
 
 constexpr int kPlanThreads = 1024;
 
-__device__ inline long long block_sum(long long v, long long* scratch) {
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+// Exclusive prefix sums of value(i), i in [0, n), by one CTA; put(i, prefix) stores them; returns the total.
+template <class Value, class Put>
+__device__ long long block_exclusive_scan(int n, Value value, Put put, long long* scratch) {
+  const int tid = threadIdx.x;
+  const int chunk = (n + kPlanThreads - 1) / kPlanThreads;
+  const int i0 = min(tid * chunk, n), i1 = min(i0 + chunk, n);
+  long long local = 0;
+  for (int i = i0; i < i1; ++i) local += value(i);
+  // inclusive scan of the per-thread sums: warp shuffles, then across warps through shared memory
+  long long inc = local;
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long x = __shfl_up_sync(0xffffffffu, inc, o);
+    if ((tid & 31) >= o) inc += x;
+  }
   __syncthreads();
-  if (l == 0) scratch[w] = v;
+  if ((tid & 31) == 31) scratch[tid >> 5] = inc;
   __syncthreads();
-  long long t = (l < (kPlanThreads >> 5)) ? scratch[l] : 0;
-  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-  return t;
+  long long before = 0, total = 0;
+  for (int w = 0; w < kPlanThreads / 32; ++w) {
+    if (w == (tid >> 5)) before = total;
+    total += scratch[w];
+  }
+  long long run = before + inc - local;
+  for (int i = i0; i < i1; ++i) {
+    const long long v = value(i);   // read before put(): put may overwrite what value reads
+    put(i, run);
+    run += v;
+  }
+  __syncthreads();
+  return total;
 }
+
+__device__ __forceinline__ long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
 
 // anc[i] = bit i | anc[parent[i]] in node order (parents come first).  Returns false on an invalid entry.
 __device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc, uint8_t* depth) {
@@ -35,17 +64,27 @@ __device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc,
   return true;
 }
 
-// work units per KV head: query tiles, or pairs of them
-__device__ __forceinline__ int units_of(int mtiles, int pair) { return pair ? (mtiles + 1) / 2 : mtiles; }
+// The unit occupies [us, ue) on the work line: `ovh` positions of fixed cost, then one position per KV tile.
+// Its interior cuts are the share boundaries floor(c * W / ctas) with us + ovh + snap <= boundary <= ue - snap:
+// a contiguous range of c.  Returns their number and the first such c.
+__device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W, int ctas, int snap, int ovh, int* first_c) {
+  const long long y = us + ovh + snap, z = ue - snap;
+  *first_c = 0;
+  if (z < y || ctas < 2) return 0;
+  long long ca = ceil_div(y * ctas, W), cb = ceil_div((z + 1) * ctas, W) - 1;
+  if (ca < 1) ca = 1;
+  if (cb > ctas - 1) cb = ctas - 1;
+  *first_c = static_cast<int>(ca);
+  return cb >= ca ? static_cast<int>(cb - ca + 1) : 0;
+}
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
-  __shared__ long long s_red[32];
-  __shared__ int s_chunk;
+  __shared__ long long s_scan[kPlanThreads / 32];
   const int tid = threadIdx.x;
   const int T = p.T_max;
+  const int ovh = p.forced_splits > 0 ? 0 : p.item_overhead_tiles;
 
   // ---- per sequence: validate, build masks, count tiles
-  long long work = 0;
   for (int b = tid; b < p.B; b += kPlanThreads) {
     int n = p.tree_sizes ? p.tree_sizes[b] : T;
     int L = p.seq_lens[b];
@@ -64,105 +103,135 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
     sp.n = n;
     sp.L = L;
     sp.mtiles = (n * p.G + kBlockM - 1) / kBlockM;
-    sp.item_base = 0;
-    sp.splits = 1;
-    sp.slot_base = -1;
     sp.ntiles = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;
-    sp.key = 0;
-    p.seq[b] = sp;
-    work += static_cast<long long>(p.Hkv) * units_of(sp.mtiles, p.pair) * sp.ntiles;
-  }
-  const long long total_work = block_sum(work, s_red);
-
-  // ---- choose the chunk length (KV tiles per item)
-  if (tid == 0) {
-    long long c = p.min_chunk_tiles;
-    if (p.forced_splits == 0) {
-      const long long target = (total_work + 2ll * p.num_ctas - 1) / (2ll * p.num_ctas);
-      if (target > c) c = target;
-    }
-    s_chunk = static_cast<int>(c < (1 << 28) ? c : (1 << 28));
-  }
-  __syncthreads();
-  if (p.forced_splits == 0) {
-    for (int iter = 0; iter < 28; ++iter) {
-      const int chunk = s_chunk;
-      long long slots = 0;
-      for (int b = tid; b < p.B; b += kPlanThreads) {
-        const SeqPlan sp = p.seq[b];
-        const int splits = (sp.ntiles + chunk - 1) / chunk;
-        if (splits > 1) slots += static_cast<long long>(p.Hkv) * units_of(sp.mtiles, p.pair) * splits * (p.pair ? 2 : 1);
-      }
-      const long long total_slots = block_sum(slots, s_red);
-      if (total_slots <= p.slot_cap) break;
-      __syncthreads();
-      if (tid == 0) s_chunk = chunk < (1 << 28) ? chunk * 2 : chunk;
-      __syncthreads();
-    }
-  }
-  const int chunk = s_chunk;
-
-  // ---- splits per sequence
-  for (int b = tid; b < p.B; b += kPlanThreads) {
-    SeqPlan sp = p.seq[b];
-    int splits;
-    if (p.forced_splits > 0) splits = sp.ntiles < p.forced_splits ? sp.ntiles : p.forced_splits;
-    else splits = (sp.ntiles + chunk - 1) / chunk;
-    if (splits < 1) splits = 1;
-    sp.splits = splits;
-    sp.key = (sp.ntiles + splits - 1) / splits;   // tiles per item: the sort key
+    sp.unit_base = 0;
+    sp.pad0 = 0;
+    sp.start = 0;
     p.seq[b] = sp;
   }
   __syncthreads();
 
-  // ---- order sequences by item length (longest first) and lay out items and partial slots
-  long long my_items = 0;
-  for (int b = tid; b < p.B; b += kPlanThreads) {
-    const SeqPlan me = p.seq[b];
-    long long item_base = 0, slot_base = 0;
-    for (int o = 0; o < p.B; ++o) {
-      // read only the planning fields: item_base / slot_base of other records are being written
-      const int o_key = p.seq[o].key, o_splits = p.seq[o].splits, o_mtiles = p.seq[o].mtiles;
-      const bool before = o_key > me.key || (o_key == me.key && o < b);
-      if (before) {
-        const long long cnt = static_cast<long long>(p.Hkv) * units_of(o_mtiles, p.pair) * o_splits;
-        item_base += cnt;
-        if (o_splits > 1) slot_base += cnt * (p.pair ? 2 : 1);
+  // ---- lay the sequences' units end to end
+  const long long W = block_exclusive_scan(
+      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * p.seq[b].mtiles * (p.seq[b].ntiles > 0 ? p.seq[b].ntiles + ovh : 0); },
+      [&](int b, long long v) { p.seq[b].start = v; }, s_scan);
+  const long long U = block_exclusive_scan(
+      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * p.seq[b].mtiles; },
+      [&](int b, long long v) { p.seq[b].unit_base = static_cast<int>(v); }, s_scan);
+  const int n_units = U <= p.unit_cap ? static_cast<int>(U) : 0;   // cannot exceed the advertised workspace
+  if (U > p.unit_cap && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);
+  const int ctas = static_cast<int>(W < p.num_ctas ? (W > 0 ? W : 1) : p.num_ctas);   // a share is at least one tile
+  const int snap = p.snap_tiles;
+
+  // unit -> sequence: the last sequence whose unit_base <= u (sequences without units share theirs with the next)
+  auto unit_seq = [&](int u) {
+    int lo = 0, hi = p.B;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (p.seq[mid].unit_base <= u) lo = mid; else hi = mid;
+    }
+    return lo;
+  };
+
+  // ---- pieces per unit
+  for (int u = tid; u < n_units; u += kPlanThreads) {
+    const int b = unit_seq(u);
+    const SeqPlan sp = p.seq[b];
+    const int ulen = sp.ntiles + ovh;
+    const long long us = sp.start + static_cast<long long>(u - sp.unit_base) * ulen;
+    int np;
+    if (p.forced_splits > 0) {
+      np = sp.ntiles < p.forced_splits ? sp.ntiles : p.forced_splits;
+    } else {
+      int c0;
+      np = 1 + unit_cuts(us, us + ulen, W, ctas, snap, ovh, &c0);
+    }
+    p.units[u].n_pieces = np;
+  }
+  __syncthreads();
+  const long long I = block_exclusive_scan(
+      n_units, [&](int u) { return static_cast<long long>(p.units[u].n_pieces); },
+      [&](int u, long long v) { p.units[u].first_item = static_cast<int>(v); }, s_scan);
+  const long long S = block_exclusive_scan(
+      n_units, [&](int u) { return p.units[u].n_pieces > 1 ? static_cast<long long>(p.units[u].n_pieces) : 0ll; },
+      [&](int u, long long v) { p.units[u].slot_base = p.units[u].n_pieces > 1 ? static_cast<int>(v) : -1; }, s_scan);
+  const bool fits = I <= p.item_cap && S <= p.slot_cap;
+  if (!fits && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);   // cannot happen with the advertised size
+
+  // ---- items
+  if (fits) {
+    for (int u = tid; u < n_units; u += kPlanThreads) {
+      const int b = unit_seq(u);
+      const SeqPlan sp = p.seq[b];
+      const int k = u - sp.unit_base;
+      const int ulen = sp.ntiles + ovh;
+      const long long us = sp.start + static_cast<long long>(k) * ulen;
+      const long long t_origin = us + ovh;          // line position of KV tile 0
+      const UnitPlan up = p.units[u];
+      int c0 = 0;
+      if (p.forced_splits == 0) unit_cuts(us, us + ulen, W, ctas, snap, ovh, &c0);
+      for (int j = 0; j < up.n_pieces; ++j) {
+        WorkItem it;
+        it.b = b;
+        it.g = k / sp.mtiles;
+        it.mt = k % sp.mtiles;
+        if (p.forced_splits > 0) {
+          it.tile_begin = static_cast<int>(static_cast<long long>(sp.ntiles) * j / up.n_pieces);
+          it.tile_end = static_cast<int>(static_cast<long long>(sp.ntiles) * (j + 1) / up.n_pieces);
+        } else {
+          it.tile_begin = j == 0 ? 0 : static_cast<int>(static_cast<long long>(c0 + j - 1) * W / ctas - t_origin);
+          it.tile_end = j == up.n_pieces - 1 ? sp.ntiles : static_cast<int>(static_cast<long long>(c0 + j) * W / ctas - t_origin);
+        }
+        it.slot = up.n_pieces > 1 ? up.slot_base + j : -1;
+        it.pad0 = it.pad1 = 0;
+        p.items[up.first_item + j] = it;
       }
     }
-    const int units = units_of(me.mtiles, p.pair), per_item = p.pair ? 2 : 1;
-    const long long cnt = static_cast<long long>(p.Hkv) * units * me.splits;
-    my_items += cnt;
-    const bool fits = item_base + cnt <= p.item_cap && (me.splits == 1 || slot_base + cnt * per_item <= p.slot_cap);
-    // cannot happen with a workspace of the advertised size; refuse rather than overrun
-    if (!fits && cnt > 0) report_status(p.status, EAGLE_ERR_WORKSPACE);
-    if (fits) {
-      int idx = static_cast<int>(item_base);
-      for (int g = 0; g < p.Hkv; ++g)
-        for (int mu = 0; mu < units; ++mu)
-          for (int s = 0; s < me.splits; ++s, ++idx) {
-            WorkItem it;
-            it.b = b;
-            it.g = g;
-            it.mt = p.pair ? 2 * mu : mu;
-            it.mode = (p.pair && 2 * mu + 1 < me.mtiles) ? 1 : 0;
-            it.tile_begin = static_cast<int>(static_cast<long long>(me.ntiles) * s / me.splits);
-            it.tile_end = static_cast<int>(static_cast<long long>(me.ntiles) * (s + 1) / me.splits);
-            it.slot = me.splits > 1 ? static_cast<int>(slot_base) + (idx - static_cast<int>(item_base)) * per_item : -1;
-            it.pad1 = 0;
-            p.items[idx] = it;
-          }
-    }
-    // item_base / slot_base are fields no other thread reads while planning
-    p.seq[b].item_base = static_cast<int>(item_base);
-    p.seq[b].slot_base = me.splits > 1 ? static_cast<int>(slot_base) : -1;
   }
-  const long long n_items = block_sum(my_items, s_red);
+
+  // ---- first item of every CTA
+  for (int c = tid; c <= p.num_ctas; c += kPlanThreads) {
+    long long first;
+    if (!fits || I == 0) {
+      first = 0;
+    } else if (p.forced_splits > 0) {
+      first = static_cast<long long>(c) * I / p.num_ctas;
+    } else if (c == 0) {
+      first = 0;
+    } else if (c >= ctas) {
+      first = I;
+    } else {
+      const long long x = static_cast<long long>(c) * W / ctas;   // 0 < x < W
+      int lo = 0, hi = p.B;          // last sequence whose start <= x (sequences without work share their start with the next)
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (p.seq[mid].start <= x) lo = mid; else hi = mid;
+      }
+      const SeqPlan sp = p.seq[lo];
+      const int ulen = sp.ntiles + ovh;
+      const int k = static_cast<int>((x - sp.start) / ulen);
+      const int u = sp.unit_base + k;
+      const long long us = sp.start + static_cast<long long>(k) * ulen, ue = us + ulen;
+      const long long d0 = x - (us + ovh), d1 = ue - x;   // distance to the first KV tile / to the unit's end
+      const UnitPlan up = p.units[u];
+      if (d0 >= snap && d1 >= snap) {
+        int c0;
+        unit_cuts(us, ue, W, ctas, snap, ovh, &c0);
+        first = up.first_item + 1 + (c - c0);        // the piece that starts at this boundary
+      } else if (x - us <= d1) {
+        first = up.first_item;                        // boundary moved to the unit's start
+      } else {
+        first = up.first_item + up.n_pieces;          // boundary moved to the unit's end
+      }
+    }
+    p.cta_first[c] = static_cast<int>(first);
+  }
   if (tid == 0) {
-    p.hdr->n_items = n_items <= p.item_cap ? static_cast<int>(n_items) : 0;
-    p.hdr->next_item = 0;
-    p.hdr->chunk_tiles = chunk;
-    p.hdr->n_slots = 0;
+    p.hdr->n_items = fits ? static_cast<int>(I) : 0;
+    p.hdr->n_slots = fits ? static_cast<int>(S) : 0;
+    p.hdr->n_units = n_units;
+    p.hdr->ctas_used = ctas;
+    p.hdr->total_tiles = W;
   }
 }
 
