@@ -98,6 +98,36 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
                            const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream);
 
 /*
+ * The same attention, for callers that cannot provide a workspace.  (The paper has no counterpart to this entry
+ * point: it exists for the way the library is embedded, not for the method.)
+ *
+ * Who needs it: code that receives device pointers for its tensors but may not allocate device memory when it
+ * runs - a serving backend whose memory pool is fixed at start-up, a plug-in living inside another engine's
+ * execution context, a decode loop that must never call cudaMalloc because that call stalls the whole device.
+ * Here the planner tables and the split partials live in a fixed array inside the library's device image,
+ * eagle_tree_verify_attn_static_capacity() bytes (24 MiB) per GPU that loads the library, held until the
+ * process ends.  `desc->workspace` and `desc->workspace_bytes` are ignored; everything else is as for
+ * eagle_tree_verify_attn, and so are the results.
+ *
+ *   - No cudaMalloc, cudaFree or other allocating call is made, on any call.
+ *   - Shapes whose tables and partials do not fit the array are refused with EAGLE_ERR_WORKSPACE and nothing is
+ *     launched.  The need grows with batch * num_kv_heads * ceil(max_tree * G / 128), and steeply with a
+ *     forced num_splits > 1; with num_splits = 0 the partials take about 2 * (number of SMs) * 128 * (D + 2) * 4
+ *     bytes (19.7 MB on a 148-SM B200 at D = 128).
+ *   - The first call on a device looks up the array's device address (once per device, with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on one GPU share the one array, and it keeps the previous call's contents.  Nothing in it needs
+ *     to start at zero (the planner kernel rewrites every table that is read, and each partial is written
+ *     before it is merged), but two calls that can overlap on the GPU - different streams, or graphs replayed
+ *     concurrently - would overwrite each other's plan: issue them on one stream, or order them yourself.
+ */
+int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream);
+
+/* Size in bytes of the fixed array used by eagle_tree_verify_attn_static (host function). */
+size_t eagle_tree_verify_attn_static_capacity(void);
+
+/*
  * Descriptor of one acceptance call.
  */
 typedef struct eagle_accept_desc {

@@ -15,7 +15,8 @@ import torch
 _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libeagle_verify.so"
 EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_tree_accept",
-           "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count"]
+           "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
+           "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity"]
 _lib = None
 
 
@@ -50,6 +51,9 @@ def load():
         lib.eagle_tree_verify_attn_workspace.restype = ctypes.c_size_t
         lib.eagle_tree_verify_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_verify_attn.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_static.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp]
+        lib.eagle_tree_verify_attn_static.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_static_capacity.restype = ctypes.c_size_t
         lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_accept.restype = ctypes.c_int
         lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
@@ -137,6 +141,27 @@ def eagle_tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, out=None,
                                     _dev(tree_parent, torch.int32, "tree_parent"), _dev(out, torch.bfloat16, "out"), _stream())
     _check(rc, "eagle_tree_verify_attn")
     return out
+
+
+def eagle_tree_verify_attn_static(q, k_cache, v_cache, seq_lens, tree_parent, out, *, tree_sizes=None, sm_scale=0.0,
+                                  num_splits=0, status=None):
+    """Tree-masked attention for callers that may not allocate: same arguments and results as
+    ``eagle_tree_verify_attn``, but no workspace is passed and none is allocated here either (the library's fixed
+    device array is used; ``out`` must be given).  Raises if the shape needs more than that array holds."""
+    lib = load()
+    B, T, Hq, D = q.shape
+    if k_cache.shape[0] != B or k_cache.shape[3] != D or tuple(tree_parent.shape) != (B, T) or tuple(seq_lens.shape) != (B,):
+        raise EagleError("inconsistent shapes")
+    d = _attn_desc(q, k_cache, tree_sizes, sm_scale, num_splits, None, status, None)
+    rc = lib.eagle_tree_verify_attn_static(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
+                                           _dev(v_cache, torch.bfloat16, "v_cache"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                           _dev(tree_parent, torch.int32, "tree_parent"), _dev(out, torch.bfloat16, "out"), _stream())
+    _check(rc, "eagle_tree_verify_attn_static")
+    return out
+
+
+def static_capacity() -> int:
+    return int(load().eagle_tree_verify_attn_static_capacity())
 
 
 def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, accepted_path=None,

@@ -191,6 +191,156 @@ int eagle_tree_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes,
   return EAGLE_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Attention without a caller-provided workspace.
+//
+// Some hosts of this library can hand over device pointers for tensors but have no way to get device scratch
+// at call time: an inference-server backend whose memory pool is frozen after start-up, a plug-in that runs
+// inside another engine's execution context, a latency-critical decode loop in which cudaMalloc (which
+// synchronises the whole device) is off limits.  For them the planner tables and split partials live in the
+// fixed array below, which every GPU that loads the library keeps until the process exits.
+constexpr size_t kStaticScratchBytes = 24u << 20;   // 24 MiB
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+// Same carving as carve_workspace(), but sized for the CTAs this device really runs (one per SM) instead of
+// the library-wide upper bound, so that the common shapes fit the fixed array.
+bool carve_static(const eagle_attn_desc& d, int num_ctas, void* base, Workspace* w) {
+  if (d.batch < 0 || d.num_kv_heads <= 0 || d.num_q_heads <= 0 || d.num_q_heads % d.num_kv_heads) return false;
+  const int G = d.num_q_heads / d.num_kv_heads;
+  if (G > kMaxGroup || d.max_tree < 0 || d.max_tree > kMaxTree || (d.head_dim != 64 && d.head_dim != 128)) return false;
+  if (d.num_splits < 0 || d.num_splits > 1024) return false;
+  const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
+  const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? mtiles : 1);
+  const long long slots = d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : 2ll * num_ctas);
+  const long long items = d.num_splits > 1 ? units * d.num_splits : units + num_ctas;
+  if (items > (1ll << 30)) return false;
+  char* p = static_cast<char*>(base);
+  size_t off = 0;
+  auto take = [&](size_t n) { char* r = p + off; off += align256(n); return r; };
+  w->hdr = reinterpret_cast<PlanHeader*>(take(sizeof(PlanHeader)));
+  w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * static_cast<size_t>(d.batch > 0 ? d.batch : 1)));
+  w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * static_cast<size_t>(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
+  w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * static_cast<size_t>(units > 0 ? units : 1)));
+  w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
+  w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * static_cast<size_t>(items > 0 ? items : 1)));
+  w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * static_cast<size_t>(slots) * kBlockM));
+  w->part_o = reinterpret_cast<float*>(take(sizeof(float) * static_cast<size_t>(slots) * kBlockM * d.head_dim));
+  w->unit_cap = static_cast<int32_t>(units);
+  w->item_cap = static_cast<int32_t>(items);
+  w->slot_cap = static_cast<int32_t>(slots);
+  w->bytes = off;
+  return true;
+}
+
+// Device address of the fixed scratch array on the current device.  The array's name is only a host-side handle:
+// the address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device current.
+void* g_static_ptr[kMaxDevices] = {nullptr};
+std::mutex g_static_mutex;
+
+void* static_scratch_ptr() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+    g_static_ptr[dev] = ptr;
+  }
+  return g_static_ptr[dev];
+}
+
+}  // namespace
+
+size_t eagle_tree_verify_attn_static_capacity(void) { return kStaticScratchBytes; }
+
+int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                                  const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const eagle_attn_desc& d = *desc;
+  if (d.kv_capacity < 0 || !(d.sm_scale >= 0.f)) return EAGLE_ERR_SHAPE;
+  int err = 0;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
+  const int num_ctas = dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas;
+  void* scratch = static_scratch_ptr();
+  if (!scratch) return EAGLE_ERR_DEVICE;
+  Workspace w;
+  if (!carve_static(d, num_ctas, scratch, &w)) return EAGLE_ERR_SHAPE;
+  if (w.bytes > kStaticScratchBytes) return EAGLE_ERR_WORKSPACE;   // this shape needs more than the fixed array holds
+  if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
+  if (!q || !k_cache || !v_cache || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(k_cache) & 15) || (reinterpret_cast<uintptr_t>(v_cache) & 15) ||
+      (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+    return EAGLE_ERR_SHAPE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int di = d.head_dim == 128 ? 1 : 0;
+  if (!dev->attn_prepared[di]) {
+    if (attn_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
+    dev->attn_prepared[di] = true;
+  }
+  const int G = d.num_q_heads / d.num_kv_heads;
+
+  PlanParams pp;
+  pp.seq_lens = seq_lens;
+  pp.tree_sizes = d.tree_sizes;
+  pp.tree_parent = tree_parent;
+  pp.B = d.batch;
+  pp.Hkv = d.num_kv_heads;
+  pp.G = G;
+  pp.T_max = d.max_tree;
+  pp.S_cap = d.kv_capacity;
+  pp.tile_keys = attn_tile_keys();
+  pp.num_ctas = num_ctas;
+  pp.forced_splits = d.num_splits;
+  pp.snap_tiles = 2;
+  pp.item_overhead_tiles = 4;
+  pp.unit_cap = w.unit_cap;
+  pp.item_cap = w.item_cap;
+  pp.slot_cap = w.slot_cap;
+  pp.hdr = w.hdr;
+  pp.seq = w.seq;
+  pp.anc = w.anc;
+  pp.units = w.units;
+  pp.cta_first = w.cta_first;
+  pp.items = w.items;
+  pp.status = d.status;
+  // Nothing in the array has to start at zero: the planner rebuilds every table it or the later kernels read, and
+  // a partial slot is always written by the attention kernel before the combine kernel reads it.
+  if (launch_plan(pp, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+
+  AttnParams ap;
+  ap.q = static_cast<const __nv_bfloat16*>(q);
+  ap.k = static_cast<const __nv_bfloat16*>(k_cache);
+  ap.v = static_cast<const __nv_bfloat16*>(v_cache);
+  ap.out = static_cast<__nv_bfloat16*>(out);
+  ap.B = d.batch;
+  ap.Hq = d.num_q_heads;
+  ap.Hkv = d.num_kv_heads;
+  ap.G = G;
+  ap.D = d.head_dim;
+  ap.T_max = d.max_tree;
+  ap.S_cap = d.kv_capacity;
+  const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
+  ap.scale_log2 = scale * 1.4426950408889634f;
+  ap.q_tma = 0;
+  ap.hdr = w.hdr;
+  ap.seq = w.seq;
+  ap.anc = w.anc;
+  ap.units = w.units;
+  ap.cta_first = w.cta_first;
+  ap.items = w.items;
+  ap.part_ml = w.part_ml;
+  ap.part_o = w.part_o;
+  ap.status = d.status;
+  if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
+
 const char* eagle_status_string(int code) {
   switch (code) {
     case EAGLE_OK: return "ok";
