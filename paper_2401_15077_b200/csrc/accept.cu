@@ -415,8 +415,9 @@ cudaError_t launch_cluster(const AcceptParams& p, cudaStream_t stream) {
 
 }  // namespace
 
-// Team width: a warp per tree for small vocabularies; otherwise CTAs of 512 threads, clustered so that
-// about one SM's worth of trees still spreads over the whole GPU.
+// Team width: a warp per tree for small vocabularies; otherwise CTAs of 512 threads in clusters as wide as still
+// fit the GPU in one wave (four such CTAs are resident per SM): the walk is a chain of dependent vocabulary
+// sweeps, so a tree finishes sooner the more SMs pull its rows.
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream) {
   if (p.B == 0) return cudaSuccess;
   cudaError_t e;
@@ -425,10 +426,10 @@ cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stre
     accept_kernel<32, 1><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
     e = cudaGetLastError();
   } else {
-    const long long per_tree = sm_count / p.B;   // SMs available per tree
-    if (per_tree >= 8) e = launch_cluster<8>(p, stream);
-    else if (per_tree >= 4) e = launch_cluster<4>(p, stream);
-    else if (per_tree >= 2) e = launch_cluster<2>(p, stream);
+    const long long resident = 4ll * sm_count;   // CTAs of 512 threads that can be resident at once
+    if (8ll * p.B <= resident) e = launch_cluster<8>(p, stream);
+    else if (4ll * p.B <= resident) e = launch_cluster<4>(p, stream);
+    else if (2ll * p.B <= resident) e = launch_cluster<2>(p, stream);
     else {
       accept_kernel<kCtaThreads, 1><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
       e = cudaGetLastError();

@@ -141,7 +141,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_combine(ap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, w.unit_cap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 
@@ -337,7 +337,7 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_combine(ap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, w.unit_cap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 

@@ -72,14 +72,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the CTA has been aborted or the time limit passed (and raises the abort flag).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_test_wait(bar, parity)) return true;     // non-blocking probe: the phase is often complete already
-  if (mbar_try_wait(bar, parity)) return true;
+// Slow path of a wait, kept out of line so that the dozen wait sites stay small (the kernel's hot loops have to
+// live in the instruction cache next to each other).  Returns false if the CTA has been aborted or the time limit
+// passed (and raises the abort flag).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   const unsigned long long t0 = global_timer();
   for (uint32_t spins = 1;; ++spins) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spins & 255u) == 0) {
+    if ((spins & 63u) == 0) {
       if (*abort_flag) return false;
       if (global_timer() - t0 > kWaitLimitNs) {
         *abort_flag = 1;
@@ -87,6 +87,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
+}
+// Bounded wait: a few non-blocking probes (most phases are complete, or complete within a few hundred cycles),
+// then the suspending form with the timer.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+#pragma unroll 1
+  for (int i = 0; i < 16; ++i)
+    if (mbar_test_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 // Same, with a verdict that is uniform over the warp (the callers go on to warp-collective tcgen05 instructions).
@@ -141,6 +149,20 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// 2^x on the FMA / ALU pipes (x <= ~8): split x into an integer n and a fraction f in [-0.5, 0.5] with the
+// add-a-large-constant trick, evaluate a cubic for 2^f (relative error 1e-4, far below the bf16 rounding of P) and put
+// n into the exponent field.  Used for a fraction of the exponentials so that the special-function unit, which takes
+// 8 cycles per warp instruction, is not the only thing the softmax waits for.
+__device__ __forceinline__ float poly_exp2(float x) {
+  const float xc = fmaxf(x, -126.f);
+  const float t = xc + 12582912.f;                    // 1.5 * 2^23: the integer part lands in the low mantissa bits
+  const float f = xc - (t - 12582912.f);
+  float r = fmaf(0.05500841f, f, 0.24220926f);
+  r = fmaf(r, f, 0.69328277f);
+  r = fmaf(r, f, 1.0f);
+  return __uint_as_float(__float_as_uint(r) + (__float_as_uint(t) << 23));   // the constant's own bits shift out
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -444,13 +466,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     const int h = warp >> 2;                              // which 64-column half of the score row this thread owns
     const int r = tid & (kBlockM - 1);                    // query row within the tile == TMEM lane
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t pair_bar = B.pair[warp & 3];   // barrier shared with the partner warp (bounded waits, like all others)
-    uint32_t pair_phase = 0;
+    // Hardware barrier shared with the partner warp.  Both warps of a pair run the same control flow on the same
+    // mbarriers, so they always reach it together: a warp leaves its loop only when a wait failed, and a wait that
+    // fails for one of them (the barrier never completes) fails for the other too.
+    const uint32_t pair_id = 1u + static_cast<uint32_t>(warp & 3);
     auto pair_sync = [&]() -> bool {
-      mbar_arrive(pair_bar);
-      const bool k = mbar_wait_warp(pair_bar, pair_phase & 1u, s_abort);
-      ++pair_phase;
-      return k;
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_id) : "memory");
+      return true;
     };
     float* xch = reinterpret_cast<float*>(smem + S::kXch);
     constexpr int HC = D / 2;                             // this thread's half of the accumulator columns
@@ -511,18 +533,21 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 
     uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps done so far
     bool ok = true;
-    for (int idx = item_lo; idx < item_hi && ok; ++idx) {
-      const WorkItem it = p.items[idx];
+    // one pass per item, plus a last pass without steps that only writes the final item's output
+    const int pass_end = item_hi > item_lo ? item_hi + 1 : item_lo;   // a CTA without items makes no pass at all
+    for (int idx = item_lo; idx < pass_end && ok; ++idx) {
+      const bool drain = idx == item_hi;
+      const WorkItem it = p.items[drain ? item_lo : idx];
       const SeqPlan sp = p.seq[it.b];
       const int L = sp.L, n = sp.n, G = p.G;
       const int m_valid = n * G, kv_end = L + n;
-      const int steps = it.tile_end - it.tile_begin;
+      const int steps = drain ? 0 : it.tile_end - it.tile_begin;
       const int R = it.mt * kBlockM + r;
       const bool row_valid = R < m_valid;
       const int node = row_valid ? R / G : 0, hh = row_valid ? R % G : 0;
       const uint64_t anc = row_valid ? p.anc[static_cast<size_t>(it.b) * p.T_max + node] : 0ull;
 
-      if (!p.q_tma) {
+      if (!p.q_tma && !drain) {
         // group sizes that do not divide 128: the softmax threads stage the query tile themselves;
         // thread (h, r) writes the h-th 64-column slab of row r (D = 64: h = 0 only)
         const uint32_t qb = item_count & 1u;
@@ -545,7 +570,8 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 
       float m_ref = -INFINITY;   // reference max (scaled, log2 domain) of every exponential taken so far
       float l_sum = 0.f;         // this thread's half of the row sum
-      for (int s = 0; s < steps && ok; ++s) {
+      for (int s = 0; s < steps + (drain ? 1 : 0) && ok; ++s) {
+        if (!drain) {
         const uint32_t gs = sg + s, buf = gs & 1u;
         ok = mbar_wait_warp(B.s_full[buf], (gs >> 1) & 1u, s_abort);
         if (!ok) break;
@@ -555,6 +581,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         tmem_ld32(tmem + lane_addr + kColS + buf * kTileN + h * 64, raw);
         tmem_ld32(tmem + lane_addr + kColS + buf * kTileN + h * 64 + 32, raw + 32);
         tc_wait_ld();
+        if (tid == 0) TRACE(2, (15 << 10) | (gs & 1023u));
         const int key0 = (it.tile_begin + s) * kTileN;
         if (key0 + kTileN > L) {          // the tile reaches past the committed prefix: tree mask + cache tail
           // visibility of this thread's 64 keys as one 64-bit word: keys before L are all visible, key L + m is
@@ -583,6 +610,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         const float half_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         // agree on the row max with the partner thread (other half of the row, same lane, warp +-4)
         xch[(buf * 2 + h) * kBlockM + r] = half_max;
+        if (tid == 0) TRACE(2, (12 << 10) | (gs & 1023u));
         ok = pair_sync();
         if (!ok) break;
         const float tmax = fmaxf(half_max, xch[(buf * 2 + (h ^ 1)) * kBlockM + r]) * p.scale_log2;   // scale > 0
@@ -600,11 +628,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           fence_proxy_async();
         }
 
+        if (tid == 0) TRACE(2, (13 << 10) | (gs & 1023u));
         // P[buf] was last read by the PV of step gs - 2 (this wait also keeps every thread within one phase of o_done)
         if (gs >= 2) {
           ok = mbar_wait_warp(B.o_done[buf], ((gs - 2) >> 1) & 1u, s_abort);
           if (!ok) break;
         }
+        if (tid == 0) TRACE(2, (17 << 10) | (gs & 1023u));
         // lazy rescale: move the reference only when the row max outgrows it by more than the threshold
         const bool grow = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         float factor = 1.f;
@@ -619,7 +649,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (!ok) break;
           tc_fence_after();
           uint32_t o[32];
-#pragma unroll
+#pragma unroll 1
           for (int c = 0; c < HC / 32; ++c) {
             const uint32_t o_addr = tmem + lane_addr + kColO + h * HC + c * 32;
             tmem_ld32(o_addr, o);
@@ -630,6 +660,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           }
           tc_wait_st();
         }
+        if (tid == 0) TRACE(2, (16 << 10) | (gs & 1023u));
         const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -637,17 +668,19 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           const float p0 = fast_exp2(fmaf(__uint_as_float(raw[2 * e]), p.scale_log2, neg_base));
           const float p1 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 1]), p.scale_log2, neg_base));
           const float p2 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 2]), p.scale_log2, neg_base));
-          const float p3 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 3]), p.scale_log2, neg_base));
+          const float p3 = poly_exp2(fmaf(__uint_as_float(raw[2 * e + 3]), p.scale_log2, neg_base));
           ls[0] += p0; ls[1] += p1; ls[2] += p2; ls[3] += p3;
           raw[e] = pack_bf16(p0, p1);          // packed P overwrites entries already consumed
           raw[e + 1] = pack_bf16(p2, p3);
         }
         l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        if (tid == 0) TRACE(2, (14 << 10) | (gs & 1023u));
         tmem_st32(tmem + lane_addr + kColP + buf * (kTileN / 2) + h * 32, raw);   // this thread's 64 P values
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(B.p_full[buf]);
         if (tid == 0) TRACE(2, (11 << 10) | (gs & 1023u));
+        }
 
         // the finished item's output is written after the first step of this one: its last PV has had time
         // to complete, and this item's second score tile is being computed meanwhile
@@ -656,7 +689,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           prev.live = false;
         }
       }
-      if (!ok) break;
+      if (!ok || drain) break;
       prev.live = true;
       prev.row_valid = row_valid;
       prev.slot = it.slot;
@@ -668,7 +701,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       sg += steps;
       ++item_count;
     }
-    if (ok && prev.live) ok = epilogue(prev);
   }
 
 #ifdef EAGLE_TRACE

@@ -38,7 +38,7 @@ struct UnitPlan {
   int32_t first_item;  // the unit's pieces are items first_item .. first_item + n_pieces - 1
   int32_t n_pieces;
   int32_t slot_base;   // first partial slot (n_pieces > 1), else -1
-  int32_t pad0;
+  int32_t pad0;        // the unit's sequence
 };
 
 struct PlanHeader {
@@ -161,7 +161,7 @@ cudaError_t launch_build_mask(const int32_t* tree_parent, const int32_t* tree_si
 cudaError_t launch_attn(const AttnParams& p, int num_ctas, cudaStream_t stream);
 int attn_tile_keys();
 cudaError_t attn_prepare(int head_dim);
-cudaError_t launch_combine(const AttnParams& p, cudaStream_t stream);
+cudaError_t launch_combine(const AttnParams& p, int unit_cap, cudaStream_t stream);
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
 void count_launch();

@@ -64,6 +64,58 @@ __device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc,
   return true;
 }
 
+// The same masks by one warp: lane l holds nodes l and l + 32.  Every node starts with its own bit and a pointer to its
+// parent; each round ORs in the mask of the node pointed to and jumps the pointer to that node's pointer, so six rounds
+// cover any path of up to 64 nodes.  Returns false (to all lanes) on an invalid entry.  anc[i >= n] is not written.
+__device__ inline bool build_masks_warp(const int32_t* par, int n, uint64_t* anc, uint8_t* depth, int lane) {
+  uint64_t mask[2];
+  int ptr[2];
+  bool ok = true;
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int i = lane + 32 * k;
+    mask[k] = 0ull;
+    ptr[k] = -1;
+    if (i < n) {
+      const int pi = par[i];
+      if (pi < -1 || pi >= i) ok = false;
+      else {
+        mask[k] = 1ull << i;
+        ptr[k] = pi;
+      }
+    }
+  }
+  if (!__all_sync(0xffffffffu, ok)) return false;
+#pragma unroll
+  for (int round = 0; round < 6; ++round) {
+    uint64_t add[2];
+    int next[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int t = ptr[k] >= 0 ? ptr[k] : 0;
+      // the pointed-to node lives in lane t & 31, slot t >> 5: fetch both slots and pick
+      const uint64_t m0 = __shfl_sync(0xffffffffu, mask[0], t & 31), m1 = __shfl_sync(0xffffffffu, mask[1], t & 31);
+      const int p0 = __shfl_sync(0xffffffffu, ptr[0], t & 31), p1 = __shfl_sync(0xffffffffu, ptr[1], t & 31);
+      add[k] = ptr[k] >= 0 ? ((t >> 5) ? m1 : m0) : 0ull;
+      next[k] = ptr[k] >= 0 ? ((t >> 5) ? p1 : p0) : -1;
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      mask[k] |= add[k];
+      ptr[k] = next[k];
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int i = lane + 32 * k;
+    if (i < n) {
+      anc[i] = mask[k];
+      if (depth) depth[i] = static_cast<uint8_t>(__popcll(mask[k]));
+    }
+  }
+  return true;
+}
+
 // The unit occupies [us, ue) on the work line: `ovh` positions of fixed cost, then one position per KV tile.
 // Its interior cuts are the share boundaries floor(c * W / ctas) with us + ovh + snap <= boundary <= ue - snap:
 // a contiguous range of c.  Returns their number and the first such c.
@@ -78,36 +130,50 @@ __device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W
   return cb >= ca ? static_cast<int>(cb - ca + 1) : 0;
 }
 
-__global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
+constexpr int kSmemSeqs = 512;     // per-sequence records kept in shared memory while planning (else in the workspace)
+constexpr int kSmemUnits = 1792;   // per-unit records kept in shared memory while planning
+
+__global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   __shared__ long long s_scan[kPlanThreads / 32];
+  __shared__ SeqPlan s_seq[kSmemSeqs];
+  __shared__ UnitPlan s_units[kSmemUnits];
   const int tid = threadIdx.x;
+  // The planning passes are chains of dependent reads and writes of these small tables; in shared memory each
+  // link costs tens of cycles instead of a trip to L2.  They are copied to the workspace once at the end.
+  PlanParams p = pg;
+  const bool seq_in_smem = p.B <= kSmemSeqs, units_in_smem = p.unit_cap <= kSmemUnits;
+  if (seq_in_smem) p.seq = s_seq;
+  if (units_in_smem) p.units = s_units;
   const int T = p.T_max;
   const int ovh = p.forced_splits > 0 ? 0 : p.item_overhead_tiles;
 
-  // ---- per sequence: validate, build masks, count tiles
-  for (int b = tid; b < p.B; b += kPlanThreads) {
+  // ---- per sequence (one warp each): validate, build masks, count tiles
+  for (int b = tid >> 5; b < p.B; b += kPlanThreads / 32) {
+    const int lane = tid & 31;
     int n = p.tree_sizes ? p.tree_sizes[b] : T;
     int L = p.seq_lens[b];
     int bad = 0;
     if (n < 0 || n > T) bad = EAGLE_ERR_TREE;
     else if (L < 0 || static_cast<long long>(L) + n > p.S_cap) bad = EAGLE_ERR_SEQ;
     uint64_t* anc = p.anc + static_cast<size_t>(b) * T;
-    if (!bad && !build_masks_one(p.tree_parent + static_cast<size_t>(b) * T, n, anc, nullptr)) bad = EAGLE_ERR_TREE;
+    if (!bad && !build_masks_warp(p.tree_parent + static_cast<size_t>(b) * T, n, anc, nullptr, lane)) bad = EAGLE_ERR_TREE;
     if (bad) {
-      report_status(p.status, bad);
+      if (lane == 0) report_status(p.status, bad);
       n = 0;
       L = 0;
     }
-    for (int i = n; i < T; ++i) anc[i] = 0ull;
-    SeqPlan sp;
-    sp.n = n;
-    sp.L = L;
-    sp.mtiles = (n * p.G + kBlockM - 1) / kBlockM;
-    sp.ntiles = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;
-    sp.unit_base = 0;
-    sp.pad0 = 0;
-    sp.start = 0;
-    p.seq[b] = sp;
+    for (int i = n + lane; i < T; i += 32) anc[i] = 0ull;
+    if (lane == 0) {
+      SeqPlan sp;
+      sp.n = n;
+      sp.L = L;
+      sp.mtiles = (n * p.G + kBlockM - 1) / kBlockM;
+      sp.ntiles = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;
+      sp.unit_base = 0;
+      sp.pad0 = 0;
+      sp.start = 0;
+      p.seq[b] = sp;
+    }
   }
   __syncthreads();
 
@@ -147,6 +213,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
       np = 1 + unit_cuts(us, us + ulen, W, ctas, snap, ovh, &c0);
     }
     p.units[u].n_pieces = np;
+    p.units[u].pad0 = b;
   }
   __syncthreads();
   const long long I = block_exclusive_scan(
@@ -226,6 +293,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams p) {
     }
     p.cta_first[c] = static_cast<int>(first);
   }
+  __syncthreads();
+  if (seq_in_smem)
+    for (int b = tid; b < p.B; b += kPlanThreads) pg.seq[b] = s_seq[b];
+  if (units_in_smem)
+    for (int u = tid; u < n_units; u += kPlanThreads) pg.units[u] = s_units[u];
   if (tid == 0) {
     p.hdr->n_items = fits ? static_cast<int>(I) : 0;
     p.hdr->n_slots = fits ? static_cast<int>(S) : 0;
