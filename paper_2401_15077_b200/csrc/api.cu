@@ -87,7 +87,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
     dev->attn_prepared[di] = true;
   }
   const int G = d.num_q_heads / d.num_kv_heads;
-  const int num_ctas = dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas;   // one persistent CTA per SM
+  const int num_ctas = (dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas) & ~1;   // one persistent CTA per SM, in pairs
 
   PlanParams pp;
   pp.seq_lens = seq_lens;
@@ -212,9 +212,10 @@ bool carve_static(const eagle_attn_desc& d, int num_ctas, void* base, Workspace*
   if (G > kMaxGroup || d.max_tree < 0 || d.max_tree > kMaxTree || (d.head_dim != 64 && d.head_dim != 128)) return false;
   if (d.num_splits < 0 || d.num_splits > 1024) return false;
   const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
-  const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? mtiles : 1);
-  const long long slots = d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : 2ll * num_ctas);
-  const long long items = d.num_splits > 1 ? units * d.num_splits : units + num_ctas;
+  const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? (mtiles + 1) / 2 : 1);   // super-units
+  const long long pieces = d.num_splits > 0 ? units * d.num_splits : units + num_ctas / 2;
+  const long long items = 2 * pieces;
+  const long long slots = items;
   if (items > (1ll << 30)) return false;
   char* p = static_cast<char*>(base);
   size_t off = 0;
@@ -263,7 +264,7 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   int err = 0;
   DeviceInfo* dev = device_info(&err);
   if (!dev) return err;
-  const int num_ctas = dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas;
+  const int num_ctas = (dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas) & ~1;
   void* scratch = static_scratch_ptr();
   if (!scratch) return EAGLE_ERR_DEVICE;
   Workspace w;

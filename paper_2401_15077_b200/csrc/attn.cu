@@ -340,8 +340,11 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
 
-  // this CTA's share of the work line: items [item_lo, item_hi)
-  const int item_lo = p.cta_first[blockIdx.x], item_hi = p.cta_first[blockIdx.x + 1];
+  // CTAs 2j and 2j+1 form team j; the team owns the team pieces [tp_lo, tp_hi) of the work line and piece tp gives
+  // this CTA the item 2 * tp + member (the two members walk the same KV range with sibling query tiles, or the two
+  // halves of a lone tile's range, so whatever one of them pulls from HBM the other finds in L2)
+  const int member = blockIdx.x & 1;
+  const int tp_lo = p.cta_first[blockIdx.x >> 1], tp_hi = p.cta_first[(blockIdx.x >> 1) + 1];
 #ifdef EAGLE_TRACE
   int trace_n = 0;
   const long long trace_t0 = clock64();
@@ -353,8 +356,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       uint32_t g = 0;   // KV tiles issued by this CTA so far
       uint32_t item_count = 0;
       bool ok = true;
-      for (int idx = item_lo; idx < item_hi && ok; ++idx, ++item_count) {
-        const WorkItem it = p.items[idx];
+      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
+        const WorkItem it = p.items[2 * tp + member];
+        if (it.tile_end <= it.tile_begin) continue;
         const int z = it.b * p.Hkv + it.g;
         TRACE(0, 1);
         if (p.q_tma) {
@@ -382,6 +386,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
                           B.full[slot]);
           }
         }
+        ++item_count;
       }
     }
   } else if (warp == 9) {
@@ -396,8 +401,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       const uint32_t q_lo0 = desc_lo(sbase + S::kQ, 16), ring_lo_k = desc_lo(sbase + S::kRing, 16);
       constexpr uint32_t kTileStep = S::kTileBytes >> 4;
       bool ok = true;
-      for (int idx = item_lo; idx < item_hi && ok; ++idx) {
-        const WorkItem it = p.items[idx];
+      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
+        const WorkItem it = p.items[2 * tp + member];
+        if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         TRACE(1, 1);
         const uint32_t qb = item_count & 1u;
@@ -436,8 +442,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       const uint32_t ring_lo_v = desc_lo(sbase + S::kRing, S::kSlabBytes);
       constexpr uint32_t kTileStep = S::kTileBytes >> 4;
       bool ok = true;
-      for (int idx = item_lo; idx < item_hi && ok; ++idx) {
-        const WorkItem it = p.items[idx];
+      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
+        const WorkItem it = p.items[2 * tp + member];
+        if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         for (int s = 0; s < steps && ok; ++s, ++gp) {
           ok = mbar_wait(B.p_full[gp & 1u], (gp >> 1) & 1u, s_abort);
@@ -534,11 +541,15 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps done so far
     bool ok = true;
     // one pass per item, plus a last pass without steps that only writes the final item's output
-    const int pass_end = item_hi > item_lo ? item_hi + 1 : item_lo;   // a CTA without items makes no pass at all
-    for (int idx = item_lo; idx < pass_end && ok; ++idx) {
-      const bool drain = idx == item_hi;
-      const WorkItem it = p.items[drain ? item_lo : idx];
-      const SeqPlan sp = p.seq[it.b];
+    for (int tp = tp_lo; tp <= tp_hi && ok; ++tp) {
+      const bool drain = tp == tp_hi;
+      if (drain && !prev.live) break;                       // nothing was processed
+      WorkItem it = WorkItem();
+      if (!drain) {
+        it = p.items[2 * tp + member];
+        if (it.tile_end <= it.tile_begin) continue;
+      }
+      const SeqPlan sp = drain ? SeqPlan() : p.seq[it.b];
       const int L = sp.L, n = sp.n, G = p.G;
       const int m_valid = n * G, kv_end = L + n;
       const int steps = drain ? 0 : it.tile_end - it.tile_begin;
@@ -706,12 +717,15 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 #ifdef EAGLE_TRACE
   if (tid == 0) {
     long long tiles = 0, tails = 0;
-    for (int idx = item_lo; idx < item_hi; ++idx) {
-      const WorkItem it = p.items[idx];
+    long long n_it = 0;
+    for (int tp = tp_lo; tp < tp_hi; ++tp) {
+      const WorkItem it = p.items[2 * tp + member];
+      if (it.tile_end <= it.tile_begin) continue;
+      ++n_it;
       tiles += it.tile_end - it.tile_begin;
       tails += (it.tile_end * kTileN > p.seq[it.b].L) ? 1 : 0;
     }
-    g_cta_stat[blockIdx.x][1] = item_hi - item_lo;
+    g_cta_stat[blockIdx.x][1] = n_it;
     g_cta_stat[blockIdx.x][2] = tiles;
     g_cta_stat[blockIdx.x][3] = tails;
   }

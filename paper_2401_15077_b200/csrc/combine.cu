@@ -1,7 +1,7 @@
 // Merge of the split-KV partials: m* = max_s m_s, l* = sum_s l_s 2^(m_s - m*), O = sum_s O_s 2^(m_s - m*) / l*,
 // and the zero rows of padded tree nodes.
-// Eight blocks per work unit (16 rows each, two rows per warp): a unit that stayed in one piece was written by the
-// attention kernel and costs one table look-up here; a cut unit has its rows merged.  One more block per sequence
+// Eight blocks per query tile (16 rows each, two rows per warp): a tile that stayed in one item was written by the
+// attention kernel and costs one table look-up here; otherwise its rows are merged from the items that hold it.  One more block per sequence
 // writes zeros to the rows of nodes past the tree size (one contiguous range of the output).
 #include "common.cuh"
 
@@ -27,34 +27,45 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p, 
     for (size_t i = threadIdx.x; i < vecs; i += kCombineThreads) dst[i] = make_uint4(0u, 0u, 0u, 0u);
     return;
   }
-  const int u = blockIdx.x / kBlocksPerUnit, row0 = (blockIdx.x % kBlocksPerUnit) * kRowsPerBlock;
-  if (u >= p.hdr->n_units) return;
-  const UnitPlan up = p.units[u];
-  if (up.n_pieces <= 1) return;   // written directly by the attention kernel
+  // blocks are laid out per query tile: (super-unit, tile-in-pair, 16-row chunk)
+  const int su = blockIdx.x / (2 * kBlocksPerUnit), which = (blockIdx.x / kBlocksPerUnit) & 1;
+  const int row0 = (blockIdx.x % kBlocksPerUnit) * kRowsPerBlock;
+  if (su >= p.hdr->n_units) return;
+  const UnitPlan up = p.units[su];
+  if (up.slot_base < 0) return;   // every query tile of this super-unit was written directly by the attention kernel
   const int b = up.pad0;
   const SeqPlan sp = p.seq[b];
-  const int k = u - sp.unit_base, g = k / sp.mtiles, mt = k % sp.mtiles;
+  const int npairs = (sp.mtiles + 1) / 2;
+  const int k = su - sp.unit_base, g = k / npairs, mp = k % npairs;
+  const bool paired = 2 * mp + 1 < sp.mtiles;
+  const int mt = 2 * mp + which;
+  if (mt >= sp.mtiles) return;    // a lone tile has no sibling
   const int m_valid = sp.n * p.G;
-  const size_t slot0 = static_cast<size_t>(up.slot_base);
+  // the items that hold this query tile: one per team piece for a pair, both for a lone tile (its two halves)
+  const int first = 2 * up.first_item, count = paired ? up.n_pieces : 2 * up.n_pieces;
   for (int r = row0 + warp; r < row0 + kRowsPerBlock; r += kCombineThreads / 32) {
     const int R = mt * kBlockM + r;
     if (R >= m_valid) break;
     const int i = R / p.G, h = g * p.G + R % p.G;
     float m_star = -INFINITY;
-    for (int s = 0; s < up.n_pieces; ++s) {
-      const float2 ml = p.part_ml[(slot0 + s) * kBlockM + r];
+    for (int s = 0; s < count; ++s) {
+      const WorkItem it = p.items[paired ? first + 2 * s + which : first + s];
+      if (it.tile_end <= it.tile_begin) continue;
+      const float2 ml = p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r];
       if (ml.y > 0.f) m_star = fmaxf(m_star, ml.x);
     }
     float acc[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) acc[e] = 0.f;
     float l_star = 0.f;
-    for (int s = 0; s < up.n_pieces; ++s) {
-      const float2 ml = p.part_ml[(slot0 + s) * kBlockM + r];
+    for (int s = 0; s < count; ++s) {
+      const WorkItem it = p.items[paired ? first + 2 * s + which : first + s];
+      if (it.tile_end <= it.tile_begin) continue;
+      const float2 ml = p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r];
       if (!(ml.y > 0.f)) continue;   // a piece in which this row saw no key
       const float w = exp2f(ml.x - m_star);
       l_star += ml.y * w;
-      const float* po = p.part_o + ((slot0 + s) * kBlockM + r) * D + lane * E;
+      const float* po = p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D + lane * E;
       if constexpr (E == 4) {
         const float4 v = *reinterpret_cast<const float4*>(po);
         acc[0] += v.x * w; acc[1] += v.y * w; acc[2] += v.z * w; acc[3] += v.w * w;
@@ -79,7 +90,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p, 
 
 cudaError_t launch_combine(const AttnParams& p, int unit_cap, cudaStream_t stream) {
   if (p.B == 0 || p.T_max == 0) return cudaSuccess;
-  const unsigned unit_blocks = static_cast<unsigned>(unit_cap) * kBlocksPerUnit;
+  const unsigned unit_blocks = static_cast<unsigned>(unit_cap) * 2 * kBlocksPerUnit;   // unit_cap super-units, two query tiles each
   const unsigned blocks = unit_blocks + static_cast<unsigned>(p.B);
   if (p.D == 128) combine_kernel<128><<<blocks, kCombineThreads, 0, stream>>>(p, static_cast<int>(unit_blocks));
   else combine_kernel<64><<<blocks, kCombineThreads, 0, stream>>>(p, static_cast<int>(unit_blocks));

@@ -13,10 +13,9 @@ constexpr int kBlockM = 128;          // query rows (tree node x head-in-group) 
 constexpr int kMaxGroup = 16;         // largest GQA group size supported
 constexpr int kMaxPlanCtas = 256;     // upper bound on the CTAs of the persistent attention kernel (one per SM)
 
-// A work unit is one 128-row query tile of one (sequence, KV head); its work is the sequence's KV tiles.
-// Units are laid end to end in (sequence, KV head, query tile) order; every CTA of the attention kernel takes
-// an equal, contiguous share of that line.  A share boundary inside a unit cuts it into pieces (work items);
-// a unit in several pieces is merged by the combine kernel.
+// A work unit is one 128-row query tile of one (sequence, KV head); its work is the sequence's KV tiles.  The
+// planner groups query tiles in pairs (super-units), lays the super-units end to end and gives every pair of CTAs
+// (a team) an equal contiguous share; see plan.cu.  A work item is what one CTA does for one team piece.
 struct WorkItem {
   int32_t b, g, mt;
   int32_t tile_begin, tile_end;  // KV tiles [begin, end) of `tile_keys` keys each
@@ -29,16 +28,16 @@ struct SeqPlan {
   int32_t L;           // committed prefix length
   int32_t mtiles;      // 128-row query tiles per KV head
   int32_t ntiles;      // KV tiles covering prefix + tree
-  int32_t unit_base;   // index of this sequence's first unit; unit = unit_base + g * mtiles + mt
+  int32_t unit_base;   // index of this sequence's first super-unit; super-unit = unit_base + g * ceil(mtiles/2) + mt/2
   int32_t pad0;
-  long long start;     // position of the first unit on the work line (in KV tiles)
+  long long start;     // position of the first super-unit on the work line
 };
 
-struct UnitPlan {
-  int32_t first_item;  // the unit's pieces are items first_item .. first_item + n_pieces - 1
+struct UnitPlan {        // one per super-unit
+  int32_t first_item;  // its team pieces are first_item .. first_item + n_pieces - 1; piece tp owns items 2*tp and 2*tp+1
   int32_t n_pieces;
-  int32_t slot_base;   // first partial slot (n_pieces > 1), else -1
-  int32_t pad0;        // the unit's sequence
+  int32_t slot_base;   // first partial slot when its query tiles end up in several items, else -1
+  int32_t pad0;        // its sequence
 };
 
 struct PlanHeader {
@@ -56,7 +55,7 @@ struct Workspace {
   SeqPlan* seq;        // [B]
   uint64_t* anc;       // [B, T_max]
   UnitPlan* units;     // [unit_cap]
-  int32_t* cta_first;  // [kMaxPlanCtas + 1]: CTA c owns items cta_first[c] .. cta_first[c+1] - 1
+  int32_t* cta_first;  // [kMaxPlanCtas + 1]: team j owns the team pieces cta_first[j] .. cta_first[j+1] - 1
   WorkItem* items;     // [item_cap]
   float2* part_ml;     // [slot_cap, 128]   (reference max in the log2 domain, row sum)
   float* part_o;       // [slot_cap, 128, D] unnormalised partial outputs
@@ -72,11 +71,12 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   if (G > kMaxGroup || d.max_tree < 0 || d.max_tree > kMaxTree || (d.head_dim != 64 && d.head_dim != 128)) return false;
   if (d.num_splits < 0 || d.num_splits > 1024) return false;
   const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
-  const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? mtiles : 1);
-  // chosen by the planner: every share boundary adds at most one piece, and a cut unit has at most
-  // (cuts + 1) <= 2 * cuts pieces; forced: every unit in num_splits pieces
-  const long long slots = d.num_splits > 1 ? units * d.num_splits : (d.num_splits == 1 ? 0 : 2 * kMaxPlanCtas);
-  const long long items = d.num_splits > 1 ? units * d.num_splits : units + kMaxPlanCtas;
+  const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? (mtiles + 1) / 2 : 1);   // super-units
+  // team pieces: one per super-unit plus at most one per share boundary (or num_splits per super-unit when forced);
+  // two items per team piece, and at most one partial slot per item
+  const long long pieces = d.num_splits > 0 ? units * d.num_splits : units + kMaxPlanCtas / 2;
+  const long long items = 2 * pieces;
+  const long long slots = items;
   if (items > (1ll << 30)) return false;
   char* p = static_cast<char*>(base);
   size_t off = 0;

@@ -3,13 +3,18 @@
 // The host never reads seq_lens or tree_sizes (they are device arrays and the call must not synchronise),
 // so one small CTA turns them into (1) the per-node ancestor-or-self bit masks that define tree attention
 // (Sec. 3.1 / 3.3: a draft token attends to the context and to its own root path) and (2) the work split of
-// the persistent attention kernel: work units (sequence, KV head, 128-row query tile) are laid end to end,
-// each as long as its sequence's KV tiles, and every CTA gets an equal contiguous share of that line.  A
-// share boundary that falls inside a unit cuts it into pieces; boundaries closer than `snap_tiles` to a
-// unit's edge move to the edge, so no piece is shorter than that.  Each CTA therefore does the same number
-// of KV tiles (to within the snap) whatever the mix of sequence lengths and tree sizes.  Every unit also
-// carries a fixed cost of `item_overhead_tiles` tile-equivalents at its start (query staging, pipeline fill,
-// epilogue), so that a share made of many short units is not mistaken for an equally cheap one.
+// the persistent attention kernel.
+//
+// Work split.  A work unit is one 128-row query tile of one (sequence, KV head); its work is the sequence's KV
+// tiles.  The CTAs of the attention kernel are taken in pairs ("teams").  The query tiles of a (sequence, KV head)
+// are taken two at a time: such a pair is a super-unit that both CTAs of a team walk together, one query tile each
+// over the same KV tiles, so the keys and values one of them pulls from HBM are still in L2 when the other asks for
+// them; an odd last query tile is a super-unit whose KV range the team's two CTAs split in halves.  All super-units
+// are laid end to end on one line (plus `item_overhead_tiles` positions of fixed cost at the start of each), and
+// every team gets an equal contiguous share of the line.  A share boundary inside a super-unit cuts it into
+// pieces (their partial results are merged by the combine kernel); boundaries closer than `snap_tiles` to an edge
+// move to the edge.  Every CTA therefore does the same number of KV tiles, to within the snap, whatever the mix of
+// sequence lengths and tree sizes.
 #include "common.cuh"
 
 namespace eagle {
@@ -116,22 +121,41 @@ __device__ inline bool build_masks_warp(const int32_t* par, int n, uint64_t* anc
   return true;
 }
 
-// The unit occupies [us, ue) on the work line: `ovh` positions of fixed cost, then one position per KV tile.
-// Its interior cuts are the share boundaries floor(c * W / ctas) with us + ovh + snap <= boundary <= ue - snap:
-// a contiguous range of c.  Returns their number and the first such c.
-__device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W, int ctas, int snap, int ovh, int* first_c) {
+// A super-unit occupies [us, ue) on the work line: `ovh` positions of fixed cost, then one position per KV tile of
+// its line.  Its interior cuts are the share boundaries floor(c * W / teams) with us + ovh + snap <= boundary <=
+// ue - snap: a contiguous range of c.  Returns their number and the first such c.
+__device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W, int teams, int snap, int ovh, int* first_c) {
   const long long y = us + ovh + snap, z = ue - snap;
   *first_c = 0;
-  if (z < y || ctas < 2) return 0;
-  long long ca = ceil_div(y * ctas, W), cb = ceil_div((z + 1) * ctas, W) - 1;
+  if (z < y || teams < 2) return 0;
+  long long ca = ceil_div(y * teams, W), cb = ceil_div((z + 1) * teams, W) - 1;
   if (ca < 1) ca = 1;
-  if (cb > ctas - 1) cb = ctas - 1;
+  if (cb > teams - 1) cb = teams - 1;
   *first_c = static_cast<int>(ca);
   return cb >= ca ? static_cast<int>(cb - ca + 1) : 0;
 }
 
 constexpr int kSmemSeqs = 512;     // per-sequence records kept in shared memory while planning (else in the workspace)
-constexpr int kSmemUnits = 1792;   // per-unit records kept in shared memory while planning
+constexpr int kSmemUnits = 1792;   // per-super-unit records kept in shared memory while planning
+
+// Geometry of a sequence's super-units.  The query tiles of one (sequence, KV head) are taken two at a time; a pair is
+// one super-unit whose line is the sequence's KV tiles (both CTAs of a team walk it, one query tile each), and an odd
+// last tile is a super-unit whose line is half the KV tiles (the team's CTAs take one half each).
+struct SeqGeom {
+  int npairs, ntiles, half, plen, glen;   // super-units per head; KV tiles; ceil(ntiles/2); paired length; per-head length
+  bool odd;
+  __device__ SeqGeom(const SeqPlan& sp, int ovh) {
+    npairs = (sp.mtiles + 1) / 2;
+    ntiles = sp.ntiles;
+    half = (sp.ntiles + 1) / 2;
+    odd = (sp.mtiles & 1) != 0;
+    plen = sp.ntiles + ovh;
+    glen = (sp.mtiles / 2) * plen + (odd ? half + ovh : 0);
+  }
+  __device__ bool paired(int mp) const { return !(odd && mp == npairs - 1); }
+  __device__ int line(int mp) const { return paired(mp) ? ntiles : half; }          // tile positions of the super-unit
+  __device__ long long offset(int k) const { return static_cast<long long>(k / npairs) * glen + static_cast<long long>(k % npairs) * plen; }
+};
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   __shared__ long long s_scan[kPlanThreads / 32];
@@ -177,19 +201,20 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   }
   __syncthreads();
 
-  // ---- lay the sequences' units end to end
+  // ---- lay the sequences' super-units end to end
   const long long W = block_exclusive_scan(
-      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * p.seq[b].mtiles * (p.seq[b].ntiles > 0 ? p.seq[b].ntiles + ovh : 0); },
+      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * SeqGeom(p.seq[b], ovh).glen; },
       [&](int b, long long v) { p.seq[b].start = v; }, s_scan);
   const long long U = block_exclusive_scan(
-      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * p.seq[b].mtiles; },
+      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * ((p.seq[b].mtiles + 1) / 2); },
       [&](int b, long long v) { p.seq[b].unit_base = static_cast<int>(v); }, s_scan);
   const int n_units = U <= p.unit_cap ? static_cast<int>(U) : 0;   // cannot exceed the advertised workspace
   if (U > p.unit_cap && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);
-  const int ctas = static_cast<int>(W < p.num_ctas ? (W > 0 ? W : 1) : p.num_ctas);   // a share is at least one tile
+  const int max_teams = p.num_ctas / 2;
+  const int teams = static_cast<int>(W < max_teams ? (W > 0 ? W : 1) : max_teams);   // a share is at least one position
   const int snap = p.snap_tiles;
 
-  // unit -> sequence: the last sequence whose unit_base <= u (sequences without units share theirs with the next)
+  // super-unit -> sequence: the last sequence whose unit_base <= u (sequences without units share theirs with the next)
   auto unit_seq = [&](int u) {
     int lo = 0, hi = p.B;
     while (hi - lo > 1) {
@@ -199,96 +224,126 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
     return lo;
   };
 
-  // ---- pieces per unit
+  // ---- team pieces per super-unit
   for (int u = tid; u < n_units; u += kPlanThreads) {
     const int b = unit_seq(u);
     const SeqPlan sp = p.seq[b];
-    const int ulen = sp.ntiles + ovh;
-    const long long us = sp.start + static_cast<long long>(u - sp.unit_base) * ulen;
+    const SeqGeom ge(sp, ovh);
+    const int k = u - sp.unit_base, mp = k % ge.npairs;
+    const int len = ge.line(mp);
+    const long long us = sp.start + ge.offset(k);
     int np;
     if (p.forced_splits > 0) {
-      np = sp.ntiles < p.forced_splits ? sp.ntiles : p.forced_splits;
+      np = len < p.forced_splits ? len : p.forced_splits;
     } else {
       int c0;
-      np = 1 + unit_cuts(us, us + ulen, W, ctas, snap, ovh, &c0);
+      np = 1 + unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0);
     }
     p.units[u].n_pieces = np;
     p.units[u].pad0 = b;
   }
   __syncthreads();
-  const long long I = block_exclusive_scan(
+  // a super-unit needs partial slots when some query tile of it ends up in more than one item:
+  // a pair cut into np > 1 team pieces (np items per tile), or a single tile (its halves: 2 * np items) with > 1 KV tile
+  auto slots_of = [&](int u) -> long long {
+    const UnitPlan up = p.units[u];
+    const SeqPlan sp = p.seq[up.pad0];
+    const SeqGeom ge(sp, ovh);
+    const int mp = (u - sp.unit_base) % ge.npairs;
+    const bool partial = ge.paired(mp) ? up.n_pieces > 1 : sp.ntiles > 1;
+    return partial ? 2ll * up.n_pieces : 0ll;
+  };
+  const long long TP = block_exclusive_scan(
       n_units, [&](int u) { return static_cast<long long>(p.units[u].n_pieces); },
       [&](int u, long long v) { p.units[u].first_item = static_cast<int>(v); }, s_scan);
   const long long S = block_exclusive_scan(
-      n_units, [&](int u) { return p.units[u].n_pieces > 1 ? static_cast<long long>(p.units[u].n_pieces) : 0ll; },
-      [&](int u, long long v) { p.units[u].slot_base = p.units[u].n_pieces > 1 ? static_cast<int>(v) : -1; }, s_scan);
-  const bool fits = I <= p.item_cap && S <= p.slot_cap;
+      n_units, slots_of, [&](int u, long long v) { p.units[u].slot_base = slots_of(u) > 0 ? static_cast<int>(v) : -1; }, s_scan);
+  const bool fits = 2 * TP <= p.item_cap && S <= p.slot_cap;
   if (!fits && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);   // cannot happen with the advertised size
 
-  // ---- items
+  // ---- items: two per team piece, one for each CTA of the team
   if (fits) {
     for (int u = tid; u < n_units; u += kPlanThreads) {
-      const int b = unit_seq(u);
-      const SeqPlan sp = p.seq[b];
-      const int k = u - sp.unit_base;
-      const int ulen = sp.ntiles + ovh;
-      const long long us = sp.start + static_cast<long long>(k) * ulen;
-      const long long t_origin = us + ovh;          // line position of KV tile 0
       const UnitPlan up = p.units[u];
+      const int b = up.pad0;
+      const SeqPlan sp = p.seq[b];
+      const SeqGeom ge(sp, ovh);
+      const int k = u - sp.unit_base, g = k / ge.npairs, mp = k % ge.npairs;
+      const bool paired = ge.paired(mp);
+      const int len = ge.line(mp), rest = sp.ntiles - len;      // single tile: second CTA's part has `rest` tiles
+      const long long us = sp.start + ge.offset(k);
+      const long long t_origin = us + ovh;          // line position of the super-unit's tile position 0
       int c0 = 0;
-      if (p.forced_splits == 0) unit_cuts(us, us + ulen, W, ctas, snap, ovh, &c0);
+      if (p.forced_splits == 0) unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0);
       for (int j = 0; j < up.n_pieces; ++j) {
-        WorkItem it;
-        it.b = b;
-        it.g = k / sp.mtiles;
-        it.mt = k % sp.mtiles;
+        int t0, t1;
         if (p.forced_splits > 0) {
-          it.tile_begin = static_cast<int>(static_cast<long long>(sp.ntiles) * j / up.n_pieces);
-          it.tile_end = static_cast<int>(static_cast<long long>(sp.ntiles) * (j + 1) / up.n_pieces);
+          t0 = static_cast<int>(static_cast<long long>(len) * j / up.n_pieces);
+          t1 = static_cast<int>(static_cast<long long>(len) * (j + 1) / up.n_pieces);
         } else {
-          it.tile_begin = j == 0 ? 0 : static_cast<int>(static_cast<long long>(c0 + j - 1) * W / ctas - t_origin);
-          it.tile_end = j == up.n_pieces - 1 ? sp.ntiles : static_cast<int>(static_cast<long long>(c0 + j) * W / ctas - t_origin);
+          t0 = j == 0 ? 0 : static_cast<int>(static_cast<long long>(c0 + j - 1) * W / teams - t_origin);
+          t1 = j == up.n_pieces - 1 ? len : static_cast<int>(static_cast<long long>(c0 + j) * W / teams - t_origin);
         }
-        it.slot = up.n_pieces > 1 ? up.slot_base + j : -1;
-        it.pad0 = it.pad1 = 0;
-        p.items[up.first_item + j] = it;
+        for (int m = 0; m < 2; ++m) {
+          WorkItem it;
+          it.b = b;
+          it.g = g;
+          if (paired) {
+            it.mt = 2 * mp + m;
+            it.tile_begin = t0;
+            it.tile_end = t1;
+            it.slot = up.slot_base >= 0 ? up.slot_base + m * up.n_pieces + j : -1;
+          } else {
+            it.mt = 2 * mp;
+            it.tile_begin = m == 0 ? t0 : len + (t0 < rest ? t0 : rest);
+            it.tile_end = m == 0 ? t1 : len + (t1 < rest ? t1 : rest);
+            it.slot = up.slot_base >= 0 ? up.slot_base + 2 * j + m : -1;
+          }
+          it.pad0 = it.pad1 = 0;
+          p.items[2 * (up.first_item + j) + m] = it;
+        }
       }
     }
   }
 
-  // ---- first item of every CTA
+  // ---- first team piece of every team (cta_first is indexed by team here; entries past the last team repeat the end)
   for (int c = tid; c <= p.num_ctas; c += kPlanThreads) {
     long long first;
-    if (!fits || I == 0) {
+    if (!fits || TP == 0) {
       first = 0;
     } else if (p.forced_splits > 0) {
-      first = static_cast<long long>(c) * I / p.num_ctas;
+      first = c >= max_teams ? TP : static_cast<long long>(c) * TP / max_teams;
     } else if (c == 0) {
       first = 0;
-    } else if (c >= ctas) {
-      first = I;
+    } else if (c >= teams) {
+      first = TP;
     } else {
-      const long long x = static_cast<long long>(c) * W / ctas;   // 0 < x < W
+      const long long x = static_cast<long long>(c) * W / teams;   // 0 < x < W
       int lo = 0, hi = p.B;          // last sequence whose start <= x (sequences without work share their start with the next)
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if (p.seq[mid].start <= x) lo = mid; else hi = mid;
       }
       const SeqPlan sp = p.seq[lo];
-      const int ulen = sp.ntiles + ovh;
-      const int k = static_cast<int>((x - sp.start) / ulen);
+      const SeqGeom ge(sp, ovh);
+      const long long off = x - sp.start;
+      const int g = static_cast<int>(off / ge.glen);
+      const long long rem = off % ge.glen;
+      int mp = static_cast<int>(rem / ge.plen);
+      if (mp > ge.npairs - 1) mp = ge.npairs - 1;
+      const int k = g * ge.npairs + mp;
       const int u = sp.unit_base + k;
-      const long long us = sp.start + static_cast<long long>(k) * ulen, ue = us + ulen;
-      const long long d0 = x - (us + ovh), d1 = ue - x;   // distance to the first KV tile / to the unit's end
+      const long long us = sp.start + ge.offset(k), ue = us + ge.line(mp) + ovh;
+      const long long d0 = x - (us + ovh), d1 = ue - x;   // distance to the first tile position / to the super-unit's end
       const UnitPlan up = p.units[u];
       if (d0 >= snap && d1 >= snap) {
         int c0;
-        unit_cuts(us, ue, W, ctas, snap, ovh, &c0);
+        unit_cuts(us, ue, W, teams, snap, ovh, &c0);
         first = up.first_item + 1 + (c - c0);        // the piece that starts at this boundary
       } else if (x - us <= d1) {
-        first = up.first_item;                        // boundary moved to the unit's start
+        first = up.first_item;                        // boundary moved to the super-unit's start
       } else {
-        first = up.first_item + up.n_pieces;          // boundary moved to the unit's end
+        first = up.first_item + up.n_pieces;          // boundary moved to the super-unit's end
       }
     }
     p.cta_first[c] = static_cast<int>(first);
@@ -299,10 +354,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   if (units_in_smem)
     for (int u = tid; u < n_units; u += kPlanThreads) pg.units[u] = s_units[u];
   if (tid == 0) {
-    p.hdr->n_items = fits ? static_cast<int>(I) : 0;
+    p.hdr->n_items = fits ? static_cast<int>(2 * TP) : 0;
     p.hdr->n_slots = fits ? static_cast<int>(S) : 0;
     p.hdr->n_units = n_units;
-    p.hdr->ctas_used = ctas;
+    p.hdr->ctas_used = 2 * teams;
     p.hdr->total_tiles = W;
   }
 }
