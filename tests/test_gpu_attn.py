@@ -56,6 +56,9 @@ CASES = {
     "mixtral_gqa_small": W.scaled(W.CONFIGS["mixtral_gqa"], batch=2, prefix=(1500, 3000)),
     "serving_mix_small": W.scaled(W.CONFIGS["serving_mix"], batch=6, prefix=(100, 1500)),
     "d64_gqa_ragged": W.scaled(W.CONFIGS["tiny"], batch=5, num_q_heads=16, num_kv_heads=4, prefix=(0, 700), tree=(1, 33)),
+    # group sizes that do not divide 128: the query tile is staged by the softmax threads instead of TMA
+    "group3_d128": W.scaled(W.CONFIGS["7b_mha"], batch=3, num_q_heads=12, num_kv_heads=4, prefix=(50, 1200), tree=(3, 64), max_depth=8),
+    "group6_d64": W.scaled(W.CONFIGS["tiny"], batch=2, num_q_heads=12, num_kv_heads=2, prefix=(0, 500), tree=(10, 50), max_depth=6),
     "big_group_full_tree": W.scaled(W.CONFIGS["70b_gqa"], batch=2, num_q_heads=32, num_kv_heads=2, prefix=(130, 400),
                                     tree=(64, 64), max_depth=64, child_cap=0),
 }
