@@ -63,7 +63,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except Exception:
             self.proc = None
@@ -72,10 +72,14 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([x.strip() for x in line.split(",")])
 
-    def stop(self):
+    def mark(self):
+        """Number of samples taken so far (to cut out the samples of the timed region)."""
+        return len(self.rows)
+
+    def stop(self, first=0, last=None):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -83,7 +87,8 @@ class ClockSampler:
             self.proc.kill()
         sm, smax, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        window = self.rows[first:last] or self.rows[-3:]
+        for r in window:
             try:
                 sm.append(float(r[0]))
                 smax = float(r[1])
@@ -149,7 +154,7 @@ def run_reference(args, cfg, rank, world):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="serving_mix", choices=list(W.CONFIGS))
@@ -174,7 +179,7 @@ def main():
         return
 
     import torch.distributed as dist
-    from paper_2401_15077_b200 import binding as E, build
+    from paper_2401_15077_b200 import binding as E, build, replicas
     if rank == 0 or world == 1:
         build.build()
     E.load()
@@ -183,7 +188,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    attn, acc = host_inputs(cfg, rank, args.rho)
+    attn, acc = host_inputs(cfg, replicas.rank_salt(rank), args.rho)
     alg_bytes, alg_flops = attn.algorithmic_bytes(), attn.algorithmic_flops()
 
     # ---- device-resident input sets; rotate over R sets so that consecutive steps never hit a warm L2
@@ -208,10 +213,12 @@ def main():
                             accept_len=alen, status=status)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()          # started early: nvidia-smi needs a while before its first sample
     for i in range(max(args.warmup, 3)):
         step(sets[i % R])
     torch.cuda.synchronize()
@@ -225,24 +232,21 @@ def main():
     ev_acc = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = E.launch_count()
-    sampler = ClockSampler(local)
     barrier()
-    if rank == 0:
-        sampler.start()
+    if rank == 0 and sampler.mark() == 0:
+        time.sleep(0.5)
+    m0 = sampler.mark()
     start.record()
     for i in range(K):
         step(sets[(args.warmup + i) % R], ev_pairs[i])
     stop.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(m0, sampler.mark() + 1) if rank == 0 else None
     launches = E.launch_count() - launches0
     elapsed_ms = start.elapsed_time(stop)
     attn_ms = statistics.mean(a.elapsed_time(b) for a, b in ev_pairs)
     assert int(status.item()) == 0
-    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    elapsed_ms = float(t.item())
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dev)
     value = world * K / (elapsed_ms * 1e-3)
 
     # ---- acceptance alone (reported, not part of the headline)
@@ -256,34 +260,28 @@ def main():
     accept_ms = statistics.mean(ev_acc[i][0].elapsed_time(ev_acc[i][1]) for i in range(min(K, 10)))
     mean_tokens = float(alen.float().mean().item()) + 1.0
 
-    # ---- end to end from pinned host buffers
-    pinned = {k: v.pin_memory() for k, v in host.items()}
-    dset = sets[0]
-    h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-    h_path, h_bonus = torch.empty(path.shape, dtype=path.dtype).pin_memory(), torch.empty(bonus.shape, dtype=bonus.dtype).pin_memory()
-    h2d = sum(v.numel() * v.element_size() for v in pinned.values())
-    d2h = sum(v.numel() * v.element_size() for v in (h_out, h_path, h_bonus))
-
-    def e2e_step():
-        for k2, v in pinned.items():
-            dset[k2].copy_(v, non_blocking=True)
-        step(dset)
-        h_out.copy_(out, non_blocking=True)
-        h_path.copy_(path, non_blocking=True)
-        h_bonus.copy_(bonus, non_blocking=True)
-
-    e2e_step()
+    # ---- end to end from pinned host buffers, through the library's host-buffer entry point: every step copies all
+    # inputs host->device, runs attention + acceptance, and copies the results back
+    pinned = dict(q=attn.q, k_cache=attn.k_cache, v_cache=attn.v_cache, seq_lens=attn.seq_lens, tree_sizes=attn.tree_sizes,
+                  tree_parent=attn.tree_parent, target_probs=acc.target_probs, draft_probs=acc.draft_probs,
+                  draft_tokens=acc.draft_tokens, uniforms=acc.uniforms, greedy=acc.greedy)
+    pinned = {k: v.pin_memory() for k, v in pinned.items()}
+    del sets
+    torch.cuda.empty_cache()
+    runner = E.HostStepRunner(pinned, dev)
+    h2d, d2h = runner.h2d_bytes, runner.d2h_bytes
+    runner.run()
     barrier()
+    assert int(runner.status.item()) == 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.e2e_steps):
-        e2e_step()
+        runner.run()
     e1.record()
     barrier()
-    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * args.e2e_steps / (float(te.item()) * 1e-3)
+    e2e_value = world * args.e2e_steps / (replicas.max_over_ranks(e0.elapsed_time(e1), dev) * 1e-3)
+    # the step driven from host buffers gives the same tokens as the device-resident one (all input sets hold the same data)
+    same_tokens = bool(torch.equal(runner.bonus_token, bonus.cpu()))
 
     if rank != 0:
         if world > 1:
@@ -301,7 +299,8 @@ def main():
                    "greedy": cfg.greedy, "rho": args.rho, "parallelism": f"replicas x{world}",
                    "l2": (f"rotating over {R} input sets" if R > 1 else "inputs larger than L2 (single set)")},
         "clocks": clocks, "gpu_launches": launches,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+                "api": "eagle_tree_verify_step_host", "same_tokens_as_device_path": same_tokens},
         "roofline": {"bound": "hbm", "kernel": "split-KV tree attention", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
                      "algorithmic_bytes": alg_bytes, "ms_per_launch": attn_ms,

@@ -171,6 +171,42 @@ int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, 
                       int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream);
 
 /*
+ * One whole verification step driven from HOST buffers (the two calls above, with the copies around them).
+ *
+ * Every input pointer below is a host pointer (pinned memory makes the copies asynchronous); the call enqueues on
+ * `stream`: host->device copies of all inputs into `arena`, eagle_tree_verify_attn, eagle_tree_accept, and
+ * device->host copies of out, accepted_path, bonus_token and accept_len.  It allocates nothing: `arena` is device
+ * memory provided by the caller, 256-byte aligned, at least eagle_tree_verify_step_host_arena() bytes (device copies
+ * of all tensors plus the attention workspace).  The results are in the host buffers once `stream` has drained.
+ * Verification phase: Sec. 3.3; acceptance: App. A.2, Algorithm 1.  Shapes and meanings as for the device calls.
+ */
+typedef struct eagle_host_step {
+  int32_t batch, num_q_heads, num_kv_heads, head_dim, max_tree, kv_capacity, vocab, path_cap;
+  float sm_scale;
+  const void* q;                 /* host bf16 [B, T_max, Hq, D] */
+  const void* k_cache;           /* host bf16 [B, Hkv, S_cap, D] */
+  const void* v_cache;
+  const int32_t* seq_lens;       /* host int32 [B] */
+  const int32_t* tree_sizes;     /* host int32 [B] or NULL */
+  const int32_t* tree_parent;    /* host int32 [B, T_max] */
+  const float* target_probs;     /* host fp32 [B, T_max+1, V] */
+  const float* draft_probs;      /* host fp32 [B, T_max, V] */
+  const int32_t* draft_tokens;   /* host int32 [B, T_max] */
+  const float* uniforms;         /* host fp32 [B, T_max+1] */
+  const uint8_t* greedy;         /* host uint8 [B] or NULL */
+  void* out;                     /* host bf16 [B, T_max, Hq, D] */
+  int32_t* accepted_path;        /* host int32 [B, path_cap] */
+  int32_t* bonus_token;          /* host int32 [B] */
+  int32_t* accept_len;           /* host int32 [B] */
+  int32_t* status;               /* host int32[1]: device-detected status of the step (0 = ok) */
+  void* arena;                   /* device */
+  size_t arena_bytes;
+} eagle_host_step;
+
+size_t eagle_tree_verify_step_host_arena(const eagle_host_step* step);
+int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stream);
+
+/*
  * Tree-mask builder alone (the mask "tree attention" implies: Sec. 3.1, Sec. 3.3): for every node the bit set
  * of its ancestors and itself, and its depth (top-level nodes: 1).
  *   tree_parent device int32 [B, T_max]; tree_sizes device int32 [B] or NULL;

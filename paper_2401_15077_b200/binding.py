@@ -16,7 +16,8 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libeagle_verify.so"
 EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_tree_accept",
            "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
-           "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity"]
+           "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
+           "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena"]
 _lib = None
 
 
@@ -38,6 +39,14 @@ class AcceptDesc(ctypes.Structure):
                 ("accept_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
 
 
+class HostStep(ctypes.Structure):
+    _fields_ = ([(n, ctypes.c_int32) for n in ("batch", "num_q_heads", "num_kv_heads", "head_dim", "max_tree", "kv_capacity",
+                                                "vocab", "path_cap")] + [("sm_scale", ctypes.c_float)] +
+                [(n, ctypes.c_void_p) for n in ("q", "k_cache", "v_cache", "seq_lens", "tree_sizes", "tree_parent", "target_probs",
+                                                "draft_probs", "draft_tokens", "uniforms", "greedy", "out", "accepted_path",
+                                                "bonus_token", "accept_len", "status", "arena")] + [("arena_bytes", ctypes.c_size_t)])
+
+
 def load():
     """Loads the shared library (once).  Raises if it has not been built."""
     global _lib
@@ -54,6 +63,10 @@ def load():
         lib.eagle_tree_verify_attn_static.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_verify_attn_static.restype = ctypes.c_int
         lib.eagle_tree_verify_attn_static_capacity.restype = ctypes.c_size_t
+        lib.eagle_tree_verify_step_host.argtypes = [ctypes.POINTER(HostStep), vp]
+        lib.eagle_tree_verify_step_host.restype = ctypes.c_int
+        lib.eagle_tree_verify_step_host_arena.argtypes = [ctypes.POINTER(HostStep)]
+        lib.eagle_tree_verify_step_host_arena.restype = ctypes.c_size_t
         lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_accept.restype = ctypes.c_int
         lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
@@ -205,3 +218,43 @@ def eagle_tree_build_mask(tree_parent, tree_sizes=None, status=None, with_depth=
                                    _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "eagle_tree_build_mask")
     return anc, depth
+
+
+class HostStepRunner:
+    """One verification step from (pinned) host tensors through ``eagle_tree_verify_step_host``.
+
+    ``host`` maps q, k_cache, v_cache, seq_lens, tree_sizes, tree_parent, target_probs, draft_probs, draft_tokens,
+    uniforms, greedy to CPU tensors; outputs land in the pinned tensors ``out``, ``accepted_path``, ``bonus_token``,
+    ``accept_len``, ``status`` of this object once the stream has drained.  The device arena is allocated once here."""
+
+    def __init__(self, host: dict, device):
+        lib = load()
+        self.host = host
+        q, k, tp = host["q"], host["k_cache"], host["target_probs"]
+        B, T, Hq, D = q.shape
+        self.out = torch.empty(q.shape, dtype=q.dtype).pin_memory()
+        self.accepted_path = torch.empty((B, T), dtype=torch.int32).pin_memory()
+        self.bonus_token = torch.empty((B,), dtype=torch.int32).pin_memory()
+        self.accept_len = torch.empty((B,), dtype=torch.int32).pin_memory()
+        self.status = torch.zeros((1,), dtype=torch.int32).pin_memory()
+        s = HostStep()
+        s.batch, s.num_q_heads, s.num_kv_heads, s.head_dim, s.max_tree = B, Hq, k.shape[1], D, T
+        s.kv_capacity, s.vocab, s.path_cap, s.sm_scale = k.shape[2], tp.shape[2], T, 0.0
+        for name in ("q", "k_cache", "v_cache", "seq_lens", "tree_sizes", "tree_parent", "target_probs", "draft_probs",
+                     "draft_tokens", "uniforms", "greedy"):
+            t = host.get(name)
+            setattr(s, name, None if t is None else t.data_ptr())
+        s.out, s.accepted_path, s.bonus_token = self.out.data_ptr(), self.accepted_path.data_ptr(), self.bonus_token.data_ptr()
+        s.accept_len, s.status = self.accept_len.data_ptr(), self.status.data_ptr()
+        n = lib.eagle_tree_verify_step_host_arena(ctypes.byref(s))
+        if n == 0:
+            raise EagleError("unsupported shape for the host step")
+        self.arena = torch.empty(n, dtype=torch.uint8, device=device)
+        s.arena, s.arena_bytes = self.arena.data_ptr(), n
+        self.step = s
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in host.values() if t is not None)
+        self.d2h_bytes = sum(t.numel() * t.element_size() for t in (self.out, self.accepted_path, self.bonus_token,
+                                                                    self.accept_len, self.status))
+
+    def run(self):
+        _check(load().eagle_tree_verify_step_host(ctypes.byref(self.step), _stream()), "eagle_tree_verify_step_host")

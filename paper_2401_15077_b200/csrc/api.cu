@@ -342,6 +342,101 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   return EAGLE_OK;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// One step from host buffers: copies in, the two device calls, copies out; everything on the caller's stream.
+namespace {
+
+struct HostStepLayout {
+  size_t q, k, v, seq_lens, tree_sizes, tree_parent, target, draft, tokens, uniforms, greedy, out, path, bonus, alen, status, ws;
+  size_t n_q, n_kv, n_target, n_draft, n_bt, n_b, n_u, n_path, ws_bytes, total;
+};
+
+bool host_step_layout(const eagle_host_step& s, HostStepLayout* L) {
+  if (s.batch < 0 || s.max_tree < 0 || s.vocab < 1 || s.path_cap < 0 || s.kv_capacity < 0) return false;
+  eagle_attn_desc d = {};
+  d.batch = s.batch; d.num_q_heads = s.num_q_heads; d.num_kv_heads = s.num_kv_heads; d.head_dim = s.head_dim;
+  d.max_tree = s.max_tree; d.kv_capacity = s.kv_capacity;
+  Workspace w;
+  if (!carve_workspace(d, nullptr, &w)) return false;
+  const size_t B = static_cast<size_t>(s.batch), T = static_cast<size_t>(s.max_tree);
+  L->n_q = B * T * s.num_q_heads * s.head_dim * 2;
+  L->n_kv = B * s.num_kv_heads * static_cast<size_t>(s.kv_capacity) * s.head_dim * 2;
+  L->n_target = B * (T + 1) * s.vocab * 4;
+  L->n_draft = B * T * s.vocab * 4;
+  L->n_bt = B * T * 4;
+  L->n_b = B * 4;
+  L->n_u = B * (T + 1) * 4;
+  L->n_path = B * static_cast<size_t>(s.path_cap) * 4;
+  L->ws_bytes = w.bytes;
+  size_t off = 0;
+  auto take = [&](size_t n) { const size_t r = off; off += align256(n > 0 ? n : 1); return r; };
+  L->q = take(L->n_q); L->k = take(L->n_kv); L->v = take(L->n_kv);
+  L->seq_lens = take(L->n_b); L->tree_sizes = take(L->n_b); L->tree_parent = take(L->n_bt);
+  L->target = take(L->n_target); L->draft = take(L->n_draft); L->tokens = take(L->n_bt);
+  L->uniforms = take(L->n_u); L->greedy = take(B);
+  L->out = take(L->n_q); L->path = take(L->n_path); L->bonus = take(L->n_b); L->alen = take(L->n_b);
+  L->status = take(4); L->ws = take(w.bytes);
+  L->total = off;
+  return true;
+}
+
+}  // namespace
+
+size_t eagle_tree_verify_step_host_arena(const eagle_host_step* step) {
+  HostStepLayout L;
+  if (!step || !host_step_layout(*step, &L)) return 0;
+  return L.total;
+}
+
+int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stream_) {
+  if (!step) return EAGLE_ERR_NULL;
+  const eagle_host_step& s = *step;
+  HostStepLayout L;
+  if (!host_step_layout(s, &L)) return EAGLE_ERR_SHAPE;
+  if (s.batch == 0) return EAGLE_OK;
+  if (!s.q || !s.k_cache || !s.v_cache || !s.seq_lens || !s.tree_parent || !s.target_probs || !s.draft_tokens || !s.out ||
+      !s.accepted_path || !s.bonus_token)
+    return EAGLE_ERR_NULL;
+  if ((!s.draft_probs || !s.uniforms) && !s.greedy) return EAGLE_ERR_NULL;
+  if (!s.arena || (reinterpret_cast<uintptr_t>(s.arena) & 255) || s.arena_bytes < L.total) return EAGLE_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char* A = static_cast<char*>(s.arena);
+  auto h2d = [&](size_t off, const void* src, size_t n) {
+    return !src || n == 0 || cudaMemcpyAsync(A + off, src, n, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  };
+  auto d2h = [&](void* dst, size_t off, size_t n) {
+    return !dst || n == 0 || cudaMemcpyAsync(dst, A + off, n, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  };
+  bool ok = cudaMemsetAsync(A + L.status, 0, 4, stream) == cudaSuccess;
+  ok = ok && h2d(L.q, s.q, L.n_q) && h2d(L.k, s.k_cache, L.n_kv) && h2d(L.v, s.v_cache, L.n_kv) &&
+       h2d(L.seq_lens, s.seq_lens, L.n_b) && h2d(L.tree_sizes, s.tree_sizes, L.n_b) && h2d(L.tree_parent, s.tree_parent, L.n_bt) &&
+       h2d(L.target, s.target_probs, L.n_target) && h2d(L.draft, s.draft_probs, L.n_draft) && h2d(L.tokens, s.draft_tokens, L.n_bt) &&
+       h2d(L.uniforms, s.uniforms, L.n_u) && h2d(L.greedy, s.greedy, static_cast<size_t>(s.batch));
+  if (!ok) return EAGLE_ERR_LAUNCH;
+  int32_t* d_status = reinterpret_cast<int32_t*>(A + L.status);
+  const int32_t* d_sizes = s.tree_sizes ? reinterpret_cast<const int32_t*>(A + L.tree_sizes) : nullptr;
+  eagle_attn_desc ad = {};
+  ad.batch = s.batch; ad.num_q_heads = s.num_q_heads; ad.num_kv_heads = s.num_kv_heads; ad.head_dim = s.head_dim;
+  ad.max_tree = s.max_tree; ad.kv_capacity = s.kv_capacity; ad.tree_sizes = d_sizes; ad.sm_scale = s.sm_scale;
+  ad.workspace = A + L.ws; ad.workspace_bytes = L.ws_bytes; ad.status = d_status;
+  int rc = eagle_tree_verify_attn(&ad, A + L.q, A + L.k, A + L.v, reinterpret_cast<const int32_t*>(A + L.seq_lens),
+                                  reinterpret_cast<const int32_t*>(A + L.tree_parent), A + L.out, stream_);
+  if (rc != EAGLE_OK) return rc;
+  eagle_accept_desc cd = {};
+  cd.batch = s.batch; cd.max_tree = s.max_tree; cd.vocab = s.vocab; cd.path_cap = s.path_cap; cd.tree_sizes = d_sizes;
+  cd.greedy = s.greedy ? reinterpret_cast<const uint8_t*>(A + L.greedy) : nullptr;
+  cd.accept_len = reinterpret_cast<int32_t*>(A + L.alen); cd.status = d_status;
+  rc = eagle_tree_accept(&cd, reinterpret_cast<const float*>(A + L.target),
+                         s.draft_probs ? reinterpret_cast<const float*>(A + L.draft) : nullptr,
+                         reinterpret_cast<const int32_t*>(A + L.tokens), reinterpret_cast<const int32_t*>(A + L.tree_parent),
+                         s.uniforms ? reinterpret_cast<const float*>(A + L.uniforms) : nullptr,
+                         reinterpret_cast<int32_t*>(A + L.path), reinterpret_cast<int32_t*>(A + L.bonus), stream_);
+  if (rc != EAGLE_OK) return rc;
+  ok = d2h(s.out, L.out, L.n_q) && d2h(s.accepted_path, L.path, L.n_path) && d2h(s.bonus_token, L.bonus, L.n_b) &&
+       d2h(s.accept_len, L.alen, L.n_b) && d2h(s.status, L.status, 4);
+  return ok ? EAGLE_OK : EAGLE_ERR_LAUNCH;
+}
+
 const char* eagle_status_string(int code) {
   switch (code) {
     case EAGLE_OK: return "ok";

@@ -135,3 +135,26 @@ def test_output_distribution_on_gpu_chi_square(E):
     first = np.where(alen > 0, tokens[np.arange(n), np.maximum(path[:, 0], 0)], bonus)
     pr = p_root.astype(np.float64) / p_root.astype(np.float64).sum()
     assert stats.chisquare(np.bincount(first, minlength=V), pr * n).pvalue > 1e-3
+
+
+def test_host_step_entry_matches_device_calls(E):
+    """eagle_tree_verify_step_host (copies in, attention, acceptance, copies out) gives what the two device calls give."""
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=5, prefix=(50, 900), vocab=3000)
+    attn = W.make_attn_inputs(cfg, salt=3)
+    acc = W.make_accept_inputs(cfg, salt=3, trees=(attn.tree_sizes, attn.tree_parent))
+    d = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    out = E.eagle_tree_verify_attn(attn.q.to(d), attn.k_cache.to(d), attn.v_cache.to(d), attn.seq_lens.to(d),
+                                   attn.tree_parent.to(d), tree_sizes=attn.tree_sizes.to(d), status=status)
+    path, bonus, alen, st = _gpu_accept(E, acc)
+    host = dict(q=attn.q, k_cache=attn.k_cache, v_cache=attn.v_cache, seq_lens=attn.seq_lens, tree_sizes=attn.tree_sizes,
+                tree_parent=attn.tree_parent, target_probs=acc.target_probs, draft_probs=acc.draft_probs,
+                draft_tokens=acc.draft_tokens, uniforms=acc.uniforms, greedy=acc.greedy)
+    runner = E.HostStepRunner({k: v.pin_memory() for k, v in host.items()}, d)
+    for _ in range(2):
+        runner.run()
+        torch.cuda.synchronize()
+        assert int(runner.status.item()) == 0 and st == 0 and int(status.item()) == 0
+        assert torch.equal(runner.out.view(torch.int16), out.cpu().view(torch.int16))
+        assert np.array_equal(runner.accepted_path.numpy(), path) and np.array_equal(runner.bonus_token.numpy(), bonus)
+        assert np.array_equal(runner.accept_len.numpy(), alen)
