@@ -39,9 +39,11 @@ METRIC = "tree_verify_steps_per_s"
 UNIT = "steps/s"
 HBM_FALLBACK_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture summarised in
-# profiles/ (bytes per launch on the named workload); None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu captures summarised in
+# profiles/attn_kernel_serving_mix_b16.md, keyed by (workload, batch); None where no capture exists.
+# Full serving_mix: 1199.8 MB read (measured at full size) + 43 MB written (output + cut-piece partials, scaled from
+# the batch-16 capture); batch 16: 314.3 MB + 17.4 MB.
+NCU_TRAFFIC_BYTES = {("serving_mix", 64): 1_199_820_032 + 43_000_000, ("serving_mix", 16): 314_316_800 + 17_369_344}
 
 
 def measured_hbm_peak():
@@ -302,7 +304,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                 "api": "eagle_tree_verify_step_host", "same_tokens_as_device_path": same_tokens},
         "roofline": {"bound": "hbm", "kernel": "split-KV tree attention", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+                     "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, cfg.batch)),
                      "algorithmic_bytes": alg_bytes, "ms_per_launch": attn_ms,
                      "tflops": alg_flops / (attn_ms * 1e-3) / 1e12},
         "breakdown": {"attn_kernel_ms": attn_ms, "accept_ms": accept_ms, "tokens_per_step": mean_tokens,
