@@ -27,9 +27,15 @@ namespace eagle {
 namespace {
 
 constexpr int kTileN = 128;          // keys per KV tile
-constexpr int kSlots = 5;            // ring slots; tile g uses slot (2g) % 5 for K and (2g+1) % 5 for V
-constexpr int kThreads = 352;
-constexpr int kSoftmaxThreads = 256;
+constexpr int kSlots = 5;            // ring slots; entry n of the load sequence (see the producer) uses slot n % 5
+constexpr int kThreads = 352;          // 8 softmax warps, TMA producer, two MMA issuers
+constexpr int kSoftmaxWarps = 8;
+constexpr int kGroupThreads = 128;     // one softmax group
+constexpr int kWarpProducer = 8, kWarpQK = 9, kWarpPV = 10;
+#ifndef EAGLE_POLY_STRIDE
+#define EAGLE_POLY_STRIDE 4
+#endif
+constexpr int kPolyStride = EAGLE_POLY_STRIDE;   // one pair of exponentials in kPolyStride is evaluated as a polynomial (0: none)
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0;        // S[b] at b*128
 constexpr uint32_t kColO = 256;
@@ -133,6 +139,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t addr, const uint32_t* r) {
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(addr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -151,18 +165,81 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-// 2^x on the FMA / ALU pipes (x <= ~8): split x into an integer n and a fraction f in [-0.5, 0.5] with the
-// add-a-large-constant trick, evaluate a cubic for 2^f (relative error 1e-4, far below the bf16 rounding of P) and put
-// n into the exponent field.  Used for a fraction of the exponentials so that the special-function unit, which takes
-// 8 cycles per warp instruction, is not the only thing the softmax waits for.
-__device__ __forceinline__ float poly_exp2(float x) {
-  const float xc = fmaxf(x, -126.f);
-  const float t = xc + 12582912.f;                    // 1.5 * 2^23: the integer part lands in the low mantissa bits
-  const float f = xc - (t - 12582912.f);
-  float r = fmaf(0.05500841f, f, 0.24220926f);
-  r = fmaf(r, f, 0.69328277f);
-  r = fmaf(r, f, 1.0f);
-  return __uint_as_float(__float_as_uint(r) + (__float_as_uint(t) << 23));   // the constant's own bits shift out
+// Packed pairs of floats (one 64-bit register) and the two-wide FP32 instructions of sm_100: one issue slot does the
+// work of two, which matters because the softmax is bound by instruction issue, not by any single pipe.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for a packed pair on the FMA / ALU pipes (x <= ~8): split x into an integer n and a fraction f in [-0.5, 0.5]
+// with the add-a-large-constant trick, evaluate a cubic for 2^f (relative error 1e-4, far below the bf16 rounding of
+// P) and put n into the exponent field.  Used for a fraction of the exponentials so that the special-function
+// unit, which takes 8 cycles per warp instruction, is not the only thing the softmax waits for.
+__device__ __forceinline__ void poly_exp2_pair(uint64_t x2, float& p0, float& p1) {
+  float a, b;
+  unpack2(x2, a, b);
+  const uint64_t xc2 = pack2(fmaxf(a, -126.f), fmaxf(b, -126.f));
+  const uint64_t t2 = add2(xc2, pack2(12582912.f, 12582912.f));
+  const uint64_t u2 = add2(t2, pack2(-12582912.f, -12582912.f));
+  const uint64_t f2 = fma2(u2, pack2(-1.f, -1.f), xc2);
+  uint64_t r2 = fma2(pack2(0.05500841f, 0.05500841f), f2, pack2(0.24220926f, 0.24220926f));
+  r2 = fma2(r2, f2, pack2(0.69328277f, 0.69328277f));
+  r2 = fma2(r2, f2, pack2(1.0f, 1.0f));
+  float ta, tb, ra, rb;
+  unpack2(t2, ta, tb);
+  unpack2(r2, ra, rb);
+  p0 = __uint_as_float(__float_as_uint(ta) * 0x800000u + __float_as_uint(ra));   // the constant's own bits shift out
+  p1 = __uint_as_float(__float_as_uint(tb) * 0x800000u + __float_as_uint(rb));
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Bounded wait for a tagged word in shared memory (low byte == want); the word is returned through *out.
+__device__ __noinline__ bool tag_wait_slow(volatile uint32_t* slot, uint32_t want, uint32_t* out, volatile int* abort_flag) {
+  const unsigned long long t0 = global_timer();
+  for (uint32_t spins = 1;; ++spins) {
+    const uint32_t t = *slot;
+    if ((t & 0xffu) == want) {
+      *out = t;
+      return true;
+    }
+    if ((spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool tag_wait(volatile uint32_t* slot, uint32_t want, uint32_t* out, volatile int* abort_flag) {
+#pragma unroll 1
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t t = *slot;
+    if ((t & 0xffu) == want) {
+      *out = t;
+      return true;
+    }
+  }
+  return tag_wait_slow(slot, want, out, abort_flag);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -179,8 +256,8 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
 
 #ifdef EAGLE_TRACE
 // Debug builds only: CTA 0 logs (tag, clock) pairs per role; read back with eagle_debug_trace().
-__device__ unsigned long long g_trace[4][1024];
-__device__ int g_trace_n[4];
+__device__ unsigned long long g_trace[5][1024];
+__device__ int g_trace_n[5];
 __device__ long long g_cta_stat[1024][4];   // per CTA: cycles, items, tiles, tail tiles
 #define TRACE(role, tag)                                                                          \
   do {                                                                                            \
@@ -269,9 +346,10 @@ struct Smem {
   static constexpr int kTileBytes = kSlabs * kSlabBytes;     // one Q / K / V tile
   static constexpr int kQ = 0;                               // two query tiles (double buffer)
   static constexpr int kRing = 2 * kTileBytes;
-  static constexpr int kXch = kRing + kSlots * kTileBytes;   // float [2 parities][2 halves][128 rows]: row-max exchange
-  static constexpr int kBar = kXch + 2 * 2 * kBlockM * 4;
-  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 5 + 4;
+  static constexpr int kTag = kRing + kSlots * kTileBytes;   // uint32 [128 rows]: reference maximum | step number
+  static constexpr int kLfin = kTag + kBlockM * 4;           // float [128 rows]: row sums on their way to the epilogue
+  static constexpr int kBar = kLfin + kBlockM * 4;
+  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 5;
   static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag
   static constexpr int kBytes = kMisc + 16;
 };
@@ -280,7 +358,6 @@ struct Bars {
   uint32_t full[kSlots], empty[kSlots];
   uint32_t s_full[2], p_full[2], o_done[2];
   uint32_t q_full[2], q_empty[2], o_free;
-  uint32_t pair[4];   // one per TMEM lane quarter: the two softmax warps that share its rows
 };
 
 template <int D>
@@ -307,7 +384,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     for (int i = 0; i < 2; ++i) { B.q_full[i] = b; b += 8; }
     for (int i = 0; i < 2; ++i) { B.q_empty[i] = b; b += 8; }
     B.o_free = b; b += 8;
-    for (int i = 0; i < 4; ++i) { B.pair[i] = b; b += 8; }
   }
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + S::kMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + S::kMisc + 4);
@@ -319,19 +395,19 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(B.s_full[i], 1);
-      mbar_init(B.p_full[i], kSoftmaxThreads);
+      mbar_init(B.p_full[i], kGroupThreads);
       mbar_init(B.o_done[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(B.q_full[i], p.q_tma ? 1 : kSoftmaxThreads);   // one TMA transaction, or every softmax thread's rows
+      mbar_init(B.q_full[i], p.q_tma ? 1 : kGroupThreads);   // one TMA transaction, or every softmax thread's rows
       mbar_init(B.q_empty[i], 1);
     }
-    mbar_init(B.o_free, kSoftmaxThreads);
-    for (int i = 0; i < 4; ++i) mbar_init(B.pair[i], 64);
+    mbar_init(B.o_free, kGroupThreads);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 9) {
+  if (tid < kBlockM) reinterpret_cast<volatile uint32_t*>(smem + S::kTag)[tid] = 0xffffffffu;   // no step carries this tag yet
+  if (warp == kWarpQK) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + S::kMisc), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -350,49 +426,83 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   const long long trace_t0 = clock64();
 #endif
 
-  if (warp == 8) {
+  if (warp == kWarpProducer) {
     // =========================================================================== TMA producer
+    // Load order: K(0), K(1), then V(g), K(g + 2) for g = 0, 1, ... (g counts this CTA's steps across items): the
+    // order in which the MMAs consume the tiles, since the score MMA runs two steps ahead of the PV MMA.  Entry n
+    // of that sequence lives in slot n % kSlots; with five slots the K tile of step g + 3 can be requested as soon as
+    // the PV of step g - 1 has finished, two steps before it is needed.
     if (lane == 0) {
-      uint32_t g = 0;   // KV tiles issued by this CTA so far
+      struct Cursor {
+        int tp, tile, tile_end, z;
+        bool valid;
+      };
+      // moves to the next KV tile of the work list; on entering an item, fills `it`
+      auto advance = [&](Cursor& c, WorkItem& it) -> bool {   // returns true when a new item was entered
+        if (++c.tile < c.tile_end) return false;
+        for (++c.tp; c.tp < tp_hi; ++c.tp) {
+          it = p.items[2 * c.tp + member];
+          if (it.tile_end > it.tile_begin) {
+            c.tile = it.tile_begin;
+            c.tile_end = it.tile_end;
+            c.z = it.b * p.Hkv + it.g;
+            return true;
+          }
+        }
+        c.valid = false;
+        return false;
+      };
       uint32_t item_count = 0;
       bool ok = true;
-      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
-        const WorkItem it = p.items[2 * tp + member];
-        if (it.tile_end <= it.tile_begin) continue;
-        const int z = it.b * p.Hkv + it.g;
-        TRACE(0, 1);
-        if (p.q_tma) {
+      uint32_t n = 0;   // position in the load sequence
+      auto load_tile = [&](const Cursor& c, bool is_v) {
+        const uint32_t slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
+        ok = mbar_wait(B.empty[slot], par, s_abort);
+        if (!ok) return;
+        TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
+        mbar_expect_tx(B.full[slot], S::kTileBytes);
+#pragma unroll
+        for (int sl = 0; sl < S::kSlabs; ++sl)
+          tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
+                      B.full[slot]);
+      };
+      // K cursor step: the query tile of an item goes out just before the item's first K tile
+      auto k_step = [&](Cursor& ck) {
+        WorkItem it;
+        if (advance(ck, it) && p.q_tma) {
           // query tile: box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
           const uint32_t qb = item_count & 1u;
           ok = mbar_wait(B.q_empty[qb], ((item_count >> 1) & 1u) ^ 1u, s_abort);
-          if (!ok) break;
+          if (!ok) return;
+          TRACE(0, 1);
           mbar_expect_tx(B.q_full[qb], S::kTileBytes);
 #pragma unroll
-          for (int s = 0; s < S::kSlabs; ++s)
-            tma_load_4d(sbase + S::kQ + qb * S::kTileBytes + s * S::kSlabBytes, &map_q, s * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b,
+          for (int sl = 0; sl < S::kSlabs; ++sl)
+            tma_load_4d(sbase + S::kQ + qb * S::kTileBytes + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b,
                         B.q_full[qb]);
+          ++item_count;
         }
-        for (int tile = it.tile_begin; tile < it.tile_end && ok; ++tile, ++g) {
-#pragma unroll
-          for (int kv = 0; kv < 2; ++kv) {
-            const uint32_t n = 2 * g + kv, slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
-            ok = mbar_wait(B.empty[slot], par, s_abort);
-            if (!ok) break;
-            TRACE(0, ((2 + kv) << 10) | (g & 1023u));
-            mbar_expect_tx(B.full[slot], S::kTileBytes);
-#pragma unroll
-            for (int s = 0; s < S::kSlabs; ++s)
-              tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + s * S::kSlabBytes, kv ? &map_v : &map_k, s * 64, tile * kTileN, z,
-                          B.full[slot]);
-          }
-        }
-        ++item_count;
+        if (ck.valid && ok) load_tile(ck, false);
+      };
+      Cursor ck = {tp_lo - 1, 0, 0, 0, true}, cv = {tp_lo - 1, 0, 0, 0, true};
+      WorkItem unused;
+      k_step(ck);                 // K(0)
+      ++n;
+      if (ok && ck.valid) k_step(ck);   // K(1)
+      ++n;
+      advance(cv, unused);
+      while (ok && cv.valid) {
+        load_tile(cv, true);      // V(g)
+        ++n;
+        advance(cv, unused);
+        if (ok && ck.valid) k_step(ck);   // K(g + 2)
+        ++n;
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == kWarpQK) {
     // =========================================================================== QK issuer
-    // Ring item n = 2*tile (+1 for V) lives in slot n % 6 with phase parity (n / 6) & 1.  Positions are kept as
-    // running counters (no divisions on the threads that keep the tensor pipe fed).
+    // Entry n of the load sequence lives in slot n % kSlots with phase parity (n / kSlots) & 1.  Positions are kept
+    // as running counters (no divisions on the threads that keep the tensor pipe fed).
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(kBlockM, kTileN, false);
       uint32_t ks = 0, kp = 0;       // slot / parity of the K tile of the next QK
@@ -417,6 +527,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             ok = mbar_wait(B.p_full[gq & 1u], ((gq - 2) >> 1) & 1u, s_abort);
             if (!ok) break;
           }
+          TRACE(1, (9 << 10) | (gq & 1023u));
           ok = mbar_wait(B.full[ks], kp, s_abort);
           if (!ok) break;
           TRACE(1, (10 << 10) | (gq & 1023u));
@@ -424,7 +535,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           issue_qk_tile<D>(tmem + kColS + (gq & 1u) * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
           tc_commit(B.s_full[gq & 1u]);
           tc_commit(B.empty[ks]);
-          ks += 2;
+          ks += gq == 0 ? 1u : 2u;   // K(g) is entry g for g < 2, entry 2g - 1 after that
           if (ks >= kSlots) { ks -= kSlots; kp ^= 1u; }
           if (s == steps - 1) tc_commit(B.q_empty[qb]);      // every QK of this item has been issued
           TRACE(1, (11 << 10) | (gq & 1023u));
@@ -432,11 +543,11 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         ++item_count;
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == kWarpPV) {
     // =========================================================================== PV issuer
     if (lane == 0) {
       constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, true);
-      uint32_t vs = 1, vp = 0;       // slot / parity of the V tile of the next PV
+      uint32_t vs = 2, vp = 0;       // slot / parity of the V tile of the next PV: V(g) is entry 2g + 2
       uint32_t gp = 0;               // steps issued so far (all items)
       uint32_t item_count = 0;
       const uint32_t ring_lo_v = desc_lo(sbase + S::kRing, S::kSlabBytes);
@@ -468,192 +579,145 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         ++item_count;
       }
     }
-  } else {
+  } else if (warp < kSoftmaxWarps) {
     // =========================================================================== softmax + epilogue (warps 0-7)
-    const int h = warp >> 2;                              // which 64-column half of the score row this thread owns
+    // Two groups of four warps; group g takes the steps whose global number is g mod 2 and owns S[g] / P[g], so the
+    // groups run half a step out of phase and each scheduler hosts one warp of either: while one waits on tensor
+    // memory or a barrier, the other computes.  Thread r of a group owns query row r (= TMEM lane r), all 128 score
+    // columns.  The two threads of a row share one reference maximum: the thread that handled step gs publishes it,
+    // tagged with gs, and the other picks it up before it takes its exponentials of step gs + 1.  Each keeps its own
+    // part of the row sum, relative to that reference.
+    const int grp = warp >> 2;                            // also the S / P buffer of this group
     const int r = tid & (kBlockM - 1);                    // query row within the tile == TMEM lane
+    const uint32_t buf = static_cast<uint32_t>(grp);
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    // Hardware barrier shared with the partner warp.  Both warps of a pair run the same control flow on the same
-    // mbarriers, so they always reach it together: a warp leaves its loop only when a wait failed, and a wait that
-    // fails for one of them (the barrier never completes) fails for the other too.
-    const uint32_t pair_id = 1u + static_cast<uint32_t>(warp & 3);
-    auto pair_sync = [&]() -> bool {
-      asm volatile("bar.sync %0, 64;" ::"r"(pair_id) : "memory");
-      return true;
-    };
-    float* xch = reinterpret_cast<float*>(smem + S::kXch);
-    constexpr int HC = D / 2;                             // this thread's half of the accumulator columns
+    volatile uint32_t* tag = reinterpret_cast<volatile uint32_t*>(smem + S::kTag) + r;   // reference | step, per row
+    volatile float* lfin = reinterpret_cast<volatile float*>(smem + S::kLfin) + r;       // row sum on its way to the epilogue
+    const uint32_t s_addr = tmem + lane_addr + kColS + buf * kTileN;
+    const uint32_t p_addr = tmem + lane_addr + kColP + buf * (kTileN / 2);
+    const uint32_t o_addr = tmem + lane_addr + kColO;
 
-    // What the epilogue of an item needs after its last softmax step.
-    struct Done {
-      bool live, row_valid;
-      int slot;
-      uint32_t last_step;      // global number of the item's last step
-      float m_ref, l_sum;
-      __nv_bfloat16* out_row;  // this thread's half of its output row
-    };
-    Done prev;
-    prev.live = false;
-    // Wait for the item's last PV (PVs complete in order), add the two halves of the row sum, then write this
-    // thread's half of the columns of its row: bf16 output, or the unnormalised fp32 partial of a cut unit.
-    auto epilogue = [&](const Done& d) -> bool {
-      if (!mbar_wait_warp(B.o_done[d.last_step & 1u], (d.last_step >> 1) & 1u, s_abort)) return false;
-      if (tid == 0) TRACE(2, 20);
-      tc_fence_after();
-      float* lx = xch;   // [half][row]; the surrounding pair syncs keep it apart from the row-max exchanges
-      if (!pair_sync()) return false;
-      lx[h * kBlockM + r] = d.l_sum;
-      if (!pair_sync()) return false;
-      const float l_row = d.l_sum + lx[(h ^ 1) * kBlockM + r];
-      const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-      float* part_row = d.slot >= 0 ? p.part_o + (static_cast<size_t>(d.slot) * kBlockM + r) * D + h * HC : nullptr;
-      uint32_t o[32];
-#pragma unroll
-      for (int c = 0; c < HC / 32; ++c) {
-        tmem_ld32(tmem + lane_addr + kColO + h * HC + c * 32, o);
-        tc_wait_ld();
-        if (d.row_valid) {
-          if (d.slot < 0) {
-#pragma unroll
-            for (int e = 0; e < 32; e += 8) {
-              uint4 v;
-              v.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
-              v.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-              v.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-              v.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-              *reinterpret_cast<uint4*>(d.out_row + c * 32 + e) = v;
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<uint4*>(part_row + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
-          }
-        }
-      }
-      if (d.row_valid && d.slot >= 0 && h == 0) p.part_ml[static_cast<size_t>(d.slot) * kBlockM + r] = make_float2(d.m_ref, l_row);
-      if (!pair_sync()) return false;   // the partner has read the exchanged sum
-      tc_fence_before();
-      mbar_arrive(B.o_free);            // the next item's first PV may overwrite the accumulator
-      if (tid == 0) TRACE(2, 21);
-      return true;
-    };
-
-    uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps done so far
+    uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps before the current item
     bool ok = true;
-    // one pass per item, plus a last pass without steps that only writes the final item's output
-    for (int tp = tp_lo; tp <= tp_hi && ok; ++tp) {
-      const bool drain = tp == tp_hi;
-      if (drain && !prev.live) break;                       // nothing was processed
-      WorkItem it = WorkItem();
-      if (!drain) {
-        it = p.items[2 * tp + member];
-        if (it.tile_end <= it.tile_begin) continue;
-      }
-      const SeqPlan sp = drain ? SeqPlan() : p.seq[it.b];
+    for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
+      const WorkItem it = p.items[2 * tp + member];
+      if (it.tile_end <= it.tile_begin) continue;
+      const SeqPlan sp = p.seq[it.b];
       const int L = sp.L, n = sp.n, G = p.G;
       const int m_valid = n * G, kv_end = L + n;
-      const int steps = drain ? 0 : it.tile_end - it.tile_begin;
+      const int steps = it.tile_end - it.tile_begin;
       const int R = it.mt * kBlockM + r;
       const bool row_valid = R < m_valid;
       const int node = row_valid ? R / G : 0, hh = row_valid ? R % G : 0;
       const uint64_t anc = row_valid ? p.anc[static_cast<size_t>(it.b) * p.T_max + node] : 0ull;
 
-      if (!p.q_tma && !drain) {
-        // group sizes that do not divide 128: the softmax threads stage the query tile themselves;
-        // thread (h, r) writes the h-th 64-column slab of row r (D = 64: h = 0 only)
+      if (!p.q_tma && grp == 0) {
+        // group sizes that do not divide 128: the first softmax group stages the query tile itself, a row per thread
         const uint32_t qb = item_count & 1u;
         ok = mbar_wait_warp(B.q_empty[qb], ((item_count >> 1) & 1u) ^ 1u, s_abort);
         if (!ok) break;
-        if (h < S::kSlabs) {
-          const uint4* src = reinterpret_cast<const uint4*>(
-              p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * 64);
-          unsigned char* qdst = smem + S::kQ + qb * S::kTileBytes + h * S::kSlabBytes + r * 128;
+        const uint4* src = reinterpret_cast<const uint4*>(p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D);
+        unsigned char* qdst = smem + S::kQ + qb * S::kTileBytes + r * 128;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(qdst + ((c ^ (r & 7)) << 4)) = v;
-          }
+        for (int c = 0; c < 8 * S::kSlabs; ++c) {
+          const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(qdst + (c >> 3) * S::kSlabBytes + (((c & 7) ^ (r & 7)) << 4)) = v;
         }
         fence_proxy_async();
         mbar_arrive(B.q_full[qb]);
       }
-      if (tid == 0) TRACE(2, 3);
+      if ((tid & 127) == 0) TRACE(2 + 2 * grp, 3);
 
-      float m_ref = -INFINITY;   // reference max (scaled, log2 domain) of every exponential taken so far
-      float l_sum = 0.f;         // this thread's half of the row sum
-      for (int s = 0; s < steps + (drain ? 1 : 0) && ok; ++s) {
-        if (!drain) {
-        const uint32_t gs = sg + s, buf = gs & 1u;
+      float m_ref = -INFINITY;   // reference (scaled, log2 domain) this thread's row sum is relative to
+      float m_in = -INFINITY;    // reference the other group left behind at the step before this group's latest one
+      float l_sum = 0.f;         // this thread's part of the row sum
+      // this group's steps of the item: those whose global number has the group's parity
+      for (int s = static_cast<int>((sg ^ buf) & 1u); s < steps; s += 2) {
+        const uint32_t gs = sg + s;
         ok = mbar_wait_warp(B.s_full[buf], (gs >> 1) & 1u, s_abort);
         if (!ok) break;
-        if (tid == 0) TRACE(2, (10 << 10) | (gs & 1023u));
+        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (10 << 10) | (gs & 1023u));
         tc_fence_after();
-        uint32_t raw[64];
-        tmem_ld32(tmem + lane_addr + kColS + buf * kTileN + h * 64, raw);
-        tmem_ld32(tmem + lane_addr + kColS + buf * kTileN + h * 64 + 32, raw + 32);
-        tc_wait_ld();
-        if (tid == 0) TRACE(2, (15 << 10) | (gs & 1023u));
         const int key0 = (it.tile_begin + s) * kTileN;
-        if (key0 + kTileN > L) {          // the tile reaches past the committed prefix: tree mask + cache tail
-          // visibility of this thread's 64 keys as one 64-bit word: keys before L are all visible, key L + m is
-          // visible iff bit m of the node's ancestor mask is set (the mask has no bits at or above the tree size)
-          const int rel = key0 + h * 64 - L;          // tree index of this thread's first key (negative: still in the prefix)
-          uint64_t vis;
-          if (rel >= 64) vis = 0ull;
-          else if (rel >= 0) vis = anc >> rel;
-          else if (rel > -64) vis = (anc << (-rel)) | ((1ull << (-rel)) - 1ull);
-          else vis = ~0ull;
-          const uint32_t vlo = static_cast<uint32_t>(vis), vhi = static_cast<uint32_t>(vis >> 32);
+        // visibility of this row's 128 keys, 32 per word: keys before L are all visible, key L + m is visible iff
+        // bit m of the node's ancestor mask is set (the mask has no bits at or above the tree size)
+        const bool tail = key0 + kTileN > L;          // the tile reaches past the committed prefix
+        uint32_t vm[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+        if (tail) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            raw[e] = (vlo >> e) & 1u ? raw[e] : 0xff800000u;            // -inf
-            raw[32 + e] = (vhi >> e) & 1u ? raw[32 + e] : 0xff800000u;
+          for (int c = 0; c < 4; ++c) {
+            const int rel = key0 + c * 32 - L;        // tree index of the word's first key (negative: still in the prefix)
+            uint32_t w;
+            if (rel >= 64) w = 0u;
+            else if (rel >= 0) w = static_cast<uint32_t>(anc >> rel);
+            else if (rel > -32) w = static_cast<uint32_t>(anc << (-rel)) | ((1u << (-rel)) - 1u);
+            else w = 0xffffffffu;
+            vm[c] = w;
           }
         }
+        // ---- pass 1: row maximum of the raw scores; the last two chunks stay in registers for pass 2
+        uint32_t ra[32], rb[32];
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int e = 0; e < 64; e += 4) {
-          mx[0] = fmaxf(mx[0], __uint_as_float(raw[e]));
-          mx[1] = fmaxf(mx[1], __uint_as_float(raw[e + 1]));
-          mx[2] = fmaxf(mx[2], __uint_as_float(raw[e + 2]));
-          mx[3] = fmaxf(mx[3], __uint_as_float(raw[e + 3]));
+        for (int c = 0; c < 4; c += 2) {
+          tmem_ld32(s_addr + c * 32, ra);
+          tmem_ld32(s_addr + c * 32 + 32, rb);
+          tc_wait_ld();
+          if (tail) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              ra[e] = (vm[c] >> e) & 1u ? ra[e] : 0xff800000u;       // -inf
+              rb[e] = (vm[c + 1] >> e) & 1u ? rb[e] : 0xff800000u;
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 4) {
+            mx[0] = max3(mx[0], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            mx[1] = max3(mx[1], __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
+            mx[2] = max3(mx[2], __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+            mx[3] = max3(mx[3], __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
+          }
         }
-        const float half_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        // agree on the row max with the partner thread (other half of the row, same lane, warp +-4)
-        xch[(buf * 2 + h) * kBlockM + r] = half_max;
-        if (tid == 0) TRACE(2, (12 << 10) | (gs & 1023u));
-        ok = pair_sync();
-        if (!ok) break;
-        const float tmax = fmaxf(half_max, xch[(buf * 2 + (h ^ 1)) * kBlockM + r]) * p.scale_log2;   // scale > 0
+        const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // scale > 0
+        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (12 << 10) | (gs & 1023u));
 
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
-          const uint32_t nv = 2 * (g_base + s) + 1, slot = nv % kSlots, par = (nv / kSlots) & 1u;
+          const uint32_t nv = 2 * (g_base + s) + 2, slot = nv % kSlots, par = (nv / kSlots) & 1u;
           ok = mbar_wait_warp(B.full[slot], par, s_abort);
           if (!ok) break;
-          if (key0 + r >= kv_end && h < S::kSlabs) {
+          if (key0 + r >= kv_end) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-              *reinterpret_cast<uint4*>(smem + S::kRing + slot * S::kTileBytes + h * S::kSlabBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+            for (int c = 0; c < 8 * S::kSlabs; ++c)
+              *reinterpret_cast<uint4*>(smem + S::kRing + slot * S::kTileBytes + (c >> 3) * S::kSlabBytes + r * 128 + (c & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
           fence_proxy_async();
         }
 
-        if (tid == 0) TRACE(2, (13 << 10) | (gs & 1023u));
-        // P[buf] was last read by the PV of step gs - 2 (this wait also keeps every thread within one phase of o_done)
-        if (gs >= 2) {
-          ok = mbar_wait_warp(B.o_done[buf], ((gs - 2) >> 1) & 1u, s_abort);
+        // the reference the other group settled on at the previous step (waited for at an item's first step too,
+        // where its value is not used: the other group must have read the tag of step gs - 2 before it is replaced)
+        float m_prev = -INFINITY;
+        if (gs > 0) {
+          uint32_t t = 0xff800000u;
+          ok = __all_sync(0xffffffffu, tag_wait(tag, (gs - 1u) & 0xffu, &t, s_abort));
           if (!ok) break;
+          if (s > 0) m_prev = __uint_as_float(t & 0xffffff00u);
         }
-        if (tid == 0) TRACE(2, (17 << 10) | (gs & 1023u));
+        if (m_prev != m_ref) {
+          l_sum *= fast_exp2(m_ref - m_prev);     // m_ref = -inf: nothing summed yet, the factor is 0
+          m_ref = m_prev;
+        }
+        m_in = m_prev;
         // lazy rescale: move the reference only when the row max outgrows it by more than the threshold
         const bool grow = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         float factor = 1.f;
         if (grow) {
-          factor = fast_exp2(m_ref - tmax);     // 0 when there was no reference yet
-          m_ref = tmax;
+          const float m_new = __uint_as_float(__float_as_uint(tmax) & 0xffffff00u);   // the low byte carries the step tag
+          factor = fast_exp2(m_ref - m_new);     // 0 when there was no reference yet
+          m_ref = m_new;
           l_sum *= factor;
         }
+        *tag = __float_as_uint(m_ref) | (gs & 0xffu);
         if (s > 0 && __any_sync(0xffffffffu, grow)) {
           // the previous step accumulated into O and may still be running
           ok = mbar_wait_warp(B.o_done[buf ^ 1u], ((gs - 1) >> 1) & 1u, s_abort);
@@ -661,53 +725,126 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           tc_fence_after();
           uint32_t o[32];
 #pragma unroll 1
-          for (int c = 0; c < HC / 32; ++c) {
-            const uint32_t o_addr = tmem + lane_addr + kColO + h * HC + c * 32;
-            tmem_ld32(o_addr, o);
+          for (int c = 0; c < D / 32; ++c) {
+            tmem_ld32(o_addr + c * 32, o);
             tc_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-            tmem_st32(o_addr, o);
+            tmem_st32(o_addr + c * 32, o);
           }
           tc_wait_st();
         }
-        if (tid == 0) TRACE(2, (16 << 10) | (gs & 1023u));
-        const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
-        float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(raw[2 * e]), p.scale_log2, neg_base));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 1]), p.scale_log2, neg_base));
-          const float p2 = fast_exp2(fmaf(__uint_as_float(raw[2 * e + 2]), p.scale_log2, neg_base));
-          const float p3 = poly_exp2(fmaf(__uint_as_float(raw[2 * e + 3]), p.scale_log2, neg_base));
-          ls[0] += p0; ls[1] += p1; ls[2] += p2; ls[3] += p3;
-          raw[e] = pack_bf16(p0, p1);          // packed P overwrites entries already consumed
-          raw[e + 1] = pack_bf16(p2, p3);
+        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (13 << 10) | (gs & 1023u));
+        // P[buf] was last read by the PV of step gs - 2 (this wait also keeps every thread within one phase of o_done)
+        if (gs >= 2) {
+          ok = mbar_wait_warp(B.o_done[buf], ((gs - 2) >> 1) & 1u, s_abort);
+          if (!ok) break;
         }
-        l_sum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-        if (tid == 0) TRACE(2, (14 << 10) | (gs & 1023u));
-        tmem_st32(tmem + lane_addr + kColP + buf * (kTileN / 2) + h * 32, raw);   // this thread's 64 P values
+        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (16 << 10) | (gs & 1023u));
+        // ---- pass 2: exponentials and packed P.  Chunks 2 and 3 are still in registers; chunks 0 and 1 are
+        // fetched again while those are being worked on.
+        const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
+        const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), base2 = pack2(neg_base, neg_base);
+        uint64_t ls2[2] = {0ull, 0ull};   // four partial sums
+        uint32_t pk[16];
+        auto exp_chunk = [&](const uint32_t* raw, int c) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint64_t x2 = fma2(pack2(__uint_as_float(raw[2 * j]), __uint_as_float(raw[2 * j + 1])), scale2, base2);
+            float p0, p1;
+            if (kPolyStride > 0 && j % (kPolyStride > 0 ? kPolyStride : 1) == (kPolyStride > 0 ? kPolyStride : 1) - 1) {
+              poly_exp2_pair(x2, p0, p1);
+            } else {
+              float a, b;
+              unpack2(x2, a, b);
+              p0 = fast_exp2(a);
+              p1 = fast_exp2(b);
+            }
+            ls2[j & 1] = add2(ls2[j & 1], pack2(p0, p1));
+            pk[j] = pack_bf16(p0, p1);
+          }
+          tmem_st16(p_addr + c * 16, pk);
+        };
+        exp_chunk(ra, 2);
+        tmem_ld32(s_addr, ra);              // chunk 0, in flight while chunk 3 is worked on
+        exp_chunk(rb, 3);
+        tmem_ld32(s_addr + 32, rb);         // chunk 1
+        tc_wait_ld();
+        if (tail) {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            ra[e] = (vm[0] >> e) & 1u ? ra[e] : 0xff800000u;
+            rb[e] = (vm[1] >> e) & 1u ? rb[e] : 0xff800000u;
+          }
+        }
+        exp_chunk(ra, 0);
+        exp_chunk(rb, 1);
+        {
+          float l0, l1, l2, l3;
+          unpack2(ls2[0], l0, l1);
+          unpack2(ls2[1], l2, l3);
+          l_sum += (l0 + l1) + (l2 + l3);
+        }
+        if (s == steps - 2) {
+          // this group's last step of the item, but not the item's: hand the row sum to the group that writes the
+          // output.  A two-step item is the one case where the slot may still be in use for the previous item.
+          if (s == 0 && item_count > 0) {
+            ok = mbar_wait_warp(B.o_free, (item_count - 1) & 1u, s_abort);
+            if (!ok) break;
+          }
+          *lfin = l_sum;
+        }
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(B.p_full[buf]);
-        if (tid == 0) TRACE(2, (11 << 10) | (gs & 1023u));
-        }
+        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (11 << 10) | (gs & 1023u));
 
-        // the finished item's output is written after the first step of this one: its last PV has had time
-        // to complete, and this item's second score tile is being computed meanwhile
-        if (s == 0 && prev.live) {
-          ok = epilogue(prev);
-          prev.live = false;
+        if (s == steps - 1) {
+          // ---- this group took the item's last step: it writes the item's output.  Wait for the last PV (PVs
+          // complete in order), add the other group's part of the row sum, then write the row: bf16 output, or
+          // the unnormalised fp32 partial of a cut piece.
+          ok = mbar_wait_warp(B.o_done[buf], (gs >> 1) & 1u, s_abort);
+          if (!ok) break;
+          if ((tid & 127) == 0) TRACE(2 + 2 * grp, 20);
+          tc_fence_after();
+          float l_row = l_sum;
+          if (steps > 1) {
+            // the other group's sum is relative to the reference it last saw
+            const float w = m_in == m_ref ? 1.f : fast_exp2(m_in - m_ref);
+            l_row = fmaf(*lfin, w, l_row);
+          }
+          const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+          uint32_t o[32];
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            tmem_ld32(o_addr + c * 32, o);
+            tc_wait_ld();
+            if (row_valid) {
+              if (it.slot < 0) {
+                __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D;
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                  uint4 v;
+                  v.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
+                  v.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+                  v.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+                  v.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
+                  *reinterpret_cast<uint4*>(out_row + c * 32 + e) = v;
+                }
+              } else {
+                float* part_row = p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D;
+#pragma unroll
+                for (int e = 0; e < 32; e += 4)
+                  *reinterpret_cast<uint4*>(part_row + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+              }
+            }
+          }
+          if (row_valid && it.slot >= 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_ref, l_row);
+          tc_fence_before();
+          mbar_arrive(B.o_free);            // the next item's first PV may overwrite the accumulator
+          if ((tid & 127) == 0) TRACE(2 + 2 * grp, 21);
         }
       }
-      if (!ok || drain) break;
-      prev.live = true;
-      prev.row_valid = row_valid;
-      prev.slot = it.slot;
-      prev.last_step = sg + steps - 1;
-      prev.m_ref = m_ref;
-      prev.l_sum = l_sum;
-      prev.out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D + h * HC;
       g_base += steps;
       sg += steps;
       ++item_count;
@@ -737,7 +874,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 #ifdef EAGLE_TRACE
   if (tid == 0) g_cta_stat[blockIdx.x][0] = clock64() - trace_t0;
 #endif
-  if (warp == 9) {
+  if (warp == kWarpQK) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
@@ -796,10 +933,10 @@ extern "C" int eagle_debug_cta_stat(long long* dst) {
   return 0;
 }
 extern "C" int eagle_debug_trace(unsigned long long* dst, int* counts) {
-  int zero[4] = {0, 0, 0, 0};
+  int zero[5] = {0, 0, 0, 0, 0};
   cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(dst, eagle::g_trace, sizeof(unsigned long long) * 4 * 1024);
-  cudaMemcpyFromSymbol(counts, eagle::g_trace_n, sizeof(int) * 4);
+  cudaMemcpyFromSymbol(dst, eagle::g_trace, sizeof(unsigned long long) * 5 * 1024);
+  cudaMemcpyFromSymbol(counts, eagle::g_trace_n, sizeof(int) * 5);
   cudaMemcpyToSymbol(eagle::g_trace_n, zero, sizeof(zero));
   return 0;
 }
