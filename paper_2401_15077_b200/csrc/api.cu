@@ -12,6 +12,17 @@ namespace eagle {
 
 namespace {
 
+// Planner cost model, in KV-tile positions: what starting an item costs the attention kernel (pipeline fill, output
+// write), and how close to a super-unit's edge a share boundary snaps to the edge.
+#ifndef EAGLE_ITEM_OVERHEAD
+#define EAGLE_ITEM_OVERHEAD 8
+#endif
+#ifndef EAGLE_SNAP_TILES
+#define EAGLE_SNAP_TILES 2
+#endif
+constexpr int kPlanItemOverheadTiles = EAGLE_ITEM_OVERHEAD;
+constexpr int kPlanSnapTiles = EAGLE_SNAP_TILES;
+
 std::atomic<uint64_t> g_launches{0};
 
 struct DeviceInfo {
@@ -101,8 +112,8 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.tile_keys = attn_tile_keys();
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
-  pp.snap_tiles = 2;
-  pp.item_overhead_tiles = 4;
+  pp.snap_tiles = kPlanSnapTiles;
+  pp.item_overhead_tiles = kPlanItemOverheadTiles;
   pp.unit_cap = w.unit_cap;
   pp.item_cap = w.item_cap;
   pp.slot_cap = w.slot_cap;
@@ -295,8 +306,8 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   pp.tile_keys = attn_tile_keys();
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
-  pp.snap_tiles = 2;
-  pp.item_overhead_tiles = 4;
+  pp.snap_tiles = kPlanSnapTiles;
+  pp.item_overhead_tiles = kPlanItemOverheadTiles;
   pp.unit_cap = w.unit_cap;
   pp.item_cap = w.item_cap;
   pp.slot_cap = w.slot_cap;

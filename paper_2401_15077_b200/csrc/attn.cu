@@ -27,19 +27,19 @@ namespace eagle {
 namespace {
 
 constexpr int kTileN = 128;          // keys per KV tile
-constexpr int kSlots = 5;            // ring slots; entry n of the load sequence (see the producer) uses slot n % 5
-constexpr int kThreads = 352;          // 8 softmax warps, TMA producer, two MMA issuers
+constexpr int kSlots = 6;            // ring slots; entry n of the load sequence (see the producer) uses slot n % 6
+constexpr int kSBufs = 3;            // score buffers in tensor memory; step g uses buffer g % 3
+constexpr int kThreads = 384;          // 8 softmax warps, K/V producer, two MMA issuers, Q producer
 constexpr int kSoftmaxWarps = 8;
 constexpr int kGroupThreads = 128;     // one softmax group
-constexpr int kWarpProducer = 8, kWarpQK = 9, kWarpPV = 10;
+constexpr int kWarpProducer = 8, kWarpQK = 9, kWarpPV = 10, kWarpQ = 11;
 #ifndef EAGLE_POLY_STRIDE
-#define EAGLE_POLY_STRIDE 4
+#define EAGLE_POLY_STRIDE 2
 #endif
 constexpr int kPolyStride = EAGLE_POLY_STRIDE;   // one pair of exponentials in kPolyStride is evaluated as a polynomial (0: none)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;        // S[b] at b*128
-constexpr uint32_t kColO = 256;
-constexpr uint32_t kColP = 384;      // P[b] (packed bf16: 64 columns) at 384 + b*64
+constexpr uint32_t kColS = 0;        // S[b] at b*128; P[b] (packed bf16, 64 columns) overwrites the front of S[b]
+constexpr uint32_t kColO = 384;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -344,20 +344,20 @@ struct Smem {
   static constexpr int kSlabs = D / 64;                     // 64 bf16 = one 128-byte swizzled row
   static constexpr int kSlabBytes = kTileN * 128;            // 128 rows x 128 bytes
   static constexpr int kTileBytes = kSlabs * kSlabBytes;     // one Q / K / V tile
-  static constexpr int kQ = 0;                               // two query tiles (double buffer)
-  static constexpr int kRing = 2 * kTileBytes;
+  static constexpr int kQ = 0;                               // the query tile of the current item
+  static constexpr int kRing = kTileBytes;
   static constexpr int kTag = kRing + kSlots * kTileBytes;   // uint32 [128 rows]: reference maximum | step number
   static constexpr int kLfin = kTag + kBlockM * 4;           // float [128 rows]: row sums on their way to the epilogue
   static constexpr int kBar = kLfin + kBlockM * 4;
-  static constexpr int kNumBars = 2 * kSlots + 2 + 2 + 2 + 5;
+  static constexpr int kNumBars = 2 * kSlots + 3 * kSBufs + 3;
   static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag
   static constexpr int kBytes = kMisc + 16;
 };
 
 struct Bars {
   uint32_t full[kSlots], empty[kSlots];
-  uint32_t s_full[2], p_full[2], o_done[2];
-  uint32_t q_full[2], q_empty[2], o_free;
+  uint32_t s_full[kSBufs], p_full[kSBufs], o_done[kSBufs];
+  uint32_t q_full, q_empty, o_free;
 };
 
 template <int D>
@@ -378,11 +378,11 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     uint32_t b = sbase + S::kBar;
     for (int i = 0; i < kSlots; ++i) { B.full[i] = b; b += 8; }
     for (int i = 0; i < kSlots; ++i) { B.empty[i] = b; b += 8; }
-    for (int i = 0; i < 2; ++i) { B.s_full[i] = b; b += 8; }
-    for (int i = 0; i < 2; ++i) { B.p_full[i] = b; b += 8; }
-    for (int i = 0; i < 2; ++i) { B.o_done[i] = b; b += 8; }
-    for (int i = 0; i < 2; ++i) { B.q_full[i] = b; b += 8; }
-    for (int i = 0; i < 2; ++i) { B.q_empty[i] = b; b += 8; }
+    for (int i = 0; i < kSBufs; ++i) { B.s_full[i] = b; b += 8; }
+    for (int i = 0; i < kSBufs; ++i) { B.p_full[i] = b; b += 8; }
+    for (int i = 0; i < kSBufs; ++i) { B.o_done[i] = b; b += 8; }
+    B.q_full = b; b += 8;
+    B.q_empty = b; b += 8;
     B.o_free = b; b += 8;
   }
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + S::kMisc);
@@ -393,15 +393,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       mbar_init(B.full[i], 1);
       mbar_init(B.empty[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kSBufs; ++i) {
       mbar_init(B.s_full[i], 1);
       mbar_init(B.p_full[i], kGroupThreads);
       mbar_init(B.o_done[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(B.q_full[i], p.q_tma ? 1 : kGroupThreads);   // one TMA transaction, or every softmax thread's rows
-      mbar_init(B.q_empty[i], 1);
-    }
+    mbar_init(B.q_full, p.q_tma ? 1 : kGroupThreads);   // one TMA transaction, or every thread of the first softmax group
+    mbar_init(B.q_empty, 1);
     mbar_init(B.o_free, kGroupThreads);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -428,31 +426,28 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 
   if (warp == kWarpProducer) {
     // =========================================================================== TMA producer
-    // Load order: K(0), K(1), then V(g), K(g + 2) for g = 0, 1, ... (g counts this CTA's steps across items): the
-    // order in which the MMAs consume the tiles, since the score MMA runs two steps ahead of the PV MMA.  Entry n
-    // of that sequence lives in slot n % kSlots; with five slots the K tile of step g + 3 can be requested as soon as
-    // the PV of step g - 1 has finished, two steps before it is needed.
+    // Load order: K(0), K(1), K(2), then V(g), K(g + 3) for g = 0, 1, ... (g counts this CTA's steps across items):
+    // the order in which the MMAs consume the tiles, since the score MMA runs three steps ahead of the PV MMA.
+    // Entry n of that sequence lives in slot n % kSlots; with six slots the K tile of step g + 3 is requested when the
+    // score MMA of step g has finished and the V tile of step g when the PV of step g - 3 has.
     if (lane == 0) {
       struct Cursor {
         int tp, tile, tile_end, z;
         bool valid;
       };
-      // moves to the next KV tile of the work list; on entering an item, fills `it`
-      auto advance = [&](Cursor& c, WorkItem& it) -> bool {   // returns true when a new item was entered
-        if (++c.tile < c.tile_end) return false;
+      auto advance = [&](Cursor& c) {   // moves to the next KV tile of the work list
+        if (++c.tile < c.tile_end) return;
         for (++c.tp; c.tp < tp_hi; ++c.tp) {
-          it = p.items[2 * c.tp + member];
+          const WorkItem it = p.items[2 * c.tp + member];
           if (it.tile_end > it.tile_begin) {
             c.tile = it.tile_begin;
             c.tile_end = it.tile_end;
             c.z = it.b * p.Hkv + it.g;
-            return true;
+            return;
           }
         }
         c.valid = false;
-        return false;
       };
-      uint32_t item_count = 0;
       bool ok = true;
       uint32_t n = 0;   // position in the load sequence
       auto load_tile = [&](const Cursor& c, bool is_v) {
@@ -466,37 +461,44 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
                       B.full[slot]);
       };
-      // K cursor step: the query tile of an item goes out just before the item's first K tile
-      auto k_step = [&](Cursor& ck) {
-        WorkItem it;
-        if (advance(ck, it) && p.q_tma) {
-          // query tile: box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
-          const uint32_t qb = item_count & 1u;
-          ok = mbar_wait(B.q_empty[qb], ((item_count >> 1) & 1u) ^ 1u, s_abort);
-          if (!ok) return;
-          TRACE(0, 1);
-          mbar_expect_tx(B.q_full[qb], S::kTileBytes);
-#pragma unroll
-          for (int sl = 0; sl < S::kSlabs; ++sl)
-            tma_load_4d(sbase + S::kQ + qb * S::kTileBytes + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b,
-                        B.q_full[qb]);
-          ++item_count;
-        }
-        if (ck.valid && ok) load_tile(ck, false);
-      };
       Cursor ck = {tp_lo - 1, 0, 0, 0, true}, cv = {tp_lo - 1, 0, 0, 0, true};
-      WorkItem unused;
-      k_step(ck);                 // K(0)
-      ++n;
-      if (ok && ck.valid) k_step(ck);   // K(1)
-      ++n;
-      advance(cv, unused);
+      advance(ck);
+      advance(cv);
+      for (int i = 0; i < 3; ++i, ++n) {   // K(0), K(1), K(2)
+        if (ok && ck.valid) {
+          load_tile(ck, false);
+          advance(ck);
+        }
+      }
       while (ok && cv.valid) {
         load_tile(cv, true);      // V(g)
         ++n;
-        advance(cv, unused);
-        if (ok && ck.valid) k_step(ck);   // K(g + 2)
+        advance(cv);
+        if (ok && ck.valid) {     // K(g + 3)
+          load_tile(ck, false);
+          advance(ck);
+        }
         ++n;
+      }
+    }
+  } else if (warp == kWarpQ) {
+    // =========================================================================== query-tile producer
+    // One buffer: the tile of the next item is fetched as soon as the last score MMA of the current one has finished;
+    // the softmax groups still have two or three steps of that item to work through meanwhile.
+    if (lane == 0 && p.q_tma) {
+      uint32_t item_count = 0;
+      bool ok = true;
+      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
+        const WorkItem it = p.items[2 * tp + member];
+        if (it.tile_end <= it.tile_begin) continue;
+        ok = mbar_wait(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        // box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
+        mbar_expect_tx(B.q_full, S::kTileBytes);
+#pragma unroll
+        for (int sl = 0; sl < S::kSlabs; ++sl)
+          tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full);
+        ++item_count;
       }
     }
   } else if (warp == kWarpQK) {
@@ -507,8 +509,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       constexpr uint32_t idesc_qk = instr_desc(kBlockM, kTileN, false);
       uint32_t ks = 0, kp = 0;       // slot / parity of the K tile of the next QK
       uint32_t gq = 0;               // steps issued so far (all items)
+      uint32_t sb = 0, sph = 0;      // gq % 3 and (gq / 3) & 1
       uint32_t item_count = 0;
-      const uint32_t q_lo0 = desc_lo(sbase + S::kQ, 16), ring_lo_k = desc_lo(sbase + S::kRing, 16);
+      const uint32_t q_lo = desc_lo(sbase + S::kQ, 16), ring_lo_k = desc_lo(sbase + S::kRing, 16);
       constexpr uint32_t kTileStep = S::kTileBytes >> 4;
       bool ok = true;
       for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
@@ -516,15 +519,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         TRACE(1, 1);
-        const uint32_t qb = item_count & 1u;
-        ok = mbar_wait(B.q_full[qb], (item_count >> 1) & 1u, s_abort);
+        ok = mbar_wait(B.q_full, item_count & 1u, s_abort);
         if (!ok) break;
         TRACE(1, 2);
-        const uint32_t q_lo = q_lo0 + qb * kTileStep;
         for (int s = 0; s < steps && ok; ++s, ++gq) {
-          // S[gq & 1] is free once the softmax warps have read the scores of step gq - 2
-          if (gq >= 2) {
-            ok = mbar_wait(B.p_full[gq & 1u], ((gq - 2) >> 1) & 1u, s_abort);
+          // S[gq % 3] also holds P of step gq - 3: it is free once that step's PV has finished
+          if (gq >= 3) {
+            ok = mbar_wait(B.o_done[sb], sph ^ 1u, s_abort);
             if (!ok) break;
           }
           TRACE(1, (9 << 10) | (gq & 1023u));
@@ -532,12 +533,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (!ok) break;
           TRACE(1, (10 << 10) | (gq & 1023u));
           tc_fence_after();
-          issue_qk_tile<D>(tmem + kColS + (gq & 1u) * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
-          tc_commit(B.s_full[gq & 1u]);
+          issue_qk_tile<D>(tmem + kColS + sb * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
+          tc_commit(B.s_full[sb]);
           tc_commit(B.empty[ks]);
-          ks += gq == 0 ? 1u : 2u;   // K(g) is entry g for g < 2, entry 2g - 1 after that
+          ks += gq < 2 ? 1u : 2u;   // K(g) is entry g for g < 3, entry 2g - 2 after that
           if (ks >= kSlots) { ks -= kSlots; kp ^= 1u; }
-          if (s == steps - 1) tc_commit(B.q_empty[qb]);      // every QK of this item has been issued
+          if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
+          if (s == steps - 1) tc_commit(B.q_empty);      // every QK of this item has been issued
           TRACE(1, (11 << 10) | (gq & 1023u));
         }
         ++item_count;
@@ -547,8 +549,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     // =========================================================================== PV issuer
     if (lane == 0) {
       constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, true);
-      uint32_t vs = 2, vp = 0;       // slot / parity of the V tile of the next PV: V(g) is entry 2g + 2
+      uint32_t vs = 3, vp = 0;       // slot / parity of the V tile of the next PV: V(g) is entry 2g + 3
       uint32_t gp = 0;               // steps issued so far (all items)
+      uint32_t sb = 0, sph = 0;      // gp % 3 and (gp / 3) & 1
       uint32_t item_count = 0;
       const uint32_t ring_lo_v = desc_lo(sbase + S::kRing, S::kSlabBytes);
       constexpr uint32_t kTileStep = S::kTileBytes >> 4;
@@ -558,7 +561,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         for (int s = 0; s < steps && ok; ++s, ++gp) {
-          ok = mbar_wait(B.p_full[gp & 1u], (gp >> 1) & 1u, s_abort);
+          ok = mbar_wait(B.p_full[sb], sph, s_abort);
           if (!ok) break;
           TRACE(3, (20 << 10) | (gp & 1023u));
           ok = mbar_wait(B.full[vs], vp, s_abort);
@@ -569,11 +572,12 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           }
           TRACE(3, (30 << 10) | (gp & 1023u));
           tc_fence_after();
-          issue_pv_tile(tmem + kColO, tmem + kColP + (gp & 1u) * (kTileN / 2), ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
-          tc_commit(B.o_done[gp & 1u]);
+          issue_pv_tile(tmem + kColO, tmem + kColS + sb * kTileN, ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
+          tc_commit(B.o_done[sb]);
           tc_commit(B.empty[vs]);
           vs += 2;
           if (vs >= kSlots) { vs -= kSlots; vp ^= 1u; }
+          if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
           TRACE(3, (31 << 10) | (gp & 1023u));
         }
         ++item_count;
@@ -581,20 +585,17 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     }
   } else if (warp < kSoftmaxWarps) {
     // =========================================================================== softmax + epilogue (warps 0-7)
-    // Two groups of four warps; group g takes the steps whose global number is g mod 2 and owns S[g] / P[g], so the
+    // Two groups of four warps; group g takes the steps whose global number is g mod 2, so the
     // groups run half a step out of phase and each scheduler hosts one warp of either: while one waits on tensor
     // memory or a barrier, the other computes.  Thread r of a group owns query row r (= TMEM lane r), all 128 score
     // columns.  The two threads of a row share one reference maximum: the thread that handled step gs publishes it,
     // tagged with gs, and the other picks it up before it takes its exponentials of step gs + 1.  Each keeps its own
     // part of the row sum, relative to that reference.
-    const int grp = warp >> 2;                            // also the S / P buffer of this group
+    const uint32_t grp = static_cast<uint32_t>(warp >> 2);
     const int r = tid & (kBlockM - 1);                    // query row within the tile == TMEM lane
-    const uint32_t buf = static_cast<uint32_t>(grp);
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     volatile uint32_t* tag = reinterpret_cast<volatile uint32_t*>(smem + S::kTag) + r;   // reference | step, per row
     volatile float* lfin = reinterpret_cast<volatile float*>(smem + S::kLfin) + r;       // row sum on its way to the epilogue
-    const uint32_t s_addr = tmem + lane_addr + kColS + buf * kTileN;
-    const uint32_t p_addr = tmem + lane_addr + kColP + buf * (kTileN / 2);
     const uint32_t o_addr = tmem + lane_addr + kColO;
 
     uint32_t g_base = 0, item_count = 0, sg = 0;   // KV tiles, items and steps before the current item
@@ -613,18 +614,17 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 
       if (!p.q_tma && grp == 0) {
         // group sizes that do not divide 128: the first softmax group stages the query tile itself, a row per thread
-        const uint32_t qb = item_count & 1u;
-        ok = mbar_wait_warp(B.q_empty[qb], ((item_count >> 1) & 1u) ^ 1u, s_abort);
+        ok = mbar_wait_warp(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
         if (!ok) break;
         const uint4* src = reinterpret_cast<const uint4*>(p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D);
-        unsigned char* qdst = smem + S::kQ + qb * S::kTileBytes + r * 128;
+        unsigned char* qdst = smem + S::kQ + r * 128;
 #pragma unroll
         for (int c = 0; c < 8 * S::kSlabs; ++c) {
           const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
           *reinterpret_cast<uint4*>(qdst + (c >> 3) * S::kSlabBytes + (((c & 7) ^ (r & 7)) << 4)) = v;
         }
         fence_proxy_async();
-        mbar_arrive(B.q_full[qb]);
+        mbar_arrive(B.q_full);
       }
       if ((tid & 127) == 0) TRACE(2 + 2 * grp, 3);
 
@@ -632,9 +632,11 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       float m_in = -INFINITY;    // reference the other group left behind at the step before this group's latest one
       float l_sum = 0.f;         // this thread's part of the row sum
       // this group's steps of the item: those whose global number has the group's parity
-      for (int s = static_cast<int>((sg ^ buf) & 1u); s < steps; s += 2) {
+      for (int s = static_cast<int>((sg ^ grp) & 1u); s < steps; s += 2) {
         const uint32_t gs = sg + s;
-        ok = mbar_wait_warp(B.s_full[buf], (gs >> 1) & 1u, s_abort);
+        const uint32_t sb = gs % kSBufs, sph = (gs / kSBufs) & 1u;     // score buffer of this step and its phase
+        const uint32_t s_addr = tmem + lane_addr + kColS + sb * kTileN;   // P goes over the front half of the same columns
+        ok = mbar_wait_warp(B.s_full[sb], sph, s_abort);
         if (!ok) break;
         if ((tid & 127) == 0) TRACE(2 + 2 * grp, (10 << 10) | (gs & 1023u));
         tc_fence_after();
@@ -655,11 +657,11 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             vm[c] = w;
           }
         }
-        // ---- pass 1: row maximum of the raw scores; the last two chunks stay in registers for pass 2
+        // ---- pass 1: row maximum of the raw scores; chunks 0 and 1, fetched last, stay in registers for pass 2
         uint32_t ra[32], rb[32];
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < 4; c += 2) {
+        for (int c = 2; c >= 0; c -= 2) {
           tmem_ld32(s_addr + c * 32, ra);
           tmem_ld32(s_addr + c * 32 + 32, rb);
           tc_wait_ld();
@@ -683,7 +685,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
-          const uint32_t nv = 2 * (g_base + s) + 2, slot = nv % kSlots, par = (nv / kSlots) & 1u;
+          const uint32_t nv = 2 * (g_base + s) + 3, slot = nv % kSlots, par = (nv / kSlots) & 1u;
           ok = mbar_wait_warp(B.full[slot], par, s_abort);
           if (!ok) break;
           if (key0 + r >= kv_end) {
@@ -720,7 +722,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         *tag = __float_as_uint(m_ref) | (gs & 0xffu);
         if (s > 0 && __any_sync(0xffffffffu, grow)) {
           // the previous step accumulated into O and may still be running
-          ok = mbar_wait_warp(B.o_done[buf ^ 1u], ((gs - 1) >> 1) & 1u, s_abort);
+          ok = mbar_wait_warp(B.o_done[(gs - 1) % kSBufs], ((gs - 1) / kSBufs) & 1u, s_abort);
           if (!ok) break;
           tc_fence_after();
           uint32_t o[32];
@@ -735,14 +737,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           tc_wait_st();
         }
         if ((tid & 127) == 0) TRACE(2 + 2 * grp, (13 << 10) | (gs & 1023u));
-        // P[buf] was last read by the PV of step gs - 2 (this wait also keeps every thread within one phase of o_done)
-        if (gs >= 2) {
-          ok = mbar_wait_warp(B.o_done[buf], ((gs - 2) >> 1) & 1u, s_abort);
-          if (!ok) break;
-        }
         if ((tid & 127) == 0) TRACE(2 + 2 * grp, (16 << 10) | (gs & 1023u));
-        // ---- pass 2: exponentials and packed P.  Chunks 2 and 3 are still in registers; chunks 0 and 1 are
-        // fetched again while those are being worked on.
+        // ---- pass 2: exponentials and packed P, in column order (P overwrites score columns that have been
+        // consumed).  Chunks 0 and 1 are still in registers; chunks 2 and 3 are fetched again meanwhile.
         const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
         const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), base2 = pack2(neg_base, neg_base);
         uint64_t ls2[2] = {0ull, 0ull};   // four partial sums
@@ -763,22 +760,22 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             ls2[j & 1] = add2(ls2[j & 1], pack2(p0, p1));
             pk[j] = pack_bf16(p0, p1);
           }
-          tmem_st16(p_addr + c * 16, pk);
+          tmem_st16(s_addr + c * 16, pk);
         };
-        exp_chunk(ra, 2);
-        tmem_ld32(s_addr, ra);              // chunk 0, in flight while chunk 3 is worked on
-        exp_chunk(rb, 3);
-        tmem_ld32(s_addr + 32, rb);         // chunk 1
+        exp_chunk(ra, 0);
+        tmem_ld32(s_addr + 64, ra);         // chunk 2, in flight while chunk 1 is worked on
+        exp_chunk(rb, 1);
+        tmem_ld32(s_addr + 96, rb);         // chunk 3
         tc_wait_ld();
         if (tail) {
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            ra[e] = (vm[0] >> e) & 1u ? ra[e] : 0xff800000u;
-            rb[e] = (vm[1] >> e) & 1u ? rb[e] : 0xff800000u;
+            ra[e] = (vm[2] >> e) & 1u ? ra[e] : 0xff800000u;
+            rb[e] = (vm[3] >> e) & 1u ? rb[e] : 0xff800000u;
           }
         }
-        exp_chunk(ra, 0);
-        exp_chunk(rb, 1);
+        exp_chunk(ra, 2);
+        exp_chunk(rb, 3);
         {
           float l0, l1, l2, l3;
           unpack2(ls2[0], l0, l1);
@@ -796,14 +793,14 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         }
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(B.p_full[buf]);
+        mbar_arrive(B.p_full[sb]);
         if ((tid & 127) == 0) TRACE(2 + 2 * grp, (11 << 10) | (gs & 1023u));
 
         if (s == steps - 1) {
           // ---- this group took the item's last step: it writes the item's output.  Wait for the last PV (PVs
           // complete in order), add the other group's part of the row sum, then write the row: bf16 output, or
           // the unnormalised fp32 partial of a cut piece.
-          ok = mbar_wait_warp(B.o_done[buf], (gs >> 1) & 1u, s_abort);
+          ok = mbar_wait_warp(B.o_done[sb], sph, s_abort);
           if (!ok) break;
           if ((tid & 127) == 0) TRACE(2 + 2 * grp, 20);
           tc_fence_after();
