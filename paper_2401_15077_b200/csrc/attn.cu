@@ -523,14 +523,16 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (!ok) break;
         TRACE(1, 2);
         for (int s = 0; s < steps && ok; ++s, ++gq) {
+          // the K tile arrives long before the score buffer frees up: look at it first, so that nothing but the
+          // MMA issue follows the wait that matters
+          ok = mbar_wait(B.full[ks], kp, s_abort);
+          if (!ok) break;
+          TRACE(1, (9 << 10) | (gq & 1023u));
           // S[gq % 3] also holds P of step gq - 3: it is free once that step's PV has finished
           if (gq >= 3) {
             ok = mbar_wait(B.o_done[sb], sph ^ 1u, s_abort);
             if (!ok) break;
           }
-          TRACE(1, (9 << 10) | (gq & 1023u));
-          ok = mbar_wait(B.full[ks], kp, s_abort);
-          if (!ok) break;
           TRACE(1, (10 << 10) | (gq & 1023u));
           tc_fence_after();
           issue_qk_tile<D>(tmem + kColS + sb * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
@@ -561,15 +563,15 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         for (int s = 0; s < steps && ok; ++s, ++gp) {
-          ok = mbar_wait(B.p_full[sb], sph, s_abort);
+          ok = mbar_wait(B.full[vs], vp, s_abort);   // (arrives well before P is ready)
           if (!ok) break;
           TRACE(3, (20 << 10) | (gp & 1023u));
-          ok = mbar_wait(B.full[vs], vp, s_abort);
-          if (!ok) break;
           if (s == 0 && item_count > 0) {
             ok = mbar_wait(B.o_free, (item_count - 1) & 1u, s_abort);   // previous epilogue has read O
             if (!ok) break;
           }
+          ok = mbar_wait(B.p_full[sb], sph, s_abort);
+          if (!ok) break;
           TRACE(3, (30 << 10) | (gp & 1023u));
           tc_fence_after();
           issue_pv_tile(tmem + kColO, tmem + kColS + sb * kTileN, ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
