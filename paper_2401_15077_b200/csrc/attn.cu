@@ -1,23 +1,24 @@
 // Split-KV tree attention for sm_100a: TMA-staged KV tiles, tcgen05 MMAs, accumulators in TMEM.
 //
-// One persistent CTA per SM walks its share of the planner's work list (equal numbers of KV tiles per CTA).  An
+// One persistent CTA per SM; CTAs 2j and 2j+1 form a team that walks its share of the planner's work list.  An
 // item is one 128-row query tile (row = tree node * G + head-in-group) of one (sequence, KV head) over a range of
-// 128-key KV tiles;
-// step s of the item handles KV tile s:
-//     S[s&1] = Q K^T   ->   softmax   ->   P[s&1] (packed bf16)   ->   O += P V.
-// S and P are double buffered in TMEM (S0 S1 | O | P0 P1 = 512 columns), so the score MMA of step s+1 and the
-// PV MMA of step s-1 run while the softmax warps work on step s.
-// Warp roles: warps 0-7 softmax (thread pair (r, r+128) shares query row r = TMEM lane r, 64 score columns
-// each; the pair agrees on the row max through shared memory), warp 8 TMA producer (K and V tiles through a
-// ring of five 32 KB slots, and the query tile of the NEXT item into the other half of a double-buffered Q
-// area; 128-byte swizzled boxes), warp 9 issues the QK MMAs and warp 10 the PV MMAs (each waits only on what
-// its own MMA needs).  Items overlap at their seams: the score MMA of the next item's first tile is issued
-// while the current item finishes, and the softmax warps take that first step before they write the finished
-// item's output, so the accumulator drain and the pipeline fill hide behind each other.  Softmax is fp32 in the log2 domain; the tree mask is applied in
-// registers only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are
-// zeroed in shared memory before the MMA reads them.  The accumulator is rescaled only when the running max
-// grows by more than 2^8.  Every wait is bounded (mbarrier try_wait + timer); on expiry the CTA raises
-// EAGLE_ERR_TIMEOUT, all roles leave their loops, TMEM is released and the kernel returns.
+// 128-key KV tiles; step g (counted over all of the CTA's items) handles one KV tile:
+//     S[g % 3] = Q K^T   ->   softmax   ->   P (packed bf16, written over the front of S[g % 3])   ->   O += P V.
+// Tensor memory holds three score buffers and the accumulator (S0 S1 S2 | O = 512 columns).  The score MMA of
+// step g + 3 is issued as soon as the PV MMA of step g has released its buffer, so up to three score tiles are in
+// flight and the MMAs never wait for the softmax of the step before them.
+// Warp roles: warps 0-7 softmax, as two groups of four warps that take alternate steps (one query row = one
+// TMEM lane per thread, all 128 score columns), so that one group computes while the other waits; warp 8 K/V
+// producer (TMA, 128-byte swizzled boxes, ring of six 32 KB slots, tiles requested in the order the MMAs consume
+// them); warp 9 issues the QK MMAs, warp 10 the PV MMAs; warp 11 fetches the query tile of the next item once the
+// last score MMA of the current one has finished.  The group that takes an item's last step writes its output
+// while the other group is already on the next item.  Softmax is fp32 in the log2 domain with two-wide FP32
+// instructions; part of the exponentials is a polynomial on the FMA pipe.  The tree mask is applied in registers
+// only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are zeroed in shared
+// memory before the MMA reads them.  The accumulator is rescaled only when the row maximum outgrows the shared
+// reference by more than 2^8.  Every wait is bounded (mbarrier try_wait + timer, or a bounded spin on a tagged
+// word); on expiry the CTA raises EAGLE_ERR_TIMEOUT, all roles leave their loops, TMEM is released and the kernel
+// returns.
 #include <cuda.h>
 
 #include "common.cuh"
