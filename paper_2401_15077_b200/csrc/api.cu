@@ -121,6 +121,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.seq = w.seq;
   pp.anc = w.anc;
   pp.units = w.units;
+  pp.cut_tiles = w.cut_tiles;
   pp.cta_first = w.cta_first;
   pp.items = w.items;
   pp.status = d.status;
@@ -144,6 +145,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.seq = w.seq;
   ap.anc = w.anc;
   ap.units = w.units;
+  ap.cut_tiles = w.cut_tiles;
   ap.cta_first = w.cta_first;
   ap.items = w.items;
   ap.part_ml = w.part_ml;
@@ -152,7 +154,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_combine(ap, w.unit_cap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, w.unit_cap, dev->sm_count, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 
@@ -235,6 +237,7 @@ bool carve_static(const eagle_attn_desc& d, int num_ctas, void* base, Workspace*
   w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * static_cast<size_t>(d.batch > 0 ? d.batch : 1)));
   w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * static_cast<size_t>(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
   w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * static_cast<size_t>(units > 0 ? units : 1)));
+  w->cut_tiles = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * 2 * static_cast<size_t>(units > 0 ? units : 1)));
   w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
   w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * static_cast<size_t>(items > 0 ? items : 1)));
   w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * static_cast<size_t>(slots) * kBlockM));
@@ -315,6 +318,7 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   pp.seq = w.seq;
   pp.anc = w.anc;
   pp.units = w.units;
+  pp.cut_tiles = w.cut_tiles;
   pp.cta_first = w.cta_first;
   pp.items = w.items;
   pp.status = d.status;
@@ -341,6 +345,7 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   ap.seq = w.seq;
   ap.anc = w.anc;
   ap.units = w.units;
+  ap.cut_tiles = w.cut_tiles;
   ap.cta_first = w.cta_first;
   ap.items = w.items;
   ap.part_ml = w.part_ml;
@@ -349,7 +354,7 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_combine(ap, w.unit_cap, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_combine(ap, w.unit_cap, dev->sm_count, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 

@@ -1,8 +1,9 @@
 // Merge of the split-KV partials: m* = max_s m_s, l* = sum_s l_s 2^(m_s - m*), O = sum_s O_s 2^(m_s - m*) / l*,
 // and the zero rows of padded tree nodes.
-// Eight blocks per query tile (16 rows each, two rows per warp): a tile that stayed in one item was written by the
-// attention kernel and costs one table look-up here; otherwise its rows are merged from the items that hold it.  One more block per sequence
-// writes zeros to the rows of nodes past the tree size (one contiguous range of the output).
+// A fixed grid (a few blocks per SM) walks the planner's list of cut query tiles, eight work items per tile
+// (16 rows each, two rows per warp), then one work item per sequence that writes zeros to the rows of nodes past
+// the tree size (one contiguous range of the output).  Query tiles that stayed in one item were written by the
+// attention kernel and do not appear in the list.
 #include "common.cuh"
 
 namespace eagle {
@@ -14,32 +15,31 @@ constexpr int kBlocksPerUnit = 8;                       // 16 rows per block
 constexpr int kRowsPerBlock = kBlockM / kBlocksPerUnit;
 
 template <int D>
-__global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p, int unit_blocks) {
+__global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) {
   constexpr int E = D / 32;  // elements per lane
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (static_cast<int>(blockIdx.x) >= unit_blocks) {
+  const int tile_items = p.hdr->n_cut * kBlocksPerUnit, total = tile_items + p.B;
+  for (int work = blockIdx.x; work < total; work += gridDim.x) {
+  if (work >= tile_items) {
     // ---- padding rows of one sequence: out[b, n:, :, :]
-    const int b = blockIdx.x - unit_blocks;
+    const int b = work - tile_items;
     const int n = p.seq[b].n;
     const size_t row_elems = static_cast<size_t>(p.Hq) * D;
     uint4* dst = reinterpret_cast<uint4*>(p.out + (static_cast<size_t>(b) * p.T_max + n) * row_elems);
     const size_t vecs = static_cast<size_t>(p.T_max - n) * row_elems / 8;   // 8 bf16 per 16 bytes; D is a multiple of 64
     for (size_t i = threadIdx.x; i < vecs; i += kCombineThreads) dst[i] = make_uint4(0u, 0u, 0u, 0u);
-    return;
+    continue;
   }
-  // blocks are laid out per query tile: (super-unit, tile-in-pair, 16-row chunk)
-  const int su = blockIdx.x / (2 * kBlocksPerUnit), which = (blockIdx.x / kBlocksPerUnit) & 1;
-  const int row0 = (blockIdx.x % kBlocksPerUnit) * kRowsPerBlock;
-  if (su >= p.hdr->n_units) return;
+  // work items of a query tile: (cut tile, 16-row chunk)
+  const int code = p.cut_tiles[work / kBlocksPerUnit];
+  const bool paired = ((code >> 30) & 1) == 0;        // a pair or twin: this tile's pieces are one CTA's items
+  const int su = (code & 0x3fffffff) >> 1, which = code & 1;
+  const int row0 = (work % kBlocksPerUnit) * kRowsPerBlock;
   const UnitPlan up = p.units[su];
-  if (up.slot_base < 0) return;   // every query tile of this super-unit was written directly by the attention kernel
-  const int b = up.pad0;
+  // which query tile this is: every item of it says so, empty or not
+  const WorkItem it0 = p.items[2 * up.first_item + (paired ? which : 0)];
+  const int b = it0.b, g = it0.g, mt = it0.mt;
   const SeqPlan sp = p.seq[b];
-  const int npairs = (sp.mtiles + 1) / 2;
-  const int k = su - sp.unit_base, g = k / npairs, mp = k % npairs;
-  const bool paired = 2 * mp + 1 < sp.mtiles;
-  const int mt = 2 * mp + which;
-  if (mt >= sp.mtiles) return;    // a lone tile has no sibling
   const int m_valid = sp.n * p.G;
   // the items that hold this query tile: one per team piece for a pair, both for a lone tile (its two halves)
   const int first = 2 * up.first_item, count = paired ? up.n_pieces : 2 * up.n_pieces;
@@ -84,16 +84,19 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p, 
       *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<uint32_t*>(&lo);
     }
   }
+  }
 }
 
 }  // namespace
 
-cudaError_t launch_combine(const AttnParams& p, int unit_cap, cudaStream_t stream) {
+cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cudaStream_t stream) {
   if (p.B == 0 || p.T_max == 0) return cudaSuccess;
-  const unsigned unit_blocks = static_cast<unsigned>(unit_cap) * 2 * kBlocksPerUnit;   // unit_cap super-units, two query tiles each
-  const unsigned blocks = unit_blocks + static_cast<unsigned>(p.B);
-  if (p.D == 128) combine_kernel<128><<<blocks, kCombineThreads, 0, stream>>>(p, static_cast<int>(unit_blocks));
-  else combine_kernel<64><<<blocks, kCombineThreads, 0, stream>>>(p, static_cast<int>(unit_blocks));
+  // the number of cut tiles is only known on the device: a few blocks per SM loop over them
+  const long long most = static_cast<long long>(unit_cap) * 2 * kBlocksPerUnit + p.B;
+  const long long want = static_cast<long long>(sm_count > 0 ? sm_count : 1) * 4;
+  const unsigned blocks = static_cast<unsigned>(want < most ? want : most);
+  if (p.D == 128) combine_kernel<128><<<blocks, kCombineThreads, 0, stream>>>(p);
+  else combine_kernel<64><<<blocks, kCombineThreads, 0, stream>>>(p);
   count_launch();
   return cudaGetLastError();
 }

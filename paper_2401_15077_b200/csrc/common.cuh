@@ -46,7 +46,8 @@ struct PlanHeader {
   int32_t n_units;
   int32_t ctas_used;
   long long total_tiles;
-  int32_t pad[10];
+  int32_t n_cut;       // query tiles whose output has to be merged from several pieces
+  int32_t pad[9];
 };
 
 // Workspace carving (all offsets multiples of 256 bytes).
@@ -55,6 +56,7 @@ struct Workspace {
   SeqPlan* seq;        // [B]
   uint64_t* anc;       // [B, T_max]
   UnitPlan* units;     // [unit_cap]
+  int32_t* cut_tiles;  // [2 * unit_cap]: the cut query tiles, as 2 * super-unit + tile-in-pair, in no particular order
   int32_t* cta_first;  // [kMaxPlanCtas + 1]: team j owns the team pieces cta_first[j] .. cta_first[j+1] - 1
   WorkItem* items;     // [item_cap]
   float2* part_ml;     // [slot_cap, 128]   (reference max in the log2 domain, row sum)
@@ -85,6 +87,7 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * (size_t)(d.batch > 0 ? d.batch : 1)));
   w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * (size_t)(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
   w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * (size_t)(units > 0 ? units : 1)));
+  w->cut_tiles = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * 2 * (size_t)(units > 0 ? units : 1)));
   w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
   w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * (size_t)(items > 0 ? items : 1)));
   w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * (size_t)slots * kBlockM));
@@ -108,6 +111,7 @@ struct AttnParams {
   const SeqPlan* seq;
   const uint64_t* anc;
   const UnitPlan* units;
+  const int32_t* cut_tiles;
   const int32_t* cta_first;
   const WorkItem* items;
   float2* part_ml;
@@ -130,6 +134,7 @@ struct PlanParams {
   SeqPlan* seq;
   uint64_t* anc;
   UnitPlan* units;
+  int32_t* cut_tiles;
   int32_t* cta_first;
   WorkItem* items;
   int32_t* status;
@@ -161,7 +166,7 @@ cudaError_t launch_build_mask(const int32_t* tree_parent, const int32_t* tree_si
 cudaError_t launch_attn(const AttnParams& p, int num_ctas, cudaStream_t stream);
 int attn_tile_keys();
 cudaError_t attn_prepare(int head_dim);
-cudaError_t launch_combine(const AttnParams& p, int unit_cap, cudaStream_t stream);
+cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cudaStream_t stream);
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
 void count_launch();

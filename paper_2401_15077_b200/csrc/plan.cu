@@ -138,30 +138,94 @@ __device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W
 constexpr int kSmemSeqs = 512;     // per-sequence records kept in shared memory while planning (else in the workspace)
 constexpr int kSmemUnits = 1792;   // per-super-unit records kept in shared memory while planning
 
-// Geometry of a sequence's super-units.  The query tiles of one (sequence, KV head) are taken two at a time; a pair is
-// one super-unit whose line is the sequence's KV tiles (both CTAs of a team walk it, one query tile each), and an odd
-// last tile is a super-unit whose line is half the KV tiles (the team's CTAs take one half each).
+// Geometry of a sequence's super-units.  The query tiles of one (sequence, KV head) are taken two at a time; such a
+// PAIR is one super-unit whose line is the sequence's KV tiles (both CTAs of a team walk it, one query tile each).
+// An odd last query tile has no sibling: the last tiles of two neighbouring KV heads form a TWIN super-unit with the
+// same line (each CTA of the team walks it for its own head), and with an odd number of KV heads the last head's
+// tile is a LONE super-unit whose line is half the KV tiles (the team's CTAs take one half each).  On the work line
+// the heads are laid out two at a time: the pairs of head 2j, the pairs of head 2j + 1, their twin.
+enum UnitKind { kPair = 0, kTwin = 1, kLone = 2 };
+struct UnitGeom {
+  int kind, g, mp, line;     // g: KV head (first of the two for a twin); mp: pair index within the head
+  long long offset;          // start on the work line, relative to the sequence's start
+};
 struct SeqGeom {
-  int npairs, ntiles, half, plen, glen;   // super-units per head; KV tiles; ceil(ntiles/2); paired length; per-head length
+  int pf, ntiles, half, plen, Hkv;   // whole pairs per head; KV tiles; ceil(ntiles/2); line + overhead of a pair or twin
+  int u1, u2;                        // super-units of a leftover single head / of two heads
+  long long len1, len2;              // line length of a leftover single head / of two heads
   bool odd;
-  __device__ SeqGeom(const SeqPlan& sp, int ovh) {
-    npairs = (sp.mtiles + 1) / 2;
+  int ovh;
+  __device__ SeqGeom(const SeqPlan& sp, int Hkv_, int ovh_) {
+    Hkv = Hkv_;
+    ovh = ovh_;
+    pf = sp.mtiles / 2;
     ntiles = sp.ntiles;
     half = (sp.ntiles + 1) / 2;
     odd = (sp.mtiles & 1) != 0;
     plen = sp.ntiles + ovh;
-    glen = (sp.mtiles / 2) * plen + (odd ? half + ovh : 0);
+    u1 = pf + (odd ? 1 : 0);
+    u2 = 2 * pf + (odd ? 1 : 0);
+    len1 = static_cast<long long>(pf) * plen + (odd ? half + ovh : 0);
+    len2 = 2ll * pf * plen + (odd ? plen : 0);
   }
-  __device__ bool paired(int mp) const { return !(odd && mp == npairs - 1); }
-  __device__ int line(int mp) const { return paired(mp) ? ntiles : half; }          // tile positions of the super-unit
-  __device__ long long offset(int k) const { return static_cast<long long>(k / npairs) * glen + static_cast<long long>(k % npairs) * plen; }
+  __device__ int units() const { return (Hkv / 2) * u2 + (Hkv & 1) * u1; }
+  __device__ long long length() const { return (Hkv / 2) * len2 + (Hkv & 1) * len1; }
+  __device__ UnitGeom unit(int k) const {
+    UnitGeom ug;
+    const int twos = Hkv / 2;
+    if (k < twos * u2) {
+      const int h2 = k / u2, j = k % u2;
+      const long long base = static_cast<long long>(h2) * len2;
+      if (j < 2 * pf) {
+        ug.kind = kPair;
+        ug.g = 2 * h2 + (j >= pf ? 1 : 0);
+        ug.mp = j >= pf ? j - pf : j;
+        ug.offset = base + static_cast<long long>(j) * plen;
+      } else {
+        ug.kind = kTwin;
+        ug.g = 2 * h2;
+        ug.mp = pf;
+        ug.offset = base + 2ll * pf * plen;
+      }
+      ug.line = ntiles;
+    } else {
+      const int j = k - twos * u2;
+      const long long base = static_cast<long long>(twos) * len2;
+      ug.g = Hkv - 1;
+      ug.mp = j;
+      ug.offset = base + static_cast<long long>(j) * plen;
+      if (j < pf) {
+        ug.kind = kPair;
+        ug.line = ntiles;
+      } else {
+        ug.kind = kLone;
+        ug.line = half;
+      }
+    }
+    return ug;
+  }
+  // the super-unit that holds line position `off` (relative to the sequence's start, 0 <= off < length())
+  __device__ int unit_at(long long off) const {
+    const int twos = Hkv / 2;
+    if (off < twos * len2) {
+      const int h2 = static_cast<int>(off / len2);
+      int j = static_cast<int>((off % len2) / plen);
+      if (j > u2 - 1) j = u2 - 1;
+      return h2 * u2 + j;
+    }
+    int j = static_cast<int>((off - twos * len2) / plen);
+    if (j > u1 - 1) j = u1 - 1;
+    return twos * u2 + j;
+  }
 };
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   __shared__ long long s_scan[kPlanThreads / 32];
+  __shared__ int s_ncut;
   __shared__ SeqPlan s_seq[kSmemSeqs];
   __shared__ UnitPlan s_units[kSmemUnits];
   const int tid = threadIdx.x;
+  if (tid == 0) s_ncut = 0;   // (the block synchronises several times before the counter is used)
   // The planning passes are chains of dependent reads and writes of these small tables; in shared memory each
   // link costs tens of cycles instead of a trip to L2.  They are copied to the workspace once at the end.
   PlanParams p = pg;
@@ -203,10 +267,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
 
   // ---- lay the sequences' super-units end to end
   const long long W = block_exclusive_scan(
-      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * SeqGeom(p.seq[b], ovh).glen; },
+      p.B, [&](int b) { return SeqGeom(p.seq[b], p.Hkv, ovh).length(); },
       [&](int b, long long v) { p.seq[b].start = v; }, s_scan);
   const long long U = block_exclusive_scan(
-      p.B, [&](int b) { return static_cast<long long>(p.Hkv) * ((p.seq[b].mtiles + 1) / 2); },
+      p.B, [&](int b) { return static_cast<long long>(SeqGeom(p.seq[b], p.Hkv, ovh).units()); },
       [&](int b, long long v) { p.seq[b].unit_base = static_cast<int>(v); }, s_scan);
   const int n_units = U <= p.unit_cap ? static_cast<int>(U) : 0;   // cannot exceed the advertised workspace
   if (U > p.unit_cap && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);
@@ -228,10 +292,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   for (int u = tid; u < n_units; u += kPlanThreads) {
     const int b = unit_seq(u);
     const SeqPlan sp = p.seq[b];
-    const SeqGeom ge(sp, ovh);
-    const int k = u - sp.unit_base, mp = k % ge.npairs;
-    const int len = ge.line(mp);
-    const long long us = sp.start + ge.offset(k);
+    const SeqGeom ge(sp, p.Hkv, ovh);
+    const UnitGeom ug = ge.unit(u - sp.unit_base);
+    const int len = ug.line;
+    const long long us = sp.start + ug.offset;
     int np;
     if (p.forced_splits > 0) {
       np = len < p.forced_splits ? len : p.forced_splits;
@@ -248,9 +312,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   auto slots_of = [&](int u) -> long long {
     const UnitPlan up = p.units[u];
     const SeqPlan sp = p.seq[up.pad0];
-    const SeqGeom ge(sp, ovh);
-    const int mp = (u - sp.unit_base) % ge.npairs;
-    const bool partial = ge.paired(mp) ? up.n_pieces > 1 : sp.ntiles > 1;
+    const SeqGeom ge(sp, p.Hkv, ovh);
+    const bool partial = ge.unit(u - sp.unit_base).kind != kLone ? up.n_pieces > 1 : sp.ntiles > 1;
     return partial ? 2ll * up.n_pieces : 0ll;
   };
   const long long TP = block_exclusive_scan(
@@ -267,14 +330,16 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
       const UnitPlan up = p.units[u];
       const int b = up.pad0;
       const SeqPlan sp = p.seq[b];
-      const SeqGeom ge(sp, ovh);
-      const int k = u - sp.unit_base, g = k / ge.npairs, mp = k % ge.npairs;
-      const bool paired = ge.paired(mp);
-      const int len = ge.line(mp), rest = sp.ntiles - len;      // single tile: second CTA's part has `rest` tiles
-      const long long us = sp.start + ge.offset(k);
+      const SeqGeom ge(sp, p.Hkv, ovh);
+      const UnitGeom ug = ge.unit(u - sp.unit_base);
+      const int g = ug.g, mp = ug.mp;
+      const bool paired = ug.kind != kLone;         // both CTAs of the team walk the same KV range
+      const int len = ug.line, rest = sp.ntiles - len;      // lone tile: the second CTA's part has `rest` tiles
+      const long long us = sp.start + ug.offset;
       const long long t_origin = us + ovh;          // line position of the super-unit's tile position 0
       int c0 = 0;
       if (p.forced_splits == 0) unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0);
+      bool live[2] = {false, false};    // query tiles of the super-unit with at least one non-empty item
       for (int j = 0; j < up.n_pieces; ++j) {
         int t0, t1;
         if (p.forced_splits > 0) {
@@ -287,9 +352,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
         for (int m = 0; m < 2; ++m) {
           WorkItem it;
           it.b = b;
-          it.g = g;
+          it.g = ug.kind == kTwin ? g + m : g;
           if (paired) {
-            it.mt = 2 * mp + m;
+            it.mt = ug.kind == kTwin ? 2 * mp : 2 * mp + m;
             it.tile_begin = t0;
             it.tile_end = t1;
             it.slot = up.slot_base >= 0 ? up.slot_base + m * up.n_pieces + j : -1;
@@ -301,7 +366,14 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
           }
           it.pad0 = it.pad1 = 0;
           p.items[2 * (up.first_item + j) + m] = it;
+          if (it.tile_end > it.tile_begin) live[paired ? m : 0] = true;
         }
+      }
+      // the query tiles whose pieces the combine kernel has to merge (bit 30: a lone tile, whose pieces are the
+      // items of both CTAs)
+      if (up.slot_base >= 0) {
+        for (int m = 0; m < 2; ++m)
+          if (live[m]) pg.cut_tiles[atomicAdd(&s_ncut, 1)] = (2 * u + m) | (paired ? 0 : 1 << 30);
       }
     }
   }
@@ -325,15 +397,11 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
         if (p.seq[mid].start <= x) lo = mid; else hi = mid;
       }
       const SeqPlan sp = p.seq[lo];
-      const SeqGeom ge(sp, ovh);
-      const long long off = x - sp.start;
-      const int g = static_cast<int>(off / ge.glen);
-      const long long rem = off % ge.glen;
-      int mp = static_cast<int>(rem / ge.plen);
-      if (mp > ge.npairs - 1) mp = ge.npairs - 1;
-      const int k = g * ge.npairs + mp;
+      const SeqGeom ge(sp, p.Hkv, ovh);
+      const int k = ge.unit_at(x - sp.start);
+      const UnitGeom ug = ge.unit(k);
       const int u = sp.unit_base + k;
-      const long long us = sp.start + ge.offset(k), ue = us + ge.line(mp) + ovh;
+      const long long us = sp.start + ug.offset, ue = us + ug.line + ovh;
       const long long d0 = x - (us + ovh), d1 = ue - x;   // distance to the first tile position / to the super-unit's end
       const UnitPlan up = p.units[u];
       if (d0 >= snap && d1 >= snap) {
@@ -357,6 +425,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
     p.hdr->n_items = fits ? static_cast<int>(2 * TP) : 0;
     p.hdr->n_slots = fits ? static_cast<int>(S) : 0;
     p.hdr->n_units = n_units;
+    p.hdr->n_cut = s_ncut;
     p.hdr->ctas_used = 2 * teams;
     p.hdr->total_tiles = W;
   }
