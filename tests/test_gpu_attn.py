@@ -97,6 +97,34 @@ def test_chain_tree_no_sizes_custom_scale(E, oracle):
     _check(out, ref, [9, 9])
 
 
+@pytest.mark.parametrize("shape", ["ramp_up", "ramp_down", "late_spike"])
+def test_reference_maximum_moves_between_steps(E, oracle, shape):
+    """Scores that grow (or fall) by far more than the lazy-rescale threshold from one KV tile to the next: the shared
+    reference maximum moves at many steps, the accumulator is rescaled, and the row sums of the softmax groups are
+    handed over relative to different references.  Several query tiles, cut pieces and direct tiles are all present."""
+    cfg = W.scaled(W.CONFIGS["70b_gqa"], batch=3, prefix=(700, 2600), tree=(20, 64))
+    inp = W.make_attn_inputs(cfg, salt=11)
+    S = inp.k_cache.shape[2]
+    pos = torch.arange(S, dtype=torch.float32)
+    if shape == "ramp_up":
+        gain = 0.4 + pos / 128.0 * 0.35          # |q.k| grows by about 45 per tile: about 6 log2 units per tile after scaling
+    elif shape == "ramp_down":
+        gain = 0.4 + (S - pos) / 128.0 * 0.35
+    else:
+        gain = torch.where((pos > 900) & (pos < 1030), torch.tensor(6.0), torch.tensor(0.5))
+    g = torch.Generator().manual_seed(21)
+    # keys share a direction with the queries so that the dot products follow the gain instead of averaging out
+    base = torch.randn(cfg.head_dim, generator=g).sign()
+    k = (base[None, None, None, :] * gain[None, None, :, None] + 0.3 * torch.randn(inp.k_cache.shape, generator=g))
+    inp.k_cache = k.to(torch.bfloat16)
+    inp.q = (base[None, None, None, :] * 0.9 + 0.3 * torch.randn(inp.q.shape, generator=g)).to(torch.bfloat16)
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    for splits in (0, 3):
+        out, status = _run(E, inp, num_splits=splits)
+        assert status == 0
+        _check(out, ref, inp.tree_sizes)
+
+
 def test_empty_prefix_empty_tree_and_single_node(E, oracle):
     cfg = W.scaled(W.CONFIGS["tiny"], batch=4, prefix=(0, 0), tree=(1, 6))
     inp = W.make_attn_inputs(cfg, salt=5)
