@@ -41,9 +41,9 @@ HBM_FALLBACK_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu captures summarised in
 # profiles/attn_kernel_serving_mix_b16.md, keyed by (workload, batch); None where no capture exists.
-# Full serving_mix: 1199.8 MB read (measured at full size) + 43 MB written (output + cut-piece partials, scaled from
-# the batch-16 capture); batch 16: 314.3 MB + 17.4 MB.
-NCU_TRAFFIC_BYTES = {("serving_mix", 64): 1_199_820_032 + 43_000_000, ("serving_mix", 16): 314_316_800 + 17_369_344}
+# Full serving_mix: 1224.3 MB read + 29.8 MB written, captured at full size with a one-pass metric list;
+# batch 16: 314.1 MB + 15.7 MB from the --set full capture.
+NCU_TRAFFIC_BYTES = {("serving_mix", 64): 1_224_349_184 + 29_797_888, ("serving_mix", 16): 314_063_104 + 15_671_296}
 
 
 def measured_hbm_peak():
