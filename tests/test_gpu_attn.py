@@ -59,6 +59,12 @@ CASES = {
     # group sizes that do not divide 128: the query tile is staged by the softmax threads instead of TMA
     "group3_d128": W.scaled(W.CONFIGS["7b_mha"], batch=3, num_q_heads=12, num_kv_heads=4, prefix=(50, 1200), tree=(3, 64), max_depth=8),
     "group6_d64": W.scaled(W.CONFIGS["tiny"], batch=2, num_q_heads=12, num_kv_heads=2, prefix=(0, 500), tree=(10, 50), max_depth=6),
+    # odd number of KV heads: heads 0 and 1 share twin super-units, head 2's odd tile is split in halves between two CTAs
+    "odd_heads_one_tile": W.scaled(W.CONFIGS["7b_mha"], batch=4, num_q_heads=12, num_kv_heads=3, prefix=(300, 2500), tree=(5, 30), max_depth=8),
+    # one KV head, three query tiles: a pair plus a lone tile per sequence
+    "single_head_three_tiles": W.scaled(W.CONFIGS["70b_gqa"], batch=3, num_q_heads=8, num_kv_heads=1, prefix=(100, 1800), tree=(36, 48)),
+    # five KV heads, three query tiles each: pairs, twins and one lone tile in the same sequence
+    "five_heads_three_tiles": W.scaled(W.CONFIGS["70b_gqa"], batch=2, num_q_heads=40, num_kv_heads=5, prefix=(400, 1500), tree=(40, 48)),
     "big_group_full_tree": W.scaled(W.CONFIGS["70b_gqa"], batch=2, num_q_heads=32, num_kv_heads=2, prefix=(130, 400),
                                     tree=(64, 64), max_depth=64, child_cap=0),
 }
