@@ -44,6 +44,8 @@ def _load():
         lib.oracle_tree_verify_attn.restype = i32
         lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 13
         lib.oracle_tree_accept.restype = i32
+        lib.oracle_tree_commit.argtypes = [i32] * 6 + [vp] * 4 + [i32] + [vp] * 4
+        lib.oracle_tree_commit.restype = i32
         lib.oracle_num_threads.restype = i32
         _lib = lib
     return _lib
@@ -133,3 +135,27 @@ def tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, 
     if rc != 0:
         raise ValueError(f"oracle_tree_accept failed: {rc}")
     return res
+
+
+def tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree: int, features=None):
+    """Commit of the accepted path (Sec. 3.3).  ``k_cache`` / ``v_cache``: bf16 [B, Hkv, S_cap, D] (torch CPU tensors
+    or uint16 arrays); they are NOT modified: copies are returned.  Returns a dict: k_cache, v_cache (uint16 arrays),
+    features_out [B, path_cap, F] (uint16, or None), new_seq_lens [B], valid [B]."""
+    k = _as(k_cache, np.uint16).copy()
+    v = _as(v_cache, np.uint16).copy()
+    sl, path = _as(seq_lens, np.int32), _as(accepted_path, np.int32)
+    B, Hkv, S_cap, D = k.shape
+    assert v.shape == k.shape and path.shape[0] == B and sl.shape == (B,)
+    cap = path.shape[1]
+    fin = _as(features, np.uint16)
+    F = 0 if fin is None else fin.shape[2]
+    if fin is not None:
+        assert fin.shape[:2] == (B, max_tree)
+    fout = None if fin is None else np.full((B, cap, F), 0xFFFF, np.uint16)
+    new_len = np.full((B,), -1, np.int32)
+    valid = np.full((B,), -1, np.int32)
+    rc = _load().oracle_tree_commit(B, Hkv, D, S_cap, max_tree, cap, _ptr(sl), _ptr(path), _ptr(k), _ptr(v), F, _ptr(fin),
+                                    _ptr(fout), _ptr(new_len), _ptr(valid))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_commit failed: {rc}")
+    return dict(k_cache=k, v_cache=v, features_out=fout, new_seq_lens=new_len, valid=valid)

@@ -15,6 +15,11 @@
  *   oracle_tree_accept       - Algorithm 1 (multi-round speculative sampling, App. A.2) applied
  *                              recursively at every node from the root (Sec. 3.3); the greedy setting
  *                              (Preliminaries) is the same rule with a one-hot target distribution.
+ *   oracle_tree_commit       - Sec. 3.3, last sentence: the accepted tokens and their features are recorded
+ *                              for the next drafting phase.  For the target's KV cache that means: the
+ *                              keys and values of the accepted tree nodes become the next slots of the
+ *                              committed prefix, in path order; the accepted nodes' feature vectors are
+ *                              gathered in the same order (plain definition: a simultaneous assignment).
  *
  * Readings taken where the paper is silent or garbled are listed next to the code that uses them.
  * Pins: see tests/test_oracle_*.py.  The sibling order, the lowest-index tie-break of argmax and the
@@ -314,6 +319,64 @@ int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const i
     free(p);
   }
   return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
+}
+
+/*
+ * Commit of the accepted path (Sec. 3.3: accepted tokens and their features are kept for the next drafting phase).
+ *
+ * Readings (the paper does not say where anything is stored): tree node m's key / value rows sit at cache slot
+ * L + m (as in oracle_tree_verify_attn); after the step the accepted nodes path[0..a-1] are part of the committed
+ * prefix, so slot L + j must hold what slot L + path[j] held, for every j < a at once, and the new prefix length
+ * is L + a.  Slots below L and from L + a on are left as they are.  features_out[b, j] = features_in[b, path[j]]
+ * for j < a and zeros for j >= a.  accepted_path rows hold node indices from the top of the tree down, then -1.
+ * A row that is not strictly increasing, leaves [0, max_tree) or points past the cache marks the sequence invalid:
+ * nothing of it is moved, its length stays L, its feature rows are zeros, valid[b] = 0.
+ *
+ * k_cache, v_cache: bf16 bit patterns [B, Hkv, S_cap, D], modified in place (either may be NULL).
+ * features_in [B, max_tree, F], features_out [B, path_cap, F]: bf16 bit patterns (both NULL when F = 0).
+ */
+int oracle_tree_commit(int batch, int num_kv_heads, int head_dim, int kv_capacity, int max_tree, int path_cap,
+                       const int32_t* seq_lens, const int32_t* accepted_path, uint16_t* k_cache, uint16_t* v_cache,
+                       int feature_dim, const uint16_t* features_in, uint16_t* features_out, int32_t* new_seq_lens,
+                       int32_t* valid) {
+  if (batch < 0 || num_kv_heads < 0 || head_dim < 0 || kv_capacity < 0 || max_tree < 0 || path_cap < 0 || feature_dim < 0)
+    return ORACLE_ERR_ARG;
+  if (!seq_lens || !accepted_path) return ORACLE_ERR_ARG;
+  const size_t row = (size_t)head_dim;
+  uint16_t* tmp = (uint16_t*)malloc(sizeof(uint16_t) * row * (size_t)(path_cap > 0 ? path_cap : 1));
+  if (!tmp) return ORACLE_ERR_NOMEM;
+  for (int b = 0; b < batch; ++b) {
+    const int32_t* path = accepted_path + (size_t)b * path_cap;
+    const int L = seq_lens[b];
+    int a = 0, ok = L >= 0;
+    while (a < path_cap && path[a] != -1) ++a;                       /* accepted length: entries before the first -1 */
+    for (int j = 0; j < a && ok; ++j) {
+      if (path[j] < 0 || path[j] >= max_tree) ok = 0;                /* a tree node */
+      else if (j > 0 && path[j] <= path[j - 1]) ok = 0;              /* a child comes after its parent */
+      else if ((long long)L + path[j] >= kv_capacity) ok = 0;        /* its slot exists */
+    }
+    if (valid) valid[b] = ok;
+    if (new_seq_lens) new_seq_lens[b] = ok ? L + a : L;
+    if (features_out)
+      memset(features_out + (size_t)b * path_cap * feature_dim, 0, sizeof(uint16_t) * (size_t)path_cap * feature_dim);
+    if (!ok) continue;
+    for (int t = 0; t < 2; ++t) {
+      uint16_t* cache = t == 0 ? k_cache : v_cache;
+      if (!cache) continue;
+      for (int g = 0; g < num_kv_heads; ++g) {
+        uint16_t* base = cache + ((size_t)b * num_kv_heads + g) * (size_t)kv_capacity * row;
+        /* simultaneous assignment: read every source row, then write every destination row */
+        for (int j = 0; j < a; ++j) memcpy(tmp + (size_t)j * row, base + (size_t)(L + path[j]) * row, sizeof(uint16_t) * row);
+        for (int j = 0; j < a; ++j) memcpy(base + (size_t)(L + j) * row, tmp + (size_t)j * row, sizeof(uint16_t) * row);
+      }
+    }
+    if (features_in && features_out)
+      for (int j = 0; j < a; ++j)
+        memcpy(features_out + ((size_t)b * path_cap + j) * feature_dim, features_in + ((size_t)b * max_tree + path[j]) * feature_dim,
+               sizeof(uint16_t) * (size_t)feature_dim);
+  }
+  free(tmp);
+  return ORACLE_OK;
 }
 
 /* Threads the OpenMP loops above use (reported next to the oracle's timing). */

@@ -16,7 +16,7 @@ from dataclasses import dataclass, field
 
 import torch
 
-STREAMS = dict(q=0, k=1, v=2, tree=3, target=4, draft=5, tokens=6, uniforms=7, lens=8, sizes=9)
+STREAMS = dict(q=0, k=1, v=2, tree=3, target=4, draft=5, tokens=6, uniforms=7, lens=8, sizes=9, paths=10, features=11)
 
 
 @dataclass(frozen=True)
@@ -186,6 +186,25 @@ def make_accept_inputs(cfg: VerifyConfig, salt: int = 0, rho: float = 0.9, rho_g
                 tokens[b, i] = int(torch.multinomial(dprob[c + 1], 1, generator=gk))
     uniforms = torch.rand((B, T + 1), generator=gu, dtype=torch.float32)
     return AcceptInputs(cfg, target, draft, tokens, parent, sizes, uniforms, gflag)
+
+
+def make_accepted_paths(sizes: torch.Tensor, parent: torch.Tensor, path_cap: int, cfg_index: int, salt: int = 0) -> torch.Tensor:
+    """One random chain per tree from a top-level node downwards (what an acceptance walk can return): at every node
+    stop with probability 1/4, else move to a random child.  int32 [B, path_cap], -1 padded; an empty tree or an
+    immediate stop gives an empty path."""
+    g = _gen(cfg_index, "paths", salt)
+    B, T = parent.shape
+    out = torch.full((B, path_cap), -1, dtype=torch.int32)
+    for b in range(B):
+        n, cur, j = int(sizes[b]), -1, 0
+        while j < path_cap:
+            kids = [i for i in range(n) if int(parent[b, i]) == cur]
+            if not kids or float(torch.rand((), generator=g)) < 0.25:
+                break
+            cur = kids[int(torch.randint(len(kids), (), generator=g))]
+            out[b, j] = cur
+            j += 1
+    return out
 
 
 def scaled(cfg: VerifyConfig, **kw) -> VerifyConfig:
