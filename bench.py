@@ -262,6 +262,24 @@ def main():
     accept_ms = statistics.mean(ev_acc[i][0].elapsed_time(ev_acc[i][1]) for i in range(min(K, 10)))
     mean_tokens = float(alen.float().mean().item()) + 1.0
 
+    # ---- commit of the accepted path for this layer's cache (the step after verification; reported, not part of the
+    # headline).  It moves rows in place, so it runs on the last input set, after everything that reads the cache.
+    s = sets[-1]
+    new_len = torch.empty((B,), dtype=torch.int32, device=dev)
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        E.eagle_tree_commit(s["k"], s["v"], s["sl"], path, T, new_seq_lens=new_len, status=status)
+    torch.cuda.synchronize()
+    c0.record()
+    for i in range(50):
+        E.eagle_tree_commit(s["k"], s["v"], s["sl"], path, T, new_seq_lens=new_len, status=status)
+    c1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    commit_ms = c0.elapsed_time(c1) / 50      # back-to-back calls: the larger of kernel time and enqueue time per call
+    moved = int(((path >= 0) & (path != torch.arange(T, device=dev, dtype=torch.int32)[None, :])).sum().item())
+    commit_bytes = moved * cfg.num_kv_heads * cfg.head_dim * 2 * 2 * 2     # rows that change slot: K and V, read + written
+
     # ---- end to end from pinned host buffers, through the library's host-buffer entry point: every step copies all
     # inputs host->device, runs attention + acceptance, and copies the results back
     pinned = dict(q=attn.q, k_cache=attn.k_cache, v_cache=attn.v_cache, seq_lens=attn.seq_lens, tree_sizes=attn.tree_sizes,
@@ -308,7 +326,9 @@ def main():
                      "algorithmic_bytes": alg_bytes, "ms_per_launch": attn_ms,
                      "tflops": alg_flops / (attn_ms * 1e-3) / 1e12},
         "breakdown": {"attn_kernel_ms": attn_ms, "accept_ms": accept_ms, "tokens_per_step": mean_tokens,
-                      "sequence_steps_per_s": value * B},
+                      "sequence_steps_per_s": value * B,
+                      "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
+                                    "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}},
     }
     if not args.no_cpu_baseline:
         done, secs, cores = oracle_step_sample(attn, acc, args.cpu_budget)

@@ -47,7 +47,8 @@ enum {
   EAGLE_ERR_SEQ = -6,        /* device-detected: seq_lens[b] < 0 or seq_lens[b] + tree size > kv_capacity */
   EAGLE_ERR_TOKEN = -7,      /* device-detected: draft token outside [0, vocab) */
   EAGLE_ERR_TIMEOUT = -8,    /* device-detected: a bounded wait inside a kernel ran out */
-  EAGLE_ERR_DEVICE = -9      /* the GPU is not an sm_100 device, or it lacks a required limit */
+  EAGLE_ERR_DEVICE = -9,     /* the GPU is not an sm_100 device, or it lacks a required limit */
+  EAGLE_ERR_PATH = -10       /* device-detected: an accepted path that is not an increasing list of tree nodes whose slots exist */
 };
 
 #define EAGLE_MAX_TREE 64
@@ -205,6 +206,41 @@ typedef struct eagle_host_step {
 
 size_t eagle_tree_verify_step_host_arena(const eagle_host_step* step);
 int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stream);
+
+typedef struct eagle_commit_desc {
+  int32_t batch;               /* B >= 0 (at most 65535) */
+  int32_t num_kv_heads;        /* Hkv >= 0 */
+  int32_t head_dim;            /* D: 64 or 128 */
+  int32_t kv_capacity;         /* S_cap: slots per (sequence, KV head) of k_cache / v_cache */
+  int32_t max_tree;            /* T_max <= 64: tree nodes are numbered 0 .. T_max-1; row count of features_in */
+  int32_t path_cap;            /* entries per row of accepted_path */
+  int32_t feature_dim;         /* F: elements per feature vector, a multiple of 8; 0 when no features are passed */
+  int32_t* status;             /* device int32 or NULL */
+} eagle_commit_desc;
+
+/*
+ * Commit of the accepted path: what the verification phase leaves behind for the next drafting phase (Sec. 3.3, last
+ * sentence: the accepted tokens and their features are recorded).  The paper does not say where anything is stored;
+ * with the cache layout of eagle_tree_verify_attn (tree node m at slot L_b + m) it is this:
+ *
+ *   k_cache, v_cache  device bf16 [B, Hkv, S_cap, D], updated IN PLACE (either may be NULL): for every sequence b with
+ *                     accepted nodes path[0..a-1], slot L_b + j <- slot L_b + path[j] for all j < a at once (the
+ *                     sources are read before any destination is written); all other slots keep their contents
+ *   seq_lens          device int32 [B]          L_b, the committed prefix before the step
+ *   accepted_path     device int32 [B, path_cap] node indices from the top of the tree down, then -1 (the output of
+ *                                               eagle_tree_accept); entries after the first -1 are ignored
+ *   features_in       device bf16 [B, T_max, F] or NULL   one vector per tree node (the target model's features)
+ *   features_out      device bf16 [B, path_cap, F] or NULL  row j <- features_in row path[j] for j < a, zeros for j >= a
+ *   new_seq_lens      device int32 [B] or NULL  L_b + a  (may alias seq_lens)
+ *
+ * One call serves one layer's cache; the token of the step's extra draw is not part of the path (its K/V do not
+ * exist yet).  A row that is not strictly increasing, leaves [0, T_max), or points at a slot >= S_cap (or L_b < 0)
+ * sets *status to EAGLE_ERR_PATH: nothing of that sequence is moved, its length is unchanged and its feature rows are
+ * zeros.  All pointers must be 16-byte aligned.  One launch, asynchronous on `stream`; no workspace.
+ */
+int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cache, const int32_t* seq_lens,
+                      const int32_t* accepted_path, const void* features_in, void* features_out,
+                      int32_t* new_seq_lens, eagle_stream_t stream);
 
 /*
  * Tree-mask builder alone (the mask "tree attention" implies: Sec. 3.1, Sec. 3.3): for every node the bit set

@@ -17,7 +17,7 @@ LIB_PATH = _PKG / "libeagle_verify.so"
 EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_tree_accept",
            "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
-           "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena"]
+           "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit"]
 _lib = None
 
 
@@ -37,6 +37,11 @@ class AcceptDesc(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("max_tree", ctypes.c_int32), ("vocab", ctypes.c_int32),
                 ("path_cap", ctypes.c_int32), ("tree_sizes", ctypes.c_void_p), ("greedy", ctypes.c_void_p),
                 ("accept_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+class CommitDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("batch", "num_kv_heads", "head_dim", "kv_capacity", "max_tree", "path_cap",
+                                              "feature_dim")] + [("status", ctypes.c_void_p)]
 
 
 class HostStep(ctypes.Structure):
@@ -69,6 +74,8 @@ def load():
         lib.eagle_tree_verify_step_host_arena.restype = ctypes.c_size_t
         lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_accept.restype = ctypes.c_int
+        lib.eagle_tree_commit.argtypes = [ctypes.POINTER(CommitDesc), vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.eagle_tree_commit.restype = ctypes.c_int
         lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
         lib.eagle_tree_build_mask.restype = ctypes.c_int
         lib.eagle_status_string.argtypes = [ctypes.c_int]
@@ -218,6 +225,27 @@ def eagle_tree_build_mask(tree_parent, tree_sizes=None, status=None, with_depth=
                                    _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "eagle_tree_build_mask")
     return anc, depth
+
+
+def eagle_tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree, features=None, features_out=None,
+                      new_seq_lens=None, status=None):
+    """Commit of the accepted path: moves the accepted nodes' K/V rows into the next prefix slots IN PLACE and gathers
+    their feature vectors.  Returns (new_seq_lens, features_out); both are allocated when not passed in."""
+    lib = load()
+    B, Hkv, S, D = k_cache.shape
+    cap = accepted_path.shape[1]
+    F = 0 if features is None else features.shape[2]
+    if new_seq_lens is None:
+        new_seq_lens = torch.empty((B,), dtype=torch.int32, device=k_cache.device)
+    if features is not None and features_out is None:
+        features_out = torch.empty((B, cap, F), dtype=torch.bfloat16, device=k_cache.device)
+    d = CommitDesc(B, Hkv, D, S, max_tree, cap, F, _dev(status, torch.int32, "status", True))
+    rc = lib.eagle_tree_commit(ctypes.byref(d), _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache", True),
+                               _dev(seq_lens, torch.int32, "seq_lens"), _dev(accepted_path, torch.int32, "accepted_path"),
+                               _dev(features, torch.bfloat16, "features", True), _dev(features_out, torch.bfloat16, "features_out", True),
+                               _dev(new_seq_lens, torch.int32, "new_seq_lens"), _stream())
+    _check(rc, "eagle_tree_commit")
+    return new_seq_lens, features_out
 
 
 class HostStepRunner:

@@ -453,6 +453,43 @@ int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stre
   return ok ? EAGLE_OK : EAGLE_ERR_LAUNCH;
 }
 
+int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cache, const int32_t* seq_lens,
+                      const int32_t* accepted_path, const void* features_in, void* features_out,
+                      int32_t* new_seq_lens, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const eagle_commit_desc& d = *desc;
+  if (d.batch < 0 || d.batch > 65535 || d.num_kv_heads < 0 || d.num_kv_heads > 65535 || (d.head_dim != 64 && d.head_dim != 128) ||
+      d.kv_capacity < 0 || d.max_tree < 0 || d.max_tree > kMaxTree || d.path_cap < 0 || d.feature_dim < 0 || d.feature_dim % 8)
+    return EAGLE_ERR_SHAPE;
+  if (d.batch == 0) return EAGLE_OK;
+  if (!seq_lens || (d.path_cap > 0 && !accepted_path)) return EAGLE_ERR_NULL;
+  const bool feats = d.feature_dim > 0 && features_out != nullptr;
+  if (feats && !features_in) return EAGLE_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(k_cache) & 15) || (reinterpret_cast<uintptr_t>(v_cache) & 15) ||
+      (reinterpret_cast<uintptr_t>(features_in) & 15) || (reinterpret_cast<uintptr_t>(features_out) & 15))
+    return EAGLE_ERR_SHAPE;
+  int err = 0;
+  if (!device_info(&err)) return err;
+  CommitParams cp;
+  cp.k = static_cast<__nv_bfloat16*>(k_cache);
+  cp.v = static_cast<__nv_bfloat16*>(v_cache);
+  cp.seq_lens = seq_lens;
+  cp.path = accepted_path;
+  cp.features_in = feats ? static_cast<const __nv_bfloat16*>(features_in) : nullptr;
+  cp.features_out = feats ? static_cast<__nv_bfloat16*>(features_out) : nullptr;
+  cp.new_seq_lens = new_seq_lens;
+  cp.B = d.batch;
+  cp.Hkv = d.num_kv_heads;
+  cp.D = d.head_dim;
+  cp.S_cap = d.kv_capacity;
+  cp.T_max = d.max_tree;
+  cp.path_cap = d.path_cap;
+  cp.F = d.feature_dim;
+  cp.status = d.status;
+  if (launch_commit(cp, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
+
 const char* eagle_status_string(int code) {
   switch (code) {
     case EAGLE_OK: return "ok";
@@ -465,6 +502,7 @@ const char* eagle_status_string(int code) {
     case EAGLE_ERR_TOKEN: return "draft token outside the vocabulary";
     case EAGLE_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case EAGLE_ERR_DEVICE: return "no usable sm_100 device is current";
+    case EAGLE_ERR_PATH: return "invalid accepted path (not increasing, outside the tree, or past the cache)";
     default: return "unknown status";
   }
 }

@@ -140,6 +140,18 @@ struct PlanParams {
   int32_t* status;
 };
 
+struct CommitParams {
+  __nv_bfloat16* k;          // [B, Hkv, S_cap, D], in place (may be null)
+  __nv_bfloat16* v;
+  const int32_t* seq_lens;   // [B]
+  const int32_t* path;       // [B, path_cap], -1 padded
+  const __nv_bfloat16* features_in;   // [B, T_max, F] or null
+  __nv_bfloat16* features_out;        // [B, path_cap, F] or null
+  int32_t* new_seq_lens;     // [B] or null
+  int32_t B, Hkv, D, S_cap, T_max, path_cap, F;
+  int32_t* status;
+};
+
 struct AcceptParams {
   const float* target;   // [B, T+1, V]
   const float* draft;    // [B, T, V]
@@ -169,6 +181,7 @@ cudaError_t attn_prepare(int head_dim);
 cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cudaStream_t stream);
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
+cudaError_t launch_commit(const CommitParams& p, cudaStream_t stream);
 void count_launch();
 
 }  // namespace eagle
