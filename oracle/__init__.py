@@ -44,6 +44,8 @@ def _load():
         lib.oracle_tree_verify_attn.restype = i32
         lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 13
         lib.oracle_tree_accept.restype = i32
+        lib.oracle_tree_accept_logits.argtypes = [i32, i32, i32, i32] + [vp] * 7 + [dbl] + [vp] * 6
+        lib.oracle_tree_accept_logits.restype = i32
         lib.oracle_tree_commit.argtypes = [i32] * 6 + [vp] * 4 + [i32] + [vp] * 4
         lib.oracle_tree_commit.restype = i32
         lib.oracle_num_threads.restype = i32
@@ -108,7 +110,7 @@ def tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, tree_sizes=None
 
 
 def tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, tree_sizes=None, greedy=None,
-                path_cap: int | None = None):
+                path_cap: int | None = None, temperature: float | None = None):
     """Acceptance walk (Algorithm 1 at every node, or the greedy rule).  Returns a dict of numpy arrays:
     accepted_path [B, path_cap], bonus_token [B], accept_len [B], min_margin [B], n_sweeps [B],
     n_zero_mass [B]."""
@@ -128,13 +130,26 @@ def tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, 
     res = dict(accepted_path=np.full((B, cap), -1, np.int32), bonus_token=np.full((B,), -1, np.int32),
                accept_len=np.zeros((B,), np.int32), min_margin=np.zeros((B,), np.float64),
                n_sweeps=np.zeros((B,), np.int32), n_zero_mass=np.zeros((B,), np.int32))
-    rc = _load().oracle_tree_accept(B, T, V, cap, _ptr(ts), _ptr(gr), _ptr(tp), _ptr(dp), _ptr(tok), _ptr(par),
-                                    _ptr(un), _ptr(res["accepted_path"]), _ptr(res["bonus_token"]),
-                                    _ptr(res["accept_len"]), _ptr(res["min_margin"]), _ptr(res["n_sweeps"]),
-                                    _ptr(res["n_zero_mass"]))
+    if temperature is None:
+        rc = _load().oracle_tree_accept(B, T, V, cap, _ptr(ts), _ptr(gr), _ptr(tp), _ptr(dp), _ptr(tok), _ptr(par),
+                                        _ptr(un), _ptr(res["accepted_path"]), _ptr(res["bonus_token"]),
+                                        _ptr(res["accept_len"]), _ptr(res["min_margin"]), _ptr(res["n_sweeps"]),
+                                        _ptr(res["n_zero_mass"]))
+    else:
+        rc = _load().oracle_tree_accept_logits(B, T, V, cap, _ptr(ts), _ptr(gr), _ptr(tp), _ptr(dp), _ptr(tok), _ptr(par),
+                                               _ptr(un), float(temperature), _ptr(res["accepted_path"]),
+                                               _ptr(res["bonus_token"]), _ptr(res["accept_len"]), _ptr(res["min_margin"]),
+                                               _ptr(res["n_sweeps"]), _ptr(res["n_zero_mass"]))
     if rc != 0:
         raise ValueError(f"oracle_tree_accept failed: {rc}")
     return res
+
+
+def tree_accept_logits(target_logits, draft_logits, draft_tokens, tree_parent, uniforms, temperature: float,
+                       tree_sizes=None, greedy=None, path_cap: int | None = None):
+    """The acceptance walk with the distributions given as fp32 logits: rows are softmax(logits / temperature) in fp64."""
+    return tree_accept(target_logits, draft_logits, draft_tokens, tree_parent, uniforms, tree_sizes=tree_sizes, greedy=greedy,
+                       path_cap=path_cap, temperature=temperature)
 
 
 def tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree: int, features=None):

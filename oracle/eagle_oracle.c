@@ -15,6 +15,7 @@
  *   oracle_tree_accept       - Algorithm 1 (multi-round speculative sampling, App. A.2) applied
  *                              recursively at every node from the root (Sec. 3.3); the greedy setting
  *                              (Preliminaries) is the same rule with a one-hot target distribution.
+ *   oracle_tree_accept_logits - the same with the distributions given as logits (softmax at a temperature, fp64).
  *   oracle_tree_commit       - Sec. 3.3, last sentence: the accepted tokens and their features are recorded
  *                              for the next drafting phase.  For the target's KV cache that means: the
  *                              keys and values of the accepted tree nodes become the next slots of the
@@ -198,11 +199,29 @@ int oracle_tree_verify_attn(int batch, int num_q_heads, int num_kv_heads, int he
  *   Greedy: a = argmax p (lowest id on ties); move to the lowest-index child whose token is a,
  *   else emit a.  Exactly one extra token is emitted per call.
  */
-int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const int32_t* tree_sizes,
+/* One row of a distribution as fp64: the fp32 probabilities as given, or (logits != 0) the softmax of the fp32
+ * logits at the given temperature, p(v) = exp((z_v - max z) / T) / sum, every operation in fp64. */
+static void load_row(double* dst, const float* row, int vocab, int logits, double temperature) {
+  if (!logits) {
+    for (int v = 0; v < vocab; ++v) dst[v] = (double)row[v];
+    return;
+  }
+  double zmax = -INFINITY;
+  for (int v = 0; v < vocab; ++v)
+    if ((double)row[v] > zmax) zmax = (double)row[v];
+  double sum = 0.0;
+  for (int v = 0; v < vocab; ++v) {
+    dst[v] = exp(((double)row[v] - zmax) / temperature);
+    sum += dst[v];
+  }
+  for (int v = 0; v < vocab; ++v) dst[v] /= sum;
+}
+
+static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const int32_t* tree_sizes,
                        const uint8_t* greedy, const float* target_probs, const float* draft_probs,
                        const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
                        int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
-                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass) {
+                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass, int logits, double temperature) {
   if (batch < 0 || max_tree < 0 || max_tree > 64 || vocab <= 0 || path_cap < 0 || !target_probs ||
       !tree_parent || !draft_tokens || !accepted_path || !bonus_token)
     return ORACLE_ERR_ARG;
@@ -226,16 +245,17 @@ int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const i
     const int32_t* tok = draft_tokens + (size_t)b * max_tree;
     int32_t* path = accepted_path + (size_t)b * path_cap;
     for (int j = 0; j < path_cap; ++j) path[j] = -1;
-    double* p = (double*)malloc(sizeof(double) * (size_t)vocab);
+    double* p = (double*)malloc(sizeof(double) * 2 * (size_t)vocab);
     if (!p) {
       failed = 1;
       continue;
     }
+    double* q = p + vocab;   /* the draft row of the candidate under test */
     int cur = -1, len = 0, sweeps = 0, zero_mass = 0, bonus = -1;
     double margin = INFINITY;
     for (;;) {
       const float* prow = target_probs + ((size_t)b * (max_tree + 1) + (size_t)(cur + 1)) * vocab;
-      for (int v = 0; v < vocab; ++v) p[v] = (double)prow[v];
+      load_row(p, prow, vocab, logits, temperature);
       int next = -1;
       if (is_greedy) {
         int a = 0;
@@ -255,7 +275,8 @@ int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const i
           const float* qrow = draft_probs + ((size_t)b * max_tree + i) * vocab;
           const int t = tok[i];
           const double r = (double)uniforms[(size_t)b * (max_tree + 1) + i];
-          const double pt = p[t], qt = (double)qrow[t];
+          load_row(q, qrow, vocab, logits, temperature);
+          const double pt = p[t], qt = q[t];
           if (qt > 0.0) {
             const double m = fabs(r - pt / qt);
             if (m < margin) margin = m;
@@ -265,13 +286,13 @@ int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const i
           } else {
             double Z = 0.0;
             for (int v = 0; v < vocab; ++v) {
-              const double d = p[v] - (double)qrow[v];
+              const double d = p[v] - q[v];
               Z += d > 0.0 ? d : 0.0;
             }
             ++sweeps;
             if (Z > 0.0) {
               for (int v = 0; v < vocab; ++v) {
-                const double d = p[v] - (double)qrow[v];
+                const double d = p[v] - q[v];
                 p[v] = (d > 0.0 ? d : 0.0) / Z;
               }
             } else {
@@ -319,6 +340,31 @@ int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const i
     free(p);
   }
   return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
+}
+
+int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const int32_t* tree_sizes,
+                       const uint8_t* greedy, const float* target_probs, const float* draft_probs,
+                       const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                       int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
+                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass) {
+  return accept_walk(batch, max_tree, vocab, path_cap, tree_sizes, greedy, target_probs, draft_probs, draft_tokens,
+                     tree_parent, uniforms, accepted_path, bonus_token, accept_len, min_margin, n_sweeps, n_zero_mass, 0, 1.0);
+}
+
+/*
+ * The same walk on LOGITS: every target / draft row is the softmax of the given fp32 logits at `temperature` > 0
+ * (Sec. 4: the experiments sample at temperature 1; temperature 0 is the greedy flag), taken in fp64.  Greedy
+ * sequences use the argmax, which the softmax does not move.
+ */
+int oracle_tree_accept_logits(int batch, int max_tree, int vocab, int path_cap, const int32_t* tree_sizes,
+                              const uint8_t* greedy, const float* target_logits, const float* draft_logits,
+                              const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                              double temperature, int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
+                              double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass) {
+  if (!(temperature > 0.0)) return ORACLE_ERR_ARG;
+  return accept_walk(batch, max_tree, vocab, path_cap, tree_sizes, greedy, target_logits, draft_logits, draft_tokens,
+                     tree_parent, uniforms, accepted_path, bonus_token, accept_len, min_margin, n_sweeps, n_zero_mass, 1,
+                     temperature);
 }
 
 /*
