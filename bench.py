@@ -262,6 +262,24 @@ def main():
     accept_ms = statistics.mean(ev_acc[i][0].elapsed_time(ev_acc[i][1]) for i in range(min(K, 10)))
     mean_tokens = float(alen.float().mean().item()) + 1.0
 
+    # ---- the same acceptance on logits (softmax fused into the walk; reported, not part of the headline).  The logits are
+    # the logarithms of the step's probabilities, so at temperature 1 the walk must return the same tokens.
+    s = sets[0]
+    path_p, bonus_p = path.clone(), bonus.clone()
+    zt, zd = s["tp"].clamp_min(1e-37).log(), s["dp"].clamp_min(1e-37).log()
+    path_l, bonus_l = torch.empty_like(path), torch.empty_like(bonus)
+    l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    E.eagle_tree_accept_logits(zt, zd, s["tok"], s["par"], s["un"], 1.0, path_l, bonus_l, tree_sizes=s["ts"], greedy=s["gr"], status=status)
+    l0.record()
+    for i in range(5):
+        E.eagle_tree_accept_logits(zt, zd, s["tok"], s["par"], s["un"], 1.0, path_l, bonus_l, tree_sizes=s["ts"], greedy=s["gr"],
+                                   status=status)
+    l1.record()
+    torch.cuda.synchronize()
+    accept_logits_ms = l0.elapsed_time(l1) / 5
+    logits_same = int(((path_l == path_p).all(dim=1) & (bonus_l == bonus_p)).sum().item())
+    del zt, zd
+
     # ---- commit of the accepted path for this layer's cache (the step after verification; reported, not part of the
     # headline).  It moves rows in place, so it runs on the last input set, after everything that reads the cache.
     s = sets[-1]
@@ -327,6 +345,8 @@ def main():
                      "tflops": alg_flops / (attn_ms * 1e-3) / 1e12},
         "breakdown": {"attn_kernel_ms": attn_ms, "accept_ms": accept_ms, "tokens_per_step": mean_tokens,
                       "sequence_steps_per_s": value * B,
+                      "accept_on_logits": {"ms": accept_logits_ms, "temperature": 1.0,
+                                           "sequences_with_the_same_tokens_as_on_probabilities": logits_same, "of": B},
                       "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
                                     "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}},
     }

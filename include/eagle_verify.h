@@ -207,6 +207,24 @@ typedef struct eagle_host_step {
 size_t eagle_tree_verify_step_host_arena(const eagle_host_step* step);
 int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stream);
 
+/*
+ * The same acceptance walk with the distributions given as LOGITS: every row the walk touches is taken as
+ * softmax(logits / temperature) without being materialised (the target and draft probability tensors, [B, T_max+1, V]
+ * and [B, T_max, V], are never written or read as a whole; only the rows on the walk are swept).  Sec. 4 runs the
+ * method at temperature 1 (and at temperature 0, which is the per-sequence `greedy` flag of the descriptor: greedy
+ * sequences use the argmax of the logits and ignore `temperature`).
+ *
+ *   target_logits device fp32 [B, T_max+1, V], draft_logits device fp32 [B, T_max, V]; temperature > 0 (else
+ *   EAGLE_ERR_SHAPE); everything else as for eagle_tree_accept.
+ *
+ * Each row costs one more sweep (its maximum and its mass).  Exponentials are taken in fp32 (2^((z - max) * log2(e) /
+ * temperature)), sums and scalars in fp64, so a decision can differ from an fp64 softmax only when it sits within
+ * about 1e-6 of its boundary.
+ */
+int eagle_tree_accept_logits(const eagle_accept_desc* desc, const float* target_logits, const float* draft_logits,
+                             const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                             float temperature, int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream);
+
 typedef struct eagle_commit_desc {
   int32_t batch;               /* B >= 0 (at most 65535) */
   int32_t num_kv_heads;        /* Hkv >= 0 */

@@ -17,7 +17,8 @@ LIB_PATH = _PKG / "libeagle_verify.so"
 EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_tree_accept",
            "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
-           "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit"]
+           "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit",
+           "eagle_tree_accept_logits"]
 _lib = None
 
 
@@ -74,6 +75,8 @@ def load():
         lib.eagle_tree_verify_step_host_arena.restype = ctypes.c_size_t
         lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_accept.restype = ctypes.c_int
+        lib.eagle_tree_accept_logits.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
+        lib.eagle_tree_accept_logits.restype = ctypes.c_int
         lib.eagle_tree_commit.argtypes = [ctypes.POINTER(CommitDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_commit.restype = ctypes.c_int
         lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
@@ -185,9 +188,11 @@ def static_capacity() -> int:
 
 
 def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, accepted_path=None,
-                      bonus_token=None, *, tree_sizes=None, greedy=None, accept_len=None, status=None, path_cap=None):
+                      bonus_token=None, *, tree_sizes=None, greedy=None, accept_len=None, status=None, path_cap=None,
+                      temperature=None):
     """Acceptance walk.  target_probs [B,T+1,V] fp32; draft_probs [B,T,V] fp32; draft_tokens/tree_parent [B,T]
-    int32; uniforms [B,T+1] fp32.  Returns (accepted_path [B,path_cap] int32, bonus_token [B] int32)."""
+    int32; uniforms [B,T+1] fp32.  Returns (accepted_path [B,path_cap] int32, bonus_token [B] int32).
+    With ``temperature`` the two tensors hold logits (``eagle_tree_accept_logits``)."""
     lib = load()
     B, T1, V = target_probs.shape
     T = T1 - 1
@@ -205,13 +210,22 @@ def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, unif
         raise EagleError("uniforms must be [B, T+1]")
     d = AcceptDesc(B, T, V, cap, _dev(tree_sizes, torch.int32, "tree_sizes", True), _dev(greedy, torch.uint8, "greedy", True),
                    _dev(accept_len, torch.int32, "accept_len", True), _dev(status, torch.int32, "status", True))
-    rc = lib.eagle_tree_accept(ctypes.byref(d), _dev(target_probs, torch.float32, "target_probs"),
-                               _dev(draft_probs, torch.float32, "draft_probs", True),
-                               _dev(draft_tokens, torch.int32, "draft_tokens"), _dev(tree_parent, torch.int32, "tree_parent"),
-                               _dev(uniforms, torch.float32, "uniforms", True), _dev(accepted_path, torch.int32, "accepted_path"),
-                               _dev(bonus_token, torch.int32, "bonus_token"), _stream())
-    _check(rc, "eagle_tree_accept")
+    head = (ctypes.byref(d), _dev(target_probs, torch.float32, "target_probs"), _dev(draft_probs, torch.float32, "draft_probs", True),
+            _dev(draft_tokens, torch.int32, "draft_tokens"), _dev(tree_parent, torch.int32, "tree_parent"),
+            _dev(uniforms, torch.float32, "uniforms", True))
+    tail = (_dev(accepted_path, torch.int32, "accepted_path"), _dev(bonus_token, torch.int32, "bonus_token"), _stream())
+    if temperature is None:
+        _check(lib.eagle_tree_accept(*head, *tail), "eagle_tree_accept")
+    else:
+        _check(lib.eagle_tree_accept_logits(*head, float(temperature), *tail), "eagle_tree_accept_logits")
     return accepted_path, bonus_token
+
+
+def eagle_tree_accept_logits(target_logits, draft_logits, draft_tokens, tree_parent, uniforms, temperature, accepted_path=None,
+                             bonus_token=None, **kw):
+    """Acceptance walk on logits: rows are softmax(logits / temperature), never materialised."""
+    return eagle_tree_accept(target_logits, draft_logits, draft_tokens, tree_parent, uniforms, accepted_path, bonus_token,
+                             temperature=temperature, **kw)
 
 
 def eagle_tree_build_mask(tree_parent, tree_sizes=None, status=None, with_depth=True):

@@ -17,6 +17,11 @@
 //   u_k(v) = max(0, u_{k-1}(v) - W_{k-1} * p^_k(v)),   W_k = sum_v u_k(v),
 // so that Algorithm 1's normalised residual is u_m / W_m, its accept test r < p(t)/p^(t) reads
 // r * p^(t) * W_m < u_m(t), and the final draw (scale-free) is taken from u_m.  No division is needed.
+//
+// Logits instead of probabilities (LOGITS = true): a row is softmax(z / T), never materialised.  Each row the walk
+// touches costs one more sweep for its maximum m and its mass Z = sum_v w(v), w(v) = 2^((z_v - m) * log2(e) / T);
+// then u_0 = w of the target row with W_0 = Z, and a draft row enters as p^ = w^ / Z^ (the scalar 1 / Z^ is folded
+// into the stored W_k).  Exponentials are fp32 (the logits are), sums fp64.
 #include "common.cuh"
 
 namespace eagle {
@@ -152,32 +157,45 @@ __device__ __forceinline__ unsigned int ordered_bits(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+__device__ __forceinline__ float from_ordered_bits(unsigned int b) {
+  return __uint_as_float((b & 0x80000000u) ? (b & 0x7fffffffu) : ~b);
+}
+
 // The residual after the rejections recorded so far, evaluated on the fly.
+template <bool LOGITS>
 struct Residual {
   const float* target_row;
   const float* draft_base;  // draft rows of this sequence
   const int* rej;           // rejected candidates at the current node, in order
-  const double* scale;      // scale[k] = W_k, the mass of the residual before rejection k+1 (W_0 = 1)
+  const double* scale;      // scale[k] = W_k, the mass of the residual before rejection k+1 (W_0 = 1); logits: W_k / Z^_k
+  const float* row_max;     // logits: maximum of the rejected candidates' draft rows
+  float t_max, c;           // logits: maximum of the target row; log2(e) / temperature
   int m;                    // rejections recorded
   int V;
 
+  // value of a row entry: the probability as given, or the unnormalised softmax weight
+  __device__ __forceinline__ double val(float z, float zmax) const {
+    if (LOGITS) return static_cast<double>(exp2f((z - zmax) * c));
+    return static_cast<double>(z);
+  }
   __device__ __forceinline__ double at(int v) const {
-    double x = static_cast<double>(__ldg(target_row + v));
+    double x = val(__ldg(target_row + v), t_max);
     for (int k = 0; k < m; ++k)
-      x = fmax(0.0, fma(-scale[k], static_cast<double>(__ldg(draft_base + static_cast<size_t>(rej[k]) * V + v)), x));
+      x = fmax(0.0, fma(-scale[k], val(__ldg(draft_base + static_cast<size_t>(rej[k]) * V + v), LOGITS ? row_max[k] : 0.f), x));
     return x;
   }
   // four consecutive tokens starting at v (v % 4 == 0, rows 16-byte aligned)
   __device__ __forceinline__ void at4(int v, double (&x)[4]) const {
     const float4 t = __ldg(reinterpret_cast<const float4*>(target_row + v));
-    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+    x[0] = val(t.x, t_max); x[1] = val(t.y, t_max); x[2] = val(t.z, t_max); x[3] = val(t.w, t_max);
     for (int k = 0; k < m; ++k) {
       const float4 q = __ldg(reinterpret_cast<const float4*>(draft_base + static_cast<size_t>(rej[k]) * V + v));
       const double w = -scale[k];
-      x[0] = fmax(0.0, fma(w, static_cast<double>(q.x), x[0]));
-      x[1] = fmax(0.0, fma(w, static_cast<double>(q.y), x[1]));
-      x[2] = fmax(0.0, fma(w, static_cast<double>(q.z), x[2]));
-      x[3] = fmax(0.0, fma(w, static_cast<double>(q.w), x[3]));
+      const float qm = LOGITS ? row_max[k] : 0.f;
+      x[0] = fmax(0.0, fma(w, val(q.x, qm), x[0]));
+      x[1] = fmax(0.0, fma(w, val(q.y, qm), x[1]));
+      x[2] = fmax(0.0, fma(w, val(q.z, qm), x[2]));
+      x[3] = fmax(0.0, fma(w, val(q.w, qm), x[3]));
     }
   }
 };
@@ -185,9 +203,10 @@ struct Residual {
 struct TreeSmem {
   int par[kMaxTree], tok[kMaxTree], rej[kMaxTree];
   double scale[kMaxTree];
+  float row_max[kMaxTree];
 };
 
-template <int NT, int CL>
+template <int NT, int CL, bool LOGITS>
 __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_kernel(AcceptParams p) {
   using TeamT = Team<NT, CL>;
   constexpr int TEAMS = NT == 32 ? kWarpTeamsPerCta : 1;
@@ -247,6 +266,35 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
   chunk = (chunk + 3) & ~3;
   const int v0 = min(team.rank() * chunk, V), v1 = min(v0 + chunk, V);
 
+  // logits: maximum and softmax mass of a row (two sweeps of the thread's range, the second from cache)
+  const float c = p.inv_temp_log2;
+  auto row_stats = [&](const float* row, float* zmax, double* mass) {
+    float mx = -INFINITY;
+    if (vec) {
+#pragma unroll 4
+      for (int v = v0; v < v1; v += 4) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(row + v));
+        mx = fmaxf(fmaxf(mx, fmaxf(t.x, t.y)), fmaxf(t.z, t.w));
+      }
+    } else {
+      for (int v = v0; v < v1; ++v) mx = fmaxf(mx, __ldg(row + v));
+    }
+    mx = from_ordered_bits(static_cast<unsigned int>(team.max_u64(static_cast<unsigned long long>(ordered_bits(mx)) << 32) >> 32));
+    double z = 0.0;
+    if (vec) {
+#pragma unroll 4
+      for (int v = v0; v < v1; v += 4) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(row + v));
+        z += static_cast<double>(exp2f((t.x - mx) * c)) + static_cast<double>(exp2f((t.y - mx) * c));
+        z += static_cast<double>(exp2f((t.z - mx) * c)) + static_cast<double>(exp2f((t.w - mx) * c));
+      }
+    } else {
+      for (int v = v0; v < v1; ++v) z += static_cast<double>(exp2f((__ldg(row + v) - mx) * c));
+    }
+    *zmax = mx;
+    *mass = team.sum(z);
+  };
+
   int cur = -1, len = 0, bonus = -1;
   for (;;) {
     const float* prow = target_b + static_cast<size_t>(cur + 1) * V;
@@ -273,15 +321,24 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
         if (ts.par[i] == cur && ts.tok[i] == a) next = i;
       if (next < 0) bonus = a;
     } else {
-      Residual res{prow, draft_b, ts.rej, ts.scale, 0, V};
+      Residual<LOGITS> res{prow, draft_b, ts.rej, ts.scale, ts.row_max, 0.f, c, 0, V};
       double W = 1.0;   // mass of the current residual
+      if (LOGITS) row_stats(prow, &res.t_max, &W);
       for (int i = 0; i < n && next < 0; ++i) {
         if (ts.par[i] != cur) continue;
         const float* qrow = draft_b + static_cast<size_t>(i) * V;
         const int t = ts.tok[i];
         const double r = static_cast<double>(uni_b[i]);
-        const double ut = res.at(t), qt = static_cast<double>(__ldg(qrow + t));
-        if (r * qt * W < ut) {
+        float q_max = 0.f;
+        double q_inv = 1.0;     // 1 / mass of the candidate's draft row
+        if (LOGITS) {
+          double q_mass;
+          row_stats(qrow, &q_max, &q_mass);
+          q_inv = 1.0 / q_mass;
+        }
+        const double Wq = W * q_inv;   // what a draft-row entry is multiplied with inside the residual
+        const double ut = res.at(t), qt = res.val(__ldg(qrow + t), q_max);
+        if (r * qt * Wq < ut) {
           next = i;
         } else {
           // mass of max(0, u - W * p^_i) over the vocabulary
@@ -292,20 +349,21 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
               double x[4];
               res.at4(v, x);
               const float4 q = __ldg(reinterpret_cast<const float4*>(qrow + v));
-              z += fmax(0.0, fma(-W, static_cast<double>(q.x), x[0]));
-              z += fmax(0.0, fma(-W, static_cast<double>(q.y), x[1]));
-              z += fmax(0.0, fma(-W, static_cast<double>(q.z), x[2]));
-              z += fmax(0.0, fma(-W, static_cast<double>(q.w), x[3]));
+              z += fmax(0.0, fma(-Wq, res.val(q.x, q_max), x[0]));
+              z += fmax(0.0, fma(-Wq, res.val(q.y, q_max), x[1]));
+              z += fmax(0.0, fma(-Wq, res.val(q.z, q_max), x[2]));
+              z += fmax(0.0, fma(-Wq, res.val(q.w, q_max), x[3]));
             }
           } else {
-            for (int v = v0; v < v1; ++v) z += fmax(0.0, fma(-W, static_cast<double>(__ldg(qrow + v)), res.at(v)));
+            for (int v = v0; v < v1; ++v) z += fmax(0.0, fma(-Wq, res.val(__ldg(qrow + v), q_max), res.at(v)));
           }
           z = team.sum(z);
           if (z > 0.0) {           // zero residual mass: the distribution is kept as it is
             // entry res.m is not read by anyone yet (readers stop at res.m), so it can be written in place
             if (team.tid == 0) {
               ts.rej[res.m] = i;
-              ts.scale[res.m] = W;
+              ts.scale[res.m] = Wq;
+              ts.row_max[res.m] = q_max;
             }
             team.sync_cta();
             res.m += 1;
@@ -410,7 +468,8 @@ cudaError_t launch_cluster(const AcceptParams& p, cudaStream_t stream) {
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, accept_kernel<kCtaThreads, CL>, p);
+  if (p.logits) return cudaLaunchKernelEx(&cfg, accept_kernel<kCtaThreads, CL, true>, p);
+  return cudaLaunchKernelEx(&cfg, accept_kernel<kCtaThreads, CL, false>, p);
 }
 
 }  // namespace
@@ -423,7 +482,8 @@ cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stre
   cudaError_t e;
   if (p.V <= 4096) {
     const unsigned blocks = static_cast<unsigned>((p.B + kWarpTeamsPerCta - 1) / kWarpTeamsPerCta);
-    accept_kernel<32, 1><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
+    if (p.logits) accept_kernel<32, 1, true><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
+    else accept_kernel<32, 1, false><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
     e = cudaGetLastError();
   } else {
     const long long resident = 4ll * sm_count;   // CTAs of 512 threads that can be resident at once
@@ -431,7 +491,8 @@ cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stre
     else if (4ll * p.B <= resident) e = launch_cluster<4>(p, stream);
     else if (2ll * p.B <= resident) e = launch_cluster<2>(p, stream);
     else {
-      accept_kernel<kCtaThreads, 1><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
+      if (p.logits) accept_kernel<kCtaThreads, 1, true><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
+      else accept_kernel<kCtaThreads, 1, false><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
       e = cudaGetLastError();
     }
   }

@@ -158,22 +158,25 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   return EAGLE_OK;
 }
 
-int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, const float* draft_probs,
-                      const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
-                      int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream_) {
+namespace {
+
+// Shared by the two acceptance entry points: `temperature` < 0 means the rows are probabilities.
+int accept_call(const eagle_accept_desc* desc, const float* target, const float* draft, const int32_t* draft_tokens,
+                const int32_t* tree_parent, const float* uniforms, float temperature, int32_t* accepted_path,
+                int32_t* bonus_token, eagle_stream_t stream_) {
   if (!desc) return EAGLE_ERR_NULL;
   const eagle_accept_desc& d = *desc;
   if (d.batch < 0 || d.max_tree < 0 || d.max_tree > kMaxTree || d.vocab < 1 || d.path_cap < 0) return EAGLE_ERR_SHAPE;
   if (d.batch == 0) return EAGLE_OK;
-  if (!target_probs || !draft_tokens || !tree_parent || !accepted_path || !bonus_token) return EAGLE_ERR_NULL;
+  if (!target || !draft_tokens || !tree_parent || !accepted_path || !bonus_token) return EAGLE_ERR_NULL;
   // stochastic sequences need the draft rows and the uniforms; only an all-greedy call may omit them
-  if ((!draft_probs || !uniforms) && !d.greedy) return EAGLE_ERR_NULL;
+  if ((!draft || !uniforms) && !d.greedy) return EAGLE_ERR_NULL;
   int err = 0;
   DeviceInfo* dev = device_info(&err);
   if (!dev) return err;
   AcceptParams ap;
-  ap.target = target_probs;
-  ap.draft = draft_probs;
+  ap.target = target;
+  ap.draft = draft;
   ap.tokens = draft_tokens;
   ap.parent = tree_parent;
   ap.uniforms = uniforms;
@@ -187,8 +190,26 @@ int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, 
   ap.T = d.max_tree;
   ap.V = d.vocab;
   ap.path_cap = d.path_cap;
+  ap.logits = temperature >= 0.f ? 1 : 0;
+  ap.inv_temp_log2 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
   if (launch_accept(ap, dev->sm_count, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
+}
+
+}  // namespace
+
+int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, const float* draft_probs,
+                      const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                      int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream_) {
+  return accept_call(desc, target_probs, draft_probs, draft_tokens, tree_parent, uniforms, -1.f, accepted_path, bonus_token, stream_);
+}
+
+int eagle_tree_accept_logits(const eagle_accept_desc* desc, const float* target_logits, const float* draft_logits,
+                             const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
+                             float temperature, int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream_) {
+  if (!(temperature > 0.f) || !(temperature < 3.0e38f)) return EAGLE_ERR_SHAPE;
+  return accept_call(desc, target_logits, draft_logits, draft_tokens, tree_parent, uniforms, temperature, accepted_path, bonus_token,
+                     stream_);
 }
 
 int eagle_tree_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int32_t batch, int32_t max_tree,

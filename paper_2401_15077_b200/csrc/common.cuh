@@ -165,6 +165,8 @@ struct AcceptParams {
   int32_t* accept_len;   // [B] or null
   int32_t* status;
   int32_t B, T, V, path_cap;
+  int32_t logits;        // target / draft hold logits: rows are softmax(logits / temperature)
+  float inv_temp_log2;   // log2(e) / temperature
 };
 
 __device__ inline void report_status(int32_t* status, int code) {

@@ -147,11 +147,12 @@ class AcceptInputs:
 
 
 def make_accept_inputs(cfg: VerifyConfig, salt: int = 0, rho: float = 0.9, rho_greedy: float = 0.98,
-                       trees=None, vocab: int | None = None, greedy: str | None = None) -> AcceptInputs:
+                       trees=None, vocab: int | None = None, greedy: str | None = None, logits: bool = False) -> AcceptInputs:
     """Target logits ~ N(0, variance 2); draft logits = rho*target + sqrt(1-rho^2)*fresh (same marginal).
     Row i of ``draft_probs`` is the softmax of the draft logits at node i's parent; stochastic sequences
     draw node tokens i.i.d. from that row, greedy sequences give the j-th child the parent's rank-j draft
-    token.  ``rho`` = 0 is the uncorrelated (rejection-heavy) case."""
+    token.  ``rho`` = 0 is the uncorrelated (rejection-heavy) case.  With ``logits`` the two tensors hold the logits
+    themselves (for the entry point that takes logits); tokens are drawn the same way."""
     B, T = cfg.batch, cfg.max_tree
     V = vocab or cfg.vocab
     sizes, parent = trees if trees is not None else make_trees(cfg, salt)
@@ -172,12 +173,12 @@ def make_accept_inputs(cfg: VerifyConfig, salt: int = 0, rho: float = 0.9, rho_g
         tl = torch.randn((T + 1, V), generator=gt, dtype=torch.float32) * sigma
         fresh = torch.randn((T + 1, V), generator=gd, dtype=torch.float32) * sigma
         dl = r * tl + math.sqrt(max(0.0, 1.0 - r * r)) * fresh
-        target[b] = torch.softmax(tl, dim=-1)
+        target[b] = tl if logits else torch.softmax(tl, dim=-1)
         dprob = torch.softmax(dl, dim=-1)          # row c+1 = draft distribution after node c
         child_rank = {}
         for i in range(n):
             c = int(parent[b, i])
-            draft[b, i] = dprob[c + 1]
+            draft[b, i] = dl[c + 1] if logits else dprob[c + 1]
             if gflag[b]:
                 j = child_rank.get(c, 0)
                 child_rank[c] = j + 1

@@ -78,6 +78,52 @@ def test_accept_matches_oracle(E, oracle, name, cfg, kw, mode):
     assert tolerated_total <= max(1, seqs // 100), tolerated_total
 
 
+LOGIT_CASES = [
+    ("tiny_t1", W.CONFIGS["tiny"], dict(rho=0.9), 1.0),
+    ("tiny_half_greedy_t07", W.CONFIGS["tiny"], dict(rho=0.9, greedy="half"), 0.7),
+    ("7b_t1", W.CONFIGS["7b_mha"], dict(rho=0.9), 1.0),
+    ("70b_t13", W.CONFIGS["70b_gqa"], dict(rho=0.9), 1.3),
+    ("70b_rho0", W.CONFIGS["70b_gqa"], dict(rho=0.0), 1.0),
+    ("mix_small_t08", W.scaled(W.CONFIGS["serving_mix"], batch=12), dict(rho=0.9), 0.8),
+    ("odd_vocab_batch", W.scaled(W.CONFIGS["tiny"], batch=300, tree=(0, 20), vocab=4099), dict(rho=0.7, greedy="half"), 1.0),
+    ("small_vocab_batch", W.scaled(W.CONFIGS["tiny"], batch=2000, tree=(0, 14), vocab=37), dict(rho=0.5, greedy="half"), 0.5),
+]
+
+
+@pytest.mark.parametrize("name,cfg,kw,temperature", LOGIT_CASES, ids=[c[0] for c in LOGIT_CASES])
+def test_accept_on_logits_matches_oracle(E, oracle, name, cfg, kw, temperature):
+    """eagle_tree_accept_logits against the oracle's fp64 softmax walk.  The kernel's exponentials are fp32, so a
+    decision may differ where the oracle's margin is below 1e-5; such sequences are counted."""
+    tolerated_total, seqs = 0, 0
+    d = torch.device("cuda:0")
+    for salt in range(3 if cfg.batch * cfg.vocab < 4_000_000 else 1):
+        inp = W.make_accept_inputs(cfg, salt=salt, logits=True, **kw)
+        ref = oracle.tree_accept_logits(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
+                                        temperature, tree_sizes=inp.tree_sizes, greedy=inp.greedy)
+        status = torch.zeros(1, dtype=torch.int32, device=d)
+        alen = torch.full((cfg.batch,), -7, dtype=torch.int32, device=d)
+        path, bonus = E.eagle_tree_accept_logits(inp.target_probs.to(d), inp.draft_probs.to(d), inp.draft_tokens.to(d),
+                                                 inp.tree_parent.to(d), inp.uniforms.to(d), temperature,
+                                                 tree_sizes=inp.tree_sizes.to(d), greedy=inp.greedy.to(d), accept_len=alen,
+                                                 status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        tolerated_total += _compare(inp, ref, path.cpu().numpy(), bonus.cpu().numpy(), alen.cpu().numpy())
+        seqs += cfg.batch
+        assert ref["accept_len"].max() >= 1
+    assert tolerated_total <= max(1, seqs // 50), tolerated_total
+
+
+def test_accept_on_logits_rejects_bad_temperature(E):
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=2, vocab=64)
+    inp = W.make_accept_inputs(cfg, logits=True)
+    d = torch.device("cuda:0")
+    for bad in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(Exception):
+            E.eagle_tree_accept_logits(inp.target_probs.to(d), inp.draft_probs.to(d), inp.draft_tokens.to(d), inp.tree_parent.to(d),
+                                       inp.uniforms.to(d), bad)
+
+
 def test_all_greedy_without_draft_rows(E, oracle):
     cfg = W.scaled(W.CONFIGS["7b_mha"], batch=3)
     inp = W.make_accept_inputs(cfg, salt=9, greedy="all")
