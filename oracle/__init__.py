@@ -46,6 +46,8 @@ def _load():
         lib.oracle_tree_accept.restype = i32
         lib.oracle_tree_accept_logits.argtypes = [i32, i32, i32, i32] + [vp] * 7 + [dbl] + [vp] * 6
         lib.oracle_tree_accept_logits.restype = i32
+        lib.oracle_tree_expand.argtypes = [i32, i32, i32, i32] + [vp] * 7
+        lib.oracle_tree_expand.restype = i32
         lib.oracle_tree_commit.argtypes = [i32] * 6 + [vp] * 4 + [i32] + [vp] * 4
         lib.oracle_tree_commit.restype = i32
         lib.oracle_num_threads.restype = i32
@@ -174,3 +176,20 @@ def tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree: int, featur
     if rc != 0:
         raise ValueError(f"oracle_tree_commit failed: {rc}")
     return dict(k_cache=k, v_cache=v, features_out=fout, new_seq_lens=new_len, valid=valid)
+
+
+def tree_expand(probs, num_children, max_children: int, uniforms=None, greedy=None):
+    """Child tokens of draft-tree nodes (App. A.1): top-k of each row for greedy sequences, k independent inverse-CDF draws
+    otherwise.  probs [B, R, V] fp32, num_children [B, R] int32, uniforms [B, R, max_children] fp32, greedy [B] uint8.
+    Returns a dict: tokens [B, R, max_children] int32 (-1 padded), token_probs fp32, min_margin [B, R]."""
+    p = _as(probs, np.float32)
+    B, R, V = p.shape
+    nc, un, gr = _as(num_children, np.int32), _as(uniforms, np.float32), _as(greedy, np.uint8)
+    assert nc.shape == (B, R) and (un is None or un.shape == (B, R, max_children))
+    res = dict(tokens=np.full((B, R, max_children), -2, np.int32), token_probs=np.full((B, R, max_children), -1, np.float32),
+               min_margin=np.zeros((B, R), np.float64))
+    rc = _load().oracle_tree_expand(B, R, V, max_children, _ptr(nc), _ptr(gr), _ptr(p), _ptr(un), _ptr(res["tokens"]),
+                                    _ptr(res["token_probs"]), _ptr(res["min_margin"]))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_expand failed: {rc}")
+    return res

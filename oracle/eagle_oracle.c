@@ -16,6 +16,8 @@
  *                              recursively at every node from the root (Sec. 3.3); the greedy setting
  *                              (Preliminaries) is the same rule with a one-hot target distribution.
  *   oracle_tree_accept_logits - the same with the distributions given as logits (softmax at a temperature, fp64).
+ *   oracle_tree_expand       - App. A.1 (tree structure): the children of a draft-tree node are the k most probable
+ *                              tokens of its draft distribution in the greedy setting, k sampled tokens otherwise.
  *   oracle_tree_commit       - Sec. 3.3, last sentence: the accepted tokens and their features are recorded
  *                              for the next drafting phase.  For the target's KV cache that means: the
  *                              keys and values of the accepted tree nodes become the next slots of the
@@ -423,6 +425,90 @@ int oracle_tree_commit(int batch, int num_kv_heads, int head_dim, int kv_capacit
   }
   free(tmp);
   return ORACLE_OK;
+}
+
+/*
+ * Child tokens of draft-tree nodes (App. A.1: in the greedy setting the k most probable tokens become the children,
+ * otherwise k tokens are sampled; k differs from node to node).
+ *
+ * probs [B, R, V] fp32: the draft distribution at each of R nodes per sequence (used as given, not renormalised);
+ * num_children [B, R]: k of each node, 0 <= k <= max_children; greedy [B] or NULL; uniforms [B, R, max_children]
+ * (needed by stochastic sequences).  Outputs: tokens [B, R, max_children] (-1 past k), token_probs (0 past k).
+ * Readings (the paper gives neither a tie rule nor a sampling scheme): top-k is by descending probability with the
+ * lower token id first among equal values; the k samples are independent draws with replacement, draw j being the
+ * smallest x with sum_{v<=x} p(v) > uniforms[j] * sum_v p(v) (the inverse CDF in ascending token id, as in
+ * oracle_tree_accept; the last token with positive mass if rounding leaves none).  min_margin [B, R] (optional):
+ * the smallest distance, as a fraction of the row's mass, between a draw's threshold and the edges of the cell it
+ * fell into; +inf for greedy rows.
+ */
+int oracle_tree_expand(int batch, int rows, int vocab, int max_children, const int32_t* num_children,
+                       const uint8_t* greedy, const float* probs, const float* uniforms, int32_t* tokens,
+                       float* token_probs, double* min_margin) {
+  if (batch < 0 || rows < 0 || vocab <= 0 || max_children < 0 || !num_children || !probs || !tokens) return ORACLE_ERR_ARG;
+  for (long long i = 0; i < (long long)batch * rows; ++i) {
+    const int g = greedy && greedy[i / rows];
+    if (num_children[i] < 0 || num_children[i] > max_children) return ORACLE_ERR_ARG;
+    if (g && num_children[i] > vocab) return ORACLE_ERR_ARG;       /* k distinct tokens */
+    if (!g && !uniforms) return ORACLE_ERR_ARG;
+  }
+  int failed = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (long long i = 0; i < (long long)batch * rows; ++i) {
+    const int b = (int)(i / rows), k = num_children[i];
+    const float* p = probs + (size_t)i * vocab;
+    int32_t* out = tokens + (size_t)i * max_children;
+    float* outp = token_probs ? token_probs + (size_t)i * max_children : NULL;
+    for (int j = 0; j < max_children; ++j) {
+      out[j] = -1;
+      if (outp) outp[j] = 0.f;
+    }
+    double margin = INFINITY;
+    if (greedy && greedy[b]) {
+      /* k rounds: the most probable token not taken yet, lowest id among equals */
+      unsigned char* taken = (unsigned char*)calloc((size_t)vocab, 1);
+      if (!taken) {
+        failed = 1;
+        continue;
+      }
+      for (int j = 0; j < k; ++j) {
+        int best = -1;
+        for (int v = 0; v < vocab; ++v)
+          if (!taken[v] && (best < 0 || p[v] > p[best])) best = v;
+        taken[best] = 1;
+        out[j] = best;
+        if (outp) outp[j] = p[best];
+      }
+      free(taken);
+    } else {
+      double total = 0.0;
+      for (int v = 0; v < vocab; ++v) total += (double)p[v];
+      for (int j = 0; j < k; ++j) {
+        const double thr = (double)uniforms[(size_t)i * max_children + j] * total;
+        double c = 0.0, c_prev = 0.0;
+        int x = -1, last_pos = -1;
+        for (int v = 0; v < vocab; ++v) {
+          if (p[v] > 0.f) last_pos = v;
+          c_prev = c;
+          c += (double)p[v];
+          if (c > thr) {
+            x = v;
+            break;
+          }
+        }
+        if (x < 0) {
+          x = last_pos >= 0 ? last_pos : vocab - 1;
+        } else if (total > 0.0) {
+          const double lo = (thr - c_prev) / total, hi = (c - thr) / total;
+          const double m = lo < hi ? lo : hi;
+          if (m < margin) margin = m;
+        }
+        out[j] = x;
+        if (outp) outp[j] = p[x];
+      }
+    }
+    if (min_margin) min_margin[i] = margin;
+  }
+  return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
 }
 
 /* Threads the OpenMP loops above use (reported next to the oracle's timing). */
