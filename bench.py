@@ -280,6 +280,24 @@ def main():
     logits_same = int(((path_l == path_p).all(dim=1) & (bonus_l == bonus_p)).sum().item())
     del zt, zd
 
+    # ---- child selection for the next drafting pass (App. A.1; reported, not part of the headline): 4 children for each
+    # of the first 8 nodes' draft rows of every sequence (top-4 for greedy sequences, 4 draws otherwise)
+    s = sets[0]
+    R_exp, K_exp = min(8, T), 4
+    rows_exp = s["dp"][:, :R_exp].contiguous()
+    nc_exp = torch.full((B, R_exp), K_exp, dtype=torch.int32, device=dev)
+    un_exp = torch.rand((B, R_exp, K_exp), device=dev)
+    x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    E.eagle_tree_expand(rows_exp, nc_exp, K_exp, uniforms=un_exp, greedy=s["gr"], status=status)
+    x0.record()
+    for i in range(10):
+        E.eagle_tree_expand(rows_exp, nc_exp, K_exp, uniforms=un_exp, greedy=s["gr"], status=status)
+    x1.record()
+    torch.cuda.synchronize()
+    expand_ms = x0.elapsed_time(x1) / 10
+    expand_bytes = rows_exp.numel() * 4
+    del rows_exp
+
     # ---- commit of the accepted path for this layer's cache (the step after verification; reported, not part of the
     # headline).  It moves rows in place, so it runs on the last input set, after everything that reads the cache.
     s = sets[-1]
@@ -347,6 +365,9 @@ def main():
                       "sequence_steps_per_s": value * B,
                       "accept_on_logits": {"ms": accept_logits_ms, "temperature": 1.0,
                                            "sequences_with_the_same_tokens_as_on_probabilities": logits_same, "of": B},
+                      "tree_expand": {"ms": expand_ms, "rows": B * R_exp, "children": K_exp, "bytes": expand_bytes,
+                                      "gbs": expand_bytes / (expand_ms * 1e-3) / 1e9,
+                                      "note": "rows are re-used back to back (warm L2); top-k re-reads a row k times"},
                       "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
                                     "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}},
     }

@@ -225,6 +225,36 @@ int eagle_tree_accept_logits(const eagle_accept_desc* desc, const float* target_
                              const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
                              float temperature, int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream);
 
+#define EAGLE_MAX_CHILDREN 16
+
+typedef struct eagle_expand_desc {
+  int32_t batch;               /* B >= 0 (at most 65535) */
+  int32_t rows;                /* R >= 0: draft-tree nodes expanded per sequence in this call */
+  int32_t vocab;               /* V >= 1 */
+  int32_t max_children;        /* K <= EAGLE_MAX_CHILDREN: row stride of the per-child arrays */
+  const uint8_t* greedy;       /* device uint8 [B] or NULL (= every sequence stochastic) */
+  int32_t* status;             /* device int32 or NULL */
+} eagle_expand_desc;
+
+/*
+ * Child tokens of draft-tree nodes (App. A.1, tree structure: in the greedy setting the k most probable tokens of a
+ * node's draft distribution become its children, otherwise k tokens are sampled; k varies from node to node).
+ *
+ *   draft_probs  device fp32 [B, R, V]   the draft distribution at each node (used as given, not renormalised)
+ *   num_children device int32 [B, R]     k of each node, 0 <= k <= K (greedy: also k <= V)
+ *   uniforms     device fp32 [B, R, K]   one uniform in [0, 1) per draw (may be NULL when every sequence is greedy)
+ *   child_tokens device int32 [B, R, K]  the k tokens, then -1
+ *   child_probs  device fp32 [B, R, K] or NULL   draft_probs at those tokens, then 0
+ *
+ * Greedy sequences: descending probability, the lower token id first among equal values (exact).  Other sequences: k
+ * independent draws (with replacement; the paper does not say), draw j = the smallest x with
+ * sum_{v<=x} p(v) > uniforms[j] * sum_v p(v), prefix sums in fp64 (the last token with positive mass if rounding
+ * leaves none).  A node whose k is out of range sets *status to EAGLE_ERR_SHAPE and gets no children.
+ * One launch, asynchronous on `stream`; no workspace.
+ */
+int eagle_tree_expand(const eagle_expand_desc* desc, const float* draft_probs, const int32_t* num_children,
+                      const float* uniforms, int32_t* child_tokens, float* child_probs, eagle_stream_t stream);
+
 typedef struct eagle_commit_desc {
   int32_t batch;               /* B >= 0 (at most 65535) */
   int32_t num_kv_heads;        /* Hkv >= 0 */

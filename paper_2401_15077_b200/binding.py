@@ -18,7 +18,7 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
            "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit",
-           "eagle_tree_accept_logits"]
+           "eagle_tree_accept_logits", "eagle_tree_expand"]
 _lib = None
 
 
@@ -43,6 +43,11 @@ class AcceptDesc(ctypes.Structure):
 class CommitDesc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in ("batch", "num_kv_heads", "head_dim", "kv_capacity", "max_tree", "path_cap",
                                               "feature_dim")] + [("status", ctypes.c_void_p)]
+
+
+class ExpandDesc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("batch", "rows", "vocab", "max_children")] + [("greedy", ctypes.c_void_p),
+                                                                                            ("status", ctypes.c_void_p)]
 
 
 class HostStep(ctypes.Structure):
@@ -77,6 +82,8 @@ def load():
         lib.eagle_tree_accept.restype = ctypes.c_int
         lib.eagle_tree_accept_logits.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
         lib.eagle_tree_accept_logits.restype = ctypes.c_int
+        lib.eagle_tree_expand.argtypes = [ctypes.POINTER(ExpandDesc), vp, vp, vp, vp, vp, vp]
+        lib.eagle_tree_expand.restype = ctypes.c_int
         lib.eagle_tree_commit.argtypes = [ctypes.POINTER(CommitDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_commit.restype = ctypes.c_int
         lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
@@ -239,6 +246,22 @@ def eagle_tree_build_mask(tree_parent, tree_sizes=None, status=None, with_depth=
                                    _dev(status, torch.int32, "status", True), _stream())
     _check(rc, "eagle_tree_build_mask")
     return anc, depth
+
+
+def eagle_tree_expand(draft_probs, num_children, max_children, uniforms=None, greedy=None, status=None, with_probs=True):
+    """Child tokens of draft-tree nodes: top-k per row for greedy sequences, k inverse-CDF draws otherwise.
+    draft_probs [B, R, V] fp32, num_children [B, R] int32, uniforms [B, R, K] fp32.  Returns (tokens, probs) [B, R, K]."""
+    lib = load()
+    B, R, V = draft_probs.shape
+    K = int(max_children)
+    tokens = torch.empty((B, R, K), dtype=torch.int32, device=draft_probs.device)
+    probs = torch.empty((B, R, K), dtype=torch.float32, device=draft_probs.device) if with_probs else None
+    d = ExpandDesc(B, R, V, K, _dev(greedy, torch.uint8, "greedy", True), _dev(status, torch.int32, "status", True))
+    rc = lib.eagle_tree_expand(ctypes.byref(d), _dev(draft_probs, torch.float32, "draft_probs"),
+                               _dev(num_children, torch.int32, "num_children"), _dev(uniforms, torch.float32, "uniforms", True),
+                               tokens.data_ptr(), None if probs is None else probs.data_ptr(), _stream())
+    _check(rc, "eagle_tree_expand")
+    return tokens, probs
 
 
 def eagle_tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree, features=None, features_out=None,

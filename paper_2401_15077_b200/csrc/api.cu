@@ -511,6 +511,33 @@ int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cach
   return EAGLE_OK;
 }
 
+int eagle_tree_expand(const eagle_expand_desc* desc, const float* draft_probs, const int32_t* num_children,
+                      const float* uniforms, int32_t* child_tokens, float* child_probs, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const eagle_expand_desc& d = *desc;
+  if (d.batch < 0 || d.batch > 65535 || d.rows < 0 || d.vocab < 1 || d.max_children < 0 || d.max_children > kMaxChildren)
+    return EAGLE_ERR_SHAPE;
+  if (d.batch == 0 || d.rows == 0 || d.max_children == 0) return EAGLE_OK;
+  if (!draft_probs || !num_children || !child_tokens) return EAGLE_ERR_NULL;
+  if (!uniforms && !d.greedy) return EAGLE_ERR_NULL;
+  int err = 0;
+  if (!device_info(&err)) return err;
+  ExpandParams ep;
+  ep.probs = draft_probs;
+  ep.num_children = num_children;
+  ep.greedy = d.greedy;
+  ep.uniforms = uniforms;
+  ep.tokens = child_tokens;
+  ep.token_probs = child_probs;
+  ep.B = d.batch;
+  ep.R = d.rows;
+  ep.V = d.vocab;
+  ep.K = d.max_children;
+  ep.status = d.status;
+  if (launch_expand(ep, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
+
 const char* eagle_status_string(int code) {
   switch (code) {
     case EAGLE_OK: return "ok";

@@ -152,6 +152,19 @@ struct CommitParams {
   int32_t* status;
 };
 
+constexpr int kMaxChildren = 16;
+
+struct ExpandParams {
+  const float* probs;          // [B, R, V]
+  const int32_t* num_children; // [B, R]
+  const uint8_t* greedy;       // [B] or null
+  const float* uniforms;       // [B, R, K] or null
+  int32_t* tokens;             // [B, R, K]
+  float* token_probs;          // [B, R, K] or null
+  int32_t B, R, V, K;
+  int32_t* status;
+};
+
 struct AcceptParams {
   const float* target;   // [B, T+1, V]
   const float* draft;    // [B, T, V]
@@ -184,6 +197,7 @@ cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cuda
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
 cudaError_t launch_commit(const CommitParams& p, cudaStream_t stream);
+cudaError_t launch_expand(const ExpandParams& p, cudaStream_t stream);
 void count_launch();
 
 }  // namespace eagle
