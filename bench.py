@@ -367,7 +367,7 @@ def main():
                                            "sequences_with_the_same_tokens_as_on_probabilities": logits_same, "of": B},
                       "tree_expand": {"ms": expand_ms, "rows": B * R_exp, "children": K_exp, "bytes": expand_bytes,
                                       "gbs": expand_bytes / (expand_ms * 1e-3) / 1e9,
-                                      "note": "rows are re-used back to back (warm L2); top-k re-reads a row k times"},
+                                      "note": "back-to-back calls on the same rows (warm L2)"},
                       "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
                                     "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}},
     }
