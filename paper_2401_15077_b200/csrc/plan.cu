@@ -9,7 +9,9 @@
 // tiles.  The CTAs of the attention kernel are taken in pairs ("teams").  The query tiles of a (sequence, KV head)
 // are taken two at a time: such a pair is a super-unit that both CTAs of a team walk together, one query tile each
 // over the same KV tiles, so the keys and values one of them pulls from HBM are still in L2 when the other asks for
-// them; an odd last query tile is a super-unit whose KV range the team's two CTAs split in halves.  All super-units
+// them; the odd last query tiles of two neighbouring KV heads form a twin super-unit (one head per CTA of the team,
+// same KV range), and with an odd number of KV heads the last head's odd tile is a lone super-unit whose KV range the
+// team's two CTAs split in halves.  All super-units
 // are laid end to end on one line (plus `item_overhead_tiles` positions of fixed cost at the start of each), and
 // every team gets an equal contiguous share of the line.  A share boundary inside a super-unit cuts it into
 // pieces (their partial results are merged by the combine kernel); boundaries closer than `snap_tiles` to an edge
