@@ -28,8 +28,8 @@ def test_every_declared_symbol_is_exported(lib):
 def test_status_strings(lib):
     from paper_2401_15077_b200 import binding
     assert binding.status_string(0) == "ok"
-    seen = {binding.status_string(c) for c in range(-9, 1)}
-    assert len(seen) == 10 and "unknown status" not in seen
+    seen = {binding.status_string(c) for c in range(-10, 1)}
+    assert len(seen) == 11 and "unknown status" not in seen
     assert binding.status_string(-1234) == "unknown status"
 
 
@@ -69,6 +69,24 @@ def test_host_checks_return_before_any_launch(lib):
     assert lib.eagle_tree_accept(ctypes.byref(a), fake, None, fake, fake, fake, fake, fake, None) == -1
     assert lib.eagle_tree_build_mask(None, None, 1, 8, None, None, None, None) == -1
     assert lib.eagle_tree_build_mask(fake, None, 1, 99, fake, None, None, None) == -2
+    # the entry points added for the steps around verification: same rules
+    assert lib.eagle_tree_accept_logits(ctypes.byref(a), fake, fake, fake, fake, fake, ctypes.c_float(0.0), fake, fake, None) == -2
+    assert lib.eagle_tree_accept_logits(ctypes.byref(a), fake, fake, fake, fake, fake, ctypes.c_float(float("nan")), fake, fake, None) == -2
+    assert lib.eagle_tree_accept_logits(ctypes.byref(a), None, fake, fake, fake, fake, ctypes.c_float(1.0), fake, fake, None) == -1
+    c = binding.CommitDesc(2, 4, 128, 512, 64, 64, 0, None)
+    assert lib.eagle_tree_commit(None, fake, fake, fake, fake, None, None, None, None) == -1
+    assert lib.eagle_tree_commit(ctypes.byref(c), fake, fake, None, fake, None, None, None, None) == -1
+    assert lib.eagle_tree_commit(ctypes.byref(c), ctypes.c_void_p(4100), fake, fake, fake, None, None, None, None) == -2   # misaligned cache
+    for bad in (binding.CommitDesc(2, 4, 96, 512, 64, 64, 0, None), binding.CommitDesc(2, 4, 128, 512, 65, 64, 0, None),
+                binding.CommitDesc(2, 4, 128, 512, 64, 64, 12, None)):
+        assert lib.eagle_tree_commit(ctypes.byref(bad), fake, fake, fake, fake, None, None, None, None) == -2
+    assert lib.eagle_tree_commit(ctypes.byref(binding.CommitDesc(0, 4, 128, 512, 64, 64, 0, None)), None, None, None, None, None, None,
+                                 None, None) == 0
+    e = binding.ExpandDesc(2, 3, 100, 4, None, None)
+    assert lib.eagle_tree_expand(ctypes.byref(e), None, fake, fake, fake, None, None) == -1
+    assert lib.eagle_tree_expand(ctypes.byref(e), fake, fake, None, fake, None, None) == -1            # stochastic rows need uniforms
+    assert lib.eagle_tree_expand(ctypes.byref(binding.ExpandDesc(2, 3, 100, 17, None, None)), fake, fake, fake, fake, None, None) == -2
+    assert lib.eagle_tree_expand(ctypes.byref(binding.ExpandDesc(2, 0, 100, 4, None, None)), None, None, None, None, None, None) == 0
     assert binding.launch_count() == before
 
 
