@@ -1,4 +1,6 @@
 """Parity of the CUDA tree attention (through the C ABI) with the fp64 oracle.  Needs a B200."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -129,6 +131,51 @@ def test_reference_maximum_moves_between_steps(E, oracle, shape):
         out, status = _run(E, inp, num_splits=splits)
         assert status == 0
         _check(out, ref, inp.tree_sizes)
+
+
+def _random_cfg(rng, i):
+    D = int(rng.choice([64, 128]))
+    Hkv = int(rng.choice([1, 2, 3, 4, 5, 8]))
+    G = int(rng.choice([1, 2, 3, 4, 8, 16]))
+    lo = int(rng.choice([0, 0, 1, 100, 127, 128, 129, 600]))
+    hi = lo + int(rng.choice([0, 1, 130, 700, 2500]))
+    t_lo = int(rng.integers(0, 40))
+    t_hi = int(rng.integers(max(t_lo, 1), 65))
+    depth = int(rng.choice([2, 5, 9, 64]))
+    shape = dict(max_depth=depth, child_cap=int(rng.choice([0, 2, 4])) if depth >= 9 else 0)   # (a capped shallow tree cannot hold 64 nodes)
+    return W.scaled(W.CONFIGS["tiny"], batch=int(rng.integers(1, 7)), num_q_heads=Hkv * G, num_kv_heads=Hkv, head_dim=D,
+                    prefix=(lo, hi), tree=(t_lo, t_hi), **shape)
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("EAGLE_RANDOM_SHAPES", "24"))))
+def test_random_shapes(E, oracle, seed):
+    """Random head counts, group sizes, head dims, prefix ranges around the tile size and tree shapes, with the default
+    split and with a forced one: every combination of pair / twin / lone super-units, one to many steps per item, empty
+    trees and prefixes."""
+    rng = np.random.default_rng(1000 + seed)
+    cfg = _random_cfg(rng, seed)
+    inp = W.make_attn_inputs(cfg, salt=seed, capacity_pad=int(rng.integers(0, 40)))
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    for splits in (0, int(rng.choice([2, 3, 5]))):
+        out, status = _run(E, inp, num_splits=splits)
+        assert status == 0, (cfg, splits)
+        _check(out, ref, inp.tree_sizes)
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("EAGLE_RANDOM_BATCHES", "2"))))
+def test_random_medium_batches(E, oracle, seed):
+    """Batches large enough that every CTA team gets several items and most share boundaries cut a super-unit."""
+    rng = np.random.default_rng(5000 + seed)
+    Hkv, G = int(rng.choice([4, 8])), int(rng.choice([2, 4, 8]))
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=int(rng.integers(12, 28)), num_q_heads=Hkv * G, num_kv_heads=Hkv,
+                   prefix=(int(rng.integers(0, 300)), int(rng.integers(1500, 5000))), tree=(int(rng.integers(1, 20)), 64))
+    inp = W.make_attn_inputs(cfg, salt=100 + seed)
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    out, status = _run(E, inp)
+    assert status == 0
+    _check(out, ref, inp.tree_sizes)
+    again, _ = _run(E, inp)
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16)), "same call twice must be bit-identical"
 
 
 def test_empty_prefix_empty_tree_and_single_node(E, oracle):
