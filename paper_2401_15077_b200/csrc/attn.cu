@@ -79,6 +79,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// (A wait gives up only after two seconds without progress; the K/V ring holds at most six tiles, so by then the
+// producers have been blocked on a full ring for all but the first microseconds of those two seconds and no copy of
+// theirs is still in flight when the CTA leaves.)
 // Slow path of a wait, kept out of line so that the dozen wait sites stay small (the kernel's hot loops have to
 // live in the instruction cache next to each other).  Returns false if the CTA has been aborted or the time limit
 // passed (and raises the abort flag).
