@@ -428,84 +428,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   const long long trace_t0 = clock64();
 #endif
 
-  if (warp == kWarpProducer) {
-    // =========================================================================== TMA producer
-    // Load order: K(0), K(1), K(2), then V(g), K(g + 3) for g = 0, 1, ... (g counts this CTA's steps across items):
-    // the order in which the MMAs consume the tiles, since the score MMA runs three steps ahead of the PV MMA.
-    // Entry n of that sequence lives in slot n % kSlots; with six slots the K tile of step g + 3 is requested when the
-    // score MMA of step g has finished and the V tile of step g when the PV of step g - 3 has.
-    if (lane == 0) {
-      struct Cursor {
-        int tp, tile, tile_end, z;
-        bool valid;
-      };
-      auto advance = [&](Cursor& c) {   // moves to the next KV tile of the work list
-        if (++c.tile < c.tile_end) return;
-        for (++c.tp; c.tp < tp_hi; ++c.tp) {
-          const WorkItem it = p.items[2 * c.tp + member];
-          if (it.tile_end > it.tile_begin) {
-            c.tile = it.tile_begin;
-            c.tile_end = it.tile_end;
-            c.z = it.b * p.Hkv + it.g;
-            return;
-          }
-        }
-        c.valid = false;
-      };
-      bool ok = true;
-      uint32_t n = 0;   // position in the load sequence
-      auto load_tile = [&](const Cursor& c, bool is_v) {
-        const uint32_t slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
-        ok = mbar_wait(B.empty[slot], par, s_abort);
-        if (!ok) return;
-        TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
-        mbar_expect_tx(B.full[slot], S::kTileBytes);
-#pragma unroll
-        for (int sl = 0; sl < S::kSlabs; ++sl)
-          tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
-                      B.full[slot]);
-      };
-      Cursor ck = {tp_lo - 1, 0, 0, 0, true}, cv = {tp_lo - 1, 0, 0, 0, true};
-      advance(ck);
-      advance(cv);
-      for (int i = 0; i < 3; ++i, ++n) {   // K(0), K(1), K(2)
-        if (ok && ck.valid) {
-          load_tile(ck, false);
-          advance(ck);
-        }
-      }
-      while (ok && cv.valid) {
-        load_tile(cv, true);      // V(g)
-        ++n;
-        advance(cv);
-        if (ok && ck.valid) {     // K(g + 3)
-          load_tile(ck, false);
-          advance(ck);
-        }
-        ++n;
-      }
-    }
-  } else if (warp == kWarpQ) {
-    // =========================================================================== query-tile producer
-    // One buffer: the tile of the next item is fetched as soon as the last score MMA of the current one has finished;
-    // the softmax groups still have two or three steps of that item to work through meanwhile.
-    if (lane == 0 && p.q_tma) {
-      uint32_t item_count = 0;
-      bool ok = true;
-      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
-        const WorkItem it = p.items[2 * tp + member];
-        if (it.tile_end <= it.tile_begin) continue;
-        ok = mbar_wait(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
-        if (!ok) break;
-        // box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
-        mbar_expect_tx(B.q_full, S::kTileBytes);
-#pragma unroll
-        for (int sl = 0; sl < S::kSlabs; ++sl)
-          tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full);
-        ++item_count;
-      }
-    }
-  } else if (warp == kWarpQK) {
+  if (warp == kWarpQK) {
     // =========================================================================== QK issuer
     // Entry n of the load sequence lives in slot n % kSlots with phase parity (n / kSlots) & 1.  Positions are kept
     // as running counters (no divisions on the threads that keep the tensor pipe fed).
@@ -851,6 +774,83 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       g_base += steps;
       sg += steps;
       ++item_count;
+    }
+  } else if (warp == kWarpQ) {
+    // =========================================================================== query-tile producer
+    // One buffer: the tile of the next item is fetched as soon as the last score MMA of the current one has finished;
+    // the softmax groups still have two or three steps of that item to work through meanwhile.
+    if (lane == 0 && p.q_tma) {
+      uint32_t item_count = 0;
+      bool ok = true;
+      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
+        const WorkItem it = p.items[2 * tp + member];
+        if (it.tile_end <= it.tile_begin) continue;
+        ok = mbar_wait(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        // box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
+        mbar_expect_tx(B.q_full, S::kTileBytes);
+#pragma unroll
+        for (int sl = 0; sl < S::kSlabs; ++sl)
+          tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full);
+        ++item_count;
+      }
+    }
+  } else if (warp == kWarpProducer) {
+    // =========================================================================== TMA producer
+    // Load order: K(0), K(1), K(2), then V(g), K(g + 3) for g = 0, 1, ... (g counts this CTA's steps across items):
+    // the order in which the MMAs consume the tiles, since the score MMA runs three steps ahead of the PV MMA.
+    // Entry n of that sequence lives in slot n % kSlots; with six slots the K tile of step g + 3 is requested when the
+    // score MMA of step g has finished and the V tile of step g when the PV of step g - 3 has.
+    if (lane == 0) {
+      struct Cursor {
+        int tp, tile, tile_end, z;
+        bool valid;
+      };
+      auto advance = [&](Cursor& c) {   // moves to the next KV tile of the work list
+        if (++c.tile < c.tile_end) return;
+        for (++c.tp; c.tp < tp_hi; ++c.tp) {
+          const WorkItem it = p.items[2 * c.tp + member];
+          if (it.tile_end > it.tile_begin) {
+            c.tile = it.tile_begin;
+            c.tile_end = it.tile_end;
+            c.z = it.b * p.Hkv + it.g;
+            return;
+          }
+        }
+        c.valid = false;
+      };
+      bool ok = true;
+      uint32_t n = 0;   // position in the load sequence
+      auto load_tile = [&](const Cursor& c, bool is_v) {
+        const uint32_t slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
+        ok = mbar_wait(B.empty[slot], par, s_abort);
+        if (!ok) return;
+        TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
+        mbar_expect_tx(B.full[slot], S::kTileBytes);
+#pragma unroll
+        for (int sl = 0; sl < S::kSlabs; ++sl)
+          tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
+                      B.full[slot]);
+      };
+      Cursor ck = {tp_lo - 1, 0, 0, 0, true}, cv = {tp_lo - 1, 0, 0, 0, true};
+      advance(ck);
+      advance(cv);
+      for (int i = 0; i < 3; ++i, ++n) {   // K(0), K(1), K(2)
+        if (ok && ck.valid) {
+          load_tile(ck, false);
+          advance(ck);
+        }
+      }
+      while (ok && cv.valid) {
+        load_tile(cv, true);      // V(g)
+        ++n;
+        advance(cv);
+        if (ok && ck.valid) {     // K(g + 3)
+          load_tile(ck, false);
+          advance(ck);
+        }
+        ++n;
+      }
     }
   }
 
