@@ -358,10 +358,18 @@ struct Smem {
   static constexpr int kBytes = kMisc + 16;
 };
 
+// The mbarriers sit next to one another in shared memory; their addresses are computed, not stored (an array of
+// addresses indexed at run time would live in local memory).
 struct Bars {
-  uint32_t full[kSlots], empty[kSlots];
-  uint32_t s_full[kSBufs], p_full[kSBufs], o_done[kSBufs];
-  uint32_t q_full, q_empty, o_free;
+  uint32_t base;
+  __device__ __forceinline__ uint32_t full(uint32_t i) const { return base + 8u * i; }
+  __device__ __forceinline__ uint32_t empty(uint32_t i) const { return base + 8u * (kSlots + i); }
+  __device__ __forceinline__ uint32_t s_full(uint32_t i) const { return base + 8u * (2 * kSlots + i); }
+  __device__ __forceinline__ uint32_t p_full(uint32_t i) const { return base + 8u * (2 * kSlots + kSBufs + i); }
+  __device__ __forceinline__ uint32_t o_done(uint32_t i) const { return base + 8u * (2 * kSlots + 2 * kSBufs + i); }
+  __device__ __forceinline__ uint32_t q_full() const { return base + 8u * (2 * kSlots + 3 * kSBufs); }
+  __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 1); }
+  __device__ __forceinline__ uint32_t o_free() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 2); }
 };
 
 template <int D>
@@ -378,33 +386,23 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   }
 
   Bars B;
-  {
-    uint32_t b = sbase + S::kBar;
-    for (int i = 0; i < kSlots; ++i) { B.full[i] = b; b += 8; }
-    for (int i = 0; i < kSlots; ++i) { B.empty[i] = b; b += 8; }
-    for (int i = 0; i < kSBufs; ++i) { B.s_full[i] = b; b += 8; }
-    for (int i = 0; i < kSBufs; ++i) { B.p_full[i] = b; b += 8; }
-    for (int i = 0; i < kSBufs; ++i) { B.o_done[i] = b; b += 8; }
-    B.q_full = b; b += 8;
-    B.q_empty = b; b += 8;
-    B.o_free = b; b += 8;
-  }
+  B.base = sbase + S::kBar;
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + S::kMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + S::kMisc + 4);
 
   if (tid == 0) {
     for (int i = 0; i < kSlots; ++i) {
-      mbar_init(B.full[i], 1);
-      mbar_init(B.empty[i], 1);
+      mbar_init(B.full(i), 1);
+      mbar_init(B.empty(i), 1);
     }
     for (int i = 0; i < kSBufs; ++i) {
-      mbar_init(B.s_full[i], 1);
-      mbar_init(B.p_full[i], kGroupThreads);
-      mbar_init(B.o_done[i], 1);
+      mbar_init(B.s_full(i), 1);
+      mbar_init(B.p_full(i), kGroupThreads);
+      mbar_init(B.o_done(i), 1);
     }
-    mbar_init(B.q_full, p.q_tma ? 1 : kGroupThreads);   // one TMA transaction, or every thread of the first softmax group
-    mbar_init(B.q_empty, 1);
-    mbar_init(B.o_free, kGroupThreads);
+    mbar_init(B.q_full(), p.q_tma ? 1 : kGroupThreads);   // one TMA transaction, or every thread of the first softmax group
+    mbar_init(B.q_empty(), 1);
+    mbar_init(B.o_free(), kGroupThreads);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -446,29 +444,29 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         TRACE(1, 1);
-        ok = mbar_wait(B.q_full, item_count & 1u, s_abort);
+        ok = mbar_wait(B.q_full(), item_count & 1u, s_abort);
         if (!ok) break;
         TRACE(1, 2);
         for (int s = 0; s < steps && ok; ++s, ++gq) {
           // the K tile arrives long before the score buffer frees up: look at it first, so that nothing but the
           // MMA issue follows the wait that matters
-          ok = mbar_wait(B.full[ks], kp, s_abort);
+          ok = mbar_wait(B.full(ks), kp, s_abort);
           if (!ok) break;
           TRACE(1, (9 << 10) | (gq & 1023u));
           // S[gq % 3] also holds P of step gq - 3: it is free once that step's PV has finished
           if (gq >= 3) {
-            ok = mbar_wait(B.o_done[sb], sph ^ 1u, s_abort);
+            ok = mbar_wait(B.o_done(sb), sph ^ 1u, s_abort);
             if (!ok) break;
           }
           TRACE(1, (10 << 10) | (gq & 1023u));
           tc_fence_after();
           issue_qk_tile<D>(tmem + kColS + sb * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
-          tc_commit(B.s_full[sb]);
-          tc_commit(B.empty[ks]);
+          tc_commit(B.s_full(sb));
+          tc_commit(B.empty(ks));
           ks += gq < 2 ? 1u : 2u;   // K(g) is entry g for g < 3, entry 2g - 2 after that
           if (ks >= kSlots) { ks -= kSlots; kp ^= 1u; }
           if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
-          if (s == steps - 1) tc_commit(B.q_empty);      // every QK of this item has been issued
+          if (s == steps - 1) tc_commit(B.q_empty());      // every QK of this item has been issued
           TRACE(1, (11 << 10) | (gq & 1023u));
         }
         ++item_count;
@@ -490,20 +488,20 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
         for (int s = 0; s < steps && ok; ++s, ++gp) {
-          ok = mbar_wait(B.full[vs], vp, s_abort);   // (arrives well before P is ready)
+          ok = mbar_wait(B.full(vs), vp, s_abort);   // (arrives well before P is ready)
           if (!ok) break;
           TRACE(3, (20 << 10) | (gp & 1023u));
           if (s == 0 && item_count > 0) {
-            ok = mbar_wait(B.o_free, (item_count - 1) & 1u, s_abort);   // previous epilogue has read O
+            ok = mbar_wait(B.o_free(), (item_count - 1) & 1u, s_abort);   // previous epilogue has read O
             if (!ok) break;
           }
-          ok = mbar_wait(B.p_full[sb], sph, s_abort);
+          ok = mbar_wait(B.p_full(sb), sph, s_abort);
           if (!ok) break;
           TRACE(3, (30 << 10) | (gp & 1023u));
           tc_fence_after();
           issue_pv_tile(tmem + kColO, tmem + kColS + sb * kTileN, ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
-          tc_commit(B.o_done[sb]);
-          tc_commit(B.empty[vs]);
+          tc_commit(B.o_done(sb));
+          tc_commit(B.empty(vs));
           vs += 2;
           if (vs >= kSlots) { vs -= kSlots; vp ^= 1u; }
           if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
@@ -543,7 +541,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
 
       if (!p.q_tma && grp == 0) {
         // group sizes that do not divide 128: the first softmax group stages the query tile itself, a row per thread
-        ok = mbar_wait_warp(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
+        ok = mbar_wait_warp(B.q_empty(), (item_count & 1u) ^ 1u, s_abort);
         if (!ok) break;
         const uint4* src = reinterpret_cast<const uint4*>(p.q + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D);
         unsigned char* qdst = smem + S::kQ + r * 128;
@@ -553,7 +551,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           *reinterpret_cast<uint4*>(qdst + (c >> 3) * S::kSlabBytes + (((c & 7) ^ (r & 7)) << 4)) = v;
         }
         fence_proxy_async();
-        mbar_arrive(B.q_full);
+        mbar_arrive(B.q_full());
       }
       if ((tid & 127) == 0) TRACE(2 + 2 * grp, 3);
 
@@ -565,7 +563,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         const uint32_t gs = sg + s;
         const uint32_t sb = gs % kSBufs, sph = (gs / kSBufs) & 1u;     // score buffer of this step and its phase
         const uint32_t s_addr = tmem + lane_addr + kColS + sb * kTileN;   // P goes over the front half of the same columns
-        ok = mbar_wait_warp(B.s_full[sb], sph, s_abort);
+        ok = mbar_wait_warp(B.s_full(sb), sph, s_abort);
         if (!ok) break;
         if ((tid & 127) == 0) TRACE(2 + 2 * grp, (10 << 10) | (gs & 1023u));
         tc_fence_after();
@@ -615,7 +613,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
           const uint32_t nv = 2 * (g_base + s) + 3, slot = nv % kSlots, par = (nv / kSlots) & 1u;
-          ok = mbar_wait_warp(B.full[slot], par, s_abort);
+          ok = mbar_wait_warp(B.full(slot), par, s_abort);
           if (!ok) break;
           if (key0 + r >= kv_end) {
 #pragma unroll
@@ -651,7 +649,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         *tag = __float_as_uint(m_ref) | (gs & 0xffu);
         if (s > 0 && __any_sync(0xffffffffu, grow)) {
           // the previous step accumulated into O and may still be running
-          ok = mbar_wait_warp(B.o_done[(gs - 1) % kSBufs], ((gs - 1) / kSBufs) & 1u, s_abort);
+          ok = mbar_wait_warp(B.o_done((gs - 1) % kSBufs), ((gs - 1) / kSBufs) & 1u, s_abort);
           if (!ok) break;
           tc_fence_after();
           uint32_t o[32];
@@ -715,21 +713,21 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           // this group's last step of the item, but not the item's: hand the row sum to the group that writes the
           // output.  A two-step item is the one case where the slot may still be in use for the previous item.
           if (s == 0 && item_count > 0) {
-            ok = mbar_wait_warp(B.o_free, (item_count - 1) & 1u, s_abort);
+            ok = mbar_wait_warp(B.o_free(), (item_count - 1) & 1u, s_abort);
             if (!ok) break;
           }
           *lfin = l_sum;
         }
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(B.p_full[sb]);
+        mbar_arrive(B.p_full(sb));
         if ((tid & 127) == 0) TRACE(2 + 2 * grp, (11 << 10) | (gs & 1023u));
 
         if (s == steps - 1) {
           // ---- this group took the item's last step: it writes the item's output.  Wait for the last PV (PVs
           // complete in order), add the other group's part of the row sum, then write the row: bf16 output, or
           // the unnormalised fp32 partial of a cut piece.
-          ok = mbar_wait_warp(B.o_done[sb], sph, s_abort);
+          ok = mbar_wait_warp(B.o_done(sb), sph, s_abort);
           if (!ok) break;
           if ((tid & 127) == 0) TRACE(2 + 2 * grp, 20);
           tc_fence_after();
@@ -767,7 +765,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           }
           if (row_valid && it.slot >= 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_ref, l_row);
           tc_fence_before();
-          mbar_arrive(B.o_free);            // the next item's first PV may overwrite the accumulator
+          mbar_arrive(B.o_free());            // the next item's first PV may overwrite the accumulator
           if ((tid & 127) == 0) TRACE(2 + 2 * grp, 21);
         }
       }
@@ -785,13 +783,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
         const WorkItem it = p.items[2 * tp + member];
         if (it.tile_end <= it.tile_begin) continue;
-        ok = mbar_wait(B.q_empty, (item_count & 1u) ^ 1u, s_abort);
+        ok = mbar_wait(B.q_empty(), (item_count & 1u) ^ 1u, s_abort);
         if (!ok) break;
         // box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
-        mbar_expect_tx(B.q_full, S::kTileBytes);
+        mbar_expect_tx(B.q_full(), S::kTileBytes);
 #pragma unroll
         for (int sl = 0; sl < S::kSlabs; ++sl)
-          tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full);
+          tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full());
         ++item_count;
       }
     }
@@ -823,14 +821,14 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       uint32_t n = 0;   // position in the load sequence
       auto load_tile = [&](const Cursor& c, bool is_v) {
         const uint32_t slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
-        ok = mbar_wait(B.empty[slot], par, s_abort);
+        ok = mbar_wait(B.empty(slot), par, s_abort);
         if (!ok) return;
         TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
-        mbar_expect_tx(B.full[slot], S::kTileBytes);
+        mbar_expect_tx(B.full(slot), S::kTileBytes);
 #pragma unroll
         for (int sl = 0; sl < S::kSlabs; ++sl)
           tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
-                      B.full[slot]);
+                      B.full(slot));
       };
       Cursor ck = {tp_lo - 1, 0, 0, 0, true}, cv = {tp_lo - 1, 0, 0, 0, true};
       advance(ck);
