@@ -216,34 +216,29 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
-// Bounded wait for a tagged word in shared memory (low byte == want); the word is returned through *out.
-__device__ __noinline__ bool tag_wait_slow(volatile uint32_t* slot, uint32_t want, uint32_t* out, volatile int* abort_flag) {
+// Bounded wait for a tagged word in shared memory (low byte == want).  The word comes back by value, with bit 32 set on
+// success (0: the CTA was aborted or the time limit passed); nothing is passed through memory.
+__device__ __noinline__ unsigned long long tag_wait_slow(volatile uint32_t* slot, uint32_t want, volatile int* abort_flag) {
   const unsigned long long t0 = global_timer();
   for (uint32_t spins = 1;; ++spins) {
     const uint32_t t = *slot;
-    if ((t & 0xffu) == want) {
-      *out = t;
-      return true;
-    }
+    if ((t & 0xffu) == want) return (1ull << 32) | t;
     if ((spins & 255u) == 0) {
-      if (*abort_flag) return false;
+      if (*abort_flag) return 0ull;
       if (global_timer() - t0 > kWaitLimitNs) {
         *abort_flag = 1;
-        return false;
+        return 0ull;
       }
     }
   }
 }
-__device__ __forceinline__ bool tag_wait(volatile uint32_t* slot, uint32_t want, uint32_t* out, volatile int* abort_flag) {
+__device__ __forceinline__ unsigned long long tag_wait(volatile uint32_t* slot, uint32_t want, volatile int* abort_flag) {
 #pragma unroll 1
   for (int i = 0; i < 8; ++i) {
     const uint32_t t = *slot;
-    if ((t & 0xffu) == want) {
-      *out = t;
-      return true;
-    }
+    if ((t & 0xffu) == want) return (1ull << 32) | t;
   }
-  return tag_wait_slow(slot, want, out, abort_flag);
+  return tag_wait_slow(slot, want, abort_flag);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -627,10 +622,10 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         // where its value is not used: the other group must have read the tag of step gs - 2 before it is replaced)
         float m_prev = -INFINITY;
         if (gs > 0) {
-          uint32_t t = 0xff800000u;
-          ok = __all_sync(0xffffffffu, tag_wait(tag, (gs - 1u) & 0xffu, &t, s_abort));
+          const unsigned long long t = tag_wait(tag, (gs - 1u) & 0xffu, s_abort);
+          ok = __all_sync(0xffffffffu, (t >> 32) != 0ull);
           if (!ok) break;
-          if (s > 0) m_prev = __uint_as_float(t & 0xffffff00u);
+          if (s > 0) m_prev = __uint_as_float(static_cast<uint32_t>(t) & 0xffffff00u);
         }
         if (m_prev != m_ref) {
           l_sum *= fast_exp2(m_ref - m_prev);     // m_ref = -inf: nothing summed yet, the factor is 0
