@@ -579,27 +579,33 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             vm[c] = w;
           }
         }
-        // ---- pass 1: row maximum of the raw scores; chunks 0 and 1, fetched last, stay in registers for pass 2
+        // ---- pass 1: row maximum of the raw scores.  All four chunks are fetched in one round trip to tensor memory;
+        // chunks 0 and 1 stay in registers for pass 2, chunks 2 and 3 are dropped after the maximum and fetched again
+        // later (keeping them would leave too few registers for pass 2).
         uint32_t ra[32], rb[32];
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int c = 2; c >= 0; c -= 2) {
-          tmem_ld32(s_addr + c * 32, ra);
-          tmem_ld32(s_addr + c * 32 + 32, rb);
+        {
+          uint32_t rc[32], rd[32];
+          tmem_ld32(s_addr + 64, rc);
+          tmem_ld32(s_addr + 96, rd);
+          tmem_ld32(s_addr, ra);
+          tmem_ld32(s_addr + 32, rb);
           tc_wait_ld();
           if (tail) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              ra[e] = (vm[c] >> e) & 1u ? ra[e] : 0xff800000u;       // -inf
-              rb[e] = (vm[c + 1] >> e) & 1u ? rb[e] : 0xff800000u;
+              ra[e] = (vm[0] >> e) & 1u ? ra[e] : 0xff800000u;       // -inf
+              rb[e] = (vm[1] >> e) & 1u ? rb[e] : 0xff800000u;
+              rc[e] = (vm[2] >> e) & 1u ? rc[e] : 0xff800000u;
+              rd[e] = (vm[3] >> e) & 1u ? rd[e] : 0xff800000u;
             }
           }
 #pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            mx[0] = max3(mx[0], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
-            mx[1] = max3(mx[1], __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
-            mx[2] = max3(mx[2], __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
-            mx[3] = max3(mx[3], __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
+          for (int e = 0; e < 32; e += 2) {
+            mx[0] = max3(mx[0], __uint_as_float(rc[e]), __uint_as_float(rc[e + 1]));
+            mx[1] = max3(mx[1], __uint_as_float(rd[e]), __uint_as_float(rd[e + 1]));
+            mx[2] = max3(mx[2], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            mx[3] = max3(mx[3], __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
           }
         }
         const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // scale > 0
