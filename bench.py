@@ -41,9 +41,9 @@ HBM_FALLBACK_GBS = 6650.0
 L2_BYTES = 126 * 2 ** 20
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu captures summarised in
 # profiles/attn_kernel_serving_mix_b16.md, keyed by (workload, batch); None where no capture exists.
-# Full serving_mix: 1224.3 MB read + 29.8 MB written, captured at full size with a one-pass metric list;
-# batch 16: 314.1 MB + 15.7 MB from the --set full capture.
-NCU_TRAFFIC_BYTES = {("serving_mix", 64): 1_224_349_184 + 29_797_888, ("serving_mix", 16): 314_063_104 + 15_671_296}
+# Full serving_mix: 1180.8 MB read + 24.7 MB written, captured at full size with a one-pass metric list;
+# batch 16: 313.0 MB + 8.9 MB from the --set full capture.
+NCU_TRAFFIC_BYTES = {("serving_mix", 64): 1_180_839_168 + 24_708_608, ("serving_mix", 16): 313_012_224 + 8_916_992}
 
 
 def measured_hbm_peak():
