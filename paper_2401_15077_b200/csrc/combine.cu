@@ -1,7 +1,7 @@
 // Merge of the split-KV partials: m* = max_s m_s, l* = sum_s l_s 2^(m_s - m*), O = sum_s O_s 2^(m_s - m*) / l*,
 // and the zero rows of padded tree nodes.
-// A fixed grid (a few blocks per SM) walks the planner's list of cut query tiles, eight work items per tile
-// (16 rows each, two rows per warp), then one work item per sequence that writes zeros to the rows of nodes past
+// A fixed grid (a few blocks per SM) walks the planner's list of cut query tiles, sixteen work items per tile
+// (8 rows each, one row per warp), then one work item per sequence that writes zeros to the rows of nodes past
 // the tree size (one contiguous range of the output).  Query tiles that stayed in one item were written by the
 // attention kernel and do not appear in the list.
 #include "common.cuh"
@@ -11,7 +11,7 @@ namespace eagle {
 namespace {
 
 constexpr int kCombineThreads = 256;
-constexpr int kBlocksPerUnit = 8;                       // 16 rows per block
+constexpr int kBlocksPerUnit = 16;                      // 8 rows per block: one per warp
 constexpr int kRowsPerBlock = kBlockM / kBlocksPerUnit;
 
 template <int D>
@@ -93,7 +93,7 @@ cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cuda
   if (p.B == 0 || p.T_max == 0) return cudaSuccess;
   // the number of cut tiles is only known on the device: a few blocks per SM loop over them
   const long long most = static_cast<long long>(unit_cap) * 2 * kBlocksPerUnit + p.B;
-  const long long want = static_cast<long long>(sm_count > 0 ? sm_count : 1) * 4;
+  const long long want = static_cast<long long>(sm_count > 0 ? sm_count : 1) * 8;
   const unsigned blocks = static_cast<unsigned>(want < most ? want : most);
   if (p.D == 128) combine_kernel<128><<<blocks, kCombineThreads, 0, stream>>>(p);
   else combine_kernel<64><<<blocks, kCombineThreads, 0, stream>>>(p);
