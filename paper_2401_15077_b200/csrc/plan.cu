@@ -26,28 +26,35 @@ namespace {
 constexpr int kPlanThreads = 1024;
 
 // Exclusive prefix sums of value(i), i in [0, n), by one CTA; put(i, prefix) stores them; returns the total.
+// Thread chunks -> warp scan -> scan of the 32 warp totals by the first warp -> back to the threads.
 template <class Value, class Put>
 __device__ long long block_exclusive_scan(int n, Value value, Put put, long long* scratch) {
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunk = (n + kPlanThreads - 1) / kPlanThreads;
   const int i0 = min(tid * chunk, n), i1 = min(i0 + chunk, n);
   long long local = 0;
   for (int i = i0; i < i1; ++i) local += value(i);
-  // inclusive scan of the per-thread sums: warp shuffles, then across warps through shared memory
   long long inc = local;
   for (int o = 1; o < 32; o <<= 1) {
     const long long x = __shfl_up_sync(0xffffffffu, inc, o);
-    if ((tid & 31) >= o) inc += x;
+    if (lane >= o) inc += x;
+  }
+  __syncthreads();                       // scratch may still be read by the previous scan
+  if (lane == 31) scratch[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    const long long mine = scratch[lane];
+    long long winc = mine;
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long x = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += x;
+    }
+    scratch[lane] = winc - mine;         // exclusive prefix of the warp totals
+    if (lane == 31) scratch[32] = winc;  // grand total
   }
   __syncthreads();
-  if ((tid & 31) == 31) scratch[tid >> 5] = inc;
-  __syncthreads();
-  long long before = 0, total = 0;
-  for (int w = 0; w < kPlanThreads / 32; ++w) {
-    if (w == (tid >> 5)) before = total;
-    total += scratch[w];
-  }
-  long long run = before + inc - local;
+  const long long total = scratch[32];
+  long long run = scratch[warp] + inc - local;
   for (int i = i0; i < i1; ++i) {
     const long long v = value(i);   // read before put(): put may overwrite what value reads
     put(i, run);
@@ -57,7 +64,12 @@ __device__ long long block_exclusive_scan(int n, Value value, Put put, long long
   return total;
 }
 
-__device__ __forceinline__ long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
+// Quotients on the work line.  Every operand is below W * teams; when that product fits 31 bits (the usual case) the
+// 32-bit divide is used, which is several times cheaper than the emulated 64-bit one.
+__device__ __forceinline__ long long qdiv(long long a, long long b, bool small) {
+  return small ? static_cast<long long>(static_cast<unsigned>(a) / static_cast<unsigned>(b)) : a / b;
+}
+__device__ __forceinline__ long long ceil_div(long long a, long long b, bool small) { return qdiv(a + b - 1, b, small); }
 
 // anc[i] = bit i | anc[parent[i]] in node order (parents come first).  Returns false on an invalid entry.
 __device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc, uint8_t* depth) {
@@ -126,11 +138,11 @@ __device__ inline bool build_masks_warp(const int32_t* par, int n, uint64_t* anc
 // A super-unit occupies [us, ue) on the work line: `ovh` positions of fixed cost, then one position per KV tile of
 // its line.  Its interior cuts are the share boundaries floor(c * W / teams) with us + ovh + snap <= boundary <=
 // ue - snap: a contiguous range of c.  Returns their number and the first such c.
-__device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W, int teams, int snap, int ovh, int* first_c) {
+__device__ __forceinline__ int unit_cuts(long long us, long long ue, long long W, int teams, int snap, int ovh, int* first_c, bool small) {
   const long long y = us + ovh + snap, z = ue - snap;
   *first_c = 0;
   if (z < y || teams < 2) return 0;
-  long long ca = ceil_div(y * teams, W), cb = ceil_div((z + 1) * teams, W) - 1;
+  long long ca = ceil_div(y * teams, W, small), cb = ceil_div((z + 1) * teams, W, small) - 1;
   if (ca < 1) ca = 1;
   if (cb > teams - 1) cb = teams - 1;
   *first_c = static_cast<int>(ca);
@@ -207,22 +219,22 @@ struct SeqGeom {
     return ug;
   }
   // the super-unit that holds line position `off` (relative to the sequence's start, 0 <= off < length())
-  __device__ int unit_at(long long off) const {
+  __device__ int unit_at(long long off, bool small) const {
     const int twos = Hkv / 2;
     if (off < twos * len2) {
-      const int h2 = static_cast<int>(off / len2);
-      int j = static_cast<int>((off % len2) / plen);
+      const int h2 = static_cast<int>(qdiv(off, len2, small));
+      int j = static_cast<int>(qdiv(off - h2 * len2, plen, small));
       if (j > u2 - 1) j = u2 - 1;
       return h2 * u2 + j;
     }
-    int j = static_cast<int>((off - twos * len2) / plen);
+    int j = static_cast<int>(qdiv(off - twos * len2, plen, small));
     if (j > u1 - 1) j = u1 - 1;
     return twos * u2 + j;
   }
 };
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
-  __shared__ long long s_scan[kPlanThreads / 32];
+  __shared__ long long s_scan[kPlanThreads / 32 + 1];
   __shared__ int s_ncut;
   __shared__ SeqPlan s_seq[kSmemSeqs];
   __shared__ UnitPlan s_units[kSmemUnits];
@@ -279,6 +291,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   const int max_teams = p.num_ctas / 2;
   const int teams = static_cast<int>(W < max_teams ? (W > 0 ? W : 1) : max_teams);   // a share is at least one position
   const int snap = p.snap_tiles;
+  const bool small = (W + ovh + snap + 1) * static_cast<long long>(max_teams + 1) < (1ll << 31);   // every dividend fits 31 bits
 
   // super-unit -> sequence: the last sequence whose unit_base <= u (sequences without units share theirs with the next)
   auto unit_seq = [&](int u) {
@@ -303,7 +316,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
       np = len < p.forced_splits ? len : p.forced_splits;
     } else {
       int c0;
-      np = 1 + unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0);
+      np = 1 + unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0, small);
     }
     p.units[u].n_pieces = np;
     p.units[u].pad0 = b;
@@ -340,7 +353,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
       const long long us = sp.start + ug.offset;
       const long long t_origin = us + ovh;          // line position of the super-unit's tile position 0
       int c0 = 0;
-      if (p.forced_splits == 0) unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0);
+      if (p.forced_splits == 0) unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0, small);
       bool live[2] = {false, false};    // query tiles of the super-unit with at least one non-empty item
       for (int j = 0; j < up.n_pieces; ++j) {
         int t0, t1;
@@ -348,8 +361,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
           t0 = static_cast<int>(static_cast<long long>(len) * j / up.n_pieces);
           t1 = static_cast<int>(static_cast<long long>(len) * (j + 1) / up.n_pieces);
         } else {
-          t0 = j == 0 ? 0 : static_cast<int>(static_cast<long long>(c0 + j - 1) * W / teams - t_origin);
-          t1 = j == up.n_pieces - 1 ? len : static_cast<int>(static_cast<long long>(c0 + j) * W / teams - t_origin);
+          t0 = j == 0 ? 0 : static_cast<int>(qdiv(static_cast<long long>(c0 + j - 1) * W, teams, small) - t_origin);
+          t1 = j == up.n_pieces - 1 ? len : static_cast<int>(qdiv(static_cast<long long>(c0 + j) * W, teams, small) - t_origin);
         }
         for (int m = 0; m < 2; ++m) {
           WorkItem it;
@@ -392,7 +405,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
     } else if (c >= teams) {
       first = TP;
     } else {
-      const long long x = static_cast<long long>(c) * W / teams;   // 0 < x < W
+      const long long x = qdiv(static_cast<long long>(c) * W, teams, small);   // 0 < x < W
       int lo = 0, hi = p.B;          // last sequence whose start <= x (sequences without work share their start with the next)
       while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -400,7 +413,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
       }
       const SeqPlan sp = p.seq[lo];
       const SeqGeom ge(sp, p.Hkv, ovh);
-      const int k = ge.unit_at(x - sp.start);
+      const int k = ge.unit_at(x - sp.start, small);
       const UnitGeom ug = ge.unit(k);
       const int u = sp.unit_base + k;
       const long long us = sp.start + ug.offset, ue = us + ug.line + ovh;
@@ -408,7 +421,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
       const UnitPlan up = p.units[u];
       if (d0 >= snap && d1 >= snap) {
         int c0;
-        unit_cuts(us, ue, W, teams, snap, ovh, &c0);
+        unit_cuts(us, ue, W, teams, snap, ovh, &c0, small);
         first = up.first_item + 1 + (c - c0);        // the piece that starts at this boundary
       } else if (x - us <= d1) {
         first = up.first_item;                        // boundary moved to the super-unit's start
