@@ -42,6 +42,8 @@ def _load():
         lib.oracle_tree_ancestors.restype = i32
         lib.oracle_tree_verify_attn.argtypes = [i32, i32, i32, i32, i32, i32, vp, dbl, vp, vp, vp, vp, vp, vp]
         lib.oracle_tree_verify_attn.restype = i32
+        lib.oracle_tree_verify_attn_paged.argtypes = [i32] * 8 + [vp, dbl] + [vp] * 7
+        lib.oracle_tree_verify_attn_paged.restype = i32
         lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 13
         lib.oracle_tree_accept.restype = i32
         lib.oracle_tree_accept_logits.argtypes = [i32, i32, i32, i32] + [vp] * 7 + [dbl] + [vp] * 6
@@ -108,6 +110,28 @@ def tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, tree_sizes=None
                                          _ptr(va), _ptr(sl), _ptr(par), _ptr(out))
     if rc != 0:
         raise ValueError(f"oracle_tree_verify_attn failed: {rc}")
+    return out
+
+
+def tree_verify_attn_paged(q, k_pages, v_pages, block_table, seq_lens, tree_parent, tree_sizes=None, sm_scale: float = 0.0):
+    """fp64 tree-masked attention over a paged cache.
+
+    q [B, T_max, Hq, D]; k_pages, v_pages [num_pages, Hkv, page_size, D]; block_table int32 [B, max_pages_per_seq];
+    returns float64 [B, T_max, Hq, D].
+    """
+    qa, ka, va = _as(q, np.uint16), _as(k_pages, np.uint16), _as(v_pages, np.uint16)
+    B, T, Hq, D = qa.shape
+    P, Hkv, ps = ka.shape[0], ka.shape[1], ka.shape[2]
+    assert ka.shape == va.shape == (P, Hkv, ps, D)
+    bt = _as(block_table, np.int32)
+    assert bt.ndim == 2 and bt.shape[0] == B
+    sl, par, ts = _as(seq_lens, np.int32), _as(tree_parent, np.int32), _as(tree_sizes, np.int32)
+    assert par.shape == (B, T)
+    out = np.zeros((B, T, Hq, D), np.float64)
+    rc = _load().oracle_tree_verify_attn_paged(B, Hq, Hkv, D, T, P, ps, bt.shape[1], _ptr(ts), float(sm_scale), _ptr(qa),
+                                               _ptr(ka), _ptr(va), _ptr(bt), _ptr(sl), _ptr(par), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_verify_attn_paged failed: {rc}")
     return out
 
 

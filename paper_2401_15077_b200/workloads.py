@@ -16,7 +16,7 @@ from dataclasses import dataclass, field
 
 import torch
 
-STREAMS = dict(q=0, k=1, v=2, tree=3, target=4, draft=5, tokens=6, uniforms=7, lens=8, sizes=9, paths=10, features=11)
+STREAMS = dict(q=0, k=1, v=2, tree=3, target=4, draft=5, tokens=6, uniforms=7, lens=8, sizes=9, paths=10, features=11, pages=12)
 
 
 @dataclass(frozen=True)
@@ -132,6 +132,41 @@ def make_attn_inputs(cfg: VerifyConfig, salt: int = 0, poison: bool = True, capa
         if poison:
             q[b, int(sizes[b]):] = float("nan")
     return AttnInputs(cfg, q, k, v, lens, sizes, parent, cap)
+
+
+@dataclass
+class PagedKV:
+    k_pages: torch.Tensor      # bf16 [num_pages, Hkv, page_size, D]
+    v_pages: torch.Tensor
+    block_table: torch.Tensor  # int32 [B, max_pages_per_seq]
+    page_size: int
+
+
+def make_paged_cache(inp: AttnInputs, page_size: int, salt: int = 0, spare_pages: int = 3, poison: bool = True) -> PagedKV:
+    """The same keys and values as ``inp`` stored in pages of ``page_size`` slots, scattered over the pool by a seeded
+    permutation.  Only pages that hold a visible slot get a table entry; the other entries are -1, and rows of slots
+    that are not visible (as well as ``spare_pages`` unused pages) hold NaN when ``poison``."""
+    cfg = inp.cfg
+    B, Hkv, D = cfg.batch, cfg.num_kv_heads, cfg.head_dim
+    vis = [int(inp.seq_lens[b] + inp.tree_sizes[b]) if int(inp.tree_sizes[b]) > 0 else 0 for b in range(B)]
+    need = [(n + page_size - 1) // page_size for n in vis]
+    max_pages = max(1, (inp.kv_capacity + page_size - 1) // page_size)
+    total = sum(need) + spare_pages
+    order = torch.randperm(total, generator=_gen(cfg.index, "pages", salt)).tolist()
+    fill = float("nan") if poison else 0.0
+    kp = torch.full((max(total, 1), Hkv, page_size, D), fill, dtype=torch.bfloat16)
+    vp = torch.full((max(total, 1), Hkv, page_size, D), fill, dtype=torch.bfloat16)
+    table = torch.full((B, max_pages), -1, dtype=torch.int32)
+    nxt = 0
+    for b in range(B):
+        for i in range(need[b]):
+            page = order[nxt]
+            nxt += 1
+            table[b, i] = page
+            rows = min(page_size, vis[b] - i * page_size)
+            kp[page, :, :rows] = inp.k_cache[b, :, i * page_size:i * page_size + rows]
+            vp[page, :, :rows] = inp.v_cache[b, :, i * page_size:i * page_size + rows]
+    return PagedKV(kp, vp, table, page_size)
 
 
 @dataclass
