@@ -48,7 +48,8 @@ enum {
   EAGLE_ERR_TOKEN = -7,      /* device-detected: draft token outside [0, vocab) */
   EAGLE_ERR_TIMEOUT = -8,    /* device-detected: a bounded wait inside a kernel ran out */
   EAGLE_ERR_DEVICE = -9,     /* the GPU is not an sm_100 device, or it lacks a required limit */
-  EAGLE_ERR_PATH = -10       /* device-detected: an accepted path that is not an increasing list of tree nodes whose slots exist */
+  EAGLE_ERR_PATH = -10,      /* device-detected: an accepted path that is not an increasing list of tree nodes whose slots exist */
+  EAGLE_ERR_PAGE = -11       /* device-detected: a block-table entry of a page in use outside [0, num_pages) */
 };
 
 #define EAGLE_MAX_TREE 64
@@ -71,6 +72,8 @@ typedef struct eagle_attn_desc {
   int32_t* status;             /* device int32 or NULL */
   eagle_event_t ev_attn_begin; /* optional: recorded on `stream` right before / after the split-KV   */
   eagle_event_t ev_attn_end;   /* attention kernel (the dominant kernel), for timing it alone; or NULL */
+  int32_t shared_tree;         /* nonzero: one tree for every sequence (the paper's experiments use one fixed tree shape,
+                                  App. A.1): tree_parent is int32 [T_max] and tree_sizes NULL or int32 [1] */
 } eagle_attn_desc;
 
 /* Bytes of scratch one call with this descriptor needs (host function, no CUDA work).
@@ -85,7 +88,7 @@ size_t eagle_tree_verify_attn_workspace(const eagle_attn_desc* desc);
  *   v_cache  device bf16 [B, Hkv, S_cap, D]       L_b + m holds tree node m; later slots are never used
  *                                                 in the result, whatever they contain (NaN included)
  *   seq_lens device int32 [B]                     L_b, the committed prefix length (tree not included)
- *   tree_parent device int32 [B, T_max]
+ *   tree_parent device int32 [B, T_max]           ([T_max] when desc->shared_tree is set)
  *   out      device bf16 [B, T_max, Hq, D]        out[b,i,h,:] = sum_j softmax_j(scale * q[b,i,h]·k[b,h/G,j]) v[b,h/G,j]
  *                                                 over j < L_b and j = L_b + m, m an ancestor of i or i itself;
  *                                                 rows of nodes i >= tree size are written as zeros
@@ -127,6 +130,32 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
 
 /* Size in bytes of the fixed array used by eagle_tree_verify_attn_static (host function). */
 size_t eagle_tree_verify_attn_static_capacity(void);
+
+/*
+ * A KV cache kept in pages (a storage layout of the same cache: the verification pass of Sec. 3.3 reads the same keys
+ * and values wherever a serving engine stores them).
+ */
+typedef struct eagle_paged_kv {
+  const void* k_pages;          /* device bf16 [num_pages, Hkv, page_size, D], 16-byte aligned */
+  const void* v_pages;          /* device bf16 [num_pages, Hkv, page_size, D], 16-byte aligned */
+  const int32_t* block_table;   /* device int32 [B, max_pages_per_seq]: slot j of sequence b is row j % page_size of page
+                                   block_table[b, j / page_size]; entries of pages that hold no slot below
+                                   seq_lens[b] + tree size are never read */
+  int32_t num_pages;            /* pages in the pool, >= 1 */
+  int32_t page_size;            /* slots per page: a power of two, >= 16 */
+  int32_t max_pages_per_seq;    /* row length of block_table; a sequence holds at most max_pages_per_seq * page_size slots */
+} eagle_paged_kv;
+
+/*
+ * eagle_tree_verify_attn over a paged cache.  Everything is as for that call (same planner, same kernels, same
+ * arithmetic and results, same workspace size) except where the keys and values are read from: each 128-slot tile
+ * is fetched page by page through the block table (one TMA box per page, or one box out of a page of 128 slots or
+ * more).  desc->kv_capacity is ignored: the capacity is max_pages_per_seq * page_size.  A sequence whose prefix + tree
+ * does not fit it reports EAGLE_ERR_SEQ, one with a block-table entry in use outside [0, num_pages) reports
+ * EAGLE_ERR_PAGE; its output rows are zeros and no page is read for it.
+ */
+int eagle_tree_verify_attn_paged(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* kv,
+                                 const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream);
 
 /*
  * Descriptor of one acceptance call.

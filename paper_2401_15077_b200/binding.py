@@ -18,7 +18,7 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
            "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit",
-           "eagle_tree_accept_logits", "eagle_tree_expand"]
+           "eagle_tree_accept_logits", "eagle_tree_expand", "eagle_tree_verify_attn_paged"]
 _lib = None
 
 
@@ -31,7 +31,12 @@ class AttnDesc(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("max_tree", ctypes.c_int32), ("kv_capacity", ctypes.c_int32),
                 ("tree_sizes", ctypes.c_void_p), ("sm_scale", ctypes.c_float), ("num_splits", ctypes.c_int32),
                 ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
-                ("ev_attn_begin", ctypes.c_void_p), ("ev_attn_end", ctypes.c_void_p)]
+                ("ev_attn_begin", ctypes.c_void_p), ("ev_attn_end", ctypes.c_void_p), ("shared_tree", ctypes.c_int32)]
+
+
+class PagedKV(ctypes.Structure):
+    _fields_ = [("k_pages", ctypes.c_void_p), ("v_pages", ctypes.c_void_p), ("block_table", ctypes.c_void_p),
+                ("num_pages", ctypes.c_int32), ("page_size", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32)]
 
 
 class AcceptDesc(ctypes.Structure):
@@ -74,6 +79,8 @@ def load():
         lib.eagle_tree_verify_attn_static.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_verify_attn_static.restype = ctypes.c_int
         lib.eagle_tree_verify_attn_static_capacity.restype = ctypes.c_size_t
+        lib.eagle_tree_verify_attn_paged.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(PagedKV), vp, vp, vp, vp]
+        lib.eagle_tree_verify_attn_paged.restype = ctypes.c_int
         lib.eagle_tree_verify_step_host.argtypes = [ctypes.POINTER(HostStep), vp]
         lib.eagle_tree_verify_step_host.restype = ctypes.c_int
         lib.eagle_tree_verify_step_host_arena.argtypes = [ctypes.POINTER(HostStep)]
@@ -122,17 +129,24 @@ def _stream():
     return torch.cuda.current_stream().cuda_stream
 
 
-def _attn_desc(q, k_cache, tree_sizes, sm_scale, num_splits, workspace, status, events):
+def _attn_desc(q, num_kv_heads, kv_capacity, tree_sizes, sm_scale, num_splits, workspace, status, events, shared_tree=False):
     B, T, Hq, D = q.shape
-    Hkv, S = k_cache.shape[1], k_cache.shape[2]
-    d = AttnDesc(B, Hq, Hkv, D, T, S, _dev(tree_sizes, torch.int32, "tree_sizes", True), float(sm_scale),
-                 int(num_splits), None, 0, _dev(status, torch.int32, "status", True), None, None)
+    d = AttnDesc(B, Hq, int(num_kv_heads), D, T, int(kv_capacity), _dev(tree_sizes, torch.int32, "tree_sizes", True), float(sm_scale),
+                 int(num_splits), None, 0, _dev(status, torch.int32, "status", True), None, None, 1 if shared_tree else 0)
     if workspace is not None:
         d.workspace = workspace.data_ptr()
         d.workspace_bytes = workspace.numel() * workspace.element_size()
     if events is not None:
         d.ev_attn_begin, d.ev_attn_end = events[0].cuda_event, events[1].cuda_event
     return d
+
+
+def _check_tree(tree_parent, tree_sizes, B, T, shared_tree):
+    want = (T,) if shared_tree else (B, T)
+    if tuple(tree_parent.shape) != want:
+        raise EagleError(f"tree_parent must be {want}")
+    if tree_sizes is not None and tree_sizes.numel() != (1 if shared_tree else B):
+        raise EagleError("tree_sizes has the wrong length")
 
 
 def eagle_tree_verify_attn_workspace(batch, num_q_heads, num_kv_heads, head_dim, max_tree, num_splits=0) -> int:
@@ -151,21 +165,23 @@ def alloc_workspace(q, k_cache, num_splits=0) -> torch.Tensor:
 
 
 def eagle_tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, out=None, *, tree_sizes=None, sm_scale=0.0,
-                           num_splits=0, workspace=None, status=None, events=None):
+                           num_splits=0, workspace=None, status=None, events=None, shared_tree=False):
     """Tree-masked attention.  q [B,T,Hq,D] bf16; k_cache/v_cache [B,Hkv,S,D] bf16; seq_lens [B] int32;
-    tree_parent [B,T] int32; returns out [B,T,Hq,D] bf16.  ``events``: optional pair of recorded-capable
-    torch.cuda.Event(enable_timing=True) placed around the attention kernel alone."""
+    tree_parent [B,T] int32 (or [T] with ``shared_tree``: one tree for every sequence, tree_sizes then [1] or None);
+    returns out [B,T,Hq,D] bf16.  ``events``: optional pair of recorded-capable torch.cuda.Event(enable_timing=True)
+    placed around the attention kernel alone."""
     lib = load()
     if q.dim() != 4 or k_cache.dim() != 4 or k_cache.shape != v_cache.shape:
         raise EagleError("bad tensor ranks / shapes")
     B, T, Hq, D = q.shape
-    if k_cache.shape[0] != B or k_cache.shape[3] != D or tuple(tree_parent.shape) != (B, T) or tuple(seq_lens.shape) != (B,):
+    if k_cache.shape[0] != B or k_cache.shape[3] != D or tuple(seq_lens.shape) != (B,):
         raise EagleError("inconsistent shapes")
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
     if out is None:
         out = torch.empty_like(q)
     if workspace is None:
         workspace = alloc_workspace(q, k_cache, num_splits)
-    d = _attn_desc(q, k_cache, tree_sizes, sm_scale, num_splits, workspace, status, events)
+    d = _attn_desc(q, k_cache.shape[1], k_cache.shape[2], tree_sizes, sm_scale, num_splits, workspace, status, events, shared_tree)
     rc = lib.eagle_tree_verify_attn(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
                                     _dev(v_cache, torch.bfloat16, "v_cache"), _dev(seq_lens, torch.int32, "seq_lens"),
                                     _dev(tree_parent, torch.int32, "tree_parent"), _dev(out, torch.bfloat16, "out"), _stream())
@@ -173,16 +189,44 @@ def eagle_tree_verify_attn(q, k_cache, v_cache, seq_lens, tree_parent, out=None,
     return out
 
 
+def eagle_tree_verify_attn_paged(q, k_pages, v_pages, block_table, seq_lens, tree_parent, out=None, *, tree_sizes=None,
+                                 sm_scale=0.0, num_splits=0, workspace=None, status=None, events=None, shared_tree=False):
+    """Tree-masked attention over a paged cache.  k_pages/v_pages [num_pages,Hkv,page_size,D] bf16; block_table
+    [B,max_pages_per_seq] int32: slot j of sequence b is row j % page_size of page block_table[b, j // page_size].
+    Everything else as for ``eagle_tree_verify_attn``."""
+    lib = load()
+    if q.dim() != 4 or k_pages.dim() != 4 or k_pages.shape != v_pages.shape or block_table.dim() != 2:
+        raise EagleError("bad tensor ranks / shapes")
+    B, T, Hq, D = q.shape
+    P, Hkv, ps = k_pages.shape[0], k_pages.shape[1], k_pages.shape[2]
+    if k_pages.shape[3] != D or block_table.shape[0] != B or tuple(seq_lens.shape) != (B,):
+        raise EagleError("inconsistent shapes")
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = alloc_workspace(q, k_pages, num_splits)
+    d = _attn_desc(q, Hkv, 0, tree_sizes, sm_scale, num_splits, workspace, status, events, shared_tree)
+    pk = PagedKV(_dev(k_pages, torch.bfloat16, "k_pages"), _dev(v_pages, torch.bfloat16, "v_pages"),
+                 _dev(block_table, torch.int32, "block_table"), P, ps, block_table.shape[1])
+    rc = lib.eagle_tree_verify_attn_paged(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), ctypes.byref(pk),
+                                          _dev(seq_lens, torch.int32, "seq_lens"), _dev(tree_parent, torch.int32, "tree_parent"),
+                                          _dev(out, torch.bfloat16, "out"), _stream())
+    _check(rc, "eagle_tree_verify_attn_paged")
+    return out
+
+
 def eagle_tree_verify_attn_static(q, k_cache, v_cache, seq_lens, tree_parent, out, *, tree_sizes=None, sm_scale=0.0,
-                                  num_splits=0, status=None):
+                                  num_splits=0, status=None, shared_tree=False):
     """Tree-masked attention for callers that may not allocate: same arguments and results as
     ``eagle_tree_verify_attn``, but no workspace is passed and none is allocated here either (the library's fixed
     device array is used; ``out`` must be given).  Raises if the shape needs more than that array holds."""
     lib = load()
     B, T, Hq, D = q.shape
-    if k_cache.shape[0] != B or k_cache.shape[3] != D or tuple(tree_parent.shape) != (B, T) or tuple(seq_lens.shape) != (B,):
+    if k_cache.shape[0] != B or k_cache.shape[3] != D or tuple(seq_lens.shape) != (B,):
         raise EagleError("inconsistent shapes")
-    d = _attn_desc(q, k_cache, tree_sizes, sm_scale, num_splits, None, status, None)
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
+    d = _attn_desc(q, k_cache.shape[1], k_cache.shape[2], tree_sizes, sm_scale, num_splits, None, status, None, shared_tree)
     rc = lib.eagle_tree_verify_attn_static(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
                                            _dev(v_cache, torch.bfloat16, "v_cache"), _dev(seq_lens, torch.int32, "seq_lens"),
                                            _dev(tree_parent, torch.int32, "tree_parent"), _dev(out, torch.bfloat16, "out"), _stream())

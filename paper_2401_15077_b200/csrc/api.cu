@@ -76,29 +76,31 @@ size_t eagle_tree_verify_attn_workspace(const eagle_attn_desc* desc) {
   return w.bytes;
 }
 
-int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
-                           const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
-  if (!desc) return EAGLE_ERR_NULL;
-  const eagle_attn_desc& d = *desc;
-  Workspace w;
-  if (d.kv_capacity < 0 || !(d.sm_scale >= 0.f) || !carve_workspace(d, d.workspace, &w)) return EAGLE_ERR_SHAPE;
-  if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
-  if (!q || !k_cache || !v_cache || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
-  if (!d.workspace || (reinterpret_cast<uintptr_t>(d.workspace) & 255) || d.workspace_bytes < w.bytes) return EAGLE_ERR_WORKSPACE;
-  if ((reinterpret_cast<uintptr_t>(k_cache) & 15) || (reinterpret_cast<uintptr_t>(v_cache) & 15) ||
-      (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
+namespace {
+
+// Where the keys and values of an attention call live: a contiguous cache, or pages behind a block table.
+struct KvSource {
+  const void* k;
+  const void* v;
+  int64_t capacity;             // slots per sequence
+  const int32_t* block_table;   // null: contiguous
+  int32_t num_pages, page_size, max_pages;
+};
+
+// Checks shared by every attention entry point, then the three launches: planner, attention, combine.
+int attention_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, DeviceInfo* dev, const void* q, const KvSource& kv,
+                   const int32_t* seq_lens, const int32_t* tree_parent, void* out, cudaStream_t stream) {
+  if (!q || !kv.k || !kv.v || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
+      (reinterpret_cast<uintptr_t>(out) & 15))
     return EAGLE_ERR_SHAPE;
-  int err = 0;
-  DeviceInfo* dev = device_info(&err);
-  if (!dev) return err;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int di = d.head_dim == 128 ? 1 : 0;
   if (!dev->attn_prepared[di]) {
     if (attn_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
     dev->attn_prepared[di] = true;
   }
   const int G = d.num_q_heads / d.num_kv_heads;
-  const int num_ctas = (dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas) & ~1;   // one persistent CTA per SM, in pairs
+  const int32_t s_cap = static_cast<int32_t>(kv.capacity < 0x7fffffff ? kv.capacity : 0x7fffffff);
 
   PlanParams pp;
   pp.seq_lens = seq_lens;
@@ -108,7 +110,7 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.Hkv = d.num_kv_heads;
   pp.G = G;
   pp.T_max = d.max_tree;
-  pp.S_cap = d.kv_capacity;
+  pp.S_cap = s_cap;
   pp.tile_keys = attn_tile_keys();
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
@@ -125,12 +127,19 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   pp.cta_first = w.cta_first;
   pp.items = w.items;
   pp.status = d.status;
+  pp.block_table = kv.block_table;
+  pp.page_size = kv.page_size;
+  pp.max_pages = kv.max_pages;
+  pp.num_pages = kv.num_pages;
+  pp.shared_tree = d.shared_tree != 0;
+  // Nothing in the workspace has to start at zero: the planner rebuilds every table it or the later kernels read, and
+  // a partial slot is always written by the attention kernel before the combine kernel reads it.
   if (launch_plan(pp, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
 
   AttnParams ap;
   ap.q = static_cast<const __nv_bfloat16*>(q);
-  ap.k = static_cast<const __nv_bfloat16*>(k_cache);
-  ap.v = static_cast<const __nv_bfloat16*>(v_cache);
+  ap.k = static_cast<const __nv_bfloat16*>(kv.k);
+  ap.v = static_cast<const __nv_bfloat16*>(kv.v);
   ap.out = static_cast<__nv_bfloat16*>(out);
   ap.B = d.batch;
   ap.Hq = d.num_q_heads;
@@ -138,9 +147,10 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.G = G;
   ap.D = d.head_dim;
   ap.T_max = d.max_tree;
-  ap.S_cap = d.kv_capacity;
+  ap.S_cap = s_cap;
   const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
   ap.scale_log2 = scale * 1.4426950408889634f;
+  ap.q_tma = 0;
   ap.hdr = w.hdr;
   ap.seq = w.seq;
   ap.anc = w.anc;
@@ -151,11 +161,56 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
   ap.part_ml = w.part_ml;
   ap.part_o = w.part_o;
   ap.status = d.status;
+  ap.block_table = kv.block_table;
+  ap.page_size = kv.block_table ? kv.page_size : 0;
+  ap.page_shift = 0;
+  while (kv.block_table && (1 << ap.page_shift) < kv.page_size) ++ap.page_shift;
+  ap.max_pages = kv.max_pages;
+  ap.num_pages = kv.num_pages;
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_combine(ap, w.unit_cap, dev->sm_count, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
+}
+
+// Entry with a caller-provided workspace, for either kind of cache.
+int attention_with_workspace(const eagle_attn_desc* desc, const void* q, const KvSource& kv, const int32_t* seq_lens,
+                             const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
+  const eagle_attn_desc& d = *desc;
+  Workspace w;
+  if (kv.capacity < 0 || !(d.sm_scale >= 0.f) || !carve_workspace(d, d.workspace, &w)) return EAGLE_ERR_SHAPE;
+  if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
+  if (!q || !kv.k || !kv.v || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
+  if (!d.workspace || (reinterpret_cast<uintptr_t>(d.workspace) & 255) || d.workspace_bytes < w.bytes) return EAGLE_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
+      (reinterpret_cast<uintptr_t>(out) & 15))
+    return EAGLE_ERR_SHAPE;
+  int err = 0;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
+  const int num_ctas = (dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas) & ~1;   // one persistent CTA per SM, in pairs
+  return attention_call(d, w, num_ctas, dev, q, kv, seq_lens, tree_parent, out, static_cast<cudaStream_t>(stream_));
+}
+
+}  // namespace
+
+int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                           const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const KvSource kv = {k_cache, v_cache, desc->kv_capacity, nullptr, 0, 0, 0};
+  return attention_with_workspace(desc, q, kv, seq_lens, tree_parent, out, stream_);
+}
+
+int eagle_tree_verify_attn_paged(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* pk, const int32_t* seq_lens,
+                                 const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
+  if (!desc || !pk) return EAGLE_ERR_NULL;
+  if (pk->num_pages < 1 || pk->page_size < 16 || (pk->page_size & (pk->page_size - 1)) || pk->max_pages_per_seq < 0) return EAGLE_ERR_SHAPE;
+  if (static_cast<int64_t>(pk->num_pages) * desc->num_kv_heads > 0x7fffffffll) return EAGLE_ERR_SHAPE;
+  if (desc->batch > 0 && desc->max_tree > 0 && !pk->block_table) return EAGLE_ERR_NULL;
+  const KvSource kv = {pk->k_pages, pk->v_pages, static_cast<int64_t>(pk->max_pages_per_seq) * pk->page_size, pk->block_table,
+                       pk->num_pages, pk->page_size, pk->max_pages_per_seq};
+  return attention_with_workspace(desc, q, kv, seq_lens, tree_parent, out, stream_);
 }
 
 namespace {
@@ -306,77 +361,8 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   if (!carve_static(d, num_ctas, scratch, &w)) return EAGLE_ERR_SHAPE;
   if (w.bytes > kStaticScratchBytes) return EAGLE_ERR_WORKSPACE;   // this shape needs more than the fixed array holds
   if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
-  if (!q || !k_cache || !v_cache || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
-  if ((reinterpret_cast<uintptr_t>(k_cache) & 15) || (reinterpret_cast<uintptr_t>(v_cache) & 15) ||
-      (reinterpret_cast<uintptr_t>(q) & 15) || (reinterpret_cast<uintptr_t>(out) & 15))
-    return EAGLE_ERR_SHAPE;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  const int di = d.head_dim == 128 ? 1 : 0;
-  if (!dev->attn_prepared[di]) {
-    if (attn_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
-    dev->attn_prepared[di] = true;
-  }
-  const int G = d.num_q_heads / d.num_kv_heads;
-
-  PlanParams pp;
-  pp.seq_lens = seq_lens;
-  pp.tree_sizes = d.tree_sizes;
-  pp.tree_parent = tree_parent;
-  pp.B = d.batch;
-  pp.Hkv = d.num_kv_heads;
-  pp.G = G;
-  pp.T_max = d.max_tree;
-  pp.S_cap = d.kv_capacity;
-  pp.tile_keys = attn_tile_keys();
-  pp.num_ctas = num_ctas;
-  pp.forced_splits = d.num_splits;
-  pp.snap_tiles = kPlanSnapTiles;
-  pp.item_overhead_tiles = kPlanItemOverheadTiles;
-  pp.unit_cap = w.unit_cap;
-  pp.item_cap = w.item_cap;
-  pp.slot_cap = w.slot_cap;
-  pp.hdr = w.hdr;
-  pp.seq = w.seq;
-  pp.anc = w.anc;
-  pp.units = w.units;
-  pp.cut_tiles = w.cut_tiles;
-  pp.cta_first = w.cta_first;
-  pp.items = w.items;
-  pp.status = d.status;
-  // Nothing in the array has to start at zero: the planner rebuilds every table it or the later kernels read, and
-  // a partial slot is always written by the attention kernel before the combine kernel reads it.
-  if (launch_plan(pp, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-
-  AttnParams ap;
-  ap.q = static_cast<const __nv_bfloat16*>(q);
-  ap.k = static_cast<const __nv_bfloat16*>(k_cache);
-  ap.v = static_cast<const __nv_bfloat16*>(v_cache);
-  ap.out = static_cast<__nv_bfloat16*>(out);
-  ap.B = d.batch;
-  ap.Hq = d.num_q_heads;
-  ap.Hkv = d.num_kv_heads;
-  ap.G = G;
-  ap.D = d.head_dim;
-  ap.T_max = d.max_tree;
-  ap.S_cap = d.kv_capacity;
-  const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
-  ap.scale_log2 = scale * 1.4426950408889634f;
-  ap.q_tma = 0;
-  ap.hdr = w.hdr;
-  ap.seq = w.seq;
-  ap.anc = w.anc;
-  ap.units = w.units;
-  ap.cut_tiles = w.cut_tiles;
-  ap.cta_first = w.cta_first;
-  ap.items = w.items;
-  ap.part_ml = w.part_ml;
-  ap.part_o = w.part_o;
-  ap.status = d.status;
-  if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  if (launch_combine(ap, w.unit_cap, dev->sm_count, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
-  return EAGLE_OK;
+  const KvSource kv = {k_cache, v_cache, d.kv_capacity, nullptr, 0, 0, 0};
+  return attention_call(d, w, num_ctas, dev, q, kv, seq_lens, tree_parent, out, static_cast<cudaStream_t>(stream_));
 }
 
 // ---------------------------------------------------------------------------------------------------------
@@ -551,6 +537,7 @@ const char* eagle_status_string(int code) {
     case EAGLE_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case EAGLE_ERR_DEVICE: return "no usable sm_100 device is current";
     case EAGLE_ERR_PATH: return "invalid accepted path (not increasing, outside the tree, or past the cache)";
+    case EAGLE_ERR_PAGE: return "block-table entry of a page in use outside the page pool";
     default: return "unknown status";
   }
 }

@@ -367,7 +367,7 @@ struct Bars {
   __device__ __forceinline__ uint32_t o_free() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 2); }
 };
 
-template <int D>
+template <int D, bool PAGED>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
             const __grid_constant__ CUtensorMap map_q) {
@@ -804,6 +804,8 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       struct Cursor {
         int tp, tile, tile_end, z;
         bool valid;
+        const int32_t* pages;   // paged cache: the sequence's row of the block table, and its last page in use
+        int last_page;
       };
       auto advance = [&](Cursor& c) {   // moves to the next KV tile of the work list
         if (++c.tile < c.tile_end) return;
@@ -812,7 +814,14 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (it.tile_end > it.tile_begin) {
             c.tile = it.tile_begin;
             c.tile_end = it.tile_end;
-            c.z = it.b * p.Hkv + it.g;
+            if constexpr (PAGED) {
+              const SeqPlan sp = p.seq[it.b];
+              c.z = it.g;
+              c.pages = p.block_table + static_cast<size_t>(it.b) * p.max_pages;
+              c.last_page = (sp.L + sp.n - 1) >> p.page_shift;
+            } else {
+              c.z = it.b * p.Hkv + it.g;
+            }
             return;
           }
         }
@@ -826,12 +835,29 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (!ok) return;
         TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
         mbar_expect_tx(B.full(slot), S::kTileBytes);
+        if constexpr (PAGED) {
+          // The tile's 128 slots come from one page (pages of 128 slots or more) or from 128 / page_size pages, one box
+          // each; the boxes land one under the other, which is the tile's layout.  A box past the sequence's last page
+          // fetches that last page again (its rows are masked), so the byte count of a tile never changes.
+          const int rows = p.page_size < kTileN ? p.page_size : kTileN;
+          for (int r0 = 0; r0 < kTileN; r0 += rows) {
+            const int key = c.tile * kTileN + r0;
+            int pi = key >> p.page_shift;
+            pi = pi < c.last_page ? pi : c.last_page;
+            const int page = __ldg(c.pages + pi);
 #pragma unroll
-        for (int sl = 0; sl < S::kSlabs; ++sl)
-          tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
-                      B.full(slot));
+            for (int sl = 0; sl < S::kSlabs; ++sl)
+              tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
+                          key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
+          }
+        } else {
+#pragma unroll
+          for (int sl = 0; sl < S::kSlabs; ++sl)
+            tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
+                        B.full(slot));
+        }
       };
-      Cursor ck = {tp_lo - 1, 0, 0, 0, true}, cv = {tp_lo - 1, 0, 0, 0, true};
+      Cursor ck = {tp_lo - 1, 0, 0, 0, true, nullptr, 0}, cv = {tp_lo - 1, 0, 0, 0, true, nullptr, 0};
       advance(ck);
       advance(cv);
       for (int i = 0; i < 3; ++i, ++n) {   // K(0), K(1), K(2)
@@ -898,13 +924,15 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [B*Hkv, S_cap, D] bf16 viewed as a 3-D tensor (d, slot, sequence-head); box = 64 x 128 x 1, 128-byte swizzle.
-bool make_kv_map(CUtensorMap* map, const void* base, int D, int S_cap, long long bh) {
+// [B*Hkv, S_cap, D] bf16 viewed as a 3-D tensor (d, slot, sequence-head); box = 64 x box_rows x 1, 128-byte swizzle.
+// A paged cache [num_pages, Hkv, page_size, D] is the same tensor with pages for sequences and page_size for S_cap;
+// its box has min(page_size, 128) rows.
+bool make_kv_map(CUtensorMap* map, const void* base, int D, int S_cap, long long bh, int box_rows = kTileN) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S_cap), static_cast<cuuint64_t>(bh)};
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D) * 2, static_cast<cuuint64_t>(S_cap) * D * 2};
-  const cuuint32_t box[3] = {64, kTileN, 1};
+  const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -948,25 +976,43 @@ namespace eagle {
 int attn_tile_keys() { return kTileN; }
 
 cudaError_t attn_prepare(int head_dim) {
-  if (head_dim == 128)
-    return cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kBytes);
-  return cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
+  cudaError_t e;
+  if (head_dim == 128) {
+    e = cudaFuncSetAttribute(attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kBytes);
+  }
+  e = cudaFuncSetAttribute(attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
 }
 
 // Returns cudaErrorInvalidValue when the tensor maps cannot be encoded.
 cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t stream) {
   AttnParams p = p_in;
   CUtensorMap mk, mv, mq;
-  const long long bh = static_cast<long long>(p.B) * p.Hkv;
-  if (!make_kv_map(&mk, p.k, p.D, p.S_cap, bh) || !make_kv_map(&mv, p.v, p.D, p.S_cap, bh)) return cudaErrorInvalidValue;
+  const bool paged = p.page_size > 0;
+  if (paged) {
+    const long long ph = static_cast<long long>(p.num_pages) * p.Hkv;
+    const int rows = p.page_size < kTileN ? p.page_size : kTileN;
+    if (!make_kv_map(&mk, p.k, p.D, p.page_size, ph, rows) || !make_kv_map(&mv, p.v, p.D, p.page_size, ph, rows)) return cudaErrorInvalidValue;
+  } else {
+    const long long bh = static_cast<long long>(p.B) * p.Hkv;
+    if (!make_kv_map(&mk, p.k, p.D, p.S_cap, bh) || !make_kv_map(&mv, p.v, p.D, p.S_cap, bh)) return cudaErrorInvalidValue;
+  }
   p.q_tma = (kBlockM % p.G == 0) ? 1 : 0;
   if (p.q_tma) {
     if (!make_q_map(&mq, p.q, p.D, p.Hq, p.T_max, p.B, p.G)) return cudaErrorInvalidValue;
   } else {
     mq = mk;   // unused by the kernel
   }
-  if (p.D == 128) attn_kernel<128><<<num_ctas, kThreads, Smem<128>::kBytes, stream>>>(p, mk, mv, mq);
-  else attn_kernel<64><<<num_ctas, kThreads, Smem<64>::kBytes, stream>>>(p, mk, mv, mq);
+  if (p.D == 128) {
+    if (paged) attn_kernel<128, true><<<num_ctas, kThreads, Smem<128>::kBytes, stream>>>(p, mk, mv, mq);
+    else attn_kernel<128, false><<<num_ctas, kThreads, Smem<128>::kBytes, stream>>>(p, mk, mv, mq);
+  } else {
+    if (paged) attn_kernel<64, true><<<num_ctas, kThreads, Smem<64>::kBytes, stream>>>(p, mk, mv, mq);
+    else attn_kernel<64, false><<<num_ctas, kThreads, Smem<64>::kBytes, stream>>>(p, mk, mv, mq);
+  }
   count_launch();
   return cudaGetLastError();
 }

@@ -117,6 +117,10 @@ struct AttnParams {
   float2* part_ml;
   float* part_o;
   int32_t* status;
+  // paged cache (page_size > 0): k / v are [num_pages, Hkv, page_size, D], slot j of sequence b is row j % page_size of
+  // page block_table[b * max_pages + j / page_size]; page_size is a power of two
+  const int32_t* block_table;
+  int32_t page_size, page_shift, max_pages, num_pages;
 };
 
 struct PlanParams {
@@ -138,6 +142,9 @@ struct PlanParams {
   int32_t* cta_first;
   WorkItem* items;
   int32_t* status;
+  const int32_t* block_table;   // paged cache: [B, max_pages] (null: contiguous cache)
+  int32_t page_size, max_pages, num_pages;
+  int32_t shared_tree;          // tree_parent is [T_max] and tree_sizes [1] (or null): one tree for every sequence
 };
 
 struct CommitParams {

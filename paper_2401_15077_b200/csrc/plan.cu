@@ -252,13 +252,24 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   // ---- per sequence (one warp each): validate, build masks, count tiles
   for (int b = tid >> 5; b < p.B; b += kPlanThreads / 32) {
     const int lane = tid & 31;
-    int n = p.tree_sizes ? p.tree_sizes[b] : T;
+    const int tb = p.shared_tree ? 0 : b;   // one tree for every sequence, or one per sequence
+    int n = p.tree_sizes ? p.tree_sizes[tb] : T;
     int L = p.seq_lens[b];
     int bad = 0;
     if (n < 0 || n > T) bad = EAGLE_ERR_TREE;
     else if (L < 0 || static_cast<long long>(L) + n > p.S_cap) bad = EAGLE_ERR_SEQ;
     uint64_t* anc = p.anc + static_cast<size_t>(b) * T;
-    if (!bad && !build_masks_warp(p.tree_parent + static_cast<size_t>(b) * T, n, anc, nullptr, lane)) bad = EAGLE_ERR_TREE;
+    if (!bad && !build_masks_warp(p.tree_parent + static_cast<size_t>(tb) * T, n, anc, nullptr, lane)) bad = EAGLE_ERR_TREE;
+    if (!bad && p.block_table && n > 0) {
+      // paged cache: every page that holds a visible slot must exist
+      const int used = (L + n + p.page_size - 1) / p.page_size;
+      bool page_ok = true;
+      for (int i = lane; i < used; i += 32) {
+        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages + i];
+        if (page < 0 || page >= p.num_pages) page_ok = false;
+      }
+      if (!__all_sync(0xffffffffu, page_ok)) bad = EAGLE_ERR_PAGE;
+    }
     if (bad) {
       if (lane == 0) report_status(p.status, bad);
       n = 0;

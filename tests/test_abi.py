@@ -28,8 +28,8 @@ def test_every_declared_symbol_is_exported(lib):
 def test_status_strings(lib):
     from paper_2401_15077_b200 import binding
     assert binding.status_string(0) == "ok"
-    seen = {binding.status_string(c) for c in range(-10, 1)}
-    assert len(seen) == 11 and "unknown status" not in seen
+    seen = {binding.status_string(c) for c in range(-11, 1)}
+    assert len(seen) == 12 and "unknown status" not in seen
     assert binding.status_string(-1234) == "unknown status"
 
 
@@ -69,6 +69,13 @@ def test_host_checks_return_before_any_launch(lib):
     assert lib.eagle_tree_accept(ctypes.byref(a), fake, None, fake, fake, fake, fake, fake, None) == -1
     assert lib.eagle_tree_build_mask(None, None, 1, 8, None, None, None, None) == -1
     assert lib.eagle_tree_build_mask(fake, None, 1, 99, fake, None, None, None) == -2
+    # paged cache: descriptor checks come first
+    assert lib.eagle_tree_verify_attn_paged(ctypes.byref(d), fake, None, fake, fake, fake, None) == -1
+    for pages, size, per_seq, want in [(0, 16, 4, -2), (4, 8, 4, -2), (4, 48, 4, -2), (4, 16, -1, -2), (4, 16, 4, -3)]:
+        pk = binding.PagedKV(4096, 4096, 4096, pages, size, per_seq)
+        assert lib.eagle_tree_verify_attn_paged(ctypes.byref(d), fake, ctypes.byref(pk), fake, fake, fake, None) == want
+    pk = binding.PagedKV(4096, 4096, None, 4, 16, 4)
+    assert lib.eagle_tree_verify_attn_paged(ctypes.byref(d), fake, ctypes.byref(pk), fake, fake, fake, None) == -1
     # the entry points added for the steps around verification: same rules
     assert lib.eagle_tree_accept_logits(ctypes.byref(a), fake, fake, fake, fake, fake, ctypes.c_float(0.0), fake, fake, None) == -2
     assert lib.eagle_tree_accept_logits(ctypes.byref(a), fake, fake, fake, fake, fake, ctypes.c_float(float("nan")), fake, fake, None) == -2
