@@ -800,7 +800,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     // the order in which the MMAs consume the tiles, since the score MMA runs three steps ahead of the PV MMA.
     // Entry n of that sequence lives in slot n % kSlots; with six slots the K tile of step g + 3 is requested when the
     // score MMA of step g has finished and the V tile of step g when the PV of step g - 3 has.
-    if (lane == 0) {
+    // Contiguous cache: one thread does it all.  Paged cache: the whole warp walks the list in step and lane i looks up
+    // and fetches the tile's i-th page, so the block-table reads of a tile are in flight together.
+    if (lane == 0 || PAGED) {
       struct Cursor {
         int tp, tile, tile_end, z;
         bool valid;
@@ -831,26 +833,33 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       uint32_t n = 0;   // position in the load sequence
       auto load_tile = [&](const Cursor& c, bool is_v) {
         const uint32_t slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
-        ok = mbar_wait(B.empty(slot), par, s_abort);
-        if (!ok) return;
-        TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
-        mbar_expect_tx(B.full(slot), S::kTileBytes);
         if constexpr (PAGED) {
           // The tile's 128 slots come from one page (pages of 128 slots or more) or from 128 / page_size pages, one box
           // each; the boxes land one under the other, which is the tile's layout.  A box past the sequence's last page
-          // fetches that last page again (its rows are masked), so the byte count of a tile never changes.
+          // fetches that last page again (its rows are masked), so the byte count of a tile never changes.  The page
+          // number is read before the wait for the slot, so that its latency is not added to the slot's turnaround.
           const int rows = p.page_size < kTileN ? p.page_size : kTileN;
-          for (int r0 = 0; r0 < kTileN; r0 += rows) {
-            const int key = c.tile * kTileN + r0;
-            int pi = key >> p.page_shift;
-            pi = pi < c.last_page ? pi : c.last_page;
-            const int page = __ldg(c.pages + pi);
+          const int r0 = lane * rows, key = c.tile * kTileN + r0;
+          int page = 0;
+          if (r0 < kTileN) {
+            const int pi = key >> p.page_shift;
+            page = __ldg(c.pages + (pi < c.last_page ? pi : c.last_page));
+          }
+          ok = mbar_wait_warp(B.empty(slot), par, s_abort);
+          if (!ok) return;
+          if (lane == 0) mbar_expect_tx(B.full(slot), S::kTileBytes);
+          __syncwarp();
+          if (r0 < kTileN) {
 #pragma unroll
             for (int sl = 0; sl < S::kSlabs; ++sl)
               tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
                           key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
           }
         } else {
+          ok = mbar_wait(B.empty(slot), par, s_abort);
+          if (!ok) return;
+          TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
+          mbar_expect_tx(B.full(slot), S::kTileBytes);
 #pragma unroll
           for (int sl = 0; sl < S::kSlabs; ++sl)
             tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes, is_v ? &map_v : &map_k, sl * 64, c.tile * kTileN, c.z,
