@@ -52,6 +52,8 @@ def _load():
         lib.oracle_tree_expand.restype = i32
         lib.oracle_tree_commit.argtypes = [i32] * 6 + [vp] * 4 + [i32] + [vp] * 4
         lib.oracle_tree_commit.restype = i32
+        lib.oracle_tree_commit_paged.argtypes = [i32] * 8 + [vp] * 7
+        lib.oracle_tree_commit_paged.restype = i32
         lib.oracle_num_threads.restype = i32
         _lib = lib
     return _lib
@@ -200,6 +202,24 @@ def tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree: int, featur
     if rc != 0:
         raise ValueError(f"oracle_tree_commit failed: {rc}")
     return dict(k_cache=k, v_cache=v, features_out=fout, new_seq_lens=new_len, valid=valid)
+
+
+def tree_commit_paged(k_pages, v_pages, block_table, seq_lens, accepted_path, max_tree: int):
+    """Commit of the accepted path on a paged cache.  ``k_pages`` / ``v_pages``: bf16 [num_pages, Hkv, page_size, D];
+    they are NOT modified: copies are returned.  Returns a dict: k_pages, v_pages (uint16 arrays), new_seq_lens, valid."""
+    k = _as(k_pages, np.uint16).copy()
+    v = _as(v_pages, np.uint16).copy()
+    bt, sl, path = _as(block_table, np.int32), _as(seq_lens, np.int32), _as(accepted_path, np.int32)
+    P, Hkv, ps, D = k.shape
+    B = sl.shape[0]
+    assert v.shape == k.shape and path.shape[0] == B and bt.shape[0] == B
+    new_len = np.full((B,), -1, np.int32)
+    valid = np.full((B,), -1, np.int32)
+    rc = _load().oracle_tree_commit_paged(B, Hkv, D, P, ps, bt.shape[1], max_tree, path.shape[1], _ptr(sl), _ptr(path), _ptr(bt),
+                                          _ptr(k), _ptr(v), _ptr(new_len), _ptr(valid))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_commit_paged failed: {rc}")
+    return dict(k_pages=k, v_pages=v, new_seq_lens=new_len, valid=valid)
 
 
 def tree_expand(probs, num_children, max_children: int, uniforms=None, greedy=None):

@@ -24,6 +24,7 @@
  *                              keys and values of the accepted tree nodes become the next slots of the
  *                              committed prefix, in path order; the accepted nodes' feature vectors are
  *                              gathered in the same order (plain definition: a simultaneous assignment).
+ *   oracle_tree_commit_paged - the same on a cache stored in pages.
  *
  * Readings taken where the paper is silent or garbled are listed next to the code that uses them.
  * Pins: see tests/test_oracle_*.py.  The sibling order, the lowest-index tie-break of argmax and the
@@ -479,6 +480,64 @@ int oracle_tree_commit(int batch, int num_kv_heads, int head_dim, int kv_capacit
       for (int j = 0; j < a; ++j)
         memcpy(features_out + ((size_t)b * path_cap + j) * feature_dim, features_in + ((size_t)b * max_tree + path[j]) * feature_dim,
                sizeof(uint16_t) * (size_t)feature_dim);
+  }
+  free(tmp);
+  return ORACLE_OK;
+}
+
+/*
+ * The same commit when the cache is kept in pages: slot j of sequence b is row j % page_size of page
+ * block_table[b, j / page_size] of k_pages / v_pages [num_pages, Hkv, page_size, D] (modified in place).  The rule is
+ * the one above with that address map; the capacity is max_pages_per_seq * page_size, and a path one of whose
+ * source or destination slots lies on a page outside [0, num_pages) is invalid as well.  Pages are not moved or
+ * allocated: the accepted rows are copied between (or within) the pages the sequence already owns.
+ */
+int oracle_tree_commit_paged(int batch, int num_kv_heads, int head_dim, int num_pages, int page_size, int max_pages_per_seq,
+                             int max_tree, int path_cap, const int32_t* seq_lens, const int32_t* accepted_path,
+                             const int32_t* block_table, uint16_t* k_pages, uint16_t* v_pages, int32_t* new_seq_lens,
+                             int32_t* valid) {
+  if (batch < 0 || num_kv_heads < 0 || head_dim < 0 || num_pages < 0 || page_size <= 0 || max_pages_per_seq < 0 || max_tree < 0 ||
+      path_cap < 0 || !seq_lens || !accepted_path || !block_table)
+    return ORACLE_ERR_ARG;
+  const size_t row = (size_t)head_dim;
+  const long long capacity = (long long)max_pages_per_seq * page_size;
+  uint16_t* tmp = (uint16_t*)malloc(sizeof(uint16_t) * row * (size_t)(path_cap > 0 ? path_cap : 1));
+  if (!tmp) return ORACLE_ERR_NOMEM;
+  for (int b = 0; b < batch; ++b) {
+    const int32_t* path = accepted_path + (size_t)b * path_cap;
+    const int32_t* table = block_table + (size_t)b * max_pages_per_seq;
+    const int L = seq_lens[b];
+    int a = 0, ok = L >= 0;
+    while (a < path_cap && path[a] != -1) ++a;
+    for (int j = 0; j < a && ok; ++j) {
+      if (path[j] < 0 || path[j] >= max_tree) ok = 0;
+      else if (j > 0 && path[j] <= path[j - 1]) ok = 0;
+      else if ((long long)L + path[j] >= capacity) ok = 0;
+      else {
+        const int src = table[(L + path[j]) / page_size], dst = table[(L + j) / page_size];
+        if (src < 0 || src >= num_pages || dst < 0 || dst >= num_pages) ok = 0;
+      }
+    }
+    if (valid) valid[b] = ok;
+    if (new_seq_lens) new_seq_lens[b] = ok ? L + a : L;
+    if (!ok) continue;
+    for (int t = 0; t < 2; ++t) {
+      uint16_t* pages = t == 0 ? k_pages : v_pages;
+      if (!pages) continue;
+      for (int g = 0; g < num_kv_heads; ++g) {
+        /* simultaneous assignment: read every source row, then write every destination row */
+        for (int j = 0; j < a; ++j) {
+          const int s = L + path[j];
+          memcpy(tmp + (size_t)j * row, pages + (((size_t)table[s / page_size] * num_kv_heads + g) * page_size + s % page_size) * row,
+                 sizeof(uint16_t) * row);
+        }
+        for (int j = 0; j < a; ++j) {
+          const int d = L + j;
+          memcpy(pages + (((size_t)table[d / page_size] * num_kv_heads + g) * page_size + d % page_size) * row, tmp + (size_t)j * row,
+                 sizeof(uint16_t) * row);
+        }
+      }
+    }
   }
   free(tmp);
   return ORACLE_OK;
