@@ -320,6 +320,17 @@ int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cach
                       int32_t* new_seq_lens, eagle_stream_t stream);
 
 /*
+ * eagle_tree_commit on a paged cache (see eagle_paged_kv): the pages named by kv->k_pages / kv->v_pages are updated IN
+ * PLACE although the struct declares them const (either may be NULL).  Rows are copied between, or within, the pages
+ * the sequence already owns; no page is allocated, freed or moved.  desc->kv_capacity is ignored (the capacity is
+ * max_pages_per_seq * page_size).  A source or destination slot whose block-table entry is outside [0, num_pages)
+ * sets *status to EAGLE_ERR_PAGE and the sequence is left alone, as for an invalid path.  Everything else as above.
+ */
+int eagle_tree_commit_paged(const eagle_commit_desc* desc, const eagle_paged_kv* kv, const int32_t* seq_lens,
+                            const int32_t* accepted_path, const void* features_in, void* features_out,
+                            int32_t* new_seq_lens, eagle_stream_t stream);
+
+/*
  * Tree-mask builder alone (the mask "tree attention" implies: Sec. 3.1, Sec. 3.3): for every node the bit set
  * of its ancestors and itself, and its depth (top-level nodes: 1).
  *   tree_parent device int32 [B, T_max]; tree_sizes device int32 [B] or NULL;

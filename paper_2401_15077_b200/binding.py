@@ -18,7 +18,8 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_build_mask", "eagle_status_string", "eagle_launch_count",
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
            "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit",
-           "eagle_tree_accept_logits", "eagle_tree_expand", "eagle_tree_verify_attn_paged"]
+           "eagle_tree_accept_logits", "eagle_tree_expand", "eagle_tree_verify_attn_paged",
+           "eagle_tree_commit_paged"]
 _lib = None
 
 
@@ -93,6 +94,8 @@ def load():
         lib.eagle_tree_expand.restype = ctypes.c_int
         lib.eagle_tree_commit.argtypes = [ctypes.POINTER(CommitDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_commit.restype = ctypes.c_int
+        lib.eagle_tree_commit_paged.argtypes = [ctypes.POINTER(CommitDesc), ctypes.POINTER(PagedKV), vp, vp, vp, vp, vp, vp]
+        lib.eagle_tree_commit_paged.restype = ctypes.c_int
         lib.eagle_tree_build_mask.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
         lib.eagle_tree_build_mask.restype = ctypes.c_int
         lib.eagle_status_string.argtypes = [ctypes.c_int]
@@ -326,6 +329,30 @@ def eagle_tree_commit(k_cache, v_cache, seq_lens, accepted_path, max_tree, featu
                                _dev(features, torch.bfloat16, "features", True), _dev(features_out, torch.bfloat16, "features_out", True),
                                _dev(new_seq_lens, torch.int32, "new_seq_lens"), _stream())
     _check(rc, "eagle_tree_commit")
+    return new_seq_lens, features_out
+
+
+def eagle_tree_commit_paged(k_pages, v_pages, block_table, seq_lens, accepted_path, max_tree, features=None, features_out=None,
+                            new_seq_lens=None, status=None):
+    """``eagle_tree_commit`` on a paged cache: k_pages / v_pages [num_pages, Hkv, page_size, D] are updated IN PLACE through
+    block_table [B, max_pages_per_seq].  Returns (new_seq_lens, features_out)."""
+    lib = load()
+    P, Hkv, ps, D = k_pages.shape
+    B = seq_lens.shape[0]
+    cap = accepted_path.shape[1]
+    F = 0 if features is None else features.shape[2]
+    if new_seq_lens is None:
+        new_seq_lens = torch.empty((B,), dtype=torch.int32, device=k_pages.device)
+    if features is not None and features_out is None:
+        features_out = torch.empty((B, cap, F), dtype=torch.bfloat16, device=k_pages.device)
+    d = CommitDesc(B, Hkv, D, 0, max_tree, cap, F, _dev(status, torch.int32, "status", True))
+    pk = PagedKV(_dev(k_pages, torch.bfloat16, "k_pages"), _dev(v_pages, torch.bfloat16, "v_pages", True),
+                 _dev(block_table, torch.int32, "block_table"), P, ps, block_table.shape[1])
+    rc = lib.eagle_tree_commit_paged(ctypes.byref(d), ctypes.byref(pk), _dev(seq_lens, torch.int32, "seq_lens"),
+                                     _dev(accepted_path, torch.int32, "accepted_path"), _dev(features, torch.bfloat16, "features", True),
+                                     _dev(features_out, torch.bfloat16, "features_out", True),
+                                     _dev(new_seq_lens, torch.int32, "new_seq_lens"), _stream())
+    _check(rc, "eagle_tree_commit_paged")
     return new_seq_lens, features_out
 
 

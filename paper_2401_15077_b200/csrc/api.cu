@@ -460,26 +460,26 @@ int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stre
   return ok ? EAGLE_OK : EAGLE_ERR_LAUNCH;
 }
 
-int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cache, const int32_t* seq_lens,
-                      const int32_t* accepted_path, const void* features_in, void* features_out,
-                      int32_t* new_seq_lens, eagle_stream_t stream_) {
-  if (!desc) return EAGLE_ERR_NULL;
+namespace {
+
+int commit_call(const eagle_commit_desc* desc, const KvSource& kv, const int32_t* seq_lens, const int32_t* accepted_path,
+                const void* features_in, void* features_out, int32_t* new_seq_lens, eagle_stream_t stream_) {
   const eagle_commit_desc& d = *desc;
   if (d.batch < 0 || d.batch > 65535 || d.num_kv_heads < 0 || d.num_kv_heads > 65535 || (d.head_dim != 64 && d.head_dim != 128) ||
-      d.kv_capacity < 0 || d.max_tree < 0 || d.max_tree > kMaxTree || d.path_cap < 0 || d.feature_dim < 0 || d.feature_dim % 8)
+      kv.capacity < 0 || d.max_tree < 0 || d.max_tree > kMaxTree || d.path_cap < 0 || d.feature_dim < 0 || d.feature_dim % 8)
     return EAGLE_ERR_SHAPE;
   if (d.batch == 0) return EAGLE_OK;
   if (!seq_lens || (d.path_cap > 0 && !accepted_path)) return EAGLE_ERR_NULL;
   const bool feats = d.feature_dim > 0 && features_out != nullptr;
   if (feats && !features_in) return EAGLE_ERR_NULL;
-  if ((reinterpret_cast<uintptr_t>(k_cache) & 15) || (reinterpret_cast<uintptr_t>(v_cache) & 15) ||
+  if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) ||
       (reinterpret_cast<uintptr_t>(features_in) & 15) || (reinterpret_cast<uintptr_t>(features_out) & 15))
     return EAGLE_ERR_SHAPE;
   int err = 0;
   if (!device_info(&err)) return err;
   CommitParams cp;
-  cp.k = static_cast<__nv_bfloat16*>(k_cache);
-  cp.v = static_cast<__nv_bfloat16*>(v_cache);
+  cp.k = static_cast<__nv_bfloat16*>(const_cast<void*>(kv.k));
+  cp.v = static_cast<__nv_bfloat16*>(const_cast<void*>(kv.v));
   cp.seq_lens = seq_lens;
   cp.path = accepted_path;
   cp.features_in = feats ? static_cast<const __nv_bfloat16*>(features_in) : nullptr;
@@ -488,13 +488,38 @@ int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cach
   cp.B = d.batch;
   cp.Hkv = d.num_kv_heads;
   cp.D = d.head_dim;
-  cp.S_cap = d.kv_capacity;
+  cp.S_cap = static_cast<int32_t>(kv.capacity < 0x7fffffff ? kv.capacity : 0x7fffffff);
   cp.T_max = d.max_tree;
   cp.path_cap = d.path_cap;
   cp.F = d.feature_dim;
   cp.status = d.status;
+  cp.block_table = kv.block_table;
+  cp.page_size = kv.page_size;
+  cp.max_pages = kv.max_pages;
+  cp.num_pages = kv.num_pages;
   if (launch_commit(cp, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
+}
+
+}  // namespace
+
+int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cache, const int32_t* seq_lens,
+                      const int32_t* accepted_path, const void* features_in, void* features_out,
+                      int32_t* new_seq_lens, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const KvSource kv = {k_cache, v_cache, desc->kv_capacity, nullptr, 0, 0, 0};
+  return commit_call(desc, kv, seq_lens, accepted_path, features_in, features_out, new_seq_lens, stream_);
+}
+
+int eagle_tree_commit_paged(const eagle_commit_desc* desc, const eagle_paged_kv* pk, const int32_t* seq_lens,
+                            const int32_t* accepted_path, const void* features_in, void* features_out,
+                            int32_t* new_seq_lens, eagle_stream_t stream_) {
+  if (!desc || !pk) return EAGLE_ERR_NULL;
+  if (pk->num_pages < 1 || pk->page_size < 16 || (pk->page_size & (pk->page_size - 1)) || pk->max_pages_per_seq < 0) return EAGLE_ERR_SHAPE;
+  if (desc->batch > 0 && !pk->block_table) return EAGLE_ERR_NULL;
+  const KvSource kv = {pk->k_pages, pk->v_pages, static_cast<int64_t>(pk->max_pages_per_seq) * pk->page_size, pk->block_table,
+                       pk->num_pages, pk->page_size, pk->max_pages_per_seq};
+  return commit_call(desc, kv, seq_lens, accepted_path, features_in, features_out, new_seq_lens, stream_);
 }
 
 int eagle_tree_expand(const eagle_expand_desc* desc, const float* draft_probs, const int32_t* num_children,

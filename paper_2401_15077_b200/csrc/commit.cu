@@ -7,6 +7,8 @@
 // then writes: at most 64 rows of 256 bytes per tensor, eight 16-byte vectors per thread.  Rows already in place
 // (path[j] == j) are skipped.  The CTA of KV head 0 also writes the new prefix length and gathers the features.
 // The work is a few hundred KB per call: the kernel is bound by launch and memory latency, not bandwidth.
+// With a paged cache (power-of-two page size) slot j of a sequence is row j % page_size of the page its block-table
+// row names; the pages of the source and destination slots are looked up once, while the path is checked.
 #include "common.cuh"
 
 namespace eagle {
@@ -18,6 +20,7 @@ constexpr int kMaxVecsPerThread = 4;   // 64 rows x 16 vectors (D = 128) / 256 t
 
 __global__ void __launch_bounds__(kCommitThreads) commit_kernel(CommitParams p) {
   __shared__ int s_path[kMaxTree];
+  __shared__ int s_src_page[kMaxTree], s_dst_page[kMaxTree];   // paged cache: page of slot L + path[j] / of slot L + j
   __shared__ int s_len, s_ok;
   const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x;
   const int L = p.seq_lens[b];
@@ -36,17 +39,26 @@ __global__ void __launch_bounds__(kCommitThreads) commit_kernel(CommitParams p) 
     // a row of more than 64 entries without a -1 cannot be a path of a tree of at most 64 nodes
     if (first_end == cap && p.path_cap > kMaxTree && path[kMaxTree] != -1) bad = 1;
     __syncwarp();
+    int bad_page = 0;
     for (int j = tid; j < first_end; j += 32) {
       const int m = s_path[j];
       if (m < 0 || m >= p.T_max) bad = 1;                                   // a tree node
       else if (j > 0 && m <= s_path[j - 1]) bad = 1;                        // a child comes after its parent
       else if (static_cast<long long>(L) + m >= p.S_cap) bad = 1;           // its slot exists
+      else if (p.block_table && L >= 0) {
+        const int32_t* table = p.block_table + static_cast<size_t>(b) * p.max_pages;
+        const int src = table[(L + m) / p.page_size], dst = table[(L + j) / p.page_size];
+        s_src_page[j] = src;
+        s_dst_page[j] = dst;
+        if (src < 0 || src >= p.num_pages || dst < 0 || dst >= p.num_pages) bad_page = 1;   // and so does its page
+      }
     }
     bad = __any_sync(0xffffffffu, bad);
+    bad_page = __any_sync(0xffffffffu, bad_page);
     if (tid == 0) {
       s_len = first_end;
-      s_ok = !bad;
-      if (bad && g == 0) report_status(p.status, EAGLE_ERR_PATH);
+      s_ok = !bad && !bad_page;
+      if (g == 0 && (bad || bad_page)) report_status(p.status, bad ? EAGLE_ERR_PATH : EAGLE_ERR_PAGE);
     }
   }
   __syncthreads();
@@ -71,14 +83,19 @@ __global__ void __launch_bounds__(kCommitThreads) commit_kernel(CommitParams p) 
   for (int t = 0; t < 2; ++t) {
     __nv_bfloat16* cache = t == 0 ? p.k : p.v;
     if (!cache) continue;                        // uniform over the CTA
-    uint4* base = reinterpret_cast<uint4*>(cache + (static_cast<size_t>(b) * p.Hkv + g) * static_cast<size_t>(p.S_cap) * p.D);
+    // row of slot `slot` (whose page is `page` when the cache is paged), as 16-byte vectors
+    auto row = [&](int slot, int page) -> uint4* {
+      const size_t r = p.block_table ? (static_cast<size_t>(page) * p.Hkv + g) * p.page_size + (slot & (p.page_size - 1))
+                                     : (static_cast<size_t>(b) * p.Hkv + g) * static_cast<size_t>(p.S_cap) + slot;
+      return reinterpret_cast<uint4*>(cache) + r * vpr;
+    };
     uint4 held[kMaxVecsPerThread];
 #pragma unroll
     for (int q = 0; q < kMaxVecsPerThread; ++q) {
       const int i = tid + q * kCommitThreads;
       if (i < total) {
         const int j = i / vpr, c = i % vpr, m = s_path[j];
-        if (m != j) held[q] = base[static_cast<size_t>(L + m) * vpr + c];
+        if (m != j) held[q] = row(L + m, s_src_page[j])[c];
       }
     }
     __syncthreads();                             // every source row has been read
@@ -87,7 +104,7 @@ __global__ void __launch_bounds__(kCommitThreads) commit_kernel(CommitParams p) 
       const int i = tid + q * kCommitThreads;
       if (i < total) {
         const int j = i / vpr, c = i % vpr, m = s_path[j];
-        if (m != j) base[static_cast<size_t>(L + j) * vpr + c] = held[q];
+        if (m != j) row(L + j, s_dst_page[j])[c] = held[q];
       }
     }
     __syncthreads();

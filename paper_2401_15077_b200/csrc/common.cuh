@@ -157,6 +157,8 @@ struct CommitParams {
   int32_t* new_seq_lens;     // [B] or null
   int32_t B, Hkv, D, S_cap, T_max, path_cap, F;
   int32_t* status;
+  const int32_t* block_table;   // paged cache: k / v are [num_pages, Hkv, page_size, D]; null: contiguous
+  int32_t page_size, max_pages, num_pages;
 };
 
 constexpr int kMaxChildren = 16;

@@ -76,6 +76,10 @@ def test_host_checks_return_before_any_launch(lib):
         assert lib.eagle_tree_verify_attn_paged(ctypes.byref(d), fake, ctypes.byref(pk), fake, fake, fake, None) == want
     pk = binding.PagedKV(4096, 4096, None, 4, 16, 4)
     assert lib.eagle_tree_verify_attn_paged(ctypes.byref(d), fake, ctypes.byref(pk), fake, fake, fake, None) == -1
+    c = binding.CommitDesc(1, 8, 64, 0, 8, 8, 0, None)
+    assert lib.eagle_tree_commit_paged(ctypes.byref(c), None, fake, fake, None, None, None, None) == -1
+    pk = binding.PagedKV(4096, 4096, 4096, 4, 24, 4)
+    assert lib.eagle_tree_commit_paged(ctypes.byref(c), ctypes.byref(pk), fake, fake, None, None, None, None) == -2
     # the entry points added for the steps around verification: same rules
     assert lib.eagle_tree_accept_logits(ctypes.byref(a), fake, fake, fake, fake, fake, ctypes.c_float(0.0), fake, fake, None) == -2
     assert lib.eagle_tree_accept_logits(ctypes.byref(a), fake, fake, fake, fake, fake, ctypes.c_float(float("nan")), fake, fake, None) == -2

@@ -160,3 +160,87 @@ def test_shared_tree_matches_oracle(E, oracle, name):
     # and identical bits to the call that is given the tree once per sequence
     per_seq = E.eagle_tree_verify_attn(qq.to(d), k.to(d), v.to(d), lens.to(d), parent.to(d), tree_sizes=sizes.to(d))
     assert torch.equal(out.view(torch.int16), per_seq.view(torch.int16))
+
+
+# ---- commit of the accepted path on a paged cache (bit exact)
+
+def _bits(t):
+    return t.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+COMMIT_CASES = {
+    "tiny": W.CONFIGS["tiny"],
+    "mix_small": W.scaled(W.CONFIGS["serving_mix"], batch=12, prefix=(0, 700)),
+    "d64_deep_chains": W.scaled(W.CONFIGS["tiny"], batch=9, num_q_heads=6, num_kv_heads=3, prefix=(0, 90), tree=(40, 64), max_depth=64,
+                                child_cap=2),
+}
+
+
+@pytest.mark.parametrize("page_size", [16, 64, 256])
+@pytest.mark.parametrize("name", list(COMMIT_CASES))
+def test_paged_commit_matches_oracle(E, oracle, name, page_size):
+    cfg = COMMIT_CASES[name]
+    d = torch.device("cuda:0")
+    moved = 0
+    for salt in range(2):
+        inp = W.make_attn_inputs(cfg, salt=salt, poison=False, capacity_pad=5)
+        pk = W.make_paged_cache(inp, page_size, salt=salt, poison=False)
+        paths = W.make_accepted_paths(inp.tree_sizes, inp.tree_parent, cfg.max_tree, cfg.index, salt)
+        g = torch.Generator().manual_seed(W.seed_for(cfg.index, "features", salt))
+        feats = torch.randn((cfg.batch, cfg.max_tree, 64), generator=g).to(torch.bfloat16)
+        ref = oracle.tree_commit_paged(pk.k_pages, pk.v_pages, pk.block_table, inp.seq_lens, paths, cfg.max_tree)
+        ref_f = oracle.tree_commit(inp.k_cache, inp.v_cache, inp.seq_lens, paths, cfg.max_tree, features=feats)["features_out"]
+        kd, vd = pk.k_pages.to(d), pk.v_pages.to(d)
+        status = torch.zeros(1, dtype=torch.int32, device=d)
+        new_len, fout = E.eagle_tree_commit_paged(kd, vd, pk.block_table.to(d), inp.seq_lens.to(d), paths.to(d), cfg.max_tree,
+                                                  features=feats.to(d), status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0 and ref["valid"].all()
+        assert np.array_equal(_bits(kd), ref["k_pages"]) and np.array_equal(_bits(vd), ref["v_pages"])
+        assert np.array_equal(new_len.cpu().numpy(), ref["new_seq_lens"])
+        assert np.array_equal(_bits(fout), ref_f)
+        moved += int((ref["new_seq_lens"] - inp.seq_lens.numpy()).sum())
+    assert moved > 0
+
+
+def test_paged_commit_bad_page_and_bad_path(E, oracle):
+    cfg = COMMIT_CASES["mix_small"]
+    d = torch.device("cuda:0")
+    inp = W.make_attn_inputs(cfg, poison=False)
+    pk = W.make_paged_cache(inp, 16, poison=False)
+    paths = W.make_accepted_paths(inp.tree_sizes, inp.tree_parent, cfg.max_tree, cfg.index)
+    lens = [int((paths[b] >= 0).sum()) for b in range(cfg.batch)]
+    victim = max(range(cfg.batch), key=lambda b: lens[b])
+    assert lens[victim] >= 1
+    L = int(inp.seq_lens[victim])
+    pk.block_table[victim, (L + int(paths[victim, lens[victim] - 1])) // 16] = -5
+    ref = oracle.tree_commit_paged(pk.k_pages, pk.v_pages, pk.block_table, inp.seq_lens, paths, cfg.max_tree)
+    assert ref["valid"][victim] == 0
+    kd, vd = pk.k_pages.to(d), pk.v_pages.to(d)
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    new_len, _ = E.eagle_tree_commit_paged(kd, vd, pk.block_table.to(d), inp.seq_lens.to(d), paths.to(d), cfg.max_tree, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == -11
+    assert np.array_equal(_bits(kd), ref["k_pages"]) and np.array_equal(_bits(vd), ref["v_pages"])
+    assert np.array_equal(new_len.cpu().numpy(), ref["new_seq_lens"])
+
+
+def test_verify_then_commit_then_verify_on_pages(E, oracle):
+    """The step as a serving loop runs it: attention over the pages, commit of a path, attention again from the new prefix."""
+    cfg = CASES["serving_mix_small"]
+    d = torch.device("cuda:0")
+    inp = W.make_attn_inputs(cfg, poison=False, capacity_pad=80)
+    pk = W.make_paged_cache(inp, 32, salt=9, poison=False)
+    paths = W.make_accepted_paths(inp.tree_sizes, inp.tree_parent, cfg.max_tree, cfg.index, 4)
+    kd, vd, bt = pk.k_pages.to(d), pk.v_pages.to(d), pk.block_table.to(d)
+    new_len, _ = E.eagle_tree_commit_paged(kd, vd, bt, inp.seq_lens.to(d), paths.to(d), cfg.max_tree)
+    # next step: a tree of the same shape hangs off the new prefix; its keys are whatever the slots hold (all finite here)
+    fits = (new_len.cpu() + inp.tree_sizes) <= (torch.tensor([(int(l) + int(n) + 31) // 32 * 32 for l, n in zip(inp.seq_lens, inp.tree_sizes)]))
+    sizes = torch.where(fits, inp.tree_sizes, torch.zeros_like(inp.tree_sizes))
+    q = inp.q.clone()
+    for b in range(cfg.batch):
+        q[b, int(sizes[b]):] = 0
+    out = E.eagle_tree_verify_attn_paged(q.to(d), kd, vd, bt, new_len, inp.tree_parent.to(d), tree_sizes=sizes.to(d))
+    torch.cuda.synchronize()
+    ref = oracle.tree_verify_attn_paged(q, kd.cpu(), vd.cpu(), pk.block_table, new_len.cpu(), inp.tree_parent, sizes)
+    _check(out.cpu(), ref, sizes)
