@@ -298,6 +298,40 @@ def main():
     expand_bytes = rows_exp.numel() * 4
     del rows_exp
 
+    # ---- the same attention over a paged cache (reported, not part of the headline): the first input set's keys and
+    # values cut into pages of 128 and of 16 slots, scattered over the pool by a seeded permutation
+    s = sets[0]
+    step(s)
+    ref_bits = out.view(torch.int16).clone()
+    paged = {}
+    for ps in (128, 16):
+        cap_p = (s["k"].shape[2] + ps - 1) // ps * ps
+        per_seq = cap_p // ps
+
+        def to_pages(x):
+            xp = torch.nn.functional.pad(x, (0, 0, 0, cap_p - x.shape[2]))
+            return xp.view(B, cfg.num_kv_heads, per_seq, ps, cfg.head_dim).permute(0, 2, 1, 3, 4).reshape(B * per_seq, cfg.num_kv_heads,
+                                                                                                      ps, cfg.head_dim)
+        gperm = torch.Generator().manual_seed(W.seed_for(cfg.index, "pages", ps))
+        perm = torch.randperm(B * per_seq, generator=gperm).to(dev)       # page i of the ordered pool goes to pool slot perm[i]
+        shape = (B * per_seq, cfg.num_kv_heads, ps, cfg.head_dim)
+        kp, vp = torch.empty(shape, dtype=torch.bfloat16, device=dev), torch.empty(shape, dtype=torch.bfloat16, device=dev)
+        kp[perm], vp[perm] = to_pages(s["k"]), to_pages(s["v"])
+        table = perm.view(B, per_seq).to(torch.int32).contiguous()
+        pe = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(8)]
+        for e in pe:
+            for x in e:
+                x.record()
+        for e in pe:
+            E.eagle_tree_verify_attn_paged(s["q"], kp, vp, table, s["sl"], s["par"], out, tree_sizes=s["ts"], workspace=ws,
+                                           status=status, num_splits=args.num_splits, events=(e[0], e[1]))
+        torch.cuda.synchronize()
+        paged[f"page_{ps}"] = {"attn_kernel_ms": statistics.median(e[0].elapsed_time(e[1]) for e in pe[3:]),
+                               "same_bits_as_contiguous": bool(torch.equal(out.view(torch.int16), ref_bits))}
+        del kp, vp
+    del ref_bits
+    assert int(status.item()) == 0
+
     # ---- commit of the accepted path for this layer's cache (the step after verification; reported, not part of the
     # headline).  It moves rows in place, so it runs on the last input set, after everything that reads the cache.
     s = sets[-1]
@@ -368,6 +402,7 @@ def main():
                       "tree_expand": {"ms": expand_ms, "rows": B * R_exp, "children": K_exp, "bytes": expand_bytes,
                                       "gbs": expand_bytes / (expand_ms * 1e-3) / 1e9,
                                       "note": "back-to-back calls on the same rows (warm L2)"},
+                      "paged_attention": paged,
                       "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
                                     "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}},
     }
