@@ -800,8 +800,8 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     // the order in which the MMAs consume the tiles, since the score MMA runs three steps ahead of the PV MMA.
     // Entry n of that sequence lives in slot n % kSlots; with six slots the K tile of step g + 3 is requested when the
     // score MMA of step g has finished and the V tile of step g when the PV of step g - 3 has.
-    // Contiguous cache: one thread does it all.  Paged cache: the whole warp walks the list in step and lane i looks up
-    // and fetches the tile's i-th page, so the block-table reads of a tile are in flight together.
+    // Contiguous cache: one thread does it all.  Paged cache: the whole warp walks the list in step and each lane looks up
+    // and fetches one box (a page, or a page's 64-column half) of the tile, so the block-table reads of a tile are in flight together.
     if (lane == 0 || PAGED) {
       struct Cursor {
         int tp, tile, tile_end, z;
@@ -839,7 +839,8 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           // fetches that last page again (its rows are masked), so the byte count of a tile never changes.  The page
           // number is read before the wait for the slot, so that its latency is not added to the slot's turnaround.
           const int rows = p.page_size < kTileN ? p.page_size : kTileN;
-          const int r0 = lane * rows, key = c.tile * kTileN + r0;
+          const int sl = lane % S::kSlabs;                      // lane = (box, 64-column slab): one TMA box per lane
+          const int r0 = (lane / S::kSlabs) * rows, key = c.tile * kTileN + r0;
           int page = 0;
           if (r0 < kTileN) {
             const int pi = key >> p.page_shift;
@@ -849,12 +850,9 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (!ok) return;
           if (lane == 0) mbar_expect_tx(B.full(slot), S::kTileBytes);
           __syncwarp();
-          if (r0 < kTileN) {
-#pragma unroll
-            for (int sl = 0; sl < S::kSlabs; ++sl)
-              tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
-                          key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
-          }
+          if (r0 < kTileN)
+            tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
+                        key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
         } else {
           ok = mbar_wait(B.empty(slot), par, s_abort);
           if (!ok) return;
