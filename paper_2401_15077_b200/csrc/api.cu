@@ -313,7 +313,7 @@ bool carve_static(const eagle_attn_desc& d, int num_ctas, void* base, Workspace*
   w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * static_cast<size_t>(d.batch > 0 ? d.batch : 1)));
   w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * static_cast<size_t>(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
   w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * static_cast<size_t>(units > 0 ? units : 1)));
-  w->cut_tiles = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * 2 * static_cast<size_t>(units > 0 ? units : 1)));
+  w->cut_tiles = reinterpret_cast<CutTile*>(take(sizeof(CutTile) * 2 * static_cast<size_t>(units > 0 ? units : 1)));
   w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
   w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * static_cast<size_t>(items > 0 ? items : 1)));
   w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * static_cast<size_t>(slots) * kBlockM));

@@ -40,6 +40,16 @@ struct UnitPlan {        // one per super-unit
   int32_t pad0;        // its sequence
 };
 
+// A query tile whose output has to be merged from several items' partials: everything the combine kernel needs, so
+// that it reads one record instead of walking unit -> item -> sequence.  The tile's pieces are the items
+// item0 + k * item_stride and the partial slots slot0 + k, k < count (an empty item's slot holds nothing).
+struct CutTile {
+  int32_t b, g, mt;
+  int32_t m_valid;     // query rows of the (sequence, KV head) that belong to tree nodes: tree size x group size
+  int32_t item0, item_stride;
+  int32_t slot0, count;
+};
+
 struct PlanHeader {
   int32_t n_items;
   int32_t n_slots;
@@ -56,7 +66,7 @@ struct Workspace {
   SeqPlan* seq;        // [B]
   uint64_t* anc;       // [B, T_max]
   UnitPlan* units;     // [unit_cap]
-  int32_t* cut_tiles;  // [2 * unit_cap]: the cut query tiles, as 2 * super-unit + tile-in-pair, in no particular order
+  CutTile* cut_tiles;  // [2 * unit_cap]: the cut query tiles, in no particular order
   int32_t* cta_first;  // [kMaxPlanCtas + 1]: team j owns the team pieces cta_first[j] .. cta_first[j+1] - 1
   WorkItem* items;     // [item_cap]
   float2* part_ml;     // [slot_cap, 128]   (reference max in the log2 domain, row sum)
@@ -87,7 +97,7 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * (size_t)(d.batch > 0 ? d.batch : 1)));
   w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * (size_t)(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
   w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * (size_t)(units > 0 ? units : 1)));
-  w->cut_tiles = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * 2 * (size_t)(units > 0 ? units : 1)));
+  w->cut_tiles = reinterpret_cast<CutTile*>(take(sizeof(CutTile) * 2 * (size_t)(units > 0 ? units : 1)));
   w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
   w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * (size_t)(items > 0 ? items : 1)));
   w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * (size_t)slots * kBlockM));
@@ -111,7 +121,7 @@ struct AttnParams {
   const SeqPlan* seq;
   const uint64_t* anc;
   const UnitPlan* units;
-  const int32_t* cut_tiles;
+  const CutTile* cut_tiles;
   const int32_t* cta_first;
   const WorkItem* items;
   float2* part_ml;
@@ -138,7 +148,7 @@ struct PlanParams {
   SeqPlan* seq;
   uint64_t* anc;
   UnitPlan* units;
-  int32_t* cut_tiles;
+  CutTile* cut_tiles;
   int32_t* cta_first;
   WorkItem* items;
   int32_t* status;

@@ -395,11 +395,22 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
           if (it.tile_end > it.tile_begin) live[paired ? m : 0] = true;
         }
       }
-      // the query tiles whose pieces the combine kernel has to merge (bit 30: a lone tile, whose pieces are the
-      // items of both CTAs)
+      // the query tiles whose pieces the combine kernel has to merge: a tile of a pair or twin is spread over one
+      // member's items (every second item), a lone tile over the items of both CTAs
       if (up.slot_base >= 0) {
-        for (int m = 0; m < 2; ++m)
-          if (live[m]) pg.cut_tiles[atomicAdd(&s_ncut, 1)] = (2 * u + m) | (paired ? 0 : 1 << 30);
+        for (int m = 0; m < 2; ++m) {
+          if (!live[m]) continue;
+          CutTile ct;
+          ct.b = b;
+          ct.g = ug.kind == kTwin ? g + m : g;
+          ct.mt = ug.kind == kPair ? 2 * mp + m : 2 * mp;
+          ct.m_valid = sp.n * p.G;
+          ct.item0 = 2 * up.first_item + (paired ? m : 0);
+          ct.item_stride = paired ? 2 : 1;
+          ct.slot0 = up.slot_base + (paired ? m * up.n_pieces : 0);
+          ct.count = paired ? up.n_pieces : 2 * up.n_pieces;
+          pg.cut_tiles[atomicAdd(&s_ncut, 1)] = ct;
+        }
       }
     }
   }
