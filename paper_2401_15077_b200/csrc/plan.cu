@@ -25,40 +25,67 @@ namespace {
 
 constexpr int kPlanThreads = 1024;
 
-// Exclusive prefix sums of value(i), i in [0, n), by one CTA; put(i, prefix) stores them; returns the total.
+// Two exclusive prefix sums at once, of value(i).a (64-bit) and value(i).b (32-bit), i in [0, n), by one CTA;
+// put(i, prefix_a, prefix_b) stores them; returns the totals.
 // Thread chunks -> warp scan -> scan of the 32 warp totals by the first warp -> back to the threads.
+struct ScanPair {
+  long long a;
+  int b;
+};
 template <class Value, class Put>
-__device__ long long block_exclusive_scan(int n, Value value, Put put, long long* scratch) {
+__device__ ScanPair block_exclusive_scan2(int n, Value value, Put put, long long* scratch_a, int* scratch_b) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunk = (n + kPlanThreads - 1) / kPlanThreads;
   const int i0 = min(tid * chunk, n), i1 = min(i0 + chunk, n);
-  long long local = 0;
-  for (int i = i0; i < i1; ++i) local += value(i);
-  long long inc = local;
-  for (int o = 1; o < 32; o <<= 1) {
-    const long long x = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += x;
+  ScanPair local = {0, 0};
+  for (int i = i0; i < i1; ++i) {
+    const ScanPair v = value(i);
+    local.a += v.a;
+    local.b += v.b;
   }
-  __syncthreads();                       // scratch may still be read by the previous scan
-  if (lane == 31) scratch[warp] = inc;
+  ScanPair inc = local;
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long xa = __shfl_up_sync(0xffffffffu, inc.a, o);
+    const int xb = __shfl_up_sync(0xffffffffu, inc.b, o);
+    if (lane >= o) {
+      inc.a += xa;
+      inc.b += xb;
+    }
+  }
+  __syncthreads();                       // the scratch arrays may still be read by the previous scan
+  if (lane == 31) {
+    scratch_a[warp] = inc.a;
+    scratch_b[warp] = inc.b;
+  }
   __syncthreads();
   if (warp == 0) {
-    const long long mine = scratch[lane];
-    long long winc = mine;
+    const long long mine_a = scratch_a[lane];
+    const int mine_b = scratch_b[lane];
+    long long wa = mine_a;
+    int wb = mine_b;
     for (int o = 1; o < 32; o <<= 1) {
-      const long long x = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += x;
+      const long long xa = __shfl_up_sync(0xffffffffu, wa, o);
+      const int xb = __shfl_up_sync(0xffffffffu, wb, o);
+      if (lane >= o) {
+        wa += xa;
+        wb += xb;
+      }
     }
-    scratch[lane] = winc - mine;         // exclusive prefix of the warp totals
-    if (lane == 31) scratch[32] = winc;  // grand total
+    scratch_a[lane] = wa - mine_a;       // exclusive prefixes of the warp totals
+    scratch_b[lane] = wb - mine_b;
+    if (lane == 31) {                    // grand totals
+      scratch_a[32] = wa;
+      scratch_b[32] = wb;
+    }
   }
   __syncthreads();
-  const long long total = scratch[32];
-  long long run = scratch[warp] + inc - local;
+  const ScanPair total = {scratch_a[32], scratch_b[32]};
+  ScanPair run = {scratch_a[warp] + inc.a - local.a, scratch_b[warp] + inc.b - local.b};
   for (int i = i0; i < i1; ++i) {
-    const long long v = value(i);   // read before put(): put may overwrite what value reads
-    put(i, run);
-    run += v;
+    const ScanPair v = value(i);   // read before put(): put may overwrite what value reads
+    put(i, run.a, run.b);
+    run.a += v.a;
+    run.b += v.b;
   }
   __syncthreads();
   return total;
@@ -83,10 +110,10 @@ __device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc,
   return true;
 }
 
-// The same masks by one warp: lane l holds nodes l and l + 32.  Every node starts with its own bit and a pointer to its
+// The same masks by one warp: lane l holds nodes l and l + 32 (and is given their parent entries).  Every node starts with its own bit and a pointer to its
 // parent; each round ORs in the mask of the node pointed to and jumps the pointer to that node's pointer, so six rounds
 // cover any path of up to 64 nodes.  Returns false (to all lanes) on an invalid entry.  anc[i >= n] is not written.
-__device__ inline bool build_masks_warp(const int32_t* par, int n, uint64_t* anc, uint8_t* depth, int lane) {
+__device__ inline bool build_masks_warp(int par_lo, int par_hi, int n, uint64_t* anc, uint8_t* depth, int lane) {
   uint64_t mask[2];
   int ptr[2];
   bool ok = true;
@@ -96,7 +123,7 @@ __device__ inline bool build_masks_warp(const int32_t* par, int n, uint64_t* anc
     mask[k] = 0ull;
     ptr[k] = -1;
     if (i < n) {
-      const int pi = par[i];
+      const int pi = k == 0 ? par_lo : par_hi;   // parent of node lane / of node lane + 32, loaded by the caller
       if (pi < -1 || pi >= i) ok = false;
       else {
         mask[k] = 1ull << i;
@@ -235,6 +262,7 @@ struct SeqGeom {
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   __shared__ long long s_scan[kPlanThreads / 32 + 1];
+  __shared__ int s_scan_b[kPlanThreads / 32 + 1];
   __shared__ int s_ncut;
   __shared__ SeqPlan s_seq[kSmemSeqs];
   __shared__ UnitPlan s_units[kSmemUnits];
@@ -249,54 +277,80 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   const int T = p.T_max;
   const int ovh = p.forced_splits > 0 ? 0 : p.item_overhead_tiles;
 
-  // ---- per sequence (one warp each): validate, build masks, count tiles
-  for (int b = tid >> 5; b < p.B; b += kPlanThreads / 32) {
+  // ---- per sequence (one warp each): validate, build masks, count tiles.  The inputs of a warp's next sequence are
+  // requested before the current one is worked on, and none of the loads depends on another's value.
+  {
     const int lane = tid & 31;
-    const int tb = p.shared_tree ? 0 : b;   // one tree for every sequence, or one per sequence
-    int n = p.tree_sizes ? p.tree_sizes[tb] : T;
-    int L = p.seq_lens[b];
-    int bad = 0;
-    if (n < 0 || n > T) bad = EAGLE_ERR_TREE;
-    else if (L < 0 || static_cast<long long>(L) + n > p.S_cap) bad = EAGLE_ERR_SEQ;
-    uint64_t* anc = p.anc + static_cast<size_t>(b) * T;
-    if (!bad && !build_masks_warp(p.tree_parent + static_cast<size_t>(tb) * T, n, anc, nullptr, lane)) bad = EAGLE_ERR_TREE;
-    if (!bad && p.block_table && n > 0) {
-      // paged cache: every page that holds a visible slot must exist
-      const int used = (L + n + p.page_size - 1) / p.page_size;
-      bool page_ok = true;
-      for (int i = lane; i < used; i += 32) {
-        const int page = p.block_table[static_cast<size_t>(b) * p.max_pages + i];
-        if (page < 0 || page >= p.num_pages) page_ok = false;
+    struct SeqIn {
+      int n, L, par_lo, par_hi;
+    };
+    auto fetch = [&](int b) {
+      SeqIn in;
+      const int tb = p.shared_tree ? 0 : b;   // one tree for every sequence, or one per sequence
+      const int32_t* par = p.tree_parent + static_cast<size_t>(tb) * T;
+      in.n = p.tree_sizes ? p.tree_sizes[tb] : T;
+      in.L = p.seq_lens[b];
+      in.par_lo = lane < T ? par[lane] : -1;
+      in.par_hi = lane + 32 < T ? par[lane + 32] : -1;
+      return in;
+    };
+    int b = tid >> 5;
+    SeqIn cur = {0, 0, -1, -1};
+    if (b < p.B) cur = fetch(b);
+    for (; b < p.B; b += kPlanThreads / 32) {
+      SeqIn next = {0, 0, -1, -1};
+      if (b + kPlanThreads / 32 < p.B) next = fetch(b + kPlanThreads / 32);
+      int n = cur.n, L = cur.L;
+      int bad = 0;
+      if (n < 0 || n > T) bad = EAGLE_ERR_TREE;
+      else if (L < 0 || static_cast<long long>(L) + n > p.S_cap) bad = EAGLE_ERR_SEQ;
+      uint64_t* anc = p.anc + static_cast<size_t>(b) * T;
+      if (!bad && !build_masks_warp(cur.par_lo, cur.par_hi, n, anc, nullptr, lane)) bad = EAGLE_ERR_TREE;
+      if (!bad && p.block_table && n > 0) {
+        // paged cache: every page that holds a visible slot must exist
+        const int used = (L + n + p.page_size - 1) / p.page_size;
+        bool page_ok = true;
+        for (int i = lane; i < used; i += 32) {
+          const int page = p.block_table[static_cast<size_t>(b) * p.max_pages + i];
+          if (page < 0 || page >= p.num_pages) page_ok = false;
+        }
+        if (!__all_sync(0xffffffffu, page_ok)) bad = EAGLE_ERR_PAGE;
       }
-      if (!__all_sync(0xffffffffu, page_ok)) bad = EAGLE_ERR_PAGE;
-    }
-    if (bad) {
-      if (lane == 0) report_status(p.status, bad);
-      n = 0;
-      L = 0;
-    }
-    for (int i = n + lane; i < T; i += 32) anc[i] = 0ull;
-    if (lane == 0) {
-      SeqPlan sp;
-      sp.n = n;
-      sp.L = L;
-      sp.mtiles = (n * p.G + kBlockM - 1) / kBlockM;
-      sp.ntiles = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;
-      sp.unit_base = 0;
-      sp.pad0 = 0;
-      sp.start = 0;
-      p.seq[b] = sp;
+      if (bad) {
+        if (lane == 0) report_status(p.status, bad);
+        n = 0;
+        L = 0;
+      }
+      for (int i = n + lane; i < T; i += 32) anc[i] = 0ull;
+      if (lane == 0) {
+        SeqPlan sp;
+        sp.n = n;
+        sp.L = L;
+        sp.mtiles = (n * p.G + kBlockM - 1) / kBlockM;
+        sp.ntiles = n > 0 ? (L + n + p.tile_keys - 1) / p.tile_keys : 0;
+        sp.unit_base = 0;
+        sp.pad0 = 0;
+        sp.start = 0;
+        p.seq[b] = sp;
+      }
+      cur = next;
     }
   }
   __syncthreads();
 
   // ---- lay the sequences' super-units end to end
-  const long long W = block_exclusive_scan(
-      p.B, [&](int b) { return SeqGeom(p.seq[b], p.Hkv, ovh).length(); },
-      [&](int b, long long v) { p.seq[b].start = v; }, s_scan);
-  const long long U = block_exclusive_scan(
-      p.B, [&](int b) { return static_cast<long long>(SeqGeom(p.seq[b], p.Hkv, ovh).units()); },
-      [&](int b, long long v) { p.seq[b].unit_base = static_cast<int>(v); }, s_scan);
+  const ScanPair WU = block_exclusive_scan2(
+      p.B,
+      [&](int b) {
+        const SeqGeom ge(p.seq[b], p.Hkv, ovh);
+        return ScanPair{ge.length(), ge.units()};
+      },
+      [&](int b, long long start, int unit_base) {
+        p.seq[b].start = start;
+        p.seq[b].unit_base = unit_base;
+      },
+      s_scan, s_scan_b);
+  const long long W = WU.a, U = WU.b;
   const int n_units = U <= p.unit_cap ? static_cast<int>(U) : 0;   // cannot exceed the advertised workspace
   if (U > p.unit_cap && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);
   const int max_teams = p.num_ctas / 2;
@@ -342,17 +396,23 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
     const bool partial = ge.unit(u - sp.unit_base).kind != kLone ? up.n_pieces > 1 : sp.ntiles > 1;
     return partial ? 2ll * up.n_pieces : 0ll;
   };
-  const long long TP = block_exclusive_scan(
-      n_units, [&](int u) { return static_cast<long long>(p.units[u].n_pieces); },
-      [&](int u, long long v) { p.units[u].first_item = static_cast<int>(v); }, s_scan);
-  const long long S = block_exclusive_scan(
-      n_units, slots_of, [&](int u, long long v) { p.units[u].slot_base = slots_of(u) > 0 ? static_cast<int>(v) : -1; }, s_scan);
+  const ScanPair TS = block_exclusive_scan2(
+      n_units, [&](int u) { return ScanPair{static_cast<long long>(p.units[u].n_pieces), static_cast<int>(slots_of(u))}; },
+      [&](int u, long long first_item, int slot_base) {
+        const bool has_slots = slots_of(u) > 0;     // (read before first_item is written: slots_of does not read it)
+        p.units[u].first_item = static_cast<int>(first_item);
+        p.units[u].slot_base = has_slots ? slot_base : -1;
+      },
+      s_scan, s_scan_b);
+  const long long TP = TS.a, S = TS.b;
   const bool fits = 2 * TP <= p.item_cap && S <= p.slot_cap;
   if (!fits && tid == 0) report_status(p.status, EAGLE_ERR_WORKSPACE);   // cannot happen with the advertised size
 
-  // ---- items: two per team piece, one for each CTA of the team
-  if (fits) {
-    for (int u = tid; u < n_units; u += kPlanThreads) {
+  // ---- items: two per team piece, one for each CTA of the team.  The last warps do not take part: they fill the
+  // teams' table and copy the tables out meanwhile (neither needs the items).
+  constexpr int kSideThreads = 160, kMainThreads = kPlanThreads - kSideThreads;
+  if (fits && tid < kMainThreads) {
+    for (int u = tid; u < n_units; u += kMainThreads) {
       const UnitPlan up = p.units[u];
       const int b = up.pad0;
       const SeqPlan sp = p.seq[b];
@@ -365,7 +425,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
       const long long t_origin = us + ovh;          // line position of the super-unit's tile position 0
       int c0 = 0;
       if (p.forced_splits == 0) unit_cuts(us, us + len + ovh, W, teams, snap, ovh, &c0, small);
-      bool live[2] = {false, false};    // query tiles of the super-unit with at least one non-empty item
+      bool live0 = false, live1 = false;    // query tiles of the super-unit with at least one non-empty item
       for (int j = 0; j < up.n_pieces; ++j) {
         int t0, t1;
         if (p.forced_splits > 0) {
@@ -392,14 +452,16 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
           }
           it.pad0 = it.pad1 = 0;
           p.items[2 * (up.first_item + j) + m] = it;
-          if (it.tile_end > it.tile_begin) live[paired ? m : 0] = true;
+          if (it.tile_end > it.tile_begin) {
+            if (paired && m == 1) live1 = true; else live0 = true;
+          }
         }
       }
       // the query tiles whose pieces the combine kernel has to merge: a tile of a pair or twin is spread over one
       // member's items (every second item), a lone tile over the items of both CTAs
       if (up.slot_base >= 0) {
         for (int m = 0; m < 2; ++m) {
-          if (!live[m]) continue;
+          if (!(m == 0 ? live0 : live1)) continue;
           CutTile ct;
           ct.b = b;
           ct.g = ug.kind == kTwin ? g + m : g;
@@ -416,7 +478,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   }
 
   // ---- first team piece of every team (cta_first is indexed by team here; entries past the last team repeat the end)
-  for (int c = tid; c <= p.num_ctas; c += kPlanThreads) {
+  for (int c = tid - kMainThreads; c >= 0 && c <= p.num_ctas; c += kSideThreads) {
     long long first;
     if (!fits || TP == 0) {
       first = 0;
@@ -453,11 +515,13 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
     }
     p.cta_first[c] = static_cast<int>(first);
   }
+  if (tid >= kMainThreads) {
+    if (seq_in_smem)
+      for (int b = tid - kMainThreads; b < p.B; b += kSideThreads) pg.seq[b] = s_seq[b];
+    if (units_in_smem)
+      for (int u = tid - kMainThreads; u < n_units; u += kSideThreads) pg.units[u] = s_units[u];
+  }
   __syncthreads();
-  if (seq_in_smem)
-    for (int b = tid; b < p.B; b += kPlanThreads) pg.seq[b] = s_seq[b];
-  if (units_in_smem)
-    for (int u = tid; u < n_units; u += kPlanThreads) pg.units[u] = s_units[u];
   if (tid == 0) {
     p.hdr->n_items = fits ? static_cast<int>(2 * TP) : 0;
     p.hdr->n_slots = fits ? static_cast<int>(S) : 0;
