@@ -169,6 +169,8 @@ typedef struct eagle_accept_desc {
   const uint8_t* greedy;       /* device uint8 [B] or NULL (= every sequence stochastic); 1: temperature-0 rule */
   int32_t* accept_len;         /* device int32 [B] or NULL: number of accepted nodes */
   int32_t* status;             /* device int32 or NULL */
+  int32_t shared_tree;         /* nonzero: one tree for every sequence: tree_parent is int32 [T_max], tree_sizes NULL or int32 [1]
+                                  (draft_tokens, the probability rows and the uniforms stay per sequence) */
 } eagle_accept_desc;
 
 /*
@@ -180,7 +182,7 @@ typedef struct eagle_accept_desc {
  *   draft_probs  device fp32 [B, T_max, V]     row i: the distribution node i's token was drawn from
  *                                              (may be NULL when every sequence is greedy)
  *   draft_tokens device int32 [B, T_max]
- *   tree_parent  device int32 [B, T_max]
+ *   tree_parent  device int32 [B, T_max]      ([T_max] when desc->shared_tree is set)
  *   uniforms     device fp32 [B, T_max+1]      entry i: the uniform of node i's accept test; entry T_max:
  *                                              the uniform of the final draw (may be NULL when all greedy)
  *   accepted_path device int32 [B, path_cap]   accepted node indices from the top of the tree down, then -1

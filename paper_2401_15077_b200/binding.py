@@ -43,7 +43,7 @@ class PagedKV(ctypes.Structure):
 class AcceptDesc(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("max_tree", ctypes.c_int32), ("vocab", ctypes.c_int32),
                 ("path_cap", ctypes.c_int32), ("tree_sizes", ctypes.c_void_p), ("greedy", ctypes.c_void_p),
-                ("accept_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+                ("accept_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("shared_tree", ctypes.c_int32)]
 
 
 class CommitDesc(ctypes.Structure):
@@ -243,7 +243,7 @@ def static_capacity() -> int:
 
 def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, accepted_path=None,
                       bonus_token=None, *, tree_sizes=None, greedy=None, accept_len=None, status=None, path_cap=None,
-                      temperature=None):
+                      temperature=None, shared_tree=False):
     """Acceptance walk.  target_probs [B,T+1,V] fp32; draft_probs [B,T,V] fp32; draft_tokens/tree_parent [B,T]
     int32; uniforms [B,T+1] fp32.  Returns (accepted_path [B,path_cap] int32, bonus_token [B] int32).
     With ``temperature`` the two tensors hold logits (``eagle_tree_accept_logits``)."""
@@ -256,14 +256,16 @@ def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, unif
         accepted_path = torch.empty((B, cap), dtype=torch.int32, device=dev)
     if bonus_token is None:
         bonus_token = torch.empty((B,), dtype=torch.int32, device=dev)
-    if tuple(draft_tokens.shape) != (B, T) or tuple(tree_parent.shape) != (B, T) or tuple(accepted_path.shape) != (B, cap):
+    if tuple(draft_tokens.shape) != (B, T) or tuple(accepted_path.shape) != (B, cap):
         raise EagleError("inconsistent shapes")
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
     if draft_probs is not None and tuple(draft_probs.shape) != (B, T, V):
         raise EagleError("draft_probs must be [B, T, V]")
     if uniforms is not None and tuple(uniforms.shape) != (B, T + 1):
         raise EagleError("uniforms must be [B, T+1]")
     d = AcceptDesc(B, T, V, cap, _dev(tree_sizes, torch.int32, "tree_sizes", True), _dev(greedy, torch.uint8, "greedy", True),
-                   _dev(accept_len, torch.int32, "accept_len", True), _dev(status, torch.int32, "status", True))
+                   _dev(accept_len, torch.int32, "accept_len", True), _dev(status, torch.int32, "status", True),
+                   1 if shared_tree else 0)
     head = (ctypes.byref(d), _dev(target_probs, torch.float32, "target_probs"), _dev(draft_probs, torch.float32, "draft_probs", True),
             _dev(draft_tokens, torch.int32, "draft_tokens"), _dev(tree_parent, torch.int32, "tree_parent"),
             _dev(uniforms, torch.float32, "uniforms", True))

@@ -224,13 +224,14 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
   TreeSmem& ts = s_tree[team_id];
 
   const int T = p.T, V = p.V;
-  int n = p.tree_sizes ? p.tree_sizes[b] : T;
+  const int tb = p.shared_tree ? 0 : b;   // one tree for every sequence, or one per sequence
+  int n = p.tree_sizes ? p.tree_sizes[tb] : T;
   const bool is_greedy = p.greedy && p.greedy[b] != 0;
   int bad = (n < 0 || n > T) ? EAGLE_ERR_TREE : 0;
   if (!bad && !is_greedy && (!p.draft || !p.uniforms)) bad = EAGLE_ERR_NULL;  // a stochastic walk needs both
   if (bad) n = 0;
   for (int i = team.tid; i < n; i += NT) {
-    ts.par[i] = p.parent[static_cast<size_t>(b) * T + i];
+    ts.par[i] = p.parent[static_cast<size_t>(tb) * T + i];
     ts.tok[i] = p.tokens[static_cast<size_t>(b) * T + i];
   }
   team.sync_cta();

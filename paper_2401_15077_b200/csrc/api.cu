@@ -247,6 +247,7 @@ int accept_call(const eagle_accept_desc* desc, const float* target, const float*
   ap.path_cap = d.path_cap;
   ap.logits = temperature >= 0.f ? 1 : 0;
   ap.inv_temp_log2 = temperature > 0.f ? 1.4426950408889634f / temperature : 0.f;
+  ap.shared_tree = d.shared_tree != 0;
   if (launch_accept(ap, dev->sm_count, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }

@@ -199,6 +199,7 @@ struct AcceptParams {
   int32_t B, T, V, path_cap;
   int32_t logits;        // target / draft hold logits: rows are softmax(logits / temperature)
   float inv_temp_log2;   // log2(e) / temperature
+  int32_t shared_tree;   // parent is [T] and tree_sizes [1] (or null): one tree for every sequence
 };
 
 __device__ inline void report_status(int32_t* status, int code) {

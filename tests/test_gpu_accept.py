@@ -204,3 +204,26 @@ def test_host_step_entry_matches_device_calls(E):
         assert torch.equal(runner.out.view(torch.int16), out.cpu().view(torch.int16))
         assert np.array_equal(runner.accepted_path.numpy(), path) and np.array_equal(runner.bonus_token.numpy(), bonus)
         assert np.array_equal(runner.accept_len.numpy(), alen)
+
+
+@pytest.mark.parametrize("mode", ["none", "half"])
+def test_one_tree_shared_by_every_sequence(E, oracle, mode):
+    """tree_parent given once ([T_max]) for all sequences: same tokens as the call that repeats it per sequence."""
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=10, vocab=5000)
+    sizes, parent = W.make_trees(cfg, 3)
+    n0 = int(sizes.max())
+    row = parent[int(sizes.argmax())]
+    trees = (torch.full((cfg.batch,), n0, dtype=torch.int32), row[None, :].expand(cfg.batch, -1).contiguous())
+    inp = W.make_accept_inputs(cfg, salt=3, trees=trees, greedy=mode)
+    ref = oracle.tree_accept(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
+                             tree_sizes=inp.tree_sizes, greedy=inp.greedy)
+    d = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    alen = torch.full((cfg.batch,), -7, dtype=torch.int32, device=d)
+    path, bonus = E.eagle_tree_accept(inp.target_probs.to(d), inp.draft_probs.to(d), inp.draft_tokens.to(d), row.contiguous().to(d),
+                                      inp.uniforms.to(d), tree_sizes=trees[0][:1].to(d), greedy=inp.greedy.to(d), accept_len=alen,
+                                      status=status, shared_tree=True)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert _compare(inp, ref, path.cpu().numpy(), bonus.cpu().numpy(), alen.cpu().numpy()) == 0
+    assert int(alen.sum()) > 0
