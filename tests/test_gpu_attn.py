@@ -160,6 +160,17 @@ def test_random_shapes(E, oracle, seed):
         out, status = _run(E, inp, num_splits=splits)
         assert status == 0, (cfg, splits)
         _check(out, ref, inp.tree_sizes)
+        # the same keys and values behind a block table, in pages of a random size: same plan, same bits
+        ps = int(rng.choice([16, 32, 64, 128, 256]))
+        pk = W.make_paged_cache(inp, ps, salt=seed)
+        d = torch.device("cuda:0")
+        st = torch.zeros(1, dtype=torch.int32, device=d)
+        paged = torch.full_like(out, float("nan")).to(d)
+        E.eagle_tree_verify_attn_paged(inp.q.to(d), pk.k_pages.to(d), pk.v_pages.to(d), pk.block_table.to(d), inp.seq_lens.to(d),
+                                       inp.tree_parent.to(d), paged, tree_sizes=inp.tree_sizes.to(d), num_splits=splits, status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0, (cfg, splits, ps)
+        assert torch.equal(paged.cpu().view(torch.int16), out.view(torch.int16)), (cfg, splits, ps)
 
 
 @pytest.mark.parametrize("seed", range(int(os.environ.get("EAGLE_RANDOM_BATCHES", "2"))))
