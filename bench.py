@@ -390,6 +390,7 @@ def main():
                    "l2": (f"rotating over {R} input sets" if R > 1 else "inputs larger than L2 (single set)")},
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+                "h2d_whole_tensor_bytes": runner.full_h2d_bytes,
                 "api": "eagle_tree_verify_step_host", "same_tokens_as_device_path": same_tokens},
         "roofline": {"bound": "hbm", "kernel": "split-KV tree attention", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, cfg.batch)),

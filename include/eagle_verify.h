@@ -206,7 +206,8 @@ int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, 
  * One whole verification step driven from HOST buffers (the two calls above, with the copies around them).
  *
  * Every input pointer below is a host pointer (pinned memory makes the copies asynchronous); the call enqueues on
- * `stream`: host->device copies of all inputs into `arena`, eagle_tree_verify_attn, eagle_tree_accept, and
+ * `stream`: host->device copies of the inputs into `arena` (see eagle_tree_verify_step_host_bytes for what is copied),
+ * eagle_tree_verify_attn, eagle_tree_accept, and
  * device->host copies of out, accepted_path, bonus_token and accept_len.  It allocates nothing: `arena` is device
  * memory provided by the caller, 256-byte aligned, at least eagle_tree_verify_step_host_arena() bytes (device copies
  * of all tensors plus the attention workspace).  The results are in the host buffers once `stream` has drained.
@@ -237,6 +238,16 @@ typedef struct eagle_host_step {
 
 size_t eagle_tree_verify_step_host_arena(const eagle_host_step* step);
 int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stream);
+
+/*
+ * Bytes one eagle_tree_verify_step_host call with these arguments copies host->device and device->host (host function,
+ * no CUDA work; reads the host arrays seq_lens and tree_sizes).  Of k_cache / v_cache only the slots a sequence can see
+ * (seq_lens[b] + tree size, clamped to the capacity; none for an empty tree) and of target_probs / draft_probs only the
+ * rows of existing nodes are ever read by the kernels, so when that saves more than the extra copy calls cost the step
+ * copies exactly those, sequence by sequence (2-D copies), and leaves the rest of the arena as it is; otherwise every
+ * tensor is copied whole.  This function reports which of the two the call does.
+ */
+int eagle_tree_verify_step_host_bytes(const eagle_host_step* step, size_t* h2d_bytes, size_t* d2h_bytes);
 
 /*
  * The same acceptance walk with the distributions given as LOGITS: every row the walk touches is taken as

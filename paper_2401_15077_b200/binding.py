@@ -19,7 +19,7 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
            "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit",
            "eagle_tree_accept_logits", "eagle_tree_expand", "eagle_tree_verify_attn_paged",
-           "eagle_tree_commit_paged"]
+           "eagle_tree_commit_paged", "eagle_tree_verify_step_host_bytes"]
 _lib = None
 
 
@@ -86,6 +86,9 @@ def load():
         lib.eagle_tree_verify_step_host.restype = ctypes.c_int
         lib.eagle_tree_verify_step_host_arena.argtypes = [ctypes.POINTER(HostStep)]
         lib.eagle_tree_verify_step_host_arena.restype = ctypes.c_size_t
+        lib.eagle_tree_verify_step_host_bytes.argtypes = [ctypes.POINTER(HostStep), ctypes.POINTER(ctypes.c_size_t),
+                                                          ctypes.POINTER(ctypes.c_size_t)]
+        lib.eagle_tree_verify_step_host_bytes.restype = ctypes.c_int
         lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_accept.restype = ctypes.c_int
         lib.eagle_tree_accept_logits.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
@@ -390,9 +393,12 @@ class HostStepRunner:
         self.arena = torch.empty(n, dtype=torch.uint8, device=device)
         s.arena, s.arena_bytes = self.arena.data_ptr(), n
         self.step = s
-        self.h2d_bytes = sum(t.numel() * t.element_size() for t in host.values() if t is not None)
-        self.d2h_bytes = sum(t.numel() * t.element_size() for t in (self.out, self.accepted_path, self.bonus_token,
-                                                                    self.accept_len, self.status))
+        # what the call copies: whole tensors, or (when that saves enough) only the visible cache slots and existing rows
+        self.full_h2d_bytes = sum(t.numel() * t.element_size() for t in host.values() if t is not None)
+        h2d, d2h = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        _check(lib.eagle_tree_verify_step_host_bytes(ctypes.byref(s), ctypes.byref(h2d), ctypes.byref(d2h)),
+               "eagle_tree_verify_step_host_bytes")
+        self.h2d_bytes, self.d2h_bytes = int(h2d.value), int(d2h.value)
 
     def run(self):
         _check(load().eagle_tree_verify_step_host(ctypes.byref(self.step), _stream()), "eagle_tree_verify_step_host")

@@ -404,12 +404,63 @@ bool host_step_layout(const eagle_host_step& s, HostStepLayout* L) {
   return true;
 }
 
+// What one host-driven step really has to bring to the device: of the caches only the slots a sequence can see
+// (prefix + tree), of the probability tensors only the rows of nodes that exist.  Slots and rows past those are never
+// read by the kernels, so they are left as they are in the arena.  Copying sequence by sequence costs one call per
+// sequence and tensor; it is done when the bytes it saves are worth more than those calls.
+struct HostStepTrim {
+  bool per_sequence;
+  size_t h2d_bytes, d2h_bytes;
+};
+
+inline void host_seq_extent(const eagle_host_step& s, int b, int* nodes, long long* slots) {
+  int n = s.tree_sizes ? s.tree_sizes[b] : s.max_tree;
+  n = n < 0 ? 0 : (n > s.max_tree ? s.max_tree : n);
+  long long vis = n > 0 ? static_cast<long long>(s.seq_lens[b]) + n : 0;   // an empty tree reads nothing
+  vis = vis < 0 ? 0 : (vis > s.kv_capacity ? s.kv_capacity : vis);
+  *nodes = n;
+  *slots = vis;
+}
+
+HostStepTrim host_step_trim(const eagle_host_step& s, const HostStepLayout& L) {
+  HostStepTrim t;
+  const size_t small = L.n_q + 2 * L.n_b + 2 * L.n_bt + L.n_u + (s.greedy ? static_cast<size_t>(s.batch) : 0) -
+                       (s.tree_sizes ? 0 : L.n_b) - (s.uniforms ? 0 : L.n_u);
+  const size_t full = small + 2 * L.n_kv + L.n_target + (s.draft_probs ? L.n_draft : 0);
+  size_t trimmed = small;
+  const size_t slot_bytes = static_cast<size_t>(s.num_kv_heads) * s.head_dim * 2, row_bytes = static_cast<size_t>(s.vocab) * 4;
+  for (int b = 0; b < s.batch; ++b) {
+    int n;
+    long long vis;
+    host_seq_extent(s, b, &n, &vis);
+    trimmed += 2 * static_cast<size_t>(vis) * slot_bytes + (static_cast<size_t>(n) + 1) * row_bytes +
+               (s.draft_probs ? static_cast<size_t>(n) * row_bytes : 0);
+  }
+  const size_t calls = static_cast<size_t>(s.batch) * 4;
+  t.per_sequence = full > trimmed && full - trimmed > calls * (200u << 10);   // a call costs about what 200 KB take on the link
+  t.h2d_bytes = t.per_sequence ? trimmed : full;
+  t.d2h_bytes = L.n_q + L.n_path + 2 * L.n_b + 4;
+  return t;
+}
+
 }  // namespace
 
 size_t eagle_tree_verify_step_host_arena(const eagle_host_step* step) {
   HostStepLayout L;
   if (!step || !host_step_layout(*step, &L)) return 0;
   return L.total;
+}
+
+int eagle_tree_verify_step_host_bytes(const eagle_host_step* step, size_t* h2d_bytes, size_t* d2h_bytes) {
+  HostStepLayout L;
+  if (!step) return EAGLE_ERR_NULL;
+  if (!host_step_layout(*step, &L)) return EAGLE_ERR_SHAPE;
+  if (step->batch > 0 && !step->seq_lens) return EAGLE_ERR_NULL;
+  HostStepTrim t = {false, 0, 0};
+  if (step->batch > 0) t = host_step_trim(*step, L);
+  if (h2d_bytes) *h2d_bytes = t.h2d_bytes;
+  if (d2h_bytes) *d2h_bytes = t.d2h_bytes;
+  return EAGLE_OK;
 }
 
 int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stream_) {
@@ -432,10 +483,33 @@ int eagle_tree_verify_step_host(const eagle_host_step* step, eagle_stream_t stre
     return !dst || n == 0 || cudaMemcpyAsync(dst, A + off, n, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
   };
   bool ok = cudaMemsetAsync(A + L.status, 0, 4, stream) == cudaSuccess;
-  ok = ok && h2d(L.q, s.q, L.n_q) && h2d(L.k, s.k_cache, L.n_kv) && h2d(L.v, s.v_cache, L.n_kv) &&
-       h2d(L.seq_lens, s.seq_lens, L.n_b) && h2d(L.tree_sizes, s.tree_sizes, L.n_b) && h2d(L.tree_parent, s.tree_parent, L.n_bt) &&
-       h2d(L.target, s.target_probs, L.n_target) && h2d(L.draft, s.draft_probs, L.n_draft) && h2d(L.tokens, s.draft_tokens, L.n_bt) &&
-       h2d(L.uniforms, s.uniforms, L.n_u) && h2d(L.greedy, s.greedy, static_cast<size_t>(s.batch));
+  ok = ok && h2d(L.q, s.q, L.n_q) && h2d(L.seq_lens, s.seq_lens, L.n_b) && h2d(L.tree_sizes, s.tree_sizes, L.n_b) &&
+       h2d(L.tree_parent, s.tree_parent, L.n_bt) && h2d(L.tokens, s.draft_tokens, L.n_bt) && h2d(L.uniforms, s.uniforms, L.n_u) &&
+       h2d(L.greedy, s.greedy, static_cast<size_t>(s.batch));
+  if (host_step_trim(s, L).per_sequence) {
+    // per sequence: the visible slots of every KV head (a 2-D copy: one row per head) and the rows of existing nodes
+    const size_t slot = static_cast<size_t>(s.head_dim) * 2, pitch = static_cast<size_t>(s.kv_capacity) * slot;
+    const size_t row = static_cast<size_t>(s.vocab) * 4, T = static_cast<size_t>(s.max_tree);
+    for (int b = 0; b < s.batch && ok; ++b) {
+      int n;
+      long long vis;
+      host_seq_extent(s, b, &n, &vis);
+      const size_t kv_off = static_cast<size_t>(b) * s.num_kv_heads * pitch;
+      if (vis > 0) {
+        ok = cudaMemcpy2DAsync(A + L.k + kv_off, pitch, static_cast<const char*>(s.k_cache) + kv_off, pitch, static_cast<size_t>(vis) * slot,
+                               static_cast<size_t>(s.num_kv_heads), cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+             cudaMemcpy2DAsync(A + L.v + kv_off, pitch, static_cast<const char*>(s.v_cache) + kv_off, pitch, static_cast<size_t>(vis) * slot,
+                               static_cast<size_t>(s.num_kv_heads), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+      }
+      const size_t t_off = static_cast<size_t>(b) * (T + 1) * row, d_off = static_cast<size_t>(b) * T * row;
+      ok = ok && h2d(L.target + t_off, static_cast<const char*>(static_cast<const void*>(s.target_probs)) + t_off, (static_cast<size_t>(n) + 1) * row);
+      if (s.draft_probs && n > 0)
+        ok = ok && h2d(L.draft + d_off, static_cast<const char*>(static_cast<const void*>(s.draft_probs)) + d_off, static_cast<size_t>(n) * row);
+    }
+  } else {
+    ok = ok && h2d(L.k, s.k_cache, L.n_kv) && h2d(L.v, s.v_cache, L.n_kv) && h2d(L.target, s.target_probs, L.n_target) &&
+         h2d(L.draft, s.draft_probs, L.n_draft);
+  }
   if (!ok) return EAGLE_ERR_LAUNCH;
   int32_t* d_status = reinterpret_cast<int32_t*>(A + L.status);
   const int32_t* d_sizes = s.tree_sizes ? reinterpret_cast<const int32_t*>(A + L.tree_sizes) : nullptr;

@@ -183,9 +183,13 @@ def test_output_distribution_on_gpu_chi_square(E):
     assert stats.chisquare(np.bincount(first, minlength=V), pr * n).pvalue > 1e-3
 
 
-def test_host_step_entry_matches_device_calls(E):
-    """eagle_tree_verify_step_host (copies in, attention, acceptance, copies out) gives what the two device calls give."""
-    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=5, prefix=(50, 900), vocab=3000)
+@pytest.mark.parametrize("ragged", [True, False])
+def test_host_step_entry_matches_device_calls(E, ragged):
+    """eagle_tree_verify_step_host (copies in, attention, acceptance, copies out) gives what the two device calls give.
+    Ragged lengths take the sequence-by-sequence copies of the visible slots and existing rows only (the arena is filled
+    with NaN bit patterns first: nothing that was not copied may be read); equal full-size sequences take whole-tensor copies."""
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=5, prefix=(50, 900) if ragged else (700, 700), tree=(16, 64) if ragged else (64, 64),
+                   max_depth=12, vocab=3000)
     attn = W.make_attn_inputs(cfg, salt=3)
     acc = W.make_accept_inputs(cfg, salt=3, trees=(attn.tree_sizes, attn.tree_parent))
     d = torch.device("cuda:0")
@@ -197,6 +201,8 @@ def test_host_step_entry_matches_device_calls(E):
                 tree_parent=attn.tree_parent, target_probs=acc.target_probs, draft_probs=acc.draft_probs,
                 draft_tokens=acc.draft_tokens, uniforms=acc.uniforms, greedy=acc.greedy)
     runner = E.HostStepRunner({k: v.pin_memory() for k, v in host.items()}, d)
+    assert (runner.h2d_bytes < runner.full_h2d_bytes) == ragged
+    runner.arena.fill_(255)
     for _ in range(2):
         runner.run()
         torch.cuda.synchronize()
