@@ -386,6 +386,10 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + S::kMisc + 4);
 
   if (tid == 0) {
+    // the descriptors of the three tensors are fetched ahead of the first copies that need them
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_k)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
     for (int i = 0; i < kSlots; ++i) {
       mbar_init(B.full(i), 1);
       mbar_init(B.empty(i), 1);
