@@ -607,7 +607,8 @@ int eagle_tree_expand(const eagle_expand_desc* desc, const float* draft_probs, c
   if (!draft_probs || !num_children || !child_tokens) return EAGLE_ERR_NULL;
   if (!uniforms && !d.greedy) return EAGLE_ERR_NULL;
   int err = 0;
-  if (!device_info(&err)) return err;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
   ExpandParams ep;
   ep.probs = draft_probs;
   ep.num_children = num_children;
@@ -620,7 +621,7 @@ int eagle_tree_expand(const eagle_expand_desc* desc, const float* draft_probs, c
   ep.V = d.vocab;
   ep.K = d.max_children;
   ep.status = d.status;
-  if (launch_expand(ep, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  if (launch_expand(ep, dev->sm_count, static_cast<cudaStream_t>(stream_)) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   return EAGLE_OK;
 }
 

@@ -217,7 +217,7 @@ cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cuda
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
 
 cudaError_t launch_commit(const CommitParams& p, cudaStream_t stream);
-cudaError_t launch_expand(const ExpandParams& p, cudaStream_t stream);
+cudaError_t launch_expand(const ExpandParams& p, int sm_count, cudaStream_t stream);
 void count_launch();
 
 }  // namespace eagle

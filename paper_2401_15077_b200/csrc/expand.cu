@@ -1,9 +1,9 @@
 // Child tokens of draft-tree nodes (App. A.1: in the greedy setting the k most probable tokens of a node's draft
 // distribution become its children, otherwise k tokens are sampled; k differs from node to node).
 //
-// One CTA per (sequence, node): 1024 threads when the row is staged in shared memory, else 256.  The row (128 KB at
-// V = 32000) is first copied into shared memory with coalesced 16-byte loads (when it fits; else it is re-read
-// through L1 / L2), so HBM is read once and everything below runs out of shared memory.
+// A row (128 KB at V = 32000) that fits shared memory is staged there by a CTA of 1024 threads with coalesced 16-byte
+// loads, so HBM is read once and everything else runs out of shared memory; one such CTA per SM walks the rows and
+// fetches its next row into registers meanwhile.  Longer rows are read through L1 / L2 by one CTA of 256 threads each.
 // Greedy: every thread keeps the largest key among its own tokens that is still available; a round is a block-wide
 // maximum over those, and only the round's winner rescans its tokens.  The key (value bits in sortable order,
 // inverted token id) is unique, so ties go to the lower id and the result is exact.
@@ -24,54 +24,52 @@ __device__ __forceinline__ unsigned int sortable_bits(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Largest key among the 32 per-warp maxima in s_red, by every warp on its own (one load per lane, five shuffles).
+__device__ __forceinline__ unsigned long long max_of_warp_maxima(const unsigned long long* s_red, int n_warps, int lane) {
+  unsigned long long best = lane < n_warps ? s_red[lane] : 0ull;
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long x = __shfl_xor_sync(0xffffffffu, best, o);
+    best = x > best ? x : best;
+  }
+  return best;
+}
+
+// One row: `row` points at its V probabilities (shared memory when staged, else global).  Called by the whole CTA.
 template <int kExpandThreads>
-__global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandParams p, int stage_row) {
+__device__ __forceinline__ void expand_row(const ExpandParams& p, size_t node, const float* row, int k, bool greedy,
+                                           unsigned long long* s_red, double* s_sum, int* s_tok, float* s_un) {
   constexpr int kExpandWarps = kExpandThreads / 32;
-  extern __shared__ __align__(16) float s_row[];
-  __shared__ unsigned long long s_red[kExpandWarps];
-  __shared__ double s_sum[kExpandWarps];
-  __shared__ int s_tok[kMaxChildren];
+  static_assert(kExpandWarps <= 32, "the warp maxima are reduced by one warp");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const size_t node = static_cast<size_t>(blockIdx.y) * p.R + blockIdx.x;
-  const int b = blockIdx.y, V = p.V, K = p.K;
-  const float* row = p.probs + node * V;
+  const int V = p.V, K = p.K;
   int32_t* out = p.tokens + node * K;
   float* outp = p.token_probs ? p.token_probs + node * K : nullptr;
-  int k = p.num_children[node];
-  const bool greedy = p.greedy && p.greedy[b] != 0;
-  bool bad = k < 0 || k > K || (greedy && k > V) || (!greedy && k > 0 && !p.uniforms);
-  if (bad) {
-    if (tid == 0) report_status(p.status, EAGLE_ERR_SHAPE);
-    k = 0;
-  }
   if (tid < K) s_tok[tid] = -1;
-  if (stage_row && k > 0) {
-    // rows start 16-byte aligned when V % 4 == 0 and the tensor does
-    if ((V & 3) == 0 && (reinterpret_cast<uintptr_t>(p.probs) & 15) == 0) {
-      const float4* src = reinterpret_cast<const float4*>(row);
-      float4* dst = reinterpret_cast<float4*>(s_row);
-#pragma unroll 8
-      for (int i = tid; i < V / 4; i += kExpandThreads) dst[i] = __ldg(src + i);
-    } else {
-      for (int v = tid; v < V; v += kExpandThreads) s_row[v] = row[v];
-    }
-    row = s_row;
-  }
   __syncthreads();
-
   if (greedy) {
-    // Every thread keeps the largest key among its own tokens that has not been taken yet; a round is a block-wide
-    // maximum over those, after which only the winning thread looks for its next one.
-    auto local_best = [&](unsigned long long below) {
-      unsigned long long best = 0ull;  // keys are never 0: the id part of a real token is at least 1
+    // Every thread keeps the two largest keys among its own tokens that have not been taken yet; a round is a
+    // block-wide maximum over the first of them, after which the winning thread moves its second key up.  Only a thread
+    // that wins twice in a row has to look through its tokens again (a one-thread chain of ~30 shared-memory reads,
+    // which used to follow every round).
+    unsigned long long mine = 0ull, second = 0ull;   // keys are never 0: the id part of a real token is at least 1
+    auto rescan = [&](unsigned long long below) {
+      mine = 0ull;
+      second = 0ull;
       for (int v = tid; v < V; v += kExpandThreads) {
         const unsigned long long key = (static_cast<unsigned long long>(sortable_bits(row[v])) << 32) |
                                        static_cast<unsigned int>(~static_cast<unsigned int>(v));
-        if (key < below && key > best) best = key;
+        if (key < below) {
+          if (key > mine) {
+            second = mine;
+            mine = key;
+          } else if (key > second) {
+            second = key;
+          }
+        }
       }
-      return best;
     };
-    unsigned long long mine = local_best(~0ull);   // every key is below ~0
+    bool second_known = true;
+    if (k > 0) rescan(~0ull);   // every key is below ~0
     for (int j = 0; j < k; ++j) {
       unsigned long long best = mine;
       for (int o = 16; o > 0; o >>= 1) {
@@ -80,12 +78,17 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandParams p, 
       }
       if (lane == 0) s_red[warp] = best;
       __syncthreads();
-      best = s_red[0];
-      for (int w = 1; w < kExpandWarps; ++w) best = s_red[w] > best ? s_red[w] : best;
+      best = max_of_warp_maxima(s_red, kExpandWarps, lane);
       __syncthreads();
       if (mine == best) {                // keys are unique: exactly one thread
         s_tok[j] = static_cast<int>(~static_cast<unsigned int>(best & 0xffffffffull));
-        mine = local_best(best);
+        if (second_known) {
+          mine = second;                 // (0 when the thread has no other token: it never wins again)
+          second_known = false;
+        } else {
+          rescan(best);
+          second_known = true;
+        }
       }
     }
   } else if (k > 0) {
@@ -112,6 +115,7 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandParams p, 
       lp = x > lp ? x : lp;
     }
     if (lane == 0) s_red[warp] = lp;
+    if (tid < k) s_un[tid] = __ldg(p.uniforms + node * K + tid);   // all draws' uniforms at once, not one load per draw
     __syncthreads();
     // prefix sums that tile [0, total) without gaps: a thread's upper bound is computed exactly as its successor's
     // lower bound (same operands, same order)
@@ -120,14 +124,13 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandParams p, 
     for (int w = 0; w < kExpandWarps; ++w) {
       if (w == warp) warp_off = total;
       total += s_sum[w];
-      lp = s_red[w] > lp ? s_red[w] : lp;
     }
+    lp = max_of_warp_maxima(s_red, kExpandWarps, lane);
     const double before = lane ? warp_off + up : warp_off;
     const double upto = lane == 31 ? warp_off + s_sum[warp] : warp_off + inc;
     const int fallback = lp > 0 ? static_cast<int>(lp) - 1 : V - 1;
-    const float* un = p.uniforms + node * K;
     for (int j = 0; j < k; ++j) {
-      const double thr = static_cast<double>(__ldg(un + j)) * total;
+      const double thr = static_cast<double>(s_un[j]) * total;
       if (before <= thr && upto > thr) {
         // this thread's range holds the threshold: repeat its additions
         double c = 0.0;
@@ -153,23 +156,103 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandParams p, 
   }
 }
 
+// k of a node after the checks (0 and a status word when it is unusable)
+__device__ __forceinline__ int checked_children(const ExpandParams& p, size_t node, bool greedy) {
+  int k = p.num_children[node];
+  const bool bad = k < 0 || k > p.K || (greedy && k > p.V) || (!greedy && k > 0 && !p.uniforms);
+  if (bad) {
+    if (threadIdx.x == 0) report_status(p.status, EAGLE_ERR_SHAPE);
+    k = 0;
+  }
+  return k;
+}
+
+// Rows read straight from global memory (they do not fit shared memory): one CTA per row.
+template <int kExpandThreads>
+__global__ void __launch_bounds__(kExpandThreads) expand_kernel_global(ExpandParams p) {
+  __shared__ unsigned long long s_red[kExpandThreads / 32];
+  __shared__ double s_sum[kExpandThreads / 32];
+  __shared__ int s_tok[kMaxChildren];
+  __shared__ float s_un[kMaxChildren];
+  const size_t node = static_cast<size_t>(blockIdx.y) * p.R + blockIdx.x;
+  const bool greedy = p.greedy && p.greedy[blockIdx.y] != 0;
+  const int k = checked_children(p, node, greedy);
+  expand_row<kExpandThreads>(p, node, p.probs + node * p.V, k, greedy, s_red, s_sum, s_tok, s_un);
+}
+
+// Rows staged in shared memory.  A fixed grid (one CTA per SM) walks the rows; while a row is worked on out of shared
+// memory, the next row of this CTA is already on its way from HBM into registers (kVecs 16-byte vectors per thread),
+// and is written to shared memory when the current row is finished: loading and selecting overlap.
+template <int kExpandThreads, int kVecs>
+__global__ void __launch_bounds__(kExpandThreads) expand_kernel_staged(ExpandParams p, int vectors) {
+  extern __shared__ __align__(16) float s_row[];
+  __shared__ unsigned long long s_red[kExpandThreads / 32];
+  __shared__ double s_sum[kExpandThreads / 32];
+  __shared__ int s_tok[kMaxChildren];
+  __shared__ float s_un[kMaxChildren];
+  const int tid = threadIdx.x, V = p.V;
+  const size_t n_rows = static_cast<size_t>(p.B) * p.R;
+  const int nvec = V / 4;   // used when `vectors` (V % 4 == 0 and the tensor is 16-byte aligned: every row is aligned)
+  float4 held[kVecs];
+  auto fetch = [&](size_t node) {
+    const float4* src = reinterpret_cast<const float4*>(p.probs + node * V);
+#pragma unroll
+    for (int j = 0; j < kVecs; ++j) {
+      const int i = tid + j * kExpandThreads;
+      if (i < nvec) held[j] = __ldg(src + i);
+    }
+  };
+  auto stash = [&]() {
+    float4* dst = reinterpret_cast<float4*>(s_row);
+#pragma unroll
+    for (int j = 0; j < kVecs; ++j) {
+      const int i = tid + j * kExpandThreads;
+      if (i < nvec) dst[i] = held[j];
+    }
+  };
+  size_t node = blockIdx.x;
+  if (node >= n_rows) return;
+  if (vectors) fetch(node);
+  while (node < n_rows) {
+    if (vectors) {
+      stash();
+    } else {
+      const float* row = p.probs + node * V;
+      for (int v = tid; v < V; v += kExpandThreads) s_row[v] = row[v];
+    }
+    const size_t next = node + gridDim.x;
+    if (vectors && next < n_rows) fetch(next);      // in flight while this row is worked on
+    const int b = static_cast<int>(node / p.R);
+    const bool greedy = p.greedy && p.greedy[b] != 0;
+    const int k = checked_children(p, node, greedy);
+    expand_row<kExpandThreads>(p, node, s_row, k, greedy, s_red, s_sum, s_tok, s_un);   // starts with a block barrier
+    __syncthreads();                                 // everyone is done with s_row
+    node = next;
+  }
+}
+
 }  // namespace
 
-cudaError_t launch_expand(const ExpandParams& p, cudaStream_t stream) {
+cudaError_t launch_expand(const ExpandParams& p, int sm_count, cudaStream_t stream) {
   if (p.B == 0 || p.R == 0 || p.K == 0) return cudaSuccess;
-  const dim3 grid(static_cast<unsigned>(p.R), static_cast<unsigned>(p.B));
   // a row is staged in shared memory when it fits one SM's shared memory with room to spare (V <= 51200)
   const size_t row_bytes = static_cast<size_t>(p.V) * sizeof(float);
-  const int stage = row_bytes <= 200 * 1024 ? 1 : 0;
-  const size_t smem = stage ? ((row_bytes + 15) & ~size_t(15)) : 0;
-  if (stage) {
+  if (row_bytes <= 200 * 1024) {
+    const size_t smem = (row_bytes + 15) & ~size_t(15);
+    const long long rows = static_cast<long long>(p.B) * p.R;
+    const unsigned blocks = static_cast<unsigned>(rows < sm_count ? rows : (sm_count > 0 ? sm_count : 1));
+    const int vectors = (p.V & 3) == 0 && (reinterpret_cast<uintptr_t>(p.probs) & 15) == 0;
+    // up to 8 vectors per thread (V <= 32768) stay in 32 registers; longer rows take 13
+    const bool short_row = p.V <= 8 * 4 * kExpandThreadsStaged;
+    auto kernel = short_row ? expand_kernel_staged<kExpandThreadsStaged, 8> : expand_kernel_staged<kExpandThreadsStaged, 13>;
     if (smem > 48 * 1024) {
-      const cudaError_t e = cudaFuncSetAttribute(expand_kernel<kExpandThreadsStaged>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
       if (e != cudaSuccess) return e;
     }
-    expand_kernel<kExpandThreadsStaged><<<grid, kExpandThreadsStaged, smem, stream>>>(p, 1);
+    kernel<<<blocks, kExpandThreadsStaged, smem, stream>>>(p, vectors);
   } else {
-    expand_kernel<kExpandThreadsGlobal><<<grid, kExpandThreadsGlobal, 0, stream>>>(p, 0);
+    const dim3 grid(static_cast<unsigned>(p.R), static_cast<unsigned>(p.B));
+    expand_kernel_global<kExpandThreadsGlobal><<<grid, kExpandThreadsGlobal, 0, stream>>>(p);
   }
   count_launch();
   return cudaGetLastError();
