@@ -24,14 +24,18 @@ __device__ __forceinline__ unsigned int sortable_bits(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Largest key among the 32 per-warp maxima in s_red, by every warp on its own (one load per lane, five shuffles).
+// Largest 64-bit key over a warp: the hardware warp reduction works on 32-bit words, so the high words go first and
+// the low words of the lanes that hold the largest high word second.
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+  const unsigned int hi = static_cast<unsigned int>(v >> 32), lo = static_cast<unsigned int>(v);
+  const unsigned int hi_max = __reduce_max_sync(0xffffffffu, hi);
+  const unsigned int lo_max = __reduce_max_sync(0xffffffffu, hi == hi_max ? lo : 0u);
+  return (static_cast<unsigned long long>(hi_max) << 32) | lo_max;
+}
+
+// Largest key among the per-warp maxima in s_red, by every warp on its own.
 __device__ __forceinline__ unsigned long long max_of_warp_maxima(const unsigned long long* s_red, int n_warps, int lane) {
-  unsigned long long best = lane < n_warps ? s_red[lane] : 0ull;
-  for (int o = 16; o > 0; o >>= 1) {
-    const unsigned long long x = __shfl_xor_sync(0xffffffffu, best, o);
-    best = x > best ? x : best;
-  }
-  return best;
+  return warp_max_u64(lane < n_warps ? s_red[lane] : 0ull);
 }
 
 // One row: `row` points at its V probabilities (shared memory when staged, else global).  Called by the whole CTA.
@@ -52,30 +56,38 @@ __device__ __forceinline__ void expand_row(const ExpandParams& p, size_t node, c
     // that wins twice in a row has to look through its tokens again (a one-thread chain of ~30 shared-memory reads,
     // which used to follow every round).
     unsigned long long mine = 0ull, second = 0ull;   // keys are never 0: the id part of a real token is at least 1
+    auto make_key = [](unsigned int bits, int v) {
+      return (static_cast<unsigned long long>(bits) << 32) | static_cast<unsigned int>(~static_cast<unsigned int>(v));
+    };
+    // the two largest keys below `below` among this thread's tokens.  Tokens are visited in ascending id, so among equal
+    // values the first one met is the larger key and strict 32-bit compares on the value bits keep the order right.
     auto rescan = [&](unsigned long long below) {
-      mine = 0ull;
-      second = 0ull;
+      const unsigned int below_bits = static_cast<unsigned int>(below >> 32);
+      const int below_v = static_cast<int>(~static_cast<unsigned int>(below & 0xffffffffull));
+      const bool all = below == ~0ull;
+      unsigned int b1 = 0u, b2 = 0u;    // value bits of the best and the second best (valid when v1 / v2 >= 0)
+      int v1 = -1, v2 = -1;
+#pragma unroll 4
       for (int v = tid; v < V; v += kExpandThreads) {
-        const unsigned long long key = (static_cast<unsigned long long>(sortable_bits(row[v])) << 32) |
-                                       static_cast<unsigned int>(~static_cast<unsigned int>(v));
-        if (key < below) {
-          if (key > mine) {
-            second = mine;
-            mine = key;
-          } else if (key > second) {
-            second = key;
-          }
+        const unsigned int u = sortable_bits(row[v]);
+        const bool ok = all || u < below_bits || (u == below_bits && v > below_v);
+        if (ok && (v1 < 0 || u > b1)) {
+          b2 = b1;
+          v2 = v1;
+          b1 = u;
+          v1 = v;
+        } else if (ok && (v2 < 0 || u > b2)) {
+          b2 = u;
+          v2 = v;
         }
       }
+      mine = v1 >= 0 ? make_key(b1, v1) : 0ull;
+      second = v2 >= 0 ? make_key(b2, v2) : 0ull;
     };
     bool second_known = true;
     if (k > 0) rescan(~0ull);   // every key is below ~0
     for (int j = 0; j < k; ++j) {
-      unsigned long long best = mine;
-      for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long x = __shfl_xor_sync(0xffffffffu, best, o);
-        best = x > best ? x : best;
-      }
+      unsigned long long best = warp_max_u64(mine);
       if (lane == 0) s_red[warp] = best;
       __syncthreads();
       best = max_of_warp_maxima(s_red, kExpandWarps, lane);
@@ -109,25 +121,26 @@ __device__ __forceinline__ void expand_row(const ExpandParams& p, size_t node, c
     }
     if (lane == 31) s_sum[warp] = inc;
     // the last token with positive mass, for draws that rounding pushes past the end
-    unsigned long long lp = static_cast<unsigned long long>(static_cast<unsigned int>(last_pos + 1));
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long x = __shfl_xor_sync(0xffffffffu, lp, o);
-      lp = x > lp ? x : lp;
-    }
+    unsigned long long lp = __reduce_max_sync(0xffffffffu, static_cast<unsigned int>(last_pos + 1));
     if (lane == 0) s_red[warp] = lp;
     if (tid < k) s_un[tid] = __ldg(p.uniforms + node * K + tid);   // all draws' uniforms at once, not one load per draw
     __syncthreads();
     // prefix sums that tile [0, total) without gaps: a thread's upper bound is computed exactly as its successor's
     // lower bound (same operands, same order)
     const double up = __shfl_up_sync(0xffffffffu, inc, 1);
-    double warp_off = 0.0, total = 0.0;
-    for (int w = 0; w < kExpandWarps; ++w) {
-      if (w == warp) warp_off = total;
-      total += s_sum[w];
+    // inclusive scan of the warps' masses, by every warp on its own; warp w starts where warp w - 1 ends (the same value)
+    double wincl = lane < kExpandWarps ? s_sum[lane] : 0.0;
+    for (int o = 1; o < 32; o <<= 1) {
+      const double x = __shfl_up_sync(0xffffffffu, wincl, o);
+      if (lane >= o) wincl += x;
     }
+    const double total = __shfl_sync(0xffffffffu, wincl, kExpandWarps - 1);
+    const double warp_end = __shfl_sync(0xffffffffu, wincl, warp);
+    const double warp_prev = __shfl_sync(0xffffffffu, wincl, warp > 0 ? warp - 1 : 0);
+    const double warp_off = warp > 0 ? warp_prev : 0.0;
     lp = max_of_warp_maxima(s_red, kExpandWarps, lane);
     const double before = lane ? warp_off + up : warp_off;
-    const double upto = lane == 31 ? warp_off + s_sum[warp] : warp_off + inc;
+    const double upto = lane == 31 ? warp_end : warp_off + inc;
     const int fallback = lp > 0 ? static_cast<int>(lp) - 1 : V - 1;
     for (int j = 0; j < k; ++j) {
       const double thr = static_cast<double>(s_un[j]) * total;
@@ -135,12 +148,10 @@ __device__ __forceinline__ void expand_row(const ExpandParams& p, size_t node, c
         // this thread's range holds the threshold: repeat its additions
         double c = 0.0;
         int x = v1 - 1;
+#pragma unroll 4
         for (int v = v0; v < v1; ++v) {
           c += static_cast<double>(row[v]);
-          if (before + c > thr) {
-            x = v;
-            break;
-          }
+          if (before + c > thr) x = min(x, v);      // no early exit: the loads of the whole range stay in flight together
         }
         s_tok[j] = x;
       }
