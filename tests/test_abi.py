@@ -107,3 +107,41 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", tmp_path / "nope.so")
     with pytest.raises(binding.EagleError):
         binding.load()
+
+
+def test_host_step_byte_count(lib):
+    """eagle_tree_verify_step_host_bytes: whole tensors when trimming would not pay, else only the visible cache slots and the
+    rows of existing nodes (counted here from the same host arrays)."""
+    import numpy as np
+    from paper_2401_15077_b200 import binding
+    B, Hq, Hkv, D, T, S, V = 6, 8, 2, 64, 16, 4000, 2048
+    fake = 4096
+
+    def make(lens, sizes):
+        s = binding.HostStep()
+        s.batch, s.num_q_heads, s.num_kv_heads, s.head_dim, s.max_tree = B, Hq, Hkv, D, T
+        s.kv_capacity, s.vocab, s.path_cap, s.sm_scale = S, V, T, 0.0
+        for name in ("q", "k_cache", "v_cache", "tree_parent", "target_probs", "draft_probs", "draft_tokens", "uniforms", "greedy"):
+            setattr(s, name, fake)
+        s.seq_lens, s.tree_sizes = lens.ctypes.data, sizes.ctypes.data
+        h2d, d2h = ctypes.c_size_t(0), ctypes.c_size_t(0)
+        assert lib.eagle_tree_verify_step_host_bytes(ctypes.byref(s), ctypes.byref(h2d), ctypes.byref(d2h)) == 0
+        return h2d.value, d2h.value
+
+    small = B * T * Hq * D * 2 + 2 * B * 4 + 2 * B * T * 4 + B * (T + 1) * 4 + B
+    full = small + 2 * B * Hkv * S * D * 2 + B * (T + 1) * V * 4 + B * T * V * 4
+    d2h_want = B * T * Hq * D * 2 + B * T * 4 + 2 * B * 4 + 4
+    # every sequence fills the cache and the tree: nothing to save
+    lens, sizes = np.full(B, S - T, np.int32), np.full(B, T, np.int32)
+    assert make(lens, sizes) == (full, d2h_want)
+    # ragged: visible slots and existing rows only; an empty tree reads nothing of its cache; bad lengths are clamped
+    lens = np.array([100, 3000, 0, 2500, -5, 50], np.int32)
+    sizes = np.array([16, 3, 7, 0, 9, 99], np.int32)
+    want = small
+    for L, n in zip(lens, sizes):
+        n = min(max(int(n), 0), T)
+        vis = min(max(int(L) + n, 0), S) if n > 0 else 0
+        want += 2 * vis * Hkv * D * 2 + (n + 1) * V * 4 + n * V * 4
+    assert want < full
+    assert make(lens, sizes) == (want, d2h_want)
+    assert lib.eagle_tree_verify_step_host_bytes(None, None, None) == -1
