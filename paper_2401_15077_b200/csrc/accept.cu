@@ -329,6 +329,13 @@ __global__ void __launch_bounds__(NT == 32 ? 32 * kWarpTeamsPerCta : NT) accept_
         if (ts.par[i] != cur) continue;
         const float* qrow = draft_b + static_cast<size_t>(i) * V;
         const int t = ts.tok[i];
+        // If the candidate is rejected, this thread's part of its draft row (and, before the first rejection at this
+        // node, of the target row) is swept next: ask for it now, together with the two scalars of the test, so that
+        // the sweep does not start with a second trip to memory.
+        if (v0 < v1) {
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(qrow + v0));
+          if (res.m == 0) asm volatile("prefetch.global.L1 [%0];" ::"l"(prow + v0));
+        }
         const double r = static_cast<double>(uni_b[i]);
         float q_max = 0.f;
         double q_inv = 1.0;     // 1 / mass of the candidate's draft row
