@@ -4,6 +4,8 @@ Greedy sequences must agree exactly.  Stochastic sequences must agree exactly gi
 except where the oracle itself reports that a decision on its walk came within 1e-5 of its boundary;
 such sequences are counted, and the count is asserted to stay small.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -12,6 +14,8 @@ from scipy import stats
 from paper_2401_15077_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
+
+SALTS = int(os.environ.get("EAGLE_ACCEPT_SALTS", "3"))   # seeds per case (more for a longer soak)
 MARGIN = 1e-5
 
 
@@ -66,7 +70,7 @@ CASES = [
 @pytest.mark.parametrize("name,cfg,kw,mode", CASES, ids=[c[0] for c in CASES])
 def test_accept_matches_oracle(E, oracle, name, cfg, kw, mode):
     tolerated_total, seqs = 0, 0
-    for salt in range(3 if cfg.batch * cfg.vocab < 4_000_000 else 1):
+    for salt in range(SALTS if cfg.batch * cfg.vocab < 4_000_000 else max(1, SALTS // 3)):
         inp = W.make_accept_inputs(cfg, salt=salt, **kw)
         ref = oracle.tree_accept(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
                                  tree_sizes=inp.tree_sizes, greedy=inp.greedy)
@@ -94,9 +98,9 @@ LOGIT_CASES = [
 def test_accept_on_logits_matches_oracle(E, oracle, name, cfg, kw, temperature):
     """eagle_tree_accept_logits against the oracle's fp64 softmax walk.  The kernel's exponentials are fp32, so a
     decision may differ where the oracle's margin is below 1e-5; such sequences are counted."""
-    tolerated_total, seqs = 0, 0
+    tolerated_total, seqs, accepted = 0, 0, 0
     d = torch.device("cuda:0")
-    for salt in range(3 if cfg.batch * cfg.vocab < 4_000_000 else 1):
+    for salt in range(SALTS if cfg.batch * cfg.vocab < 4_000_000 else max(1, SALTS // 3)):
         inp = W.make_accept_inputs(cfg, salt=salt, logits=True, **kw)
         ref = oracle.tree_accept_logits(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
                                         temperature, tree_sizes=inp.tree_sizes, greedy=inp.greedy)
@@ -110,7 +114,8 @@ def test_accept_on_logits_matches_oracle(E, oracle, name, cfg, kw, temperature):
         assert int(status.item()) == 0
         tolerated_total += _compare(inp, ref, path.cpu().numpy(), bonus.cpu().numpy(), alen.cpu().numpy())
         seqs += cfg.batch
-        assert ref["accept_len"].max() >= 1
+        accepted += int(ref["accept_len"].sum())
+    assert accepted >= 1        # the walks went somewhere (a single short sequence may accept nothing under one seed)
     assert tolerated_total <= max(1, seqs // 50), tolerated_total
 
 
