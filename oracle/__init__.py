@@ -19,6 +19,7 @@ _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "eagle_oracle.c"
 _LIB = _HERE / "liboracle.so"
 _lib = None
+DEC_ACCEPT, DEC_REJECT, DEC_BONUS, DEC_ARGMAX = 0, 1, 2, 3   # kinds of decision in the acceptance walk's trace
 
 
 def build(force: bool = False) -> Path:
@@ -44,9 +45,9 @@ def _load():
         lib.oracle_tree_verify_attn.restype = i32
         lib.oracle_tree_verify_attn_paged.argtypes = [i32] * 8 + [vp, dbl] + [vp] * 7
         lib.oracle_tree_verify_attn_paged.restype = i32
-        lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 13
+        lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 17
         lib.oracle_tree_accept.restype = i32
-        lib.oracle_tree_accept_logits.argtypes = [i32, i32, i32, i32] + [vp] * 7 + [dbl] + [vp] * 6
+        lib.oracle_tree_accept_logits.argtypes = [i32, i32, i32, i32] + [vp] * 7 + [dbl] + [vp] * 10
         lib.oracle_tree_accept_logits.restype = i32
         lib.oracle_tree_expand.argtypes = [i32, i32, i32, i32] + [vp] * 7
         lib.oracle_tree_expand.restype = i32
@@ -141,7 +142,8 @@ def tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, 
                 path_cap: int | None = None, temperature: float | None = None):
     """Acceptance walk (Algorithm 1 at every node, or the greedy rule).  Returns a dict of numpy arrays:
     accepted_path [B, path_cap], bonus_token [B], accept_len [B], min_margin [B], n_sweeps [B],
-    n_zero_mass [B]."""
+    n_zero_mass [B], and the walk's decisions in order: n_dec [B], dec_kind / dec_node / dec_margin [B, T+1]
+    (kinds: DEC_ACCEPT, DEC_REJECT, DEC_BONUS, DEC_ARGMAX)."""
     tp = _as(target_probs, np.float32)
     B, T1, V = tp.shape
     T = T1 - 1
@@ -157,17 +159,20 @@ def tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, uniforms, 
     cap = T if path_cap is None else path_cap
     res = dict(accepted_path=np.full((B, cap), -1, np.int32), bonus_token=np.full((B,), -1, np.int32),
                accept_len=np.zeros((B,), np.int32), min_margin=np.zeros((B,), np.float64),
-               n_sweeps=np.zeros((B,), np.int32), n_zero_mass=np.zeros((B,), np.int32))
+               n_sweeps=np.zeros((B,), np.int32), n_zero_mass=np.zeros((B,), np.int32),
+               n_dec=np.zeros((B,), np.int32), dec_kind=np.full((B, T + 1), -1, np.int32),
+               dec_node=np.full((B, T + 1), -2, np.int32), dec_margin=np.full((B, T + 1), np.nan, np.float64))
+    trace = (_ptr(res["n_dec"]), _ptr(res["dec_kind"]), _ptr(res["dec_node"]), _ptr(res["dec_margin"]))
     if temperature is None:
         rc = _load().oracle_tree_accept(B, T, V, cap, _ptr(ts), _ptr(gr), _ptr(tp), _ptr(dp), _ptr(tok), _ptr(par),
                                         _ptr(un), _ptr(res["accepted_path"]), _ptr(res["bonus_token"]),
                                         _ptr(res["accept_len"]), _ptr(res["min_margin"]), _ptr(res["n_sweeps"]),
-                                        _ptr(res["n_zero_mass"]))
+                                        _ptr(res["n_zero_mass"]), *trace)
     else:
         rc = _load().oracle_tree_accept_logits(B, T, V, cap, _ptr(ts), _ptr(gr), _ptr(tp), _ptr(dp), _ptr(tok), _ptr(par),
                                                _ptr(un), float(temperature), _ptr(res["accepted_path"]),
                                                _ptr(res["bonus_token"]), _ptr(res["accept_len"]), _ptr(res["min_margin"]),
-                                               _ptr(res["n_sweeps"]), _ptr(res["n_zero_mass"]))
+                                               _ptr(res["n_sweeps"]), _ptr(res["n_zero_mass"]), *trace)
     if rc != 0:
         raise ValueError(f"oracle_tree_accept failed: {rc}")
     return res

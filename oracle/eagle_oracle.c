@@ -44,6 +44,12 @@
 #define ORACLE_ERR_TREE (-2)
 #define ORACLE_ERR_NOMEM (-3)
 
+/* kinds of decision in the acceptance walk's trace */
+#define ORACLE_DEC_ACCEPT 0
+#define ORACLE_DEC_REJECT 1
+#define ORACLE_DEC_BONUS 2
+#define ORACLE_DEC_ARGMAX 3
+
 static double bf16_to_f64(uint16_t h) {
   uint32_t u = ((uint32_t)h) << 16;
   float f;
@@ -246,6 +252,14 @@ int oracle_tree_verify_attn_paged(int batch, int num_q_heads, int num_kv_heads, 
  *   n_sweeps     int32 [batch] or NULL: vocabulary-wide passes the walk needed (rejections + final draw,
  *                or one argmax per visited node)
  *   n_zero_mass  int32 [batch] or NULL: rejections whose residual had zero mass (distribution kept)
+ *   n_dec, dec_kind, dec_node, dec_margin (all or none; int32 [batch], int32 / int32 / fp64 [batch, max_tree + 1]):
+ *                the walk's decisions one by one, in the order they were taken, so that a differing result can be
+ *                traced to the first decision that differs.  kind ORACLE_DEC_ACCEPT / ORACLE_DEC_REJECT: the accept
+ *                test of candidate `node` and its outcome, margin |r - p(t)/p^(t)| (+inf when p^(t) = 0);
+ *                ORACLE_DEC_BONUS: the final draw at `node` (-1 = the context), margin = distance of u to the nearer
+ *                edge of the chosen cell of the normalised CDF; ORACLE_DEC_ARGMAX: the greedy argmax at `node`,
+ *                margin = gap between the two largest probabilities.  A walk takes at most max_tree + 1 decisions
+ *                (every node is tested at most once, then one draw; or one argmax per visited node).
  *
  * Walk (Sec. 3.3: Algorithm 1 applied at every node, starting from the root):
  *   cur = context.  p = target row of cur (used as given, each node starts from its own row).
@@ -281,10 +295,12 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
                        const uint8_t* greedy, const float* target_probs, const float* draft_probs,
                        const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
                        int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
-                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass, int logits, double temperature) {
+                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass, int32_t* n_dec, int32_t* dec_kind,
+                       int32_t* dec_node, double* dec_margin, int logits, double temperature) {
   if (batch < 0 || max_tree < 0 || max_tree > 64 || vocab <= 0 || path_cap < 0 || !target_probs ||
       !tree_parent || !draft_tokens || !accepted_path || !bonus_token)
     return ORACLE_ERR_ARG;
+  if (n_dec && (!dec_kind || !dec_node || !dec_margin)) return ORACLE_ERR_ARG;
   for (int b = 0; b < batch; ++b) {
     const int n = tree_size_of(tree_sizes, b, max_tree);
     if (n < 0 || n > max_tree) return ORACLE_ERR_ARG;
@@ -311,8 +327,9 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
       continue;
     }
     double* q = p + vocab;   /* the draft row of the candidate under test */
-    int cur = -1, len = 0, sweeps = 0, zero_mass = 0, bonus = -1;
+    int cur = -1, len = 0, sweeps = 0, zero_mass = 0, bonus = -1, decisions = 0;
     double margin = INFINITY;
+    const size_t dec0 = (size_t)b * (max_tree + 1);
     for (;;) {
       const float* prow = target_probs + ((size_t)b * (max_tree + 1) + (size_t)(cur + 1)) * vocab;
       load_row(p, prow, vocab, logits, temperature);
@@ -325,6 +342,12 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
         for (int v = 0; v < vocab; ++v)
           if (v != a && p[v] > second) second = p[v];
         if (vocab > 1 && p[a] - second < margin) margin = p[a] - second;
+        if (n_dec) {
+          dec_kind[dec0 + decisions] = ORACLE_DEC_ARGMAX;
+          dec_node[dec0 + decisions] = cur;
+          dec_margin[dec0 + decisions] = vocab > 1 ? p[a] - second : INFINITY;
+          ++decisions;
+        }
         ++sweeps;
         for (int i = 0; i < n && next < 0; ++i)
           if (par[i] == cur && tok[i] == a) next = i;
@@ -337,9 +360,13 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
           const double r = (double)uniforms[(size_t)b * (max_tree + 1) + i];
           load_row(q, qrow, vocab, logits, temperature);
           const double pt = p[t], qt = q[t];
-          if (qt > 0.0) {
-            const double m = fabs(r - pt / qt);
-            if (m < margin) margin = m;
+          const double m_test = qt > 0.0 ? fabs(r - pt / qt) : INFINITY;
+          if (m_test < margin) margin = m_test;
+          if (n_dec) {
+            dec_kind[dec0 + decisions] = r * qt < pt ? ORACLE_DEC_ACCEPT : ORACLE_DEC_REJECT;
+            dec_node[dec0 + decisions] = i;
+            dec_margin[dec0 + decisions] = m_test;
+            ++decisions;
           }
           if (r * qt < pt) {
             next = i;
@@ -367,6 +394,7 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
           const double thr = u * total;
           double c = 0.0, c_prev = 0.0;
           int x = -1, last_pos = -1;
+          double m_draw = 0.0;   /* rounding left no cell above the threshold: the draw sits on the last edge */
           for (int v = 0; v < vocab; ++v) {
             if (p[v] > 0.0) last_pos = v;
             c_prev = c;
@@ -380,8 +408,14 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
             x = last_pos >= 0 ? last_pos : vocab - 1;
           } else if (total > 0.0) {
             const double lo = (thr - c_prev) / total, hi = (c - thr) / total;
-            const double m = lo < hi ? lo : hi;
-            if (m < margin) margin = m;
+            m_draw = lo < hi ? lo : hi;
+            if (m_draw < margin) margin = m_draw;
+          }
+          if (n_dec) {
+            dec_kind[dec0 + decisions] = ORACLE_DEC_BONUS;
+            dec_node[dec0 + decisions] = cur;
+            dec_margin[dec0 + decisions] = m_draw;
+            ++decisions;
           }
           ++sweeps;
           bonus = x;
@@ -397,6 +431,7 @@ static int accept_walk(int batch, int max_tree, int vocab, int path_cap, const i
     if (min_margin) min_margin[b] = margin;
     if (n_sweeps) n_sweeps[b] = sweeps;
     if (n_zero_mass) n_zero_mass[b] = zero_mass;
+    if (n_dec) n_dec[b] = decisions;
     free(p);
   }
   return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
@@ -406,9 +441,11 @@ int oracle_tree_accept(int batch, int max_tree, int vocab, int path_cap, const i
                        const uint8_t* greedy, const float* target_probs, const float* draft_probs,
                        const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
                        int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
-                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass) {
+                       double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass, int32_t* n_dec, int32_t* dec_kind,
+                       int32_t* dec_node, double* dec_margin) {
   return accept_walk(batch, max_tree, vocab, path_cap, tree_sizes, greedy, target_probs, draft_probs, draft_tokens,
-                     tree_parent, uniforms, accepted_path, bonus_token, accept_len, min_margin, n_sweeps, n_zero_mass, 0, 1.0);
+                     tree_parent, uniforms, accepted_path, bonus_token, accept_len, min_margin, n_sweeps, n_zero_mass, n_dec,
+                     dec_kind, dec_node, dec_margin, 0, 1.0);
 }
 
 /*
@@ -420,11 +457,12 @@ int oracle_tree_accept_logits(int batch, int max_tree, int vocab, int path_cap, 
                               const uint8_t* greedy, const float* target_logits, const float* draft_logits,
                               const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
                               double temperature, int32_t* accepted_path, int32_t* bonus_token, int32_t* accept_len,
-                              double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass) {
+                              double* min_margin, int32_t* n_sweeps, int32_t* n_zero_mass, int32_t* n_dec, int32_t* dec_kind,
+                              int32_t* dec_node, double* dec_margin) {
   if (!(temperature > 0.0)) return ORACLE_ERR_ARG;
   return accept_walk(batch, max_tree, vocab, path_cap, tree_sizes, greedy, target_logits, draft_logits, draft_tokens,
-                     tree_parent, uniforms, accepted_path, bonus_token, accept_len, min_margin, n_sweeps, n_zero_mass, 1,
-                     temperature);
+                     tree_parent, uniforms, accepted_path, bonus_token, accept_len, min_margin, n_sweeps, n_zero_mass, n_dec,
+                     dec_kind, dec_node, dec_margin, 1, temperature);
 }
 
 /*

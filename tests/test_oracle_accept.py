@@ -459,3 +459,102 @@ def test_worked_example_fixture(oracle):
     t, d, tk, par, un, sz = _single_node_batch(P4B, [Q4] * 3, toks, r, u, 4)
     res = oracle.tree_accept(t, d, tk, par, un, tree_sizes=sz)
     assert list(_first_token(res, tk)) == want
+
+
+# --------------------------------------------------------- the decision trace (what the parity tests classify mismatches with)
+
+def test_trace_of_worked_example(oracle):
+    """The decisions of the hand-derived example, one by one: kinds, nodes and margins follow from its thresholds
+    (1/3, 0, 8/15) and from the final distributions (one-hot on token 0 at the context; uniform at an accepted leaf)."""
+    toks = [1, 3, 2]
+    r = np.array([[0.3333, 0.9, 0.9], [0.3334, 0.0, 0.5333], [0.3334, 0.0, 0.5334]], np.float32)
+    u = np.array([0.9, 0.5, 0.0], np.float32)
+    t, d, tk, par, un, sz = _single_node_batch(P4B, [Q4] * 3, toks, r, u, 4)
+    res = oracle.tree_accept(t, d, tk, par, un, tree_sizes=sz)
+    A, R, B = oracle.DEC_ACCEPT, oracle.DEC_REJECT, oracle.DEC_BONUS
+    want = [
+        # accepted at once; node 0 is then a leaf whose row is uniform: u = 0.9 lies in cell [0.75, 1)
+        [(A, 0, abs(float(r[0, 0]) - 1 / 3)), (B, 0, 0.1)],
+        # first rejected; second has residual mass 0 (ratio 0, r = 0: on the boundary); third accepted; leaf: u = 0.5 on an edge
+        [(R, 0, abs(float(r[1, 0]) - 1 / 3)), (R, 1, 0.0), (A, 2, abs(float(r[1, 2]) - 8 / 15)), (B, 2, 0.0)],
+        # all three rejected: final draw at the context from a one-hot distribution, u = 0 on the lower edge
+        [(R, 0, abs(float(r[2, 0]) - 1 / 3)), (R, 1, 0.0), (R, 2, abs(float(r[2, 2]) - 8 / 15)), (B, -1, 0.0)],
+    ]
+    for b, decs in enumerate(want):
+        assert res["n_dec"][b] == len(decs)
+        for j, (kind, node, margin) in enumerate(decs):
+            assert (res["dec_kind"][b, j], res["dec_node"][b, j]) == (kind, node), (b, j)
+            assert abs(res["dec_margin"][b, j] - margin) < 1e-6, (b, j, res["dec_margin"][b, j], margin)
+        assert abs(res["min_margin"][b] - min(m for _, _, m in decs)) < 1e-6
+
+
+def _replay(oracle_mod, res, b, parent):
+    """Path and 'a final draw / argmax ended the walk' rebuilt from the decision list alone."""
+    path, cur = [], -1
+    for j in range(int(res["n_dec"][b])):
+        kind, node = int(res["dec_kind"][b, j]), int(res["dec_node"][b, j])
+        if kind in (oracle_mod.DEC_ACCEPT, oracle_mod.DEC_REJECT):
+            assert int(parent[node]) == cur            # a candidate is a child of the current node
+            if kind == oracle_mod.DEC_ACCEPT:
+                path.append(node)
+                cur = node
+        elif kind == oracle_mod.DEC_BONUS:
+            assert node == cur and j == int(res["n_dec"][b]) - 1
+        else:
+            assert node == cur
+            if j + 1 < int(res["n_dec"][b]):           # not the last argmax: it matched a child
+                nxt = int(res["dec_node"][b, j + 1])
+                assert int(parent[nxt]) == cur
+                path.append(nxt)
+                cur = nxt
+    return path
+
+
+def test_trace_replays_to_the_result_and_tolerance_helper_finds_first_difference(oracle):
+    from accept_trace import first_differing_decision, compare_with_oracle
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=40, tree=(3, 30), max_depth=6, vocab=50)
+    inp = W.make_accept_inputs(cfg, salt=5, rho=0.9, greedy="half")
+    res = oracle.tree_accept(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
+                             tree_sizes=inp.tree_sizes, greedy=inp.greedy)
+    par = inp.tree_parent.numpy()
+    T = cfg.max_tree
+    flipped = 0
+    for b in range(cfg.batch):
+        n = int(res["n_dec"][b])
+        assert 1 <= n <= T + 1
+        path = _replay(oracle, res, b, par[b])
+        assert path == [int(x) for x in res["accepted_path"][b] if x >= 0]
+        finite = res["dec_margin"][b, :n]
+        assert np.isclose(finite.min(), res["min_margin"][b]) or (np.isinf(finite.min()) and np.isinf(res["min_margin"][b]))
+        # identical outputs contradict no decision
+        assert first_differing_decision(res, b, res["accepted_path"][b], res["bonus_token"][b]) is None
+        if inp.greedy[b]:
+            continue
+        # pretend the other side took decision j the other way, for every accept test j: the helper must point at j
+        for j in range(n):
+            kind, node = int(res["dec_kind"][b, j]), int(res["dec_node"][b, j])
+            depth = sum(1 for i in range(j) if res["dec_kind"][b, i] == oracle.DEC_ACCEPT)
+            fake = res["accepted_path"][b].copy()
+            if kind == oracle.DEC_ACCEPT:
+                fake[depth:] = -1                                  # it rejected the candidate and every later one
+            elif kind == oracle.DEC_REJECT:
+                fake[depth:] = -1
+                fake[depth] = node                                 # it accepted the candidate and stopped there
+            else:
+                continue
+            assert first_differing_decision(res, b, fake, (int(res["bonus_token"][b]) + 1) % cfg.vocab) == j
+            flipped += 1
+        fake_bonus = (int(res["bonus_token"][b]) + 1) % cfg.vocab   # same path, another final draw: the last decision
+        assert first_differing_decision(res, b, res["accepted_path"][b], fake_bonus) == n - 1
+    assert flipped > 50
+    # the tolerance applies at the first differing decision only
+    b = next(b for b in range(cfg.batch) if not inp.greedy[b] and res["accept_len"][b] >= 1)
+    path, bonus, alen = res["accepted_path"].copy(), res["bonus_token"].copy(), res["accept_len"].copy()
+    path[b, :] = -1
+    alen[b] = 0
+    with pytest.raises(AssertionError):
+        compare_with_oracle(res, path, bonus, alen, inp.greedy)      # a wrong decision far from its boundary
+    d = first_differing_decision(res, b, path[b], bonus[b])
+    res2 = {k: v.copy() for k, v in res.items()}
+    res2["dec_margin"][b, d] = 1e-7
+    assert compare_with_oracle(res2, path, bonus, alen, inp.greedy) == 1
