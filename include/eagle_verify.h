@@ -77,7 +77,8 @@ typedef struct eagle_attn_desc {
 } eagle_attn_desc;
 
 /* Bytes of scratch one call with this descriptor needs (host function, no CUDA work).
- * Depends on batch, heads, head_dim and max_tree only.  Returns 0 if the shape is unsupported. */
+ * Depends on batch, heads, head_dim, max_tree and num_splits only.  Returns 0 if the shape is unsupported.
+ * With num_splits = 0 it is about 35 MB whatever the batch (plus some 100 bytes per (sequence, KV head, 256 query rows)). */
 size_t eagle_tree_verify_attn_workspace(const eagle_attn_desc* desc);
 
 /*
@@ -116,8 +117,9 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
  *   - No cudaMalloc, cudaFree or other allocating call is made, on any call.
  *   - Shapes whose tables and partials do not fit the array are refused with EAGLE_ERR_WORKSPACE and nothing is
  *     launched.  The need grows with batch * num_kv_heads * ceil(max_tree * G / 128), and steeply with a
- *     forced num_splits > 1; with num_splits = 0 the partials take about 2 * (number of SMs) * 128 * (D + 2) * 4
- *     bytes (19.7 MB on a 148-SM B200 at D = 128).
+ *     forced num_splits > 1; with num_splits = 0 the partials take (2 * (number of SMs) + 2 * batch if num_kv_heads is
+ *     odd) * 128 * (D + 2) * 4 bytes (19.7 MB on a 148-SM B200 at D = 128), which leaves room for the tables of some 30 000
+ *     (sequence, KV head, 256 query rows) units.
  *   - The first call on a device looks up the array's device address (once per device, with that device
  *     current).  Make that first call outside any stream capture.
  *   - All calls on one GPU share the one array, and it keeps the previous call's contents.  Nothing in it needs
@@ -156,6 +158,56 @@ typedef struct eagle_paged_kv {
  */
 int eagle_tree_verify_attn_paged(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* kv,
                                  const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream);
+
+/*
+ * The same call in two halves, for a verification pass over many layers.  The verification phase is one target
+ * forward pass over every layer with the same draft tree and the same prefix lengths (Sec. 3.3, App. A.1); the tree
+ * masks and the work split depend on nothing else, so they are made once per pass and reused by every layer:
+ *
+ *   eagle_tree_verify_plan          the planner alone: masks + work list into desc->workspace (one launch).
+ *                                   `paged` is NULL for a contiguous cache; for a paged cache it names the block table
+ *                                   (its page pointers are not read), so that the pages in use are validated.
+ *   eagle_tree_verify_attn_planned  attention + combine of one layer over the plan in desc->workspace (two launches).
+ *   eagle_tree_verify_attn_planned_paged   the same over a paged cache.
+ *
+ * The descriptor of the planned calls must equal the one the plan was made with (shape fields, num_splits, workspace),
+ * on the same GPU; sm_scale, status and the events may differ.  Plan followed by planned gives bit for bit what
+ * eagle_tree_verify_attn gives.  The plan stays valid until the workspace is written by another plan; the split
+ * partials in the workspace are reused by every planned call, so planned calls that share a workspace must not overlap
+ * on the GPU.  Arguments, results and errors as for eagle_tree_verify_attn (device-detected errors of the trees and
+ * lengths are reported by the plan call; the planned calls then write zeros for the affected sequences).
+ */
+int eagle_tree_verify_plan(const eagle_attn_desc* desc, const int32_t* seq_lens, const int32_t* tree_parent,
+                           const eagle_paged_kv* paged, eagle_stream_t stream);
+int eagle_tree_verify_attn_planned(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                                   void* out, eagle_stream_t stream);
+int eagle_tree_verify_attn_planned_paged(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* kv, void* out,
+                                         eagle_stream_t stream);
+
+/*
+ * Where a plan keeps its tree masks (host function, no CUDA work): device uint64 [B, T_max] inside desc->workspace,
+ * bit m of entry [b, i] set iff node m is node i or one of its ancestors (the mask tree attention implies, Sec. 3.1 /
+ * 3.3); entries of nodes >= tree size and of invalid sequences are 0.  Valid after eagle_tree_verify_plan or
+ * eagle_tree_verify_attn on that workspace has run.  NULL if the descriptor is unusable.
+ */
+const uint64_t* eagle_tree_verify_plan_masks(const eagle_attn_desc* desc);
+
+/*
+ * How long a wait inside the attention kernel may go without progress before the kernel gives up, in nanoseconds
+ * (host function; process-wide; applies to launches made after the call; 0 restores the default of two seconds).
+ * Every wait in the kernels is bounded: when one runs out the kernel sets *status to EAGLE_ERR_TIMEOUT, releases what
+ * it holds and returns, and the context stays usable.  Keep the limit far above the time a copy takes (milliseconds
+ * are safe): a kernel that gives up while its own copies are still in flight would leave them writing into shared
+ * memory it no longer owns.
+ */
+void eagle_set_wait_limit_ns(uint64_t ns);
+
+/*
+ * Test hook (fault injection for the time-out path; not for production use): attention launches made after this call
+ * have their K/V producer stop issuing copies after `after_tiles` tiles per CTA, so the consumers' waits run out and
+ * the kernel reports EAGLE_ERR_TIMEOUT.  Nothing is in flight when it returns.  A negative value switches it off.
+ */
+void eagle_test_stall_kv_producer(int32_t after_tiles);
 
 /*
  * Descriptor of one acceptance call.
@@ -201,6 +253,15 @@ typedef struct eagle_accept_desc {
 int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, const float* draft_probs,
                       const int32_t* draft_tokens, const int32_t* tree_parent, const float* uniforms,
                       int32_t* accepted_path, int32_t* bonus_token, eagle_stream_t stream);
+
+/*
+ * How an acceptance call of this batch size and vocabulary is laid out on the current GPU (host function, launches
+ * nothing): 0 when one warp walks each tree (vocabularies up to 4096), else the number of 512-thread CTAs, 1, 2, 4 or
+ * 8, that form the thread-block cluster walking one tree (the fewer trees, the wider the cluster).  The result of
+ * eagle_tree_accept does not depend on it; it is reported so that every variant can be told apart and exercised.
+ * Negative EAGLE_ERR_* on a bad argument or when no sm_100 device is current.
+ */
+int eagle_tree_accept_cluster_width(int32_t batch, int32_t vocab);
 
 /*
  * One whole verification step driven from HOST buffers (the two calls above, with the copies around them).

@@ -19,7 +19,9 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_verify_attn_static", "eagle_tree_verify_attn_static_capacity",
            "eagle_tree_verify_step_host", "eagle_tree_verify_step_host_arena", "eagle_tree_commit",
            "eagle_tree_accept_logits", "eagle_tree_expand", "eagle_tree_verify_attn_paged",
-           "eagle_tree_commit_paged", "eagle_tree_verify_step_host_bytes"]
+           "eagle_tree_commit_paged", "eagle_tree_verify_step_host_bytes", "eagle_tree_accept_cluster_width",
+           "eagle_tree_verify_plan", "eagle_tree_verify_attn_planned", "eagle_tree_verify_attn_planned_paged",
+           "eagle_tree_verify_plan_masks", "eagle_set_wait_limit_ns", "eagle_test_stall_kv_producer"]
 _lib = None
 
 
@@ -82,6 +84,18 @@ def load():
         lib.eagle_tree_verify_attn_static_capacity.restype = ctypes.c_size_t
         lib.eagle_tree_verify_attn_paged.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(PagedKV), vp, vp, vp, vp]
         lib.eagle_tree_verify_attn_paged.restype = ctypes.c_int
+        lib.eagle_tree_verify_plan.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, ctypes.POINTER(PagedKV), vp]
+        lib.eagle_tree_verify_plan.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_planned.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp]
+        lib.eagle_tree_verify_attn_planned.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_planned_paged.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(PagedKV), vp, vp]
+        lib.eagle_tree_verify_attn_planned_paged.restype = ctypes.c_int
+        lib.eagle_tree_verify_plan_masks.argtypes = [ctypes.POINTER(AttnDesc)]
+        lib.eagle_tree_verify_plan_masks.restype = ctypes.c_void_p
+        lib.eagle_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
+        lib.eagle_set_wait_limit_ns.restype = None
+        lib.eagle_test_stall_kv_producer.argtypes = [i32]
+        lib.eagle_test_stall_kv_producer.restype = None
         lib.eagle_tree_verify_step_host.argtypes = [ctypes.POINTER(HostStep), vp]
         lib.eagle_tree_verify_step_host.restype = ctypes.c_int
         lib.eagle_tree_verify_step_host_arena.argtypes = [ctypes.POINTER(HostStep)]
@@ -91,6 +105,8 @@ def load():
         lib.eagle_tree_verify_step_host_bytes.restype = ctypes.c_int
         lib.eagle_tree_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, vp, vp, vp]
         lib.eagle_tree_accept.restype = ctypes.c_int
+        lib.eagle_tree_accept_cluster_width.argtypes = [i32, i32]
+        lib.eagle_tree_accept_cluster_width.restype = ctypes.c_int
         lib.eagle_tree_accept_logits.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
         lib.eagle_tree_accept_logits.restype = ctypes.c_int
         lib.eagle_tree_expand.argtypes = [ctypes.POINTER(ExpandDesc), vp, vp, vp, vp, vp, vp]
@@ -222,6 +238,88 @@ def eagle_tree_verify_attn_paged(q, k_pages, v_pages, block_table, seq_lens, tre
     return out
 
 
+class VerifyPlan:
+    """The plan of one verification pass (tree masks + work split), made once by ``eagle_tree_verify_plan`` and used by
+    every layer's ``attend`` / ``attend_paged``.  Holds the descriptor fields and the workspace; marshalling only."""
+
+    def __init__(self, shape, num_kv_heads, kv_capacity, tree_sizes, num_splits, workspace, shared_tree, paged):
+        self.shape, self.num_kv_heads, self.kv_capacity = tuple(shape), int(num_kv_heads), int(kv_capacity)
+        self.tree_sizes, self.num_splits, self.workspace = tree_sizes, int(num_splits), workspace
+        self.shared_tree, self.paged = bool(shared_tree), paged
+
+    def _desc(self, q_like_shape, sm_scale, status, events):
+        B, T, Hq, D = q_like_shape
+        d = AttnDesc(B, Hq, self.num_kv_heads, D, T, self.kv_capacity, _dev(self.tree_sizes, torch.int32, "tree_sizes", True),
+                     float(sm_scale), self.num_splits, self.workspace.data_ptr(), self.workspace.numel(),
+                     _dev(status, torch.int32, "status", True), None, None, 1 if self.shared_tree else 0)
+        if events is not None:
+            d.ev_attn_begin, d.ev_attn_end = events[0].cuda_event, events[1].cuda_event
+        return d
+
+    def masks(self):
+        """Device address of the plan's ancestor masks (uint64 [B, T_max]) as an int64 tensor copy."""
+        B, T = self.shape[0], self.shape[1]
+        d = self._desc(self.shape, 0.0, None, None)
+        ptr = load().eagle_tree_verify_plan_masks(ctypes.byref(d))
+        if not ptr:
+            raise EagleError("eagle_tree_verify_plan_masks failed")
+        off = ptr - self.workspace.data_ptr()
+        return self.workspace[off:off + B * T * 8].view(torch.int64).view(B, T).clone()
+
+    def attend(self, q, k_cache, v_cache, out=None, *, sm_scale=0.0, status=None, events=None):
+        if tuple(q.shape) != self.shape or k_cache.shape != v_cache.shape or k_cache.shape[2] != self.kv_capacity:
+            raise EagleError("tensors do not match the plan")
+        if out is None:
+            out = torch.empty_like(q)
+        d = self._desc(q.shape, sm_scale, status, events)
+        rc = load().eagle_tree_verify_attn_planned(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
+                                                   _dev(v_cache, torch.bfloat16, "v_cache"), _dev(out, torch.bfloat16, "out"), _stream())
+        _check(rc, "eagle_tree_verify_attn_planned")
+        return out
+
+    def attend_paged(self, q, k_pages, v_pages, block_table, out=None, *, sm_scale=0.0, status=None, events=None):
+        if tuple(q.shape) != self.shape:
+            raise EagleError("tensors do not match the plan")
+        if out is None:
+            out = torch.empty_like(q)
+        d = self._desc(q.shape, sm_scale, status, events)
+        pk = PagedKV(_dev(k_pages, torch.bfloat16, "k_pages"), _dev(v_pages, torch.bfloat16, "v_pages"),
+                     _dev(block_table, torch.int32, "block_table"), k_pages.shape[0], k_pages.shape[2], block_table.shape[1])
+        rc = load().eagle_tree_verify_attn_planned_paged(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), ctypes.byref(pk),
+                                                         _dev(out, torch.bfloat16, "out"), _stream())
+        _check(rc, "eagle_tree_verify_attn_planned_paged")
+        return out
+
+
+def eagle_tree_verify_plan(shape, num_kv_heads, kv_capacity, seq_lens, tree_parent, *, tree_sizes=None, num_splits=0,
+                           workspace=None, status=None, shared_tree=False, paged=None) -> VerifyPlan:
+    """Plans one verification pass: ``shape`` = (B, T_max, Hq, D) of q / out.  ``paged`` = (block_table, num_pages,
+    page_size) for a paged cache (``kv_capacity`` is then ignored).  Returns the plan that ``attend`` takes."""
+    B, T, Hq, D = shape
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
+    if workspace is None:
+        n = eagle_tree_verify_attn_workspace(B, Hq, num_kv_heads, D, T, num_splits)
+        workspace = torch.empty(n, dtype=torch.uint8, device=seq_lens.device)
+    plan = VerifyPlan(shape, num_kv_heads, 0 if paged else kv_capacity, tree_sizes, num_splits, workspace, shared_tree, paged)
+    d = plan._desc(shape, 0.0, status, None)
+    pk = None
+    if paged is not None:
+        table, num_pages, page_size = paged
+        pk = ctypes.byref(PagedKV(None, None, _dev(table, torch.int32, "block_table"), int(num_pages), int(page_size), table.shape[1]))
+    rc = load().eagle_tree_verify_plan(ctypes.byref(d), _dev(seq_lens, torch.int32, "seq_lens"), _dev(tree_parent, torch.int32, "tree_parent"),
+                                       pk, _stream())
+    _check(rc, "eagle_tree_verify_plan")
+    return plan
+
+
+def set_wait_limit_ns(ns: int):
+    load().eagle_set_wait_limit_ns(int(ns))
+
+
+def test_stall_kv_producer(after_tiles: int):
+    load().eagle_test_stall_kv_producer(int(after_tiles))
+
+
 def eagle_tree_verify_attn_static(q, k_cache, v_cache, seq_lens, tree_parent, out, *, tree_sizes=None, sm_scale=0.0,
                                   num_splits=0, status=None, shared_tree=False):
     """Tree-masked attention for callers that may not allocate: same arguments and results as
@@ -278,6 +376,14 @@ def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, unif
     else:
         _check(lib.eagle_tree_accept_logits(*head, float(temperature), *tail), "eagle_tree_accept_logits")
     return accepted_path, bonus_token
+
+
+def eagle_tree_accept_cluster_width(batch: int, vocab: int) -> int:
+    """0 when a warp walks each tree, else the CTAs per cluster (1, 2, 4, 8) an acceptance call of this size uses here."""
+    rc = load().eagle_tree_accept_cluster_width(int(batch), int(vocab))
+    if rc < 0:
+        _check(rc, "eagle_tree_accept_cluster_width")
+    return rc
 
 
 def eagle_tree_accept_logits(target_logits, draft_logits, draft_tokens, tree_parent, uniforms, temperature, accepted_path=None,

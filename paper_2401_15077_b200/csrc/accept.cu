@@ -482,30 +482,38 @@ cudaError_t launch_cluster(const AcceptParams& p, cudaStream_t stream) {
 
 }  // namespace
 
-// Team width: a warp per tree for small vocabularies; otherwise CTAs of 512 threads in clusters as wide as still
-// fit the GPU in one wave (four such CTAs are resident per SM): the walk is a chain of dependent vocabulary
-// sweeps, so a tree finishes sooner the more SMs pull its rows.
+// Team width: a warp per tree for small vocabularies (returned as 0); otherwise CTAs of 512 threads in clusters as
+// wide as still fit the GPU with at most four CTAs per SM: the walk is a chain of dependent vocabulary sweeps, so a
+// tree finishes sooner the more SMs pull its rows.  (With 64 registers per thread only two CTAs of 512 threads are
+// resident per SM, so at batch 64 the clusters of eight run in two waves; measured, that is still faster than clusters
+// of four in one wave: 52 against 57 us on the 64-sequence mix.)
+int accept_cluster_width(int batch, int vocab, int sm_count) {
+  if (vocab <= 4096) return 0;
+  const long long resident = 4ll * sm_count;
+  if (8ll * batch <= resident) return 8;
+  if (4ll * batch <= resident) return 4;
+  if (2ll * batch <= resident) return 2;
+  return 1;
+}
+
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream) {
   if (p.B == 0) return cudaSuccess;
   cudaError_t e;
-  if (p.V <= 4096) {
-    const unsigned blocks = static_cast<unsigned>((p.B + kWarpTeamsPerCta - 1) / kWarpTeamsPerCta);
-    if (p.logits) accept_kernel<32, 1, true><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
-    else accept_kernel<32, 1, false><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
-    e = cudaGetLastError();
-  } else {
-    // Team width: the widest cluster whose CTAs number at most four per SM.  (With 64 registers per thread only two
-    // CTAs of 512 threads are resident per SM, so at batch 64 the clusters of eight run in two waves; measured, that is
-    // still faster than clusters of four in one wave: 52 against 57 us on the 64-sequence mix.)
-    const long long resident = 4ll * sm_count;
-    if (8ll * p.B <= resident) e = launch_cluster<8>(p, stream);
-    else if (4ll * p.B <= resident) e = launch_cluster<4>(p, stream);
-    else if (2ll * p.B <= resident) e = launch_cluster<2>(p, stream);
-    else {
+  switch (accept_cluster_width(p.B, p.V, sm_count)) {
+    case 0: {
+      const unsigned blocks = static_cast<unsigned>((p.B + kWarpTeamsPerCta - 1) / kWarpTeamsPerCta);
+      if (p.logits) accept_kernel<32, 1, true><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
+      else accept_kernel<32, 1, false><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);
+      e = cudaGetLastError();
+      break;
+    }
+    case 8: e = launch_cluster<8>(p, stream); break;
+    case 4: e = launch_cluster<4>(p, stream); break;
+    case 2: e = launch_cluster<2>(p, stream); break;
+    default:
       if (p.logits) accept_kernel<kCtaThreads, 1, true><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
       else accept_kernel<kCtaThreads, 1, false><<<static_cast<unsigned>(p.B), kCtaThreads, 0, stream>>>(p);
       e = cudaGetLastError();
-    }
   }
   count_launch();
   return e;

@@ -24,6 +24,11 @@ constexpr int kPlanItemOverheadTiles = EAGLE_ITEM_OVERHEAD;
 constexpr int kPlanSnapTiles = EAGLE_SNAP_TILES;
 
 std::atomic<uint64_t> g_launches{0};
+// How long a wait inside the attention kernel may last before the kernel gives up (EAGLE_ERR_TIMEOUT), and the
+// fault-injection hook of the time-out test: the K/V producer issues no copy after this many tiles (negative: off).
+constexpr uint64_t kDefaultWaitLimitNs = 2000000000ull;
+std::atomic<uint64_t> g_wait_limit_ns{kDefaultWaitLimitNs};
+std::atomic<int32_t> g_stall_after_tiles{-1};
 
 struct DeviceInfo {
   bool ready = false;
@@ -87,30 +92,20 @@ struct KvSource {
   int32_t num_pages, page_size, max_pages;
 };
 
-// Checks shared by every attention entry point, then the three launches: planner, attention, combine.
-int attention_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, DeviceInfo* dev, const void* q, const KvSource& kv,
-                   const int32_t* seq_lens, const int32_t* tree_parent, void* out, cudaStream_t stream) {
-  if (!q || !kv.k || !kv.v || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
-  if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
-      (reinterpret_cast<uintptr_t>(out) & 15))
-    return EAGLE_ERR_SHAPE;
-  const int di = d.head_dim == 128 ? 1 : 0;
-  if (!dev->attn_prepared[di]) {
-    if (attn_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
-    dev->attn_prepared[di] = true;
-  }
-  const int G = d.num_q_heads / d.num_kv_heads;
-  const int32_t s_cap = static_cast<int32_t>(kv.capacity < 0x7fffffff ? kv.capacity : 0x7fffffff);
-
+// The planner launch: tree masks and work list into the workspace.  Depends on the lengths, the trees and the shape
+// only, so one plan serves every layer of a verification pass.
+int plan_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, const KvSource& kv, const int32_t* seq_lens,
+              const int32_t* tree_parent, cudaStream_t stream) {
+  if (!seq_lens || !tree_parent) return EAGLE_ERR_NULL;
   PlanParams pp;
   pp.seq_lens = seq_lens;
   pp.tree_sizes = d.tree_sizes;
   pp.tree_parent = tree_parent;
   pp.B = d.batch;
   pp.Hkv = d.num_kv_heads;
-  pp.G = G;
+  pp.G = d.num_q_heads / d.num_kv_heads;
   pp.T_max = d.max_tree;
-  pp.S_cap = s_cap;
+  pp.S_cap = static_cast<int32_t>(kv.capacity < 0x7fffffff ? kv.capacity : 0x7fffffff);
   pp.tile_keys = attn_tile_keys();
   pp.num_ctas = num_ctas;
   pp.forced_splits = d.num_splits;
@@ -135,7 +130,21 @@ int attention_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, D
   // Nothing in the workspace has to start at zero: the planner rebuilds every table it or the later kernels read, and
   // a partial slot is always written by the attention kernel before the combine kernel reads it.
   if (launch_plan(pp, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
+  return EAGLE_OK;
+}
 
+// The attention and combine launches over a plan that is already in the workspace.
+int attend_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, DeviceInfo* dev, const void* q, const KvSource& kv,
+                void* out, cudaStream_t stream) {
+  if (!q || !kv.k || !kv.v || !out) return EAGLE_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
+      (reinterpret_cast<uintptr_t>(out) & 15))
+    return EAGLE_ERR_SHAPE;
+  const int di = d.head_dim == 128 ? 1 : 0;
+  if (!dev->attn_prepared[di]) {
+    if (attn_prepare(d.head_dim) != cudaSuccess) return EAGLE_ERR_DEVICE;
+    dev->attn_prepared[di] = true;
+  }
   AttnParams ap;
   ap.q = static_cast<const __nv_bfloat16*>(q);
   ap.k = static_cast<const __nv_bfloat16*>(kv.k);
@@ -144,10 +153,10 @@ int attention_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, D
   ap.B = d.batch;
   ap.Hq = d.num_q_heads;
   ap.Hkv = d.num_kv_heads;
-  ap.G = G;
+  ap.G = d.num_q_heads / d.num_kv_heads;
   ap.D = d.head_dim;
   ap.T_max = d.max_tree;
-  ap.S_cap = s_cap;
+  ap.S_cap = static_cast<int32_t>(kv.capacity < 0x7fffffff ? kv.capacity : 0x7fffffff);
   const float scale = d.sm_scale != 0.f ? d.sm_scale : 1.0f / std::sqrt(static_cast<float>(d.head_dim));
   ap.scale_log2 = scale * 1.4426950408889634f;
   ap.q_tma = 0;
@@ -167,6 +176,8 @@ int attention_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, D
   while (kv.block_table && (1 << ap.page_shift) < kv.page_size) ++ap.page_shift;
   ap.max_pages = kv.max_pages;
   ap.num_pages = kv.num_pages;
+  ap.wait_limit_ns = g_wait_limit_ns.load(std::memory_order_relaxed);
+  ap.stall_after_tiles = g_stall_after_tiles.load(std::memory_order_relaxed);
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (launch_attn(ap, num_ctas, stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
   if (d.ev_attn_end && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_end), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
@@ -174,23 +185,44 @@ int attention_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, D
   return EAGLE_OK;
 }
 
+// Which of the two halves of an attention call an entry point runs.
+enum AttnPhase { kPlanOnly = 1, kAttendOnly = 2, kPlanAndAttend = 3 };
+
 // Entry with a caller-provided workspace, for either kind of cache.
-int attention_with_workspace(const eagle_attn_desc* desc, const void* q, const KvSource& kv, const int32_t* seq_lens,
+int attention_with_workspace(const eagle_attn_desc* desc, int phase, const void* q, const KvSource& kv, const int32_t* seq_lens,
                              const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
   const eagle_attn_desc& d = *desc;
   Workspace w;
   if (kv.capacity < 0 || !(d.sm_scale >= 0.f) || !carve_workspace(d, d.workspace, &w)) return EAGLE_ERR_SHAPE;
   if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
-  if (!q || !kv.k || !kv.v || !seq_lens || !tree_parent || !out) return EAGLE_ERR_NULL;
+  if ((phase & kPlanOnly) && (!seq_lens || !tree_parent)) return EAGLE_ERR_NULL;
+  if ((phase & kAttendOnly) && (!q || !kv.k || !kv.v || !out)) return EAGLE_ERR_NULL;
   if (!d.workspace || (reinterpret_cast<uintptr_t>(d.workspace) & 255) || d.workspace_bytes < w.bytes) return EAGLE_ERR_WORKSPACE;
-  if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
-      (reinterpret_cast<uintptr_t>(out) & 15))
+  if ((phase & kAttendOnly) &&
+      ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
+       (reinterpret_cast<uintptr_t>(out) & 15)))
     return EAGLE_ERR_SHAPE;
   int err = 0;
   DeviceInfo* dev = device_info(&err);
   if (!dev) return err;
   const int num_ctas = (dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas) & ~1;   // one persistent CTA per SM, in pairs
-  return attention_call(d, w, num_ctas, dev, q, kv, seq_lens, tree_parent, out, static_cast<cudaStream_t>(stream_));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (phase & kPlanOnly) {
+    const int rc = plan_call(d, w, num_ctas, kv, seq_lens, tree_parent, stream);
+    if (rc != EAGLE_OK) return rc;
+  }
+  if (phase & kAttendOnly) return attend_call(d, w, num_ctas, dev, q, kv, out, stream);
+  return EAGLE_OK;
+}
+
+bool paged_source(const eagle_attn_desc* desc, const eagle_paged_kv* pk, KvSource* kv, int* rc) {
+  if (!desc || !pk) { *rc = EAGLE_ERR_NULL; return false; }
+  if (pk->num_pages < 1 || pk->page_size < 16 || (pk->page_size & (pk->page_size - 1)) || pk->max_pages_per_seq < 0) { *rc = EAGLE_ERR_SHAPE; return false; }
+  if (static_cast<int64_t>(pk->num_pages) * desc->num_kv_heads > 0x7fffffffll) { *rc = EAGLE_ERR_SHAPE; return false; }
+  if (desc->batch > 0 && desc->max_tree > 0 && !pk->block_table) { *rc = EAGLE_ERR_NULL; return false; }
+  *kv = {pk->k_pages, pk->v_pages, static_cast<int64_t>(pk->max_pages_per_seq) * pk->page_size, pk->block_table,
+         pk->num_pages, pk->page_size, pk->max_pages_per_seq};
+  return true;
 }
 
 }  // namespace
@@ -199,19 +231,50 @@ int eagle_tree_verify_attn(const eagle_attn_desc* desc, const void* q, const voi
                            const int32_t* seq_lens, const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
   if (!desc) return EAGLE_ERR_NULL;
   const KvSource kv = {k_cache, v_cache, desc->kv_capacity, nullptr, 0, 0, 0};
-  return attention_with_workspace(desc, q, kv, seq_lens, tree_parent, out, stream_);
+  return attention_with_workspace(desc, kPlanAndAttend, q, kv, seq_lens, tree_parent, out, stream_);
 }
 
 int eagle_tree_verify_attn_paged(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* pk, const int32_t* seq_lens,
                                  const int32_t* tree_parent, void* out, eagle_stream_t stream_) {
-  if (!desc || !pk) return EAGLE_ERR_NULL;
-  if (pk->num_pages < 1 || pk->page_size < 16 || (pk->page_size & (pk->page_size - 1)) || pk->max_pages_per_seq < 0) return EAGLE_ERR_SHAPE;
-  if (static_cast<int64_t>(pk->num_pages) * desc->num_kv_heads > 0x7fffffffll) return EAGLE_ERR_SHAPE;
-  if (desc->batch > 0 && desc->max_tree > 0 && !pk->block_table) return EAGLE_ERR_NULL;
-  const KvSource kv = {pk->k_pages, pk->v_pages, static_cast<int64_t>(pk->max_pages_per_seq) * pk->page_size, pk->block_table,
-                       pk->num_pages, pk->page_size, pk->max_pages_per_seq};
-  return attention_with_workspace(desc, q, kv, seq_lens, tree_parent, out, stream_);
+  KvSource kv;
+  int rc = EAGLE_OK;
+  if (!paged_source(desc, pk, &kv, &rc)) return rc;
+  return attention_with_workspace(desc, kPlanAndAttend, q, kv, seq_lens, tree_parent, out, stream_);
 }
+
+int eagle_tree_verify_plan(const eagle_attn_desc* desc, const int32_t* seq_lens, const int32_t* tree_parent,
+                           const eagle_paged_kv* pk, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  KvSource kv = {nullptr, nullptr, desc->kv_capacity, nullptr, 0, 0, 0};
+  int rc = EAGLE_OK;
+  if (pk && !paged_source(desc, pk, &kv, &rc)) return rc;
+  return attention_with_workspace(desc, kPlanOnly, nullptr, kv, seq_lens, tree_parent, nullptr, stream_);
+}
+
+int eagle_tree_verify_attn_planned(const eagle_attn_desc* desc, const void* q, const void* k_cache, const void* v_cache,
+                                   void* out, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  const KvSource kv = {k_cache, v_cache, desc->kv_capacity, nullptr, 0, 0, 0};
+  return attention_with_workspace(desc, kAttendOnly, q, kv, nullptr, nullptr, out, stream_);
+}
+
+int eagle_tree_verify_attn_planned_paged(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* pk, void* out,
+                                         eagle_stream_t stream_) {
+  KvSource kv;
+  int rc = EAGLE_OK;
+  if (!paged_source(desc, pk, &kv, &rc)) return rc;
+  return attention_with_workspace(desc, kAttendOnly, q, kv, nullptr, nullptr, out, stream_);
+}
+
+const uint64_t* eagle_tree_verify_plan_masks(const eagle_attn_desc* desc) {
+  Workspace w;
+  if (!desc || !desc->workspace || !carve_workspace(*desc, desc->workspace, &w)) return nullptr;
+  return w.anc;
+}
+
+void eagle_set_wait_limit_ns(uint64_t ns) { g_wait_limit_ns.store(ns ? ns : kDefaultWaitLimitNs, std::memory_order_relaxed); }
+
+void eagle_test_stall_kv_producer(int32_t after_tiles) { g_stall_after_tiles.store(after_tiles, std::memory_order_relaxed); }
 
 namespace {
 
@@ -268,6 +331,14 @@ int eagle_tree_accept_logits(const eagle_accept_desc* desc, const float* target_
                      stream_);
 }
 
+int eagle_tree_accept_cluster_width(int32_t batch, int32_t vocab) {
+  if (batch < 0 || vocab < 1) return EAGLE_ERR_SHAPE;
+  int err = 0;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
+  return accept_cluster_width(batch, vocab, dev->sm_count);
+}
+
 int eagle_tree_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int32_t batch, int32_t max_tree,
                           uint64_t* anc_mask, uint8_t* depth, int32_t* status, eagle_stream_t stream_) {
   if (batch < 0 || max_tree < 0 || max_tree > kMaxTree) return EAGLE_ERR_SHAPE;
@@ -293,38 +364,6 @@ constexpr size_t kStaticScratchBytes = 24u << 20;   // 24 MiB
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {
-
-// Same carving as carve_workspace(), but sized for the CTAs this device really runs (one per SM) instead of
-// the library-wide upper bound, so that the common shapes fit the fixed array.
-bool carve_static(const eagle_attn_desc& d, int num_ctas, void* base, Workspace* w) {
-  if (d.batch < 0 || d.num_kv_heads <= 0 || d.num_q_heads <= 0 || d.num_q_heads % d.num_kv_heads) return false;
-  const int G = d.num_q_heads / d.num_kv_heads;
-  if (G > kMaxGroup || d.max_tree < 0 || d.max_tree > kMaxTree || (d.head_dim != 64 && d.head_dim != 128)) return false;
-  if (d.num_splits < 0 || d.num_splits > 1024) return false;
-  const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
-  const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? (mtiles + 1) / 2 : 1);   // super-units
-  const long long pieces = d.num_splits > 0 ? units * d.num_splits : units + num_ctas / 2;
-  const long long items = 2 * pieces;
-  const long long slots = items;
-  if (items > (1ll << 30)) return false;
-  char* p = static_cast<char*>(base);
-  size_t off = 0;
-  auto take = [&](size_t n) { char* r = p + off; off += align256(n); return r; };
-  w->hdr = reinterpret_cast<PlanHeader*>(take(sizeof(PlanHeader)));
-  w->seq = reinterpret_cast<SeqPlan*>(take(sizeof(SeqPlan) * static_cast<size_t>(d.batch > 0 ? d.batch : 1)));
-  w->anc = reinterpret_cast<uint64_t*>(take(sizeof(uint64_t) * static_cast<size_t>(d.batch > 0 ? d.batch : 1) * (d.max_tree > 0 ? d.max_tree : 1)));
-  w->units = reinterpret_cast<UnitPlan*>(take(sizeof(UnitPlan) * static_cast<size_t>(units > 0 ? units : 1)));
-  w->cut_tiles = reinterpret_cast<CutTile*>(take(sizeof(CutTile) * 2 * static_cast<size_t>(units > 0 ? units : 1)));
-  w->cta_first = reinterpret_cast<int32_t*>(take(sizeof(int32_t) * (kMaxPlanCtas + 1)));
-  w->items = reinterpret_cast<WorkItem*>(take(sizeof(WorkItem) * static_cast<size_t>(items > 0 ? items : 1)));
-  w->part_ml = reinterpret_cast<float2*>(take(sizeof(float2) * static_cast<size_t>(slots) * kBlockM));
-  w->part_o = reinterpret_cast<float*>(take(sizeof(float) * static_cast<size_t>(slots) * kBlockM * d.head_dim));
-  w->unit_cap = static_cast<int32_t>(units);
-  w->item_cap = static_cast<int32_t>(items);
-  w->slot_cap = static_cast<int32_t>(slots);
-  w->bytes = off;
-  return true;
-}
 
 // Device address of the fixed scratch array on the current device.  The array's name is only a host-side handle:
 // the address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device current.
@@ -358,12 +397,16 @@ int eagle_tree_verify_attn_static(const eagle_attn_desc* desc, const void* q, co
   const int num_ctas = (dev->sm_count < kMaxPlanCtas ? dev->sm_count : kMaxPlanCtas) & ~1;
   void* scratch = static_scratch_ptr();
   if (!scratch) return EAGLE_ERR_DEVICE;
+  // carved for the CTAs this device really runs (one per SM) instead of the library-wide bound, so that common shapes fit
   Workspace w;
-  if (!carve_static(d, num_ctas, scratch, &w)) return EAGLE_ERR_SHAPE;
+  if (!carve_workspace(d, scratch, &w, num_ctas)) return EAGLE_ERR_SHAPE;
   if (w.bytes > kStaticScratchBytes) return EAGLE_ERR_WORKSPACE;   // this shape needs more than the fixed array holds
   if (d.batch == 0 || d.max_tree == 0) return EAGLE_OK;
   const KvSource kv = {k_cache, v_cache, d.kv_capacity, nullptr, 0, 0, 0};
-  return attention_call(d, w, num_ctas, dev, q, kv, seq_lens, tree_parent, out, static_cast<cudaStream_t>(stream_));
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int rc = plan_call(d, w, num_ctas, kv, seq_lens, tree_parent, stream);
+  if (rc != EAGLE_OK) return rc;
+  return attend_call(d, w, num_ctas, dev, q, kv, out, stream);
 }
 
 // ---------------------------------------------------------------------------------------------------------

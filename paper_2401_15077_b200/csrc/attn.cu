@@ -42,7 +42,6 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0;        // S[b] at b*128; P[b] (packed bf16, 64 columns) overwrites the front of S[b]
 constexpr uint32_t kColO = 384;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // ---------------------------------------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -79,9 +78,13 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// (A wait gives up only after two seconds without progress; the K/V ring holds at most six tiles, so by then the
-// producers have been blocked on a full ring for all but the first microseconds of those two seconds and no copy of
-// theirs is still in flight when the CTA leaves.)
+// (A wait gives up only after the time limit has passed without progress, two seconds unless the host changed it, and
+// never less than far longer than a copy takes; the K/V ring holds at most six tiles, so by then the producers have been
+// blocked for all but the first microseconds of that time and no copy of theirs is still in flight when the CTA leaves.)
+// The limit sits in shared memory right after the abort flag, so the wait sites pass one pointer.
+__device__ __forceinline__ unsigned long long wait_limit_of(volatile int* abort_flag) {
+  return *reinterpret_cast<volatile unsigned long long*>(abort_flag + 1);
+}
 // Slow path of a wait, kept out of line so that the dozen wait sites stay small (the kernel's hot loops have to
 // live in the instruction cache next to each other).  Returns false if the CTA has been aborted or the time limit
 // passed (and raises the abort flag).
@@ -91,7 +94,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
     if (mbar_try_wait(bar, parity)) return true;
     if ((spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if (global_timer() - t0 > kWaitLimitNs) {
+      if (global_timer() - t0 > wait_limit_of(abort_flag)) {
         *abort_flag = 1;
         return false;
       }
@@ -225,7 +228,7 @@ __device__ __noinline__ unsigned long long tag_wait_slow(volatile uint32_t* slot
     if ((t & 0xffu) == want) return (1ull << 32) | t;
     if ((spins & 255u) == 0) {
       if (*abort_flag) return 0ull;
-      if (global_timer() - t0 > kWaitLimitNs) {
+      if (global_timer() - t0 > wait_limit_of(abort_flag)) {
         *abort_flag = 1;
         return 0ull;
       }
@@ -252,22 +255,6 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major)
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
-
-#ifdef EAGLE_TRACE
-// Debug builds only: CTA 0 logs (tag, clock) pairs per role; read back with eagle_debug_trace().
-__device__ unsigned long long g_trace[5][1024];
-__device__ int g_trace_n[5];
-__device__ long long g_cta_stat[1024][4];   // per CTA: cycles, items, tiles, tail tiles
-#define TRACE(role, tag)                                                                          \
-  do {                                                                                            \
-    if (blockIdx.x == 0 && trace_n < 1024) {                                                      \
-      g_trace[role][trace_n] = (static_cast<unsigned long long>(tag) << 48) | (static_cast<unsigned long long>(clock64()) & 0xffffffffffffull); \
-      g_trace_n[role] = ++trace_n;                                                                \
-    }                                                                                             \
-  } while (0)
-#else
-#define TRACE(role, tag) do { } while (0)
-#endif
 
 // Descriptor halves.  The low word holds the start address (>>4) and the leading-dimension offset, so stepping along
 // the contraction is a 32-bit add on the low word; the high word (8-row-group stride, version, swizzle) is constant.
@@ -349,7 +336,7 @@ struct Smem {
   static constexpr int kLfin = kTag + kBlockM * 4;           // float [128 rows]: row sums on their way to the epilogue
   static constexpr int kBar = kLfin + kBlockM * 4;
   static constexpr int kNumBars = 2 * kSlots + 3 * kSBufs + 3;
-  static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag
+  static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag, wait limit (8 bytes)
   static constexpr int kBytes = kMisc + 16;
 };
 
@@ -403,6 +390,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     mbar_init(B.q_empty(), 1);
     mbar_init(B.o_free(), kGroupThreads);
     *s_abort = 0;
+    *reinterpret_cast<volatile unsigned long long*>(smem + S::kMisc + 8) = p.wait_limit_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < kBlockM) reinterpret_cast<volatile uint32_t*>(smem + S::kTag)[tid] = 0xffffffffu;   // no step carries this tag yet
@@ -420,10 +408,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   // halves of a lone tile's range, so whatever one of them pulls from HBM the other finds in L2)
   const int member = blockIdx.x & 1;
   const int tp_lo = p.cta_first[blockIdx.x >> 1], tp_hi = p.cta_first[(blockIdx.x >> 1) + 1];
-#ifdef EAGLE_TRACE
-  int trace_n = 0;
-  const long long trace_t0 = clock64();
-#endif
 
   if (warp == kWarpQK) {
     // =========================================================================== QK issuer
@@ -442,22 +426,18 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         const WorkItem it = p.items[2 * tp + member];
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
-        TRACE(1, 1);
         ok = mbar_wait(B.q_full(), item_count & 1u, s_abort);
         if (!ok) break;
-        TRACE(1, 2);
         for (int s = 0; s < steps && ok; ++s, ++gq) {
           // the K tile arrives long before the score buffer frees up: look at it first, so that nothing but the
           // MMA issue follows the wait that matters
           ok = mbar_wait(B.full(ks), kp, s_abort);
           if (!ok) break;
-          TRACE(1, (9 << 10) | (gq & 1023u));
           // S[gq % 3] also holds P of step gq - 3: it is free once that step's PV has finished
           if (gq >= 3) {
             ok = mbar_wait(B.o_done(sb), sph ^ 1u, s_abort);
             if (!ok) break;
           }
-          TRACE(1, (10 << 10) | (gq & 1023u));
           tc_fence_after();
           issue_qk_tile<D>(tmem + kColS + sb * kTileN, q_lo, ring_lo_k + ks * kTileStep, idesc_qk);
           tc_commit(B.s_full(sb));
@@ -466,7 +446,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (ks >= kSlots) { ks -= kSlots; kp ^= 1u; }
           if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
           if (s == steps - 1) tc_commit(B.q_empty());      // every QK of this item has been issued
-          TRACE(1, (11 << 10) | (gq & 1023u));
         }
         ++item_count;
       }
@@ -489,14 +468,12 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         for (int s = 0; s < steps && ok; ++s, ++gp) {
           ok = mbar_wait(B.full(vs), vp, s_abort);   // (arrives well before P is ready)
           if (!ok) break;
-          TRACE(3, (20 << 10) | (gp & 1023u));
           if (s == 0 && item_count > 0) {
             ok = mbar_wait(B.o_free(), (item_count - 1) & 1u, s_abort);   // previous epilogue has read O
             if (!ok) break;
           }
           ok = mbar_wait(B.p_full(sb), sph, s_abort);
           if (!ok) break;
-          TRACE(3, (30 << 10) | (gp & 1023u));
           tc_fence_after();
           issue_pv_tile(tmem + kColO, tmem + kColS + sb * kTileN, ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
           tc_commit(B.o_done(sb));
@@ -504,7 +481,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           vs += 2;
           if (vs >= kSlots) { vs -= kSlots; vp ^= 1u; }
           if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
-          TRACE(3, (31 << 10) | (gp & 1023u));
         }
         ++item_count;
       }
@@ -552,7 +528,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         fence_proxy_async();
         mbar_arrive(B.q_full());
       }
-      if ((tid & 127) == 0) TRACE(2 + 2 * grp, 3);
 
       float m_ref = -INFINITY;   // reference (scaled, log2 domain) this thread's row sum is relative to
       float m_in = -INFINITY;    // reference the other group left behind at the step before this group's latest one
@@ -564,7 +539,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         const uint32_t s_addr = tmem + lane_addr + kColS + sb * kTileN;   // P goes over the front half of the same columns
         ok = mbar_wait_warp(B.s_full(sb), sph, s_abort);
         if (!ok) break;
-        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (10 << 10) | (gs & 1023u));
         tc_fence_after();
         const int key0 = (it.tile_begin + s) * kTileN;
         // visibility of this row's 128 keys, 32 per word: keys before L are all visible, key L + m is visible iff
@@ -613,7 +587,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           }
         }
         const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // scale > 0
-        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (12 << 10) | (gs & 1023u));
 
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
@@ -668,8 +641,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           }
           tc_wait_st();
         }
-        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (13 << 10) | (gs & 1023u));
-        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (16 << 10) | (gs & 1023u));
         // ---- pass 2: exponentials and packed P, in column order (P overwrites score columns that have been
         // consumed).  Chunks 0 and 1 are still in registers; chunks 2 and 3 are fetched again meanwhile.
         const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
@@ -726,7 +697,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(B.p_full(sb));
-        if ((tid & 127) == 0) TRACE(2 + 2 * grp, (11 << 10) | (gs & 1023u));
 
         if (s == steps - 1) {
           // ---- this group took the item's last step: it writes the item's output.  Wait for the last PV (PVs
@@ -734,7 +704,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           // the unnormalised fp32 partial of a cut piece.
           ok = mbar_wait_warp(B.o_done(sb), sph, s_abort);
           if (!ok) break;
-          if ((tid & 127) == 0) TRACE(2 + 2 * grp, 20);
           tc_fence_after();
           float l_row = l_sum;
           if (steps > 1) {
@@ -771,7 +740,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (row_valid && it.slot >= 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_ref, l_row);
           tc_fence_before();
           mbar_arrive(B.o_free());            // the next item's first PV may overwrite the accumulator
-          if ((tid & 127) == 0) TRACE(2 + 2 * grp, 21);
         }
       }
       g_base += steps;
@@ -837,6 +805,10 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       uint32_t n = 0;   // position in the load sequence
       auto load_tile = [&](const Cursor& c, bool is_v) {
         const uint32_t slot = n % kSlots, par = ((n / kSlots) & 1u) ^ 1u;
+        if (p.stall_after_tiles >= 0 && n >= static_cast<uint32_t>(p.stall_after_tiles)) {
+          ok = false;   // test hook: the producer falls silent (nothing further is issued), so the consumers' waits run out
+          return;
+        }
         if constexpr (PAGED) {
           // The tile's 128 slots come from one page (pages of 128 slots or more) or from 128 / page_size pages, one box
           // each; the boxes land one under the other, which is the tile's layout.  A box past the sequence's last page
@@ -860,7 +832,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         } else {
           ok = mbar_wait(B.empty(slot), par, s_abort);
           if (!ok) return;
-          TRACE(0, ((2 + (is_v ? 1 : 0)) << 10) | (n & 1023u));
           mbar_expect_tx(B.full(slot), S::kTileBytes);
 #pragma unroll
           for (int sl = 0; sl < S::kSlabs; ++sl)
@@ -890,29 +861,10 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     }
   }
 
-#ifdef EAGLE_TRACE
-  if (tid == 0) {
-    long long tiles = 0, tails = 0;
-    long long n_it = 0;
-    for (int tp = tp_lo; tp < tp_hi; ++tp) {
-      const WorkItem it = p.items[2 * tp + member];
-      if (it.tile_end <= it.tile_begin) continue;
-      ++n_it;
-      tiles += it.tile_end - it.tile_begin;
-      tails += (it.tile_end * kTileN > p.seq[it.b].L) ? 1 : 0;
-    }
-    g_cta_stat[blockIdx.x][1] = n_it;
-    g_cta_stat[blockIdx.x][2] = tiles;
-    g_cta_stat[blockIdx.x][3] = tails;
-  }
-#endif
   // ---- teardown: everyone arrives here (normally or after an abort); release TMEM
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && *s_abort) report_status(p.status, EAGLE_ERR_TIMEOUT);
-#ifdef EAGLE_TRACE
-  if (tid == 0) g_cta_stat[blockIdx.x][0] = clock64() - trace_t0;
-#endif
   if (warp == kWarpQK) {
     __syncwarp();
     tc_fence_after();
@@ -965,24 +917,6 @@ bool make_q_map(CUtensorMap* map, const void* base, int D, int Hq, int T_max, in
 }
 
 }  // namespace
-
-#ifdef EAGLE_TRACE
-}  // namespace eagle
-extern "C" int eagle_debug_cta_stat(long long* dst) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(dst, eagle::g_cta_stat, sizeof(long long) * 1024 * 4);
-  return 0;
-}
-extern "C" int eagle_debug_trace(unsigned long long* dst, int* counts) {
-  int zero[5] = {0, 0, 0, 0, 0};
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(dst, eagle::g_trace, sizeof(unsigned long long) * 5 * 1024);
-  cudaMemcpyFromSymbol(counts, eagle::g_trace_n, sizeof(int) * 5);
-  cudaMemcpyToSymbol(eagle::g_trace_n, zero, sizeof(zero));
-  return 0;
-}
-namespace eagle {
-#endif
 
 int attn_tile_keys() { return kTileN; }
 

@@ -69,11 +69,12 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
       }
     }
     // a piece counts when its item is not empty (an empty item never wrote its slot) and the row saw a key in it
+    // (a row all of whose keys in the piece were masked keeps the reference -inf; its sum may hold rounding dust)
     bool use[kPiecesAtOnce];
     float m_new = m_star;
 #pragma unroll
     for (int u = 0; u < kPiecesAtOnce; ++u) {
-      use[u] = s0 + u < ct.count && t1[u] > t0[u] && ml[u].y > 0.f;
+      use[u] = s0 + u < ct.count && t1[u] > t0[u] && ml[u].y > 0.f && ml[u].x > -INFINITY;
       if (use[u]) m_new = fmaxf(m_new, ml[u].x);
     }
     if (m_new == -INFINITY) continue;

@@ -77,7 +77,9 @@ struct Workspace {
 
 __host__ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
-__host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Workspace* w) {
+// `num_ctas` bounds the CTAs of the attention kernel the plan may be made for (the library-wide bound by default; the
+// fixed-array entry point passes the current device's count so that common shapes fit its array).
+__host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Workspace* w, int num_ctas = kMaxPlanCtas) {
   if (d.batch < 0 || d.num_kv_heads <= 0 || d.num_q_heads <= 0 || d.num_q_heads % d.num_kv_heads) return false;
   const int G = d.num_q_heads / d.num_kv_heads;
   if (G > kMaxGroup || d.max_tree < 0 || d.max_tree > kMaxTree || (d.head_dim != 64 && d.head_dim != 128)) return false;
@@ -85,10 +87,19 @@ __host__ inline bool carve_workspace(const eagle_attn_desc& d, void* base, Works
   const long long mtiles = (static_cast<long long>(d.max_tree) * G + kBlockM - 1) / kBlockM;
   const long long units = static_cast<long long>(d.batch) * d.num_kv_heads * (mtiles > 0 ? (mtiles + 1) / 2 : 1);   // super-units
   // team pieces: one per super-unit plus at most one per share boundary (or num_splits per super-unit when forced);
-  // two items per team piece, and at most one partial slot per item
-  const long long pieces = d.num_splits > 0 ? units * d.num_splits : units + kMaxPlanCtas / 2;
+  // two items per team piece
+  const long long teams = num_ctas / 2;
+  const long long pieces = d.num_splits > 0 ? units * d.num_splits : units + teams;
   const long long items = 2 * pieces;
-  const long long slots = items;
+  // Partial slots: one per item when the split is forced.  With equal shares only cut super-units and lone tiles take
+  // slots, two per piece: a share boundary cuts at most one super-unit, so the cut pairs and twins hold at most
+  // 2 * (cuts + cut units) <= 4 * (teams - 1) slots, and a lone tile (one per sequence, only with an odd number of
+  // KV heads) holds 2 * (its cuts + 1).
+  long long slots = items;
+  if (d.num_splits == 0) {
+    const long long bound = 4 * teams + 2ll * d.batch * (d.num_kv_heads & 1);
+    if (bound < slots) slots = bound;
+  }
   if (items > (1ll << 30)) return false;
   char* p = static_cast<char*>(base);
   size_t off = 0;
@@ -131,6 +142,8 @@ struct AttnParams {
   // page block_table[b * max_pages + j / page_size]; page_size is a power of two
   const int32_t* block_table;
   int32_t page_size, page_shift, max_pages, num_pages;
+  unsigned long long wait_limit_ns;   // a wait that makes no progress for this long aborts the CTA (EAGLE_ERR_TIMEOUT)
+  int32_t stall_after_tiles;          // test hook: the K/V producer stops issuing after this many tiles (negative: off)
 };
 
 struct PlanParams {
@@ -215,6 +228,7 @@ int attn_tile_keys();
 cudaError_t attn_prepare(int head_dim);
 cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cudaStream_t stream);
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
+int accept_cluster_width(int batch, int vocab, int sm_count);   // 0: a warp per tree; else CTAs per cluster
 
 cudaError_t launch_commit(const CommitParams& p, cudaStream_t stream);
 cudaError_t launch_expand(const ExpandParams& p, int sm_count, cudaStream_t stream);

@@ -98,19 +98,7 @@ __device__ __forceinline__ long long qdiv(long long a, long long b, bool small) 
 }
 __device__ __forceinline__ long long ceil_div(long long a, long long b, bool small) { return qdiv(a + b - 1, b, small); }
 
-// anc[i] = bit i | anc[parent[i]] in node order (parents come first).  Returns false on an invalid entry.
-__device__ inline bool build_masks_one(const int32_t* par, int n, uint64_t* anc, uint8_t* depth) {
-  for (int i = 0; i < n; ++i) {
-    const int pi = par[i];
-    if (pi < -1 || pi >= i) return false;
-    const uint64_t up = pi >= 0 ? anc[pi] : 0ull;
-    anc[i] = up | (1ull << i);
-    if (depth) depth[i] = static_cast<uint8_t>(__popcll(up) + 1);
-  }
-  return true;
-}
-
-// The same masks by one warp: lane l holds nodes l and l + 32 (and is given their parent entries).  Every node starts with its own bit and a pointer to its
+// Ancestor-or-self masks of one tree by one warp: lane l holds nodes l and l + 32 (and is given their parent entries).  Every node starts with its own bit and a pointer to its
 // parent; each round ORs in the mask of the node pointed to and jumps the pointer to that node's pointer, so six rounds
 // cover any path of up to 64 nodes.  Returns false (to all lanes) on an invalid entry.  anc[i >= n] is not written.
 __device__ inline bool build_masks_warp(int par_lo, int par_hi, int n, uint64_t* anc, uint8_t* depth, int lane) {
@@ -532,21 +520,25 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(PlanParams pg) {
   }
 }
 
-__global__ void build_mask_kernel(const int32_t* __restrict__ tree_parent, const int32_t* __restrict__ tree_sizes,
-                                  int batch, int T, uint64_t* __restrict__ anc, uint8_t* __restrict__ depth,
-                                  int32_t* status) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= batch) return;
+// The stand-alone mask builder: one warp per tree, the same routine the planner runs.
+constexpr int kMaskWarps = 4;
+__global__ void __launch_bounds__(32 * kMaskWarps)
+build_mask_kernel(const int32_t* __restrict__ tree_parent, const int32_t* __restrict__ tree_sizes, int batch, int T,
+                  uint64_t* __restrict__ anc, uint8_t* __restrict__ depth, int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int b = blockIdx.x * kMaskWarps + (threadIdx.x >> 5);
+  if (b >= batch) return;   // uniform over the warp
   int n = tree_sizes ? tree_sizes[b] : T;
+  const int32_t* par = tree_parent + static_cast<size_t>(b) * T;
   uint64_t* a = anc + static_cast<size_t>(b) * T;
   uint8_t* d = depth ? depth + static_cast<size_t>(b) * T : nullptr;
   bool ok = n >= 0 && n <= T;
-  if (ok) ok = build_masks_one(tree_parent + static_cast<size_t>(b) * T, n, a, d);
+  if (ok) ok = build_masks_warp(lane < n ? par[lane] : -1, lane + 32 < n ? par[lane + 32] : -1, n, a, d, lane);
   if (!ok) {
-    report_status(status, EAGLE_ERR_TREE);
+    if (lane == 0) report_status(status, EAGLE_ERR_TREE);
     n = 0;
   }
-  for (int i = n; i < T; ++i) {
+  for (int i = n + lane; i < T; i += 32) {
     a[i] = 0ull;
     if (d) d[i] = 0;
   }
@@ -562,9 +554,8 @@ cudaError_t launch_plan(const PlanParams& p, cudaStream_t stream) {
 
 cudaError_t launch_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int batch, int max_tree,
                               uint64_t* anc, uint8_t* depth, int32_t* status, cudaStream_t stream) {
-  const int threads = 128;
-  build_mask_kernel<<<(batch + threads - 1) / threads, threads, 0, stream>>>(tree_parent, tree_sizes, batch, max_tree,
-                                                                               anc, depth, status);
+  build_mask_kernel<<<(batch + kMaskWarps - 1) / kMaskWarps, 32 * kMaskWarps, 0, stream>>>(tree_parent, tree_sizes, batch, max_tree,
+                                                                                            anc, depth, status);
   count_launch();
   return cudaGetLastError();
 }

@@ -54,7 +54,7 @@ def _check(out, ref, sizes):
 CASES = {
     "tiny": W.CONFIGS["tiny"],
     "7b_mha": W.CONFIGS["7b_mha"],
-    "70b_gqa_b2": W.scaled(W.CONFIGS["70b_gqa"], batch=2),
+    "70b_gqa": W.CONFIGS["70b_gqa"],
     "mixtral_gqa_small": W.scaled(W.CONFIGS["mixtral_gqa"], batch=2, prefix=(1500, 3000)),
     "serving_mix_small": W.scaled(W.CONFIGS["serving_mix"], batch=6, prefix=(100, 1500)),
     "d64_gqa_ragged": W.scaled(W.CONFIGS["tiny"], batch=5, num_q_heads=16, num_kv_heads=4, prefix=(0, 700), tree=(1, 33)),
@@ -228,6 +228,105 @@ def test_invalid_inputs_are_reported_not_trapped(E, oracle):
     bad2.seq_lens[0] = bad2.kv_capacity   # prefix + tree does not fit the cache
     out, status = _run(E, bad2)
     assert status == -6 and np.all(out.double().numpy()[0] == 0.0)
+
+
+def test_piece_in_which_a_row_sees_no_key(E, oracle):
+    """Prefix of 100 slots and a star tree of 64 nodes (every node sees the prefix and itself only), cut into two pieces
+    at the KV-tile boundary: in the second piece (tree nodes 28..63) the rows of nodes 0..27 have every key masked, so
+    their partial must not count in the merge.  Also with a chain, where the late rows see everything."""
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=3, num_q_heads=8, num_kv_heads=2, head_dim=128, prefix=(100, 100), tree=(64, 64), max_depth=64)
+    for shape in ("star", "chain"):
+        inp = W.make_attn_inputs(cfg, salt=31)
+        inp.tree_parent[:] = -1 if shape == "star" else torch.arange(-1, 63, dtype=torch.int32)
+        ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+        for splits in (2, 0):
+            out, status = _run(E, inp, num_splits=splits)
+            assert status == 0
+            _check(out, ref, inp.tree_sizes)
+
+
+def test_plan_once_attend_many_layers(E, oracle):
+    """One plan for a verification pass, then attention + combine per layer on that plan: bit for bit what the one-call
+    form gives for every layer's K/V, and the oracle's result; the plan's own tree masks equal the oracle's bit for bit."""
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=9, prefix=(30, 2500), tree=(0, 64), max_depth=64)
+    layers = [W.make_attn_inputs(cfg, salt=40)]
+    for l in (1, 2):
+        other = W.make_attn_inputs(cfg, salt=40)
+        g = torch.Generator().manual_seed(400 + l)
+        for name in ("q", "k_cache", "v_cache"):
+            t = getattr(other, name)
+            fresh = torch.randn(t.shape, generator=g).to(torch.bfloat16)
+            setattr(other, name, torch.where(torch.isnan(t), t, fresh))     # same lengths and trees, other values
+        layers.append(other)
+    base = layers[0]
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    for splits in (0, 3):
+        plan = E.eagle_tree_verify_plan(tuple(base.q.shape), cfg.num_kv_heads, base.k_cache.shape[2], base.seq_lens.to(d),
+                                        base.tree_parent.to(d), tree_sizes=base.tree_sizes.to(d), num_splits=splits, status=status)
+        torch.cuda.synchronize()
+        anc_ref, _ = oracle.tree_ancestors(base.tree_parent.numpy(), base.tree_sizes.numpy())
+        assert np.array_equal(plan.masks().cpu().numpy().view(np.uint64), anc_ref)
+        for inp in layers:
+            out = torch.full(inp.q.shape, float("nan"), dtype=torch.bfloat16, device=d)
+            plan.attend(inp.q.to(d), inp.k_cache.to(d), inp.v_cache.to(d), out, status=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            whole, st = _run(E, inp, num_splits=splits)
+            assert st == 0 and torch.equal(out.cpu().view(torch.int16), whole.view(torch.int16))
+            ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+            _check(out.cpu(), ref, inp.tree_sizes)
+    # the same over a paged cache
+    pk = W.make_paged_cache(base, 64, salt=3)
+    plan = E.eagle_tree_verify_plan(tuple(base.q.shape), cfg.num_kv_heads, 0, base.seq_lens.to(d), base.tree_parent.to(d),
+                                    tree_sizes=base.tree_sizes.to(d), status=status,
+                                    paged=(pk.block_table.to(d), pk.k_pages.shape[0], pk.page_size))
+    out = plan.attend_paged(base.q.to(d), pk.k_pages.to(d), pk.v_pages.to(d), pk.block_table.to(d), status=status)
+    torch.cuda.synchronize()
+    whole, st = _run(E, base)
+    assert int(status.item()) == 0 and torch.equal(out.cpu().view(torch.int16), whole.view(torch.int16))
+
+
+def test_planner_masks_match_oracle(E, oracle):
+    """The masks the attention kernel really reads (built by the planner, left in the workspace), bit for bit; trees of
+    every size up to 64 and depth up to 64, per sequence and one tree shared by all."""
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=70, num_q_heads=8, num_kv_heads=2, prefix=(0, 300), tree=(0, 64), max_depth=64)
+    sizes, parent = W.make_trees(cfg, salt=8)
+    lens = torch.randint(0, 300, (cfg.batch,), dtype=torch.int32)
+    anc_ref, _ = oracle.tree_ancestors(parent.numpy(), sizes.numpy())
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    plan = E.eagle_tree_verify_plan((cfg.batch, 64, 8, 128), 2, 400, lens.to(d), parent.to(d), tree_sizes=sizes.to(d), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(plan.masks().cpu().numpy().view(np.uint64), anc_ref)
+    b = int(sizes.argmax())
+    plan = E.eagle_tree_verify_plan((cfg.batch, 64, 8, 128), 2, 400, lens.to(d), parent[b].contiguous().to(d),
+                                    tree_sizes=sizes[b:b + 1].to(d), status=status, shared_tree=True)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(plan.masks().cpu().numpy().view(np.uint64), np.broadcast_to(anc_ref[b], anc_ref.shape))
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_fine(E, oracle):
+    """Failure handling: every wait in the attention kernel is bounded.  The K/V producer is told (test hook) to fall
+    silent after two tiles and the limit is lowered to 2 ms: the kernel must return by itself with EAGLE_ERR_TIMEOUT,
+    and an ordinary call right after must be correct."""
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=2, prefix=(600, 900))
+    inp = W.make_attn_inputs(cfg, salt=12)
+    ref = oracle.tree_verify_attn(inp.q, inp.k_cache, inp.v_cache, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    try:
+        E.set_wait_limit_ns(2_000_000)
+        E.test_stall_kv_producer(2)
+        out, status = _run(E, inp)
+    finally:
+        E.test_stall_kv_producer(-1)
+        E.set_wait_limit_ns(0)
+    assert status == -8, E.status_string(status)
+    out, status = _run(E, inp)
+    assert status == 0
+    _check(out, ref, inp.tree_sizes)
 
 
 def test_mask_builder_matches_oracle(E, oracle):
