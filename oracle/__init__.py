@@ -56,6 +56,8 @@ def _load():
         lib.oracle_tree_commit_paged.argtypes = [i32] * 8 + [vp] * 7
         lib.oracle_tree_commit_paged.restype = i32
         lib.oracle_num_threads.restype = i32
+        lib.oracle_set_num_threads.argtypes = [i32]
+        lib.oracle_set_num_threads.restype = None
         _lib = lib
     return _lib
 
@@ -82,6 +84,11 @@ def _as(a, dtype):
 
 def num_threads() -> int:
     return int(_load().oracle_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    """Threads for the oracle's OpenMP loops from now on (0: the default).  For timing; results do not depend on it."""
+    _load().oracle_set_num_threads(int(n))
 
 
 def tree_ancestors(tree_parent, tree_sizes=None):

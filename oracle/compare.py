@@ -1,4 +1,5 @@
-"""Comparison of an acceptance result with the oracle's, decision by decision (helper of the parity tests).
+"""Comparison of an acceptance result with the oracle's, decision by decision (test infrastructure, like the oracle:
+used by the parity tests, the smoke check and the bench's parity record; holds none of the method's arithmetic).
 
 With fixed uniforms the walk has one correct result; a floating-point decision that sits within rounding of its
 boundary may still fall either way.  The stated rule: results must be identical, except that a difference is tolerated

@@ -677,3 +677,13 @@ int oracle_num_threads(void) {
 #endif
   return n;
 }
+
+/* Number of threads the OpenMP loops above use from now on (0 or less: the OpenMP default).  Timing aid only: the
+ * results do not depend on it (every unit is computed by one thread, in the same order of operations). */
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+  omp_set_num_threads(n > 0 ? n : omp_get_num_procs());
+#else
+  (void)n;
+#endif
+}

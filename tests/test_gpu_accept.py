@@ -2,7 +2,7 @@
 
 Greedy sequences must agree exactly.  Stochastic sequences must agree exactly given the same uniforms,
 except where the oracle's margin at the FIRST decision that differs is below 1e-5 (the decisions are
-compared one by one, see accept_trace.py); such sequences are counted, and the count is asserted to stay small.
+compared one by one, see oracle/compare.py); such sequences are counted, and the count is asserted to stay small.
 """
 import os
 
@@ -11,7 +11,7 @@ import pytest
 import torch
 from scipy import stats
 
-from accept_trace import compare_with_oracle
+from oracle.compare import compare_with_oracle
 from paper_2401_15077_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu

@@ -511,7 +511,7 @@ def _replay(oracle_mod, res, b, parent):
 
 
 def test_trace_replays_to_the_result_and_tolerance_helper_finds_first_difference(oracle):
-    from accept_trace import first_differing_decision, compare_with_oracle
+    from oracle.compare import first_differing_decision, compare_with_oracle
     cfg = W.scaled(W.CONFIGS["tiny"], batch=40, tree=(3, 30), max_depth=6, vocab=50)
     inp = W.make_accept_inputs(cfg, salt=5, rho=0.9, greedy="half")
     res = oracle.tree_accept(inp.target_probs, inp.draft_probs, inp.draft_tokens, inp.tree_parent, inp.uniforms,
