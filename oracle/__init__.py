@@ -45,6 +45,10 @@ def _load():
         lib.oracle_tree_verify_attn.restype = i32
         lib.oracle_tree_verify_attn_paged.argtypes = [i32] * 8 + [vp, dbl] + [vp] * 7
         lib.oracle_tree_verify_attn_paged.restype = i32
+        lib.oracle_tree_verify_attn_fp8.argtypes = [i32, i32, i32, i32, i32, i32, vp, dbl] + [vp] * 8
+        lib.oracle_tree_verify_attn_fp8.restype = i32
+        lib.oracle_e4m3_table.argtypes = [vp]
+        lib.oracle_e4m3_table.restype = None
         lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 17
         lib.oracle_tree_accept.restype = i32
         lib.oracle_tree_accept_logits.argtypes = [i32, i32, i32, i32] + [vp] * 7 + [dbl] + [vp] * 10
@@ -142,6 +146,32 @@ def tree_verify_attn_paged(q, k_pages, v_pages, block_table, seq_lens, tree_pare
                                                _ptr(ka), _ptr(va), _ptr(bt), _ptr(sl), _ptr(par), _ptr(out))
     if rc != 0:
         raise ValueError(f"oracle_tree_verify_attn_paged failed: {rc}")
+    return out
+
+
+def e4m3_table():
+    """The 256 values of the fp8 e4m3 codes as the oracle decodes them (float64; the two NaN codes are NaN)."""
+    out = np.zeros(256, np.float64)
+    _load().oracle_e4m3_table(_ptr(out))
+    return out
+
+
+def tree_verify_attn_fp8(q, k_codes, v_codes, k_scale, v_scale, seq_lens, tree_parent, tree_sizes=None, sm_scale: float = 0.0):
+    """fp64 tree-masked attention over a cache stored as e4m3 codes (uint8 [B, Hkv, S_cap, D]) with fp32 scales [B, Hkv]:
+    key = code value * k_scale, value = code value * v_scale.  q is bf16.  Returns float64 [B, T_max, Hq, D]."""
+    qa = _as(q, np.uint16)
+    ka, va = _as(k_codes, np.uint8), _as(v_codes, np.uint8)
+    B, T, Hq, D = qa.shape
+    Hkv, S = ka.shape[1], ka.shape[2]
+    assert ka.shape == va.shape == (B, Hkv, S, D)
+    ks, vs = _as(k_scale, np.float32), _as(v_scale, np.float32)
+    assert ks.shape == vs.shape == (B, Hkv)
+    sl, par, ts = _as(seq_lens, np.int32), _as(tree_parent, np.int32), _as(tree_sizes, np.int32)
+    out = np.zeros((B, T, Hq, D), np.float64)
+    rc = _load().oracle_tree_verify_attn_fp8(B, Hq, Hkv, D, T, S, _ptr(ts), float(sm_scale), _ptr(qa), _ptr(ka), _ptr(va),
+                                             _ptr(ks), _ptr(vs), _ptr(sl), _ptr(par), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_verify_attn_fp8 failed: {rc}")
     return out
 
 

@@ -13,6 +13,7 @@
  *                              for one attention layer that is softmax attention over the committed
  *                              prefix plus the node's ancestors and itself (plain definition).
  *   oracle_tree_verify_attn_paged - the same over a cache stored in pages addressed through a block table.
+ *   oracle_tree_verify_attn_fp8 - the same over a cache stored as fp8 (e4m3) codes with one scale per (sequence, KV head).
  *   oracle_tree_accept       - Algorithm 1 (multi-round speculative sampling, App. A.2) applied
  *                              recursively at every node from the root (Sec. 3.3); the greedy setting
  *                              (Preliminaries) is the same rule with a one-hot target distribution.
@@ -232,6 +233,101 @@ int oracle_tree_verify_attn_paged(int batch, int num_q_heads, int num_kv_heads, 
   free(kc);
   free(vc);
   return rc;
+}
+
+/*
+ * Value of an fp8 "e4m3" code (the 8-bit float with 1 sign, 4 exponent and 3 mantissa bits, exponent bias 7, no
+ * infinities; the two codes with all exponent and mantissa bits set are NaN), written from that definition:
+ * exponent field 0 -> (mantissa / 8) * 2^-6 (zero and the subnormals), else (1 + mantissa / 8) * 2^(exponent - 7).
+ */
+static double e4m3_to_f64(uint8_t c) {
+  const int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+  double v;
+  if (e == 15 && m == 7) return NAN;
+  if (e == 0) v = ldexp((double)m / 8.0, -6);
+  else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+  return sign ? -v : v;
+}
+
+/* The 256 values of the code above (for the test that pins the table against a library's conversion). */
+void oracle_e4m3_table(double* out256) {
+  for (int c = 0; c < 256; ++c) out256[c] = e4m3_to_f64((uint8_t)c);
+}
+
+/*
+ * The same attention when the cache is STORED in fp8 (a storage format of the same cache: Sec. 4.4 notes that the
+ * decoding being sped up is bound by memory traffic, and Sec. 4.2 reports the method on a quantised deployment; the
+ * paper gives no quantisation scheme, so the convention is this library's): k_cache / v_cache hold e4m3 codes
+ * [batch, num_kv_heads, kv_capacity, head_dim] and every (sequence, KV head) has one fp32 scale for its keys and one
+ * for its values, k_scale / v_scale [batch, num_kv_heads]: key = code value * k_scale, value = code value * v_scale,
+ * exactly (fp64).  Everything after that is the definition of oracle_tree_verify_attn, written out again on those
+ * values: queries stay bf16, scores / softmax / sums are fp64.  Slots that are not visible are never read.
+ */
+int oracle_tree_verify_attn_fp8(int batch, int num_q_heads, int num_kv_heads, int head_dim, int max_tree,
+                                int kv_capacity, const int32_t* tree_sizes, double sm_scale, const uint16_t* q,
+                                const uint8_t* k_cache, const uint8_t* v_cache, const float* k_scale, const float* v_scale,
+                                const int32_t* seq_lens, const int32_t* tree_parent, double* out) {
+  if (batch < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || head_dim <= 0 || max_tree < 0 || max_tree > 64 ||
+      num_q_heads % num_kv_heads != 0 || !seq_lens || !tree_parent || !out || !k_scale || !v_scale)
+    return ORACLE_ERR_ARG;
+  const int G = num_q_heads / num_kv_heads;
+  const int D = head_dim;
+  if (sm_scale == 0.0) sm_scale = 1.0 / sqrt((double)D);
+  for (int b = 0; b < batch; ++b) {
+    const int n = tree_size_of(tree_sizes, b, max_tree);
+    if (n < 0 || n > max_tree || seq_lens[b] < 0 || seq_lens[b] + n > kv_capacity) return ORACLE_ERR_ARG;
+    if (!tree_valid(tree_parent + (size_t)b * max_tree, n)) return ORACLE_ERR_TREE;
+  }
+  memset(out, 0, sizeof(double) * (size_t)batch * max_tree * num_q_heads * D);
+  int failed = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+  for (int b = 0; b < batch; ++b) {
+    for (int h = 0; h < num_q_heads; ++h) {
+      const int n = tree_size_of(tree_sizes, b, max_tree);
+      const int L = seq_lens[b];
+      const int g = h / G;
+      const int32_t* par = tree_parent + (size_t)b * max_tree;
+      const uint8_t* kb = k_cache + ((size_t)b * num_kv_heads + g) * (size_t)kv_capacity * D;
+      const uint8_t* vb = v_cache + ((size_t)b * num_kv_heads + g) * (size_t)kv_capacity * D;
+      const double ks = (double)k_scale[(size_t)b * num_kv_heads + g], vs = (double)v_scale[(size_t)b * num_kv_heads + g];
+      int* slots = (int*)malloc(sizeof(int) * (size_t)(L + max_tree + 1));
+      double* s = (double*)malloc(sizeof(double) * (size_t)(L + max_tree + 1));
+      if (!slots || !s) {
+        failed = 1;
+        free(slots);
+        free(s);
+        continue;
+      }
+      for (int i = 0; i < n; ++i) {
+        const uint16_t* qi = q + (((size_t)b * max_tree + i) * num_q_heads + h) * D;
+        double* oi = out + (((size_t)b * max_tree + i) * num_q_heads + h) * D;
+        int cnt = 0;
+        for (int j = 0; j < L; ++j) slots[cnt++] = j;                      /* the whole prefix */
+        for (int c = i; c >= 0; c = par[c]) slots[cnt++] = L + c;          /* then the root path of node i */
+        double smax = -INFINITY;
+        for (int t = 0; t < cnt; ++t) {
+          const uint8_t* kj = kb + (size_t)slots[t] * D;
+          double acc = 0.0;
+          for (int d = 0; d < D; ++d) acc += bf16_to_f64(qi[d]) * (e4m3_to_f64(kj[d]) * ks);
+          s[t] = sm_scale * acc;
+          if (s[t] > smax) smax = s[t];
+        }
+        double denom = 0.0;
+        for (int t = 0; t < cnt; ++t) {
+          s[t] = exp(s[t] - smax);
+          denom += s[t];
+        }
+        for (int d = 0; d < D; ++d) {
+          double acc = 0.0;
+          for (int t = 0; t < cnt; ++t) acc += s[t] * (e4m3_to_f64(vb[(size_t)slots[t] * D + d]) * vs);
+          oi[d] = acc / denom;
+        }
+      }
+      free(slots);
+      free(s);
+    }
+  }
+  return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
 }
 
 /*

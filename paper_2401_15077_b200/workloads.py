@@ -170,6 +170,38 @@ def make_paged_cache(inp: AttnInputs, page_size: int, salt: int = 0, spare_pages
 
 
 @dataclass
+class Fp8KV:
+    k_codes: torch.Tensor      # uint8 [B, Hkv, S_cap, D]: fp8 e4m3 codes
+    v_codes: torch.Tensor
+    k_scale: torch.Tensor      # fp32 [B, Hkv]
+    v_scale: torch.Tensor
+
+
+def make_fp8_cache(inp: AttnInputs, poison: bool = True, power_of_two_scales: bool = False) -> Fp8KV:
+    """The keys and values of ``inp`` as a serving engine would store them in fp8: per (sequence, KV head) a scale
+    amax / 448 over the visible slots and the codes of round(x / scale) to e4m3 (the library's conversion; this is input
+    preparation, not part of the verification step).  Slots that are not visible hold the NaN code when ``poison``."""
+    cfg = inp.cfg
+    B, Hkv = cfg.batch, cfg.num_kv_heads
+    out = []
+    for x in (inp.k_cache, inp.v_cache):
+        codes = torch.full(x.shape, 0x7F if poison else 0, dtype=torch.uint8)
+        scale = torch.ones((B, Hkv), dtype=torch.float32)
+        for b in range(B):
+            n = int(inp.seq_lens[b] + inp.tree_sizes[b])
+            if n == 0:
+                continue
+            vis = x[b, :, :n].float()
+            s = vis.abs().amax(dim=(1, 2)).clamp_min(1e-12) / 448.0
+            if power_of_two_scales:
+                s = torch.exp2(torch.ceil(torch.log2(s)))
+            scale[b] = s
+            codes[b, :, :n] = (vis / s[:, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)
+        out += [codes, scale]
+    return Fp8KV(out[0], out[2], out[1], out[3])
+
+
+@dataclass
 class AcceptInputs:
     cfg: VerifyConfig
     target_probs: torch.Tensor   # fp32 [B, T_max+1, V]
