@@ -275,6 +275,34 @@ class StepContext:
         return {"layers": layers, "plan_ms": e[0].elapsed_time(e[1]), "ms_per_layer": e[1].elapsed_time(e[2]) / layers,
                 "note": "eagle_tree_verify_plan once, then eagle_tree_verify_attn_planned per layer"}
 
+    def fp8_leg(self, attn_ms_bf16, pk, calls=12):
+        """The same attention over the same cache stored as fp8 (e4m3) codes with a scale per (sequence, KV head): the
+        attention kernel's time (library events), against the bf16 call's, and its own HBM fraction (half the cache bytes)."""
+        cfg = self.cfg
+        if cfg.head_dim != 128:
+            return None
+        f8 = W.make_fp8_cache(self.attn)
+        dev, s = self.dev, self.sets[0]
+        sets = [(f8.k_codes.to(dev), f8.v_codes.to(dev)) for _ in range(max(1, min(self.R, 24)))]
+        ks, vs = f8.k_scale.to(dev), f8.v_scale.to(dev)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(calls)]
+        for a, b in evs:
+            a.record()
+            b.record()
+        for i in range(3 + calls):
+            kc, vc = sets[i % len(sets)]
+            self.E.eagle_tree_verify_attn_fp8(s["q"], kc, vc, ks, vs, s["sl"], s["par"], self.out, tree_sizes=s["ts"], workspace=self.ws,
+                                              status=self.status, num_splits=self.num_splits, events=evs[i - 3] if i >= 3 else None)
+        torch.cuda.synchronize()
+        self.check()
+        ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
+        kv_rows = int((self.attn.seq_lens.long() + self.attn.tree_sizes.long()).sum()) * cfg.num_kv_heads
+        alg = kv_rows * cfg.head_dim * 2 + int(self.attn.tree_sizes.long().sum()) * cfg.num_q_heads * cfg.head_dim * 4 + \
+            2 * 4 * cfg.batch * cfg.num_kv_heads
+        gbs = alg / (ms * 1e-3) / 1e9
+        return {"attn_kernel_ms": ms, "ratio_to_bf16": ms / attn_ms_bf16, "algorithmic_bytes": alg, "gbs": gbs, "hbm_frac": gbs / pk["hbm"],
+                "note": "e4m3 codes + fp32 scale per (sequence, KV head); codes widened exactly to bf16 in shared memory"}
+
     def free(self):
         self.sets = None
         self.out = self.ws = None
@@ -470,6 +498,9 @@ def main():
         per_layer = ctx.per_layer()
         per_layer["attn_kernel_share_of_layer"] = attn_ms / per_layer["ms_per_layer"]
 
+        # ---- the same attention over an fp8 copy of the cache (reported, not part of the headline)
+        fp8_kv = ctx.fp8_leg(attn_ms, pk)
+
         # ---- the same attention over a paged cache (reported, not part of the headline): the first input set's keys and
         # values cut into pages of 128 and of 16 slots, scattered over the pool by a seeded permutation
         ctx.step(0)
@@ -527,7 +558,7 @@ def main():
                                  "sequences_with_the_same_tokens_as_on_probabilities": logits_same, "of": B},
             "tree_expand": {"ms": expand_ms, "rows": B * R_exp, "children": K_exp, "bytes": expand_bytes,
                             "gbs": expand_bytes / (expand_ms * 1e-3) / 1e9, "note": "back-to-back calls on the same rows (warm L2)"},
-            "per_layer": per_layer, "paged_attention": paged,
+            "per_layer": per_layer, "fp8_kv": fp8_kv, "paged_attention": paged,
             "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
                           "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}})
     ctx.free()
@@ -578,6 +609,7 @@ def main():
             pl = o.per_layer()
             pl["attn_kernel_share_of_layer"] = a_ms / pl["ms_per_layer"]
             rec["per_layer"] = pl
+            rec["fp8_kv"] = o.fp8_leg(a_ms, pk)
             o.check()
             others[name] = rec
             o.free()

@@ -185,6 +185,26 @@ int eagle_tree_verify_attn_planned_paged(const eagle_attn_desc* desc, const void
                                          eagle_stream_t stream);
 
 /*
+ * The same attention over a cache STORED in fp8.  The decoding this method speeds up is bound by memory traffic (Sec. 4.4)
+ * and the paper reports the method on a quantised deployment (Sec. 4.2); it fixes no quantisation scheme, so the
+ * convention here is this library's: k_codes / v_codes are device uint8 [B, Hkv, S_cap, D] holding fp8 "e4m3" codes (1
+ * sign, 4 exponent, 3 mantissa bits, bias 7, no infinities), and every (sequence, KV head) has one fp32 scale for its keys
+ * and one for its values, k_scale / v_scale device fp32 [B, Hkv]:  key = value(code) * k_scale[b, h],  value =
+ * value(code) * v_scale[b, h].  Only the storage changes: the codes are widened exactly (every e4m3 number is a bf16
+ * number) on their way to the tensor cores, the keys' scale is folded into the softmax scale and the values' scale into
+ * the output, and everything else (queries in bf16, fp32 scores / softmax / accumulation, bf16 output, planner, work split,
+ * errors) is as for eagle_tree_verify_attn.  What it saves is half of the cache bytes read.  head_dim must be 128 and the
+ * cache contiguous (else EAGLE_ERR_SHAPE).  Slots that are not visible may hold any code; the two NaN codes (0x7f, 0xff)
+ * in a VISIBLE slot are not propagated as NaN (they are read as +-480 times the scale): do not store them.
+ * eagle_tree_verify_attn_planned_fp8 is the per-layer half over a plan made by eagle_tree_verify_plan (paged = NULL).
+ */
+int eagle_tree_verify_attn_fp8(const eagle_attn_desc* desc, const void* q, const void* k_codes, const void* v_codes,
+                               const float* k_scale, const float* v_scale, const int32_t* seq_lens, const int32_t* tree_parent,
+                               void* out, eagle_stream_t stream);
+int eagle_tree_verify_attn_planned_fp8(const eagle_attn_desc* desc, const void* q, const void* k_codes, const void* v_codes,
+                                       const float* k_scale, const float* v_scale, void* out, eagle_stream_t stream);
+
+/*
  * Where a plan keeps its tree masks (host function, no CUDA work): device uint64 [B, T_max] inside desc->workspace,
  * bit m of entry [b, i] set iff node m is node i or one of its ancestors (the mask tree attention implies, Sec. 3.1 /
  * 3.3); entries of nodes >= tree size and of invalid sequences are 0.  Valid after eagle_tree_verify_plan or

@@ -21,7 +21,8 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_accept_logits", "eagle_tree_expand", "eagle_tree_verify_attn_paged",
            "eagle_tree_commit_paged", "eagle_tree_verify_step_host_bytes", "eagle_tree_accept_cluster_width",
            "eagle_tree_verify_plan", "eagle_tree_verify_attn_planned", "eagle_tree_verify_attn_planned_paged",
-           "eagle_tree_verify_plan_masks", "eagle_set_wait_limit_ns", "eagle_test_stall_kv_producer"]
+           "eagle_tree_verify_plan_masks", "eagle_set_wait_limit_ns", "eagle_test_stall_kv_producer",
+           "eagle_tree_verify_attn_fp8", "eagle_tree_verify_attn_planned_fp8"]
 _lib = None
 
 
@@ -84,6 +85,10 @@ def load():
         lib.eagle_tree_verify_attn_static_capacity.restype = ctypes.c_size_t
         lib.eagle_tree_verify_attn_paged.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(PagedKV), vp, vp, vp, vp]
         lib.eagle_tree_verify_attn_paged.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_fp8.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 9
+        lib.eagle_tree_verify_attn_fp8.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_planned_fp8.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 7
+        lib.eagle_tree_verify_attn_planned_fp8.restype = ctypes.c_int
         lib.eagle_tree_verify_plan.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, ctypes.POINTER(PagedKV), vp]
         lib.eagle_tree_verify_plan.restype = ctypes.c_int
         lib.eagle_tree_verify_attn_planned.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp]
@@ -238,6 +243,32 @@ def eagle_tree_verify_attn_paged(q, k_pages, v_pages, block_table, seq_lens, tre
     return out
 
 
+def eagle_tree_verify_attn_fp8(q, k_codes, v_codes, k_scale, v_scale, seq_lens, tree_parent, out=None, *, tree_sizes=None,
+                               sm_scale=0.0, num_splits=0, workspace=None, status=None, events=None, shared_tree=False):
+    """Tree-masked attention over a cache stored as fp8 e4m3 codes: k_codes / v_codes uint8 [B,Hkv,S,D] (D = 128),
+    k_scale / v_scale fp32 [B,Hkv].  Everything else as for ``eagle_tree_verify_attn``."""
+    lib = load()
+    if q.dim() != 4 or k_codes.dim() != 4 or k_codes.shape != v_codes.shape:
+        raise EagleError("bad tensor ranks / shapes")
+    B, T, Hq, D = q.shape
+    Hkv = k_codes.shape[1]
+    if k_codes.shape[0] != B or k_codes.shape[3] != D or tuple(seq_lens.shape) != (B,) or tuple(k_scale.shape) != (B, Hkv) or \
+            tuple(v_scale.shape) != (B, Hkv):
+        raise EagleError("inconsistent shapes")
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = alloc_workspace(q, k_codes, num_splits)
+    d = _attn_desc(q, Hkv, k_codes.shape[2], tree_sizes, sm_scale, num_splits, workspace, status, events, shared_tree)
+    rc = lib.eagle_tree_verify_attn_fp8(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+                                        _dev(v_codes, torch.uint8, "v_codes"), _dev(k_scale, torch.float32, "k_scale"),
+                                        _dev(v_scale, torch.float32, "v_scale"), _dev(seq_lens, torch.int32, "seq_lens"),
+                                        _dev(tree_parent, torch.int32, "tree_parent"), _dev(out, torch.bfloat16, "out"), _stream())
+    _check(rc, "eagle_tree_verify_attn_fp8")
+    return out
+
+
 class VerifyPlan:
     """The plan of one verification pass (tree masks + work split), made once by ``eagle_tree_verify_plan`` and used by
     every layer's ``attend`` / ``attend_paged``.  Holds the descriptor fields and the workspace; marshalling only."""
@@ -275,6 +306,18 @@ class VerifyPlan:
         rc = load().eagle_tree_verify_attn_planned(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
                                                    _dev(v_cache, torch.bfloat16, "v_cache"), _dev(out, torch.bfloat16, "out"), _stream())
         _check(rc, "eagle_tree_verify_attn_planned")
+        return out
+
+    def attend_fp8(self, q, k_codes, v_codes, k_scale, v_scale, out=None, *, sm_scale=0.0, status=None, events=None):
+        if tuple(q.shape) != self.shape or k_codes.shape != v_codes.shape or k_codes.shape[2] != self.kv_capacity:
+            raise EagleError("tensors do not match the plan")
+        if out is None:
+            out = torch.empty_like(q)
+        d = self._desc(q.shape, sm_scale, status, events)
+        rc = load().eagle_tree_verify_attn_planned_fp8(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), _dev(k_codes, torch.uint8, "k_codes"),
+                                                       _dev(v_codes, torch.uint8, "v_codes"), _dev(k_scale, torch.float32, "k_scale"),
+                                                       _dev(v_scale, torch.float32, "v_scale"), _dev(out, torch.bfloat16, "out"), _stream())
+        _check(rc, "eagle_tree_verify_attn_planned_fp8")
         return out
 
     def attend_paged(self, q, k_pages, v_pages, block_table, out=None, *, sm_scale=0.0, status=None, events=None):

@@ -90,6 +90,8 @@ struct KvSource {
   int64_t capacity;             // slots per sequence
   const int32_t* block_table;   // null: contiguous
   int32_t num_pages, page_size, max_pages;
+  const float* k_scale = nullptr;   // non-null: k / v hold fp8 (e4m3) codes with these scales per (sequence, KV head)
+  const float* v_scale = nullptr;
 };
 
 // The planner launch: tree masks and work list into the workspace.  Depends on the lengths, the trees and the shape
@@ -176,6 +178,8 @@ int attend_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, Devi
   while (kv.block_table && (1 << ap.page_shift) < kv.page_size) ++ap.page_shift;
   ap.max_pages = kv.max_pages;
   ap.num_pages = kv.num_pages;
+  ap.k_scale = kv.k_scale;
+  ap.v_scale = kv.v_scale;
   ap.wait_limit_ns = g_wait_limit_ns.load(std::memory_order_relaxed);
   ap.stall_after_tiles = g_stall_after_tiles.load(std::memory_order_relaxed);
   if (d.ev_attn_begin && cudaEventRecord(static_cast<cudaEvent_t>(d.ev_attn_begin), stream) != cudaSuccess) return EAGLE_ERR_LAUNCH;
@@ -240,6 +244,29 @@ int eagle_tree_verify_attn_paged(const eagle_attn_desc* desc, const void* q, con
   int rc = EAGLE_OK;
   if (!paged_source(desc, pk, &kv, &rc)) return rc;
   return attention_with_workspace(desc, kPlanAndAttend, q, kv, seq_lens, tree_parent, out, stream_);
+}
+
+int eagle_tree_verify_attn_fp8(const eagle_attn_desc* desc, const void* q, const void* k_codes, const void* v_codes,
+                               const float* k_scale, const float* v_scale, const int32_t* seq_lens, const int32_t* tree_parent,
+                               void* out, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  if (desc->head_dim != 128) return EAGLE_ERR_SHAPE;
+  if (desc->batch > 0 && desc->max_tree > 0 && (!k_scale || !v_scale)) return EAGLE_ERR_NULL;
+  KvSource kv = {k_codes, v_codes, desc->kv_capacity, nullptr, 0, 0, 0};
+  kv.k_scale = k_scale;
+  kv.v_scale = v_scale;
+  return attention_with_workspace(desc, kPlanAndAttend, q, kv, seq_lens, tree_parent, out, stream_);
+}
+
+int eagle_tree_verify_attn_planned_fp8(const eagle_attn_desc* desc, const void* q, const void* k_codes, const void* v_codes,
+                                       const float* k_scale, const float* v_scale, void* out, eagle_stream_t stream_) {
+  if (!desc) return EAGLE_ERR_NULL;
+  if (desc->head_dim != 128) return EAGLE_ERR_SHAPE;
+  if (desc->batch > 0 && desc->max_tree > 0 && (!k_scale || !v_scale)) return EAGLE_ERR_NULL;
+  KvSource kv = {k_codes, v_codes, desc->kv_capacity, nullptr, 0, 0, 0};
+  kv.k_scale = k_scale;
+  kv.v_scale = v_scale;
+  return attention_with_workspace(desc, kAttendOnly, q, kv, nullptr, nullptr, out, stream_);
 }
 
 int eagle_tree_verify_plan(const eagle_attn_desc* desc, const int32_t* seq_lens, const int32_t* tree_parent,

@@ -28,9 +28,14 @@ namespace eagle {
 namespace {
 
 constexpr int kTileN = 128;          // keys per KV tile
-constexpr int kSlots = 6;            // ring slots; entry n of the load sequence (see the producer) uses slot n % 6
+// Ring slots of K/V tiles; entry n of the load sequence (see the producer) uses slot n % slots.  A cache stored as fp8
+// codes has four slots of bf16 tiles plus four staging slots of raw codes instead of six slots.
+template <bool FP8>
+constexpr int slots_of() { return FP8 ? 4 : 6; }
 constexpr int kSBufs = 3;            // score buffers in tensor memory; step g uses buffer g % 3
 constexpr int kThreads = 384;          // 8 softmax warps, K/V producer, two MMA issuers, Q producer
+constexpr int kThreadsFp8 = 512;       // the same plus four warps that widen fp8 codes to bf16 tiles
+constexpr int kWarpConvert = 12;
 constexpr int kSoftmaxWarps = 8;
 constexpr int kGroupThreads = 128;     // one softmax group
 constexpr int kWarpProducer = 8, kWarpQK = 9, kWarpPV = 10, kWarpQ = 11;
@@ -325,23 +330,27 @@ __device__ __forceinline__ void issue_pv_tile(uint32_t o_tmem, uint32_t p_tmem, 
       ::"r"(o_tmem), "r"(p_tmem), "r"(v_lo), "r"(idesc), "r"(kDescHi), "r"(acc0) : "memory");
 }
 
-template <int D>
+template <int D, bool FP8>
 struct Smem {
+  static constexpr int kSlots = slots_of<FP8>();
   static constexpr int kSlabs = D / 64;                     // 64 bf16 = one 128-byte swizzled row
   static constexpr int kSlabBytes = kTileN * 128;            // 128 rows x 128 bytes
   static constexpr int kTileBytes = kSlabs * kSlabBytes;     // one Q / K / V tile
+  static constexpr int kCodeBytes = kTileN * D;              // one K / V tile of fp8 codes (128 rows x D bytes)
   static constexpr int kQ = 0;                               // the query tile of the current item
   static constexpr int kRing = kTileBytes;
-  static constexpr int kTag = kRing + kSlots * kTileBytes;   // uint32 [128 rows]: reference maximum | step number
+  static constexpr int kStage = kRing + kSlots * kTileBytes; // fp8 only: raw code tiles on their way to the ring
+  static constexpr int kTag = kStage + (FP8 ? kSlots * kCodeBytes : 0);   // uint32 [128 rows]: reference maximum | step number
   static constexpr int kLfin = kTag + kBlockM * 4;           // float [128 rows]: row sums on their way to the epilogue
   static constexpr int kBar = kLfin + kBlockM * 4;
-  static constexpr int kNumBars = 2 * kSlots + 3 * kSBufs + 3;
+  static constexpr int kNumBars = 2 * kSlots + 3 * kSBufs + 3 + (FP8 ? 2 * kSlots : 0);
   static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag, wait limit (8 bytes)
   static constexpr int kBytes = kMisc + 16;
 };
 
 // The mbarriers sit next to one another in shared memory; their addresses are computed, not stored (an array of
 // addresses indexed at run time would live in local memory).
+template <int kSlots>
 struct Bars {
   uint32_t base;
   __device__ __forceinline__ uint32_t full(uint32_t i) const { return base + 8u * i; }
@@ -352,13 +361,18 @@ struct Bars {
   __device__ __forceinline__ uint32_t q_full() const { return base + 8u * (2 * kSlots + 3 * kSBufs); }
   __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 1); }
   __device__ __forceinline__ uint32_t o_free() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 2); }
+  // fp8 only: a staging slot holds a tile of codes / the converter warps are done with it
+  __device__ __forceinline__ uint32_t st_full(uint32_t i) const { return base + 8u * (2 * kSlots + 3 * kSBufs + 3 + i); }
+  __device__ __forceinline__ uint32_t st_empty(uint32_t i) const { return base + 8u * (3 * kSlots + 3 * kSBufs + 3 + i); }
 };
 
-template <int D, bool PAGED>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int D, bool PAGED, bool FP8>
+__global__ void __launch_bounds__(FP8 ? kThreadsFp8 : kThreads, 1)
 attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
             const __grid_constant__ CUtensorMap map_q) {
-  using S = Smem<D>;
+  static_assert(!(FP8 && PAGED) && !(FP8 && D != 128), "the fp8 cache form is built for contiguous caches with 128-wide heads");
+  using S = Smem<D, FP8>;
+  constexpr int kSlots = S::kSlots;
   extern __shared__ __align__(1024) unsigned char smem[];
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -367,7 +381,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     return;
   }
 
-  Bars B;
+  Bars<kSlots> B;
   B.base = sbase + S::kBar;
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(smem + S::kMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + S::kMisc + 4);
@@ -378,8 +392,12 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
     for (int i = 0; i < kSlots; ++i) {
-      mbar_init(B.full(i), 1);
+      mbar_init(B.full(i), FP8 ? kGroupThreads : 1);   // one TMA transaction, or every thread of the converter warps
       mbar_init(B.empty(i), 1);
+      if constexpr (FP8) {
+        mbar_init(B.st_full(i), 1);
+        mbar_init(B.st_empty(i), kGroupThreads);
+      }
     }
     for (int i = 0; i < kSBufs; ++i) {
       mbar_init(B.s_full(i), 1);
@@ -513,6 +531,12 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       const bool row_valid = R < m_valid;
       const int node = row_valid ? R / G : 0, hh = row_valid ? R % G : 0;
       const uint64_t anc = row_valid ? p.anc[static_cast<size_t>(it.b) * p.T_max + node] : 0ull;
+      // fp8 cache: the keys' scale of this (sequence, KV head) goes into the softmax scale, the values' into the output
+      float scale_log2 = p.scale_log2, v_scale = 1.f;
+      if constexpr (FP8) {
+        scale_log2 *= p.k_scale[it.b * p.Hkv + it.g];
+        v_scale = p.v_scale[it.b * p.Hkv + it.g];
+      }
 
       if (!p.q_tma && grp == 0) {
         // group sizes that do not divide 128: the first softmax group stages the query tile itself, a row per thread
@@ -559,9 +583,42 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         }
         // ---- pass 1: row maximum of the raw scores.  All four chunks are fetched in one round trip to tensor memory;
         // chunks 0 and 1 stay in registers for pass 2, chunks 2 and 3 are dropped after the maximum and fetched again
-        // later (keeping them would leave too few registers for pass 2).
+        // later (keeping them would leave too few registers for pass 2).  (With an fp8 cache the CTA has 512 threads and
+        // 128 registers each: two round trips, chunks 2 and 3 first, then chunks 0 and 1, which stay.)
         uint32_t ra[32], rb[32];
         float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if constexpr (FP8) {
+          tmem_ld32(s_addr + 64, ra);
+          tmem_ld32(s_addr + 96, rb);
+          tc_wait_ld();
+          if (tail) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              ra[e] = (vm[2] >> e) & 1u ? ra[e] : 0xff800000u;       // -inf
+              rb[e] = (vm[3] >> e) & 1u ? rb[e] : 0xff800000u;
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            mx[0] = max3(mx[0], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            mx[1] = max3(mx[1], __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+          }
+          tmem_ld32(s_addr, ra);
+          tmem_ld32(s_addr + 32, rb);
+          tc_wait_ld();
+          if (tail) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              ra[e] = (vm[0] >> e) & 1u ? ra[e] : 0xff800000u;
+              rb[e] = (vm[1] >> e) & 1u ? rb[e] : 0xff800000u;
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            mx[2] = max3(mx[2], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            mx[3] = max3(mx[3], __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+          }
+        } else
         {
           uint32_t rc[32], rd[32];
           tmem_ld32(s_addr + 64, rc);
@@ -586,7 +643,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             mx[3] = max3(mx[3], __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
           }
         }
-        const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;   // scale > 0
+        const float tmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;   // scale > 0
 
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
@@ -644,7 +701,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         // ---- pass 2: exponentials and packed P, in column order (P overwrites score columns that have been
         // consumed).  Chunks 0 and 1 are still in registers; chunks 2 and 3 are fetched again meanwhile.
         const float neg_base = m_ref == -INFINITY ? 0.f : -m_ref;
-        const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), base2 = pack2(neg_base, neg_base);
+        const uint64_t scale2 = pack2(scale_log2, scale_log2), base2 = pack2(neg_base, neg_base);
         uint64_t ls2[2] = {0ull, 0ull};   // four partial sums
         uint32_t pk[16];
         auto exp_chunk = [&](const uint32_t* raw, int c) {
@@ -711,7 +768,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             const float w = m_in == m_ref ? 1.f : fast_exp2(m_in - m_ref);
             l_row = fmaf(*lfin, w, l_row);
           }
-          const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+          const float inv = l_row > 0.f ? v_scale / l_row : 0.f;   // (v_scale is 1 unless the cache is fp8)
           uint32_t o[32];
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
@@ -731,6 +788,10 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
                 }
               } else {
                 float* part_row = p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D;
+                if constexpr (FP8) {
+#pragma unroll
+                  for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * v_scale);
+                }
 #pragma unroll
                 for (int e = 0; e < 32; e += 4)
                   *reinterpret_cast<uint4*>(part_row + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
@@ -829,6 +890,12 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           if (r0 < kTileN)
             tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
                         key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
+        } else if constexpr (FP8) {
+          // the tile of codes goes to the staging slot; the converter warps widen it into ring slot `slot`
+          ok = mbar_wait(B.st_empty(slot), par, s_abort);
+          if (!ok) return;
+          mbar_expect_tx(B.st_full(slot), S::kCodeBytes);
+          tma_load_3d(sbase + S::kStage + slot * S::kCodeBytes, is_v ? &map_v : &map_k, 0, c.tile * kTileN, c.z, B.st_full(slot));
         } else {
           ok = mbar_wait(B.empty(slot), par, s_abort);
           if (!ok) return;
@@ -857,6 +924,61 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           advance(ck);
         }
         ++n;
+      }
+    }
+  } else if (FP8 && warp >= kWarpConvert) {
+    // =========================================================================== fp8 -> bf16 converter (warps 12-15)
+    // Thread r owns row r of every K / V tile: it reads the row's 128 codes from the staging slot (eight 16-byte chunks,
+    // 128-byte swizzled as the copy laid them down), widens them, and writes the row's 256 bytes into the ring slot in
+    // the swizzled two-slab layout the MMAs read.  Every e4m3 number is a bf16 number, so this is exact: the code's
+    // exponent and mantissa bits are moved into place (which leaves the value 2^-120 times too small, subnormals
+    // included) and one bf16 multiplication by 2^120 restores it.  The scales are applied elsewhere.
+    if constexpr (FP8) {
+      const int r = tid & (kBlockM - 1);
+      uint32_t steps_total = 0;     // this CTA's steps over all its items
+      for (int tp = tp_lo; tp < tp_hi; ++tp) {
+        const WorkItem it = p.items[2 * tp + member];
+        if (it.tile_end > it.tile_begin) steps_total += static_cast<uint32_t>(it.tile_end - it.tile_begin);
+      }
+      const __nv_bfloat162 two120 = __halves2bfloat162(__ushort_as_bfloat16(0x7B80), __ushort_as_bfloat16(0x7B80));
+      auto widen = [&](uint32_t w, uint32_t& lo, uint32_t& hi) {
+        const uint32_t m = w & 0x7f7f7f7fu, sg = w & 0x80808080u;
+        uint32_t a = (__byte_perm(m, 0u, 0x4140) << 4) | __byte_perm(sg, 0u, 0x1404);   // codes 0 and 1 of the word
+        uint32_t b = (__byte_perm(m, 0u, 0x4342) << 4) | __byte_perm(sg, 0u, 0x3424);   // codes 2 and 3
+        __nv_bfloat162 x = __hmul2(*reinterpret_cast<__nv_bfloat162*>(&a), two120);
+        __nv_bfloat162 y = __hmul2(*reinterpret_cast<__nv_bfloat162*>(&b), two120);
+        lo = *reinterpret_cast<uint32_t*>(&x);
+        hi = *reinterpret_cast<uint32_t*>(&y);
+      };
+      // Entry n of the load sequence is K(n) for n < 3, V((n - 3) / 2) for odd n and K((n + 2) / 2) for even n after
+      // that; the K entries of the last three steps do not exist (the producer skips them, the numbering keeps its gaps).
+      bool ok = true;
+      uint32_t slot = 0, par = 0;
+      const uint32_t n_end = steps_total ? 2u * steps_total + 2u : 0u;
+      for (uint32_t n = 0; n < n_end && ok; ++n, slot = (slot + 1 == kSlots ? 0 : slot + 1), par ^= (slot == 0 ? 1u : 0u)) {
+        const uint32_t g = n < 3 ? n : ((n & 1u) ? (n - 3u) / 2u : (n + 2u) / 2u);
+        if (g >= steps_total) continue;
+        ok = mbar_wait_warp(B.st_full(slot), par, s_abort);
+        if (!ok) break;
+        ok = mbar_wait_warp(B.empty(slot), par ^ 1u, s_abort);    // the MMA that read the ring slot last has finished
+        if (!ok) break;
+        const unsigned char* src = smem + S::kStage + slot * S::kCodeBytes + r * 128;
+        unsigned char* dst = smem + S::kRing + slot * S::kTileBytes + r * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {                              // codes 16c .. 16c + 15 of the row
+          const uint4 w = *reinterpret_cast<const uint4*>(src + ((c ^ (r & 7)) << 4));
+          uint4 u, v;
+          widen(w.x, u.x, u.y);
+          widen(w.y, u.z, u.w);
+          widen(w.z, v.x, v.y);
+          widen(w.w, v.z, v.w);
+          unsigned char* d = dst + (c >> 2) * S::kSlabBytes;       // 64 columns per slab: chunks 2c and 2c + 1 of the slab's row
+          *reinterpret_cast<uint4*>(d + ((((2 * c) & 7) ^ (r & 7)) << 4)) = u;
+          *reinterpret_cast<uint4*>(d + ((((2 * c + 1) & 7) ^ (r & 7)) << 4)) = v;
+        }
+        fence_proxy_async();                                       // the MMAs read the slot through the async proxy
+        mbar_arrive(B.full(slot));
+        mbar_arrive(B.st_empty(slot));
       }
     }
   }
@@ -901,6 +1023,18 @@ bool make_kv_map(CUtensorMap* map, const void* base, int D, int S_cap, long long
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A cache of fp8 codes [B*Hkv, S_cap, D] uint8: box = D x 128 rows x 1 (D = 128: one 128-byte swizzled row per slot).
+bool make_code_map(CUtensorMap* map, const void* base, int D, int S_cap, long long bh) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S_cap), static_cast<cuuint64_t>(bh)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S_cap) * D};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(D), static_cast<cuuint32_t>(kTileN), 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // q [B, T_max, Hq, D] bf16 viewed as (d, head, node, sequence); box = 64 x G x 128/G x 1: the 128 query rows of one
 // (sequence, KV head, query tile) in (node, head-in-group) order.  Needs 128 % G == 0.
 bool make_q_map(CUtensorMap* map, const void* base, int D, int Hq, int T_max, int B, int G) {
@@ -923,21 +1057,27 @@ int attn_tile_keys() { return kTileN; }
 cudaError_t attn_prepare(int head_dim) {
   cudaError_t e;
   if (head_dim == 128) {
-    e = cudaFuncSetAttribute(attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kBytes);
+    e = cudaFuncSetAttribute(attn_kernel<128, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128, false>::kBytes);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::kBytes);
+    e = cudaFuncSetAttribute(attn_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128, true>::kBytes);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(attn_kernel<128, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128, false>::kBytes);
   }
-  e = cudaFuncSetAttribute(attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
+  e = cudaFuncSetAttribute(attn_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64, false>::kBytes);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::kBytes);
+  return cudaFuncSetAttribute(attn_kernel<64, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64, false>::kBytes);
 }
 
 // Returns cudaErrorInvalidValue when the tensor maps cannot be encoded.
 cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t stream) {
   AttnParams p = p_in;
   CUtensorMap mk, mv, mq;
-  const bool paged = p.page_size > 0;
-  if (paged) {
+  const bool paged = p.page_size > 0, fp8 = p.k_scale != nullptr;
+  if (fp8) {
+    if (paged || p.D != 128) return cudaErrorInvalidValue;
+    const long long bh = static_cast<long long>(p.B) * p.Hkv;
+    if (!make_code_map(&mk, p.k, p.D, p.S_cap, bh) || !make_code_map(&mv, p.v, p.D, p.S_cap, bh)) return cudaErrorInvalidValue;
+  } else if (paged) {
     const long long ph = static_cast<long long>(p.num_pages) * p.Hkv;
     const int rows = p.page_size < kTileN ? p.page_size : kTileN;
     if (!make_kv_map(&mk, p.k, p.D, p.page_size, ph, rows) || !make_kv_map(&mv, p.v, p.D, p.page_size, ph, rows)) return cudaErrorInvalidValue;
@@ -951,12 +1091,14 @@ cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t strea
   } else {
     mq = mk;   // unused by the kernel
   }
-  if (p.D == 128) {
-    if (paged) attn_kernel<128, true><<<num_ctas, kThreads, Smem<128>::kBytes, stream>>>(p, mk, mv, mq);
-    else attn_kernel<128, false><<<num_ctas, kThreads, Smem<128>::kBytes, stream>>>(p, mk, mv, mq);
+  if (fp8) {
+    attn_kernel<128, false, true><<<num_ctas, kThreadsFp8, Smem<128, true>::kBytes, stream>>>(p, mk, mv, mq);
+  } else if (p.D == 128) {
+    if (paged) attn_kernel<128, true, false><<<num_ctas, kThreads, Smem<128, false>::kBytes, stream>>>(p, mk, mv, mq);
+    else attn_kernel<128, false, false><<<num_ctas, kThreads, Smem<128, false>::kBytes, stream>>>(p, mk, mv, mq);
   } else {
-    if (paged) attn_kernel<64, true><<<num_ctas, kThreads, Smem<64>::kBytes, stream>>>(p, mk, mv, mq);
-    else attn_kernel<64, false><<<num_ctas, kThreads, Smem<64>::kBytes, stream>>>(p, mk, mv, mq);
+    if (paged) attn_kernel<64, true, false><<<num_ctas, kThreads, Smem<64, false>::kBytes, stream>>>(p, mk, mv, mq);
+    else attn_kernel<64, false, false><<<num_ctas, kThreads, Smem<64, false>::kBytes, stream>>>(p, mk, mv, mq);
   }
   count_launch();
   return cudaGetLastError();

@@ -142,6 +142,10 @@ struct AttnParams {
   // page block_table[b * max_pages + j / page_size]; page_size is a power of two
   const int32_t* block_table;
   int32_t page_size, page_shift, max_pages, num_pages;
+  // cache stored as fp8 (e4m3) codes: k / v point to uint8 [B, Hkv, S_cap, D] and every (sequence, KV head) has one scale
+  // for its keys and one for its values, fp32 [B, Hkv] (null: the cache is bf16)
+  const float* k_scale;
+  const float* v_scale;
   unsigned long long wait_limit_ns;   // a wait that makes no progress for this long aborts the CTA (EAGLE_ERR_TIMEOUT)
   int32_t stall_after_tiles;          // test hook: the K/V producer stops issuing after this many tiles (negative: off)
 };

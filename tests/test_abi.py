@@ -19,7 +19,7 @@ def lib():
 def test_every_declared_symbol_is_exported(lib):
     from paper_2401_15077_b200 import binding
     header = (ROOT / "include" / "eagle_verify.h").read_text()
-    declared = set(re.findall(r"\b(eagle_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(eagle_[a-z0-9_]+)\s*\(", header))
     assert declared == set(binding.EXPORTS)
     for name in declared:
         assert getattr(lib, name) is not None

@@ -1,0 +1,149 @@
+"""Parity of the tree attention over an fp8 (e4m3) cache (through the C ABI) with the oracle's fp8 form.  Needs a B200.
+
+Only the storage differs from the bf16 call: the codes are widened exactly, the scales are applied in fp32, so the same
+bounds hold against the oracle evaluated on the same codes and scales."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2401_15077_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2401_15077_b200 import build, binding
+    build.build()
+    binding.load()
+    assert torch.cuda.is_available()
+    return binding
+
+
+def _run(E, inp, f8, num_splits=0, sm_scale=0.0):
+    d = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    out = torch.full(inp.q.shape, float("nan"), dtype=torch.bfloat16, device=d)
+    E.eagle_tree_verify_attn_fp8(inp.q.to(d), f8.k_codes.to(d), f8.v_codes.to(d), f8.k_scale.to(d), f8.v_scale.to(d), inp.seq_lens.to(d),
+                                 inp.tree_parent.to(d), out, tree_sizes=inp.tree_sizes.to(d), num_splits=num_splits, status=status,
+                                 sm_scale=sm_scale)
+    torch.cuda.synchronize()
+    return out.cpu(), int(status.item())
+
+
+def _check(out, ref, sizes, scale=1.0):
+    got = out.double().numpy()
+    assert np.isfinite(got).all()
+    rows = np.zeros(ref.shape[:2], bool)
+    for b, n in enumerate(sizes):
+        rows[b, :int(n)] = True
+        assert np.all(got[b, int(n):] == 0.0)
+    if rows.any():
+        err = np.abs(got - ref)[rows]
+        assert err.max() <= MAX_ABS * scale and err.mean() <= MEAN_ABS * scale, (err.max(), err.mean())
+
+
+CASES = {
+    "7b_mha": W.CONFIGS["7b_mha"],
+    "70b_gqa_b2": W.scaled(W.CONFIGS["70b_gqa"], batch=2),
+    "mixtral_gqa_small": W.scaled(W.CONFIGS["mixtral_gqa"], batch=2, prefix=(1500, 3000)),
+    "serving_mix_small": W.scaled(W.CONFIGS["serving_mix"], batch=6, prefix=(100, 1500)),
+    "ragged_small_trees": W.scaled(W.CONFIGS["7b_mha"], batch=5, num_q_heads=16, num_kv_heads=4, prefix=(0, 700), tree=(0, 33)),
+    "group3": W.scaled(W.CONFIGS["7b_mha"], batch=3, num_q_heads=12, num_kv_heads=4, prefix=(50, 1200), tree=(3, 64), max_depth=8),
+    "odd_heads": W.scaled(W.CONFIGS["7b_mha"], batch=4, num_q_heads=12, num_kv_heads=3, prefix=(300, 2500), tree=(5, 30), max_depth=8),
+    "five_heads_three_tiles": W.scaled(W.CONFIGS["70b_gqa"], batch=2, num_q_heads=40, num_kv_heads=5, prefix=(400, 1500), tree=(40, 48)),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_fp8_attention_matches_oracle(E, oracle, name):
+    cfg = CASES[name]
+    inp = W.make_attn_inputs(cfg, salt=3, capacity_pad=19)
+    f8 = W.make_fp8_cache(inp)
+    ref = oracle.tree_verify_attn_fp8(inp.q, f8.k_codes, f8.v_codes, f8.k_scale, f8.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    for splits in (0, 3):
+        out, status = _run(E, inp, f8, num_splits=splits)
+        assert status == 0
+        _check(out, ref, inp.tree_sizes)
+    again, _ = _run(E, inp, f8, num_splits=3)
+    assert torch.equal(out.view(torch.int16), again.view(torch.int16))
+
+
+def test_every_code_is_widened_exactly(E, oracle):
+    """Keys of zeros (uniform softmax) and values that run through all 254 number codes, subnormals included: the output
+    is the mean of the decoded values, so a wrongly widened code shows.  Large and small scales per head."""
+    cfg = W.scaled(W.CONFIGS["7b_mha"], batch=2, num_q_heads=4, num_kv_heads=2, prefix=(508, 508), tree=(4, 4))
+    inp = W.make_attn_inputs(cfg, salt=1)
+    S = inp.k_cache.shape[2]
+    codes = torch.tensor([c for c in range(256) if c not in (0x7F, 0xFF)], dtype=torch.uint8)
+    g = torch.Generator().manual_seed(9)
+    v_codes = codes[torch.randint(0, 254, (2, 2, S, 128), generator=g)]
+    # column d of slot j holds a code that depends on (j + d): every column's mean runs over all codes
+    k_codes = torch.zeros((2, 2, S, 128), dtype=torch.uint8)
+    k_scale = torch.ones((2, 2))
+    v_scale = torch.tensor([[1.0, 2.0 ** -7], [3.0, 0.011]])
+    f8 = W.Fp8KV(k_codes, v_codes, k_scale, v_scale)
+    ref = oracle.tree_verify_attn_fp8(inp.q, k_codes, v_codes, k_scale, v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    out, status = _run(E, inp, f8)
+    assert status == 0
+    got = out.double().numpy()
+    for b in range(2):
+        for h in range(4):
+            s = float(v_scale[b, h // 2])
+            err = np.abs(got[b, :4, h] - ref[b, :4, h])
+            assert err.max() <= 2e-2 * s * 16, (b, h, err.max())         # values up to 448 * scale: bf16 rounding of means ~ 10 * scale
+            assert err.max() <= np.abs(ref[b, :4, h]).max() * 2.0 ** -7 + 1e-6 * s
+    # only subnormal codes (|value| <= 7 * 2^-9): a flush to zero in the widening would return zeros
+    sub = torch.tensor([1, 2, 3, 4, 5, 6, 7], dtype=torch.uint8)
+    v_sub = sub[torch.randint(0, 7, (2, 2, S, 128), generator=g)]
+    f8s = W.Fp8KV(k_codes, v_sub, k_scale, torch.full((2, 2), 64.0))
+    ref = oracle.tree_verify_attn_fp8(inp.q, k_codes, v_sub, k_scale, f8s.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    out, status = _run(E, inp, f8s)
+    got = out.double().numpy()[:, :4]
+    assert status == 0 and ref[:, :4].min() > 0.3 and np.abs(got - ref[:, :4]).max() <= 2e-2
+
+
+def test_fp8_plan_once_attend_many(E, oracle):
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=7, prefix=(30, 2000), tree=(0, 64), max_depth=64)
+    inp = W.make_attn_inputs(cfg, salt=5)
+    f8 = W.make_fp8_cache(inp)
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    plan = E.eagle_tree_verify_plan(tuple(inp.q.shape), cfg.num_kv_heads, inp.k_cache.shape[2], inp.seq_lens.to(d), inp.tree_parent.to(d),
+                                    tree_sizes=inp.tree_sizes.to(d), status=status)
+    out = plan.attend_fp8(inp.q.to(d), f8.k_codes.to(d), f8.v_codes.to(d), f8.k_scale.to(d), f8.v_scale.to(d), status=status)
+    torch.cuda.synchronize()
+    whole, st = _run(E, inp, f8)
+    assert st == 0 and int(status.item()) == 0 and torch.equal(out.cpu().view(torch.int16), whole.view(torch.int16))
+    ref = oracle.tree_verify_attn_fp8(inp.q, f8.k_codes, f8.v_codes, f8.k_scale, f8.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    _check(whole, ref, inp.tree_sizes)
+
+
+def test_fp8_full_size_mixtral_sampled(E, oracle):
+    cfg = W.CONFIGS["mixtral_gqa"]
+    inp = W.make_attn_inputs(cfg)
+    f8 = W.make_fp8_cache(inp)
+    out, status = _run(E, inp, f8)
+    assert status == 0
+    got = out.double().numpy()
+    assert np.isfinite(got).all()
+    G = cfg.num_q_heads // cfg.num_kv_heads
+    for b, g in [(0, 0), (7, 7), (3, 5)]:
+        n, end = int(inp.tree_sizes[b]), int(inp.seq_lens[b] + inp.tree_sizes[b])
+        ref = oracle.tree_verify_attn_fp8(inp.q[b:b + 1, :, g * G:(g + 1) * G].contiguous(), f8.k_codes[b:b + 1, g:g + 1, :end].contiguous(),
+                                          f8.v_codes[b:b + 1, g:g + 1, :end].contiguous(), f8.k_scale[b:b + 1, g:g + 1].contiguous(),
+                                          f8.v_scale[b:b + 1, g:g + 1].contiguous(), inp.seq_lens[b:b + 1], inp.tree_parent[b:b + 1],
+                                          inp.tree_sizes[b:b + 1])
+        err = np.abs(got[b, :n, g * G:(g + 1) * G] - ref[0, :n])
+        assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, (b, g, err.max(), err.mean())
+
+
+def test_fp8_refuses_unsupported_shapes(E):
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["tiny"], batch=1)                     # head_dim 64
+    inp = W.make_attn_inputs(cfg)
+    f8 = W.make_fp8_cache(inp)
+    with pytest.raises(E.EagleError):
+        E.eagle_tree_verify_attn_fp8(inp.q.to(d), f8.k_codes.to(d), f8.v_codes.to(d), f8.k_scale.to(d), f8.v_scale.to(d),
+                                     inp.seq_lens.to(d), inp.tree_parent.to(d))
