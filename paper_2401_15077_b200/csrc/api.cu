@@ -15,7 +15,7 @@ namespace {
 // Planner cost model, in KV-tile positions: what starting an item costs the attention kernel (pipeline fill, output
 // write), and how close to a super-unit's edge a share boundary snaps to the edge.
 #ifndef EAGLE_ITEM_OVERHEAD
-#define EAGLE_ITEM_OVERHEAD 5
+#define EAGLE_ITEM_OVERHEAD 6
 #endif
 #ifndef EAGLE_SNAP_TILES
 #define EAGLE_SNAP_TILES 2

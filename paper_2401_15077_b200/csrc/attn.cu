@@ -10,8 +10,8 @@
 // Warp roles: warps 0-7 softmax, as two groups of four warps that take alternate steps (one query row = one
 // TMEM lane per thread, all 128 score columns), so that one group computes while the other waits; warp 8 K/V
 // producer (TMA, 128-byte swizzled boxes, ring of six 32 KB slots, tiles requested in the order the MMAs consume
-// them); warp 9 issues the QK MMAs, warp 10 the PV MMAs; warp 11 fetches the query tile of the next item once the
-// last score MMA of the current one has finished.  The group that takes an item's last step writes its output
+// them); warp 9 issues the QK MMAs (and fetches the query tile of the next item once the last score MMA of the
+// current one has finished), warp 10 the PV MMAs.  The group that takes an item's last step writes its output
 // while the other group is already on the next item.  Softmax is fp32 in the log2 domain with two-wide FP32
 // instructions; part of the exponentials is a polynomial on the FMA pipe.  The tree mask is applied in registers
 // only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are zeroed in shared
@@ -33,14 +33,17 @@ constexpr int kTileN = 128;          // keys per KV tile
 template <bool FP8>
 constexpr int slots_of() { return FP8 ? 4 : 6; }
 constexpr int kSBufs = 3;            // score buffers in tensor memory; step g uses buffer g % 3
-constexpr int kThreads = 384;          // 8 softmax warps, K/V producer, two MMA issuers, Q producer
-constexpr int kThreadsFp8 = 512;       // the same plus four warps that widen fp8 codes to bf16 tiles
-constexpr int kWarpConvert = 12;
+constexpr int kThreads = 352;          // 8 softmax warps, K/V producer, two MMA issuers: 186 registers for every thread
+constexpr int kThreadsFp8 = 480;       // the same plus four warps that widen fp8 codes to bf16 tiles
+constexpr int kWarpConvert = 11;
 constexpr int kSoftmaxWarps = 8;
 constexpr int kGroupThreads = 128;     // one softmax group
-constexpr int kWarpProducer = 8, kWarpQK = 9, kWarpPV = 10, kWarpQ = 11;
+constexpr int kWarpProducer = 8, kWarpQK = 9, kWarpPV = 10;
+// One pair of exponentials in three goes through the polynomial.  The softmax loop runs at the register limit (three
+// warps per scheduler: 168 registers): a variant that spills even a few values is a fifth slower, and shares of 1/4 and
+// below (more exponentials in flight on the special-function unit) or 1/2 with the masking code in the loop did.
 #ifndef EAGLE_POLY_STRIDE
-#define EAGLE_POLY_STRIDE 2
+#define EAGLE_POLY_STRIDE 3
 #endif
 constexpr int kPolyStride = EAGLE_POLY_STRIDE;   // one pair of exponentials in kPolyStride is evaluated as a polynomial (0: none)
 constexpr uint32_t kTmemCols = 512;
@@ -444,6 +447,17 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         const WorkItem it = p.items[2 * tp + member];
         if (it.tile_end <= it.tile_begin) continue;
         const int steps = it.tile_end - it.tile_begin;
+        if (p.q_tma) {
+          // This thread also fetches the item's query tile, as soon as the last score MMA of the item before has
+          // finished with the single 32 KB buffer (the softmax groups still have two or three steps of that item to work
+          // through meanwhile): box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order.
+          ok = mbar_wait(B.q_empty(), (item_count & 1u) ^ 1u, s_abort);
+          if (!ok) break;
+          mbar_expect_tx(B.q_full(), S::kTileBytes);
+#pragma unroll
+          for (int sl = 0; sl < S::kSlabs; ++sl)
+            tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full());
+        }
         ok = mbar_wait(B.q_full(), item_count & 1u, s_abort);
         if (!ok) break;
         for (int s = 0; s < steps && ok; ++s, ++gq) {
@@ -565,21 +579,29 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (!ok) break;
         tc_fence_after();
         const int key0 = (it.tile_begin + s) * kTileN;
-        // visibility of this row's 128 keys, 32 per word: keys before L are all visible, key L + m is visible iff
-        // bit m of the node's ancestor mask is set (the mask has no bits at or above the tree size)
-        const bool tail = key0 + kTileN > L;          // the tile reaches past the committed prefix
-        uint32_t vm[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
-        if (tail) {
-#pragma unroll
+        // Tiles that reach past the committed prefix (an item's last one or two): a compact pre-pass writes -inf over the
+        // scores of this row's invisible keys in tensor memory, so that the two passes below carry no masking code (the
+        // loop they form has to stay small: the instruction cache decides a fifth of this kernel's speed).  Keys before L
+        // are all visible; key L + m is visible iff bit m of the node's ancestor mask is set (the mask has no bits at or
+        // above the tree size).
+        if (key0 + kTileN > L) {
+#pragma unroll 1
           for (int c = 0; c < 4; ++c) {
-            const int rel = key0 + c * 32 - L;        // tree index of the word's first key (negative: still in the prefix)
+            const int rel = key0 + c * 32 - L;        // tree index of the chunk's first key (negative: still in the prefix)
             uint32_t w;
             if (rel >= 64) w = 0u;
             else if (rel >= 0) w = static_cast<uint32_t>(anc >> rel);
             else if (rel > -32) w = static_cast<uint32_t>(anc << (-rel)) | ((1u << (-rel)) - 1u);
             else w = 0xffffffffu;
-            vm[c] = w;
+            if (rel <= -32) continue;                 // wholly in the prefix (uniform over the warp: the loads below are collective)
+            uint32_t t[32];
+            tmem_ld32(s_addr + c * 32, t);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) t[e] = (w >> e) & 1u ? t[e] : 0xff800000u;       // -inf
+            tmem_st32(s_addr + c * 32, t);
           }
+          tc_wait_st();
         }
         // ---- pass 1: row maximum of the raw scores.  All four chunks are fetched in one round trip to tensor memory;
         // chunks 0 and 1 stay in registers for pass 2, chunks 2 and 3 are dropped after the maximum and fetched again
@@ -591,13 +613,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           tmem_ld32(s_addr + 64, ra);
           tmem_ld32(s_addr + 96, rb);
           tc_wait_ld();
-          if (tail) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              ra[e] = (vm[2] >> e) & 1u ? ra[e] : 0xff800000u;       // -inf
-              rb[e] = (vm[3] >> e) & 1u ? rb[e] : 0xff800000u;
-            }
-          }
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             mx[0] = max3(mx[0], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
@@ -606,13 +621,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           tmem_ld32(s_addr, ra);
           tmem_ld32(s_addr + 32, rb);
           tc_wait_ld();
-          if (tail) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              ra[e] = (vm[0] >> e) & 1u ? ra[e] : 0xff800000u;
-              rb[e] = (vm[1] >> e) & 1u ? rb[e] : 0xff800000u;
-            }
-          }
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             mx[2] = max3(mx[2], __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
@@ -626,15 +634,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           tmem_ld32(s_addr, ra);
           tmem_ld32(s_addr + 32, rb);
           tc_wait_ld();
-          if (tail) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              ra[e] = (vm[0] >> e) & 1u ? ra[e] : 0xff800000u;       // -inf
-              rb[e] = (vm[1] >> e) & 1u ? rb[e] : 0xff800000u;
-              rc[e] = (vm[2] >> e) & 1u ? rc[e] : 0xff800000u;
-              rd[e] = (vm[3] >> e) & 1u ? rd[e] : 0xff800000u;
-            }
-          }
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             mx[0] = max3(mx[0], __uint_as_float(rc[e]), __uint_as_float(rc[e + 1]));
@@ -727,13 +726,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         exp_chunk(rb, 1);
         tmem_ld32(s_addr + 96, rb);         // chunk 3
         tc_wait_ld();
-        if (tail) {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            ra[e] = (vm[2] >> e) & 1u ? ra[e] : 0xff800000u;
-            rb[e] = (vm[3] >> e) & 1u ? rb[e] : 0xff800000u;
-          }
-        }
         exp_chunk(ra, 2);
         exp_chunk(rb, 3);
         {
@@ -806,26 +798,6 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       g_base += steps;
       sg += steps;
       ++item_count;
-    }
-  } else if (warp == kWarpQ) {
-    // =========================================================================== query-tile producer
-    // One buffer: the tile of the next item is fetched as soon as the last score MMA of the current one has finished;
-    // the softmax groups still have two or three steps of that item to work through meanwhile.
-    if (lane == 0 && p.q_tma) {
-      uint32_t item_count = 0;
-      bool ok = true;
-      for (int tp = tp_lo; tp < tp_hi && ok; ++tp) {
-        const WorkItem it = p.items[2 * tp + member];
-        if (it.tile_end <= it.tile_begin) continue;
-        ok = mbar_wait(B.q_empty(), (item_count & 1u) ^ 1u, s_abort);
-        if (!ok) break;
-        // box (64 columns, G heads, 128/G nodes); rows land in (node, head) order = query row order
-        mbar_expect_tx(B.q_full(), S::kTileBytes);
-#pragma unroll
-        for (int sl = 0; sl < S::kSlabs; ++sl)
-          tma_load_4d(sbase + S::kQ + sl * S::kSlabBytes, &map_q, sl * 64, it.g * p.G, it.mt * (kBlockM / p.G), it.b, B.q_full());
-        ++item_count;
-      }
     }
   } else if (warp == kWarpProducer) {
     // =========================================================================== TMA producer
