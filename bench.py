@@ -51,8 +51,9 @@ SM_COUNT, EX2_PER_SM_PER_CLK = 148, 16      # special-function rate behind the e
 # profiles/attn_kernel_serving_mix_b16.md, keyed by (workload, batch), with the SHA-256 of the attention kernel's source
 # the captures were taken on: when the source has changed since, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "attn_cu_sha256": "",
-    "bytes": {("serving_mix", 64): 1_180_839_168 + 24_708_608, ("serving_mix", 16): 313_012_224 + 8_916_992},
+    "attn_cu_sha256": "1e270d6f4248e68775b94c17eecbdad4764e6ed35b280f389fed860a40a96c0c",
+    # full size: one-pass metric list, two launches averaged (1181.1 MB read + 22.8 MB written); batch 16: --set full
+    "bytes": {("serving_mix", 64): 1_181_139_328 + 22_816_256, ("serving_mix", 16): 313_046_528 + 9_554_304},
 }
 
 
@@ -453,6 +454,20 @@ def main():
         accept_ms = statistics.mean(a.elapsed_time(b) for a, b in ev_acc)
         path, bonus, alen, status = ctx.path, ctx.bonus, ctx.alen, ctx.status
 
+        # ---- the same acceptance with uncorrelated draft and target logits (rho = 0: rejection-heavy, the longest walks)
+        acc0 = W.make_accept_inputs(cfg, salt=replicas.rank_salt(rank), rho=0.0, trees=(attn.tree_sizes, attn.tree_parent))
+        t0 = {k: v.to(dev) for k, v in dict(tp=acc0.target_probs, dp=acc0.draft_probs, tok=acc0.draft_tokens, un=acc0.uniforms).items()}
+        s0 = ctx.sets[0]
+        ev0 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(6)]
+        for a, b in ev0:
+            a.record()
+            E.eagle_tree_accept(t0["tp"], t0["dp"], t0["tok"], s0["par"], t0["un"], path, bonus, tree_sizes=s0["ts"], greedy=s0["gr"],
+                                accept_len=alen, status=status)
+            b.record()
+        torch.cuda.synchronize()
+        accept_rho0 = {"ms": statistics.mean(a.elapsed_time(b) for a, b in ev0[1:]), "tokens_per_step": float(alen.float().mean().item()) + 1.0}
+        del t0, acc0
+
         # ---- the device path's outputs on input set 0, kept for the parity record
         ctx.step(0)
         torch.cuda.synchronize()
@@ -553,7 +568,7 @@ def main():
         moved = int(((path >= 0) & (path != torch.arange(T, device=dev, dtype=torch.int32)[None, :])).sum().item())
         commit_bytes = moved * cfg.num_kv_heads * cfg.head_dim * 2 * 2 * 2     # rows that change slot: K and V, read + written
         extras.update({
-            "accept_ms": accept_ms, "tokens_per_step": mean_tokens,
+            "accept_ms": accept_ms, "tokens_per_step": mean_tokens, "accept_rho0": accept_rho0,
             "accept_on_logits": {"ms": accept_logits_ms, "temperature": 1.0,
                                  "sequences_with_the_same_tokens_as_on_probabilities": logits_same, "of": B},
             "tree_expand": {"ms": expand_ms, "rows": B * R_exp, "children": K_exp, "bytes": expand_bytes,
