@@ -253,6 +253,35 @@ class StepContext:
         torch.cuda.synchronize()
         return start.elapsed_time(stop), statistics.mean(a.elapsed_time(b) for a, b in evs), self.E.launch_count() - launches0
 
+    def graph_leg(self, K=50):
+        """The same step captured once in a CUDA graph (all R input sets in turn, so that no replay finds its inputs in L2) and
+        replayed: what the step costs without the host's launch gaps."""
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            for i in range(self.R):
+                self.step(i)                       # (every first-call set-up of the library has long happened)
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(self.R):
+                    self.step(i)
+        torch.cuda.current_stream().wait_stream(side)
+        reps = max(1, K // self.R)
+        for _ in range(2):
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        self.check()
+        ms = a.elapsed_time(b) / (reps * self.R)
+        return {"ms_per_step": ms, "steps_per_s": 1e3 / ms, "steps": reps * self.R,
+                "note": "the four launches of a step replayed from one CUDA graph"}
+
     def per_layer(self, layers=32):
         """One plan for the verification pass, then attention + combine for each of ``layers`` layers (rotating K/V sets)."""
         s0 = self.sets[0]
@@ -509,6 +538,9 @@ def main():
         expand_bytes = rows_exp.numel() * 4
         del rows_exp
 
+        # ---- the step replayed from a CUDA graph (no launch gaps)
+        cuda_graph = ctx.graph_leg()
+
         # ---- one plan per verification pass, attention + combine per layer
         per_layer = ctx.per_layer()
         per_layer["attn_kernel_share_of_layer"] = attn_ms / per_layer["ms_per_layer"]
@@ -573,7 +605,7 @@ def main():
                                  "sequences_with_the_same_tokens_as_on_probabilities": logits_same, "of": B},
             "tree_expand": {"ms": expand_ms, "rows": B * R_exp, "children": K_exp, "bytes": expand_bytes,
                             "gbs": expand_bytes / (expand_ms * 1e-3) / 1e9, "note": "back-to-back calls on the same rows (warm L2)"},
-            "per_layer": per_layer, "fp8_kv": fp8_kv, "paged_attention": paged,
+            "cuda_graph": cuda_graph, "per_layer": per_layer, "fp8_kv": fp8_kv, "paged_attention": paged,
             "kv_commit": {"ms": commit_ms, "rows_moved_per_kv_head": moved, "bytes": commit_bytes,
                           "gbs": commit_bytes / (commit_ms * 1e-3) / 1e9, "bound": "launch + memory latency"}})
     ctx.free()
@@ -624,6 +656,7 @@ def main():
             pl = o.per_layer()
             pl["attn_kernel_share_of_layer"] = a_ms / pl["ms_per_layer"]
             rec["per_layer"] = pl
+            rec["cuda_graph"] = o.graph_leg()
             rec["fp8_kv"] = o.fp8_leg(a_ms, pk)
             o.check()
             others[name] = rec

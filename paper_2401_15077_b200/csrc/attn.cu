@@ -647,6 +647,16 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (key0 + kTileN > kv_end) {
           // rows of the V tile past prefix + tree may hold anything: zero them so that 0 * garbage cannot reach O
           const uint32_t nv = 2 * (g_base + s) + 3, slot = nv % kSlots, par = (nv / kSlots) & 1u;
+          if constexpr (FP8) {
+            // With four ring slots this V tile shares its slot with the V tile of two steps ago, which need not have
+            // been consumed, or even converted, when this step's scores are ready; the parity wait below would then
+            // take that older phase for this one and the zeros would land in the wrong tile.  Wait for that PV first.
+            // (With six slots the slot's previous tile is three steps back: its PV freed this step's score buffer.)
+            if (gs >= 2u) {
+              ok = mbar_wait_warp(B.o_done((gs - 2u) % kSBufs), ((gs - 2u) / kSBufs) & 1u, s_abort);
+              if (!ok) break;
+            }
+          }
           ok = mbar_wait_warp(B.full(slot), par, s_abort);
           if (!ok) break;
           if (key0 + r >= kv_end) {

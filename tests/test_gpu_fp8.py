@@ -147,3 +147,22 @@ def test_fp8_refuses_unsupported_shapes(E):
     with pytest.raises(E.EagleError):
         E.eagle_tree_verify_attn_fp8(inp.q.to(d), f8.k_codes.to(d), f8.v_codes.to(d), f8.k_scale.to(d), f8.v_scale.to(d),
                                      inp.seq_lens.to(d), inp.tree_parent.to(d))
+
+
+def test_fp8_many_short_items_repeatedly(E, oracle):
+    """A small ragged batch gives every CTA items of one or two KV tiles; the last tile of a sequence (whose V rows past
+    prefix + tree are zeroed in shared memory) then shares its ring slot with a tile that may not have been consumed yet.
+    The call is repeated: every run must be within the bounds and bit-identical to the first (a race here showed as a
+    wrong (sequence, KV head) unit in about half of the runs)."""
+    cfg = CASES["ragged_small_trees"]
+    inp = W.make_attn_inputs(cfg, salt=3, capacity_pad=19)
+    f8 = W.make_fp8_cache(inp)
+    ref = oracle.tree_verify_attn_fp8(inp.q, f8.k_codes, f8.v_codes, f8.k_scale, f8.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    first = None
+    for rep in range(30):
+        out, status = _run(E, inp, f8)
+        assert status == 0
+        _check(out, ref, inp.tree_sizes)
+        if first is None:
+            first = out
+        assert torch.equal(out.view(torch.int16), first.view(torch.int16)), rep
