@@ -145,3 +145,14 @@ def test_host_step_byte_count(lib):
     assert want < full
     assert make(lens, sizes) == (want, d2h_want)
     assert lib.eagle_tree_verify_step_host_bytes(None, None, None) == -1
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header compiles as C99 with warnings as errors, without CUDA or C++."""
+    import subprocess
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "eagle_verify.h"\n'
+                   'int main(void) { eagle_attn_desc d; eagle_accept_desc a; eagle_paged_kv k; (void)d; (void)a; (void)k;\n'
+                   '  return sizeof(eagle_host_step) > 0 && EAGLE_MAX_TREE == 64 ? 0 : 1; }\n')
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only", "-I", str(ROOT / "include"), str(src)],
+                   check=True)

@@ -166,3 +166,23 @@ def test_fp8_many_short_items_repeatedly(E, oracle):
         if first is None:
             first = out
         assert torch.equal(out.view(torch.int16), first.view(torch.int16)), rep
+
+
+def test_fp8_wait_that_runs_out_is_reported(E, oracle):
+    """The converter warps' waits are bounded like every other: with the K/V producer silenced after two tiles (test hook)
+    and the limit lowered to 2 ms the call returns by itself with EAGLE_ERR_TIMEOUT; the next call is correct."""
+    cfg = W.scaled(W.CONFIGS["7b_mha"], batch=2, num_q_heads=8, num_kv_heads=2, prefix=(600, 900), tree=(8, 8))
+    inp = W.make_attn_inputs(cfg, salt=12)
+    f8 = W.make_fp8_cache(inp)
+    ref = oracle.tree_verify_attn_fp8(inp.q, f8.k_codes, f8.v_codes, f8.k_scale, f8.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    try:
+        E.set_wait_limit_ns(2_000_000)
+        E.test_stall_kv_producer(2)
+        out, status = _run(E, inp, f8)
+    finally:
+        E.test_stall_kv_producer(-1)
+        E.set_wait_limit_ns(0)
+    assert status == -8, E.status_string(status)
+    out, status = _run(E, inp, f8)
+    assert status == 0
+    _check(out, ref, inp.tree_sizes)
