@@ -13,12 +13,15 @@
 // them); warp 9 issues the QK MMAs (and fetches the query tile of the next item once the last score MMA of the
 // current one has finished), warp 10 the PV MMAs.  The group that takes an item's last step writes its output
 // while the other group is already on the next item.  Softmax is fp32 in the log2 domain with two-wide FP32
-// instructions; part of the exponentials is a polynomial on the FMA pipe.  The tree mask is applied in registers
-// only on tiles that reach past the committed prefix; rows of a V tile past prefix + tree are zeroed in shared
-// memory before the MMA reads them.  The accumulator is rescaled only when the row maximum outgrows the shared
-// reference by more than 2^8.  Every wait is bounded (mbarrier try_wait + timer, or a bounded spin on a tagged
-// word); on expiry the CTA raises EAGLE_ERR_TIMEOUT, all roles leave their loops, TMEM is released and the kernel
-// returns.
+// instructions; part of the exponentials is a polynomial on the FMA pipe.  The tree mask is applied only on tiles
+// that reach past the committed prefix, by a pre-pass that writes -inf over the invisible scores in tensor memory;
+// rows of a V tile past prefix + tree are zeroed in shared memory before the MMA reads them.  The accumulator is
+// rescaled only when the row maximum outgrows the shared reference by more than 2^8.  Every wait is bounded
+// (mbarrier try_wait + timer, or a bounded spin on a tagged word); on expiry the CTA raises EAGLE_ERR_TIMEOUT, all
+// roles leave their loops, TMEM is released and the kernel returns.
+// Instantiations: PAGED (the K/V producer gathers a tile page by page through a block table) and FP8 (the cache holds
+// e4m3 codes: tiles of codes land in a staging ring, four more warps widen them exactly into a ring of four bf16
+// slots, the scales go into the softmax scale and the output).
 #include <cuda.h>
 
 #include "common.cuh"
