@@ -331,7 +331,7 @@ class StepContext:
             2 * 4 * cfg.batch * cfg.num_kv_heads
         gbs = alg / (ms * 1e-3) / 1e9
         return {"attn_kernel_ms": ms, "ratio_to_bf16": ms / attn_ms_bf16, "algorithmic_bytes": alg, "gbs": gbs, "hbm_frac": gbs / pk["hbm"],
-                "note": "e4m3 codes + fp32 scale per (sequence, KV head); codes widened exactly to bf16 in shared memory"}
+                "note": "e4m3 codes + fp32 scale per (sequence, KV head); codes widened exactly to fp16 in shared memory, fp16 x fp16 MMAs"}
 
     def free(self):
         self.sets = None

@@ -190,12 +190,15 @@ int eagle_tree_verify_attn_planned_paged(const eagle_attn_desc* desc, const void
  * convention here is this library's: k_codes / v_codes are device uint8 [B, Hkv, S_cap, D] holding fp8 "e4m3" codes (1
  * sign, 4 exponent, 3 mantissa bits, bias 7, no infinities), and every (sequence, KV head) has one fp32 scale for its keys
  * and one for its values, k_scale / v_scale device fp32 [B, Hkv]:  key = value(code) * k_scale[b, h],  value =
- * value(code) * v_scale[b, h].  Only the storage changes: the codes are widened exactly (every e4m3 number is a bf16
+ * value(code) * v_scale[b, h].  Only the storage changes: the codes are widened exactly (every e4m3 number is an fp16
  * number) on their way to the tensor cores, the keys' scale is folded into the softmax scale and the values' scale into
- * the output, and everything else (queries in bf16, fp32 scores / softmax / accumulation, bf16 output, planner, work split,
- * errors) is as for eagle_tree_verify_attn.  What it saves is half of the cache bytes read.  head_dim must be 128 and the
- * cache contiguous (else EAGLE_ERR_SHAPE).  Slots that are not visible may hold any code; the two NaN codes (0x7f, 0xff)
- * in a VISIBLE slot are not propagated as NaN (they are read as +-480 times the scale): do not store them.
+ * the output.  A tensor-core instruction takes one 16-bit type for both operands, so this form multiplies in fp16: the
+ * bf16 queries are converted to fp16 (exact for magnitudes from 2^-14 to 65504; smaller ones are rounded to multiples of
+ * 2^-24, larger ones become infinite) and the probabilities are rounded to fp16 instead of bf16.  Everything else (fp32
+ * scores / softmax / accumulation, bf16 output, planner, work split, errors) is as for eagle_tree_verify_attn.  What it
+ * saves is half of the cache bytes held and read.  head_dim must be 128 and the cache contiguous (else EAGLE_ERR_SHAPE).
+ * Slots that are not visible may hold any code; one of the two NaN codes (0x7f, 0xff) in a VISIBLE slot makes the output
+ * rows that see it NaN.
  * eagle_tree_verify_attn_planned_fp8 is the per-layer half over a plan made by eagle_tree_verify_plan (paged = NULL).
  */
 int eagle_tree_verify_attn_fp8(const eagle_attn_desc* desc, const void* q, const void* k_codes, const void* v_codes,

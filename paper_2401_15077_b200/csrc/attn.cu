@@ -20,8 +20,8 @@
 // (mbarrier try_wait + timer, or a bounded spin on a tagged word); on expiry the CTA raises EAGLE_ERR_TIMEOUT, all
 // roles leave their loops, TMEM is released and the kernel returns.
 // Instantiations: PAGED (the K/V producer gathers a tile page by page through a block table) and FP8 (the cache holds
-// e4m3 codes: tiles of codes land in a staging ring, four more warps widen them exactly into a ring of four bf16
-// slots, the scales go into the softmax scale and the output).
+// e4m3 codes: tiles of codes land in a staging ring, four more warps widen them exactly into a ring of four fp16
+// slots and the MMAs run fp16 x fp16; the scales go into the softmax scale and the output).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -32,12 +32,13 @@ namespace {
 
 constexpr int kTileN = 128;          // keys per KV tile
 // Ring slots of K/V tiles; entry n of the load sequence (see the producer) uses slot n % slots.  A cache stored as fp8
-// codes has four slots of bf16 tiles plus four staging slots of raw codes instead of six slots.
+// codes has four slots of fp16 tiles plus four staging slots of raw codes instead of six slots.
 template <bool FP8>
 constexpr int slots_of() { return FP8 ? 4 : 6; }
 constexpr int kSBufs = 3;            // score buffers in tensor memory; step g uses buffer g % 3
 constexpr int kThreads = 352;          // 8 softmax warps, K/V producer, two MMA issuers: 186 registers for every thread
-constexpr int kThreadsFp8 = 480;       // the same plus four warps that widen fp8 codes to bf16 tiles
+constexpr int kConvWarps = 4;           // fp8 cache: warps that widen tiles of codes to fp16 tiles
+constexpr int kThreadsFp8 = kThreads + 32 * kConvWarps;   // (a fifth warp per scheduler: 128 registers for every thread)
 constexpr int kWarpConvert = 11;
 constexpr int kSoftmaxWarps = 8;
 constexpr int kGroupThreads = 128;     // one softmax group
@@ -260,10 +261,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// kind::f16 instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(N >> 3) << 17) |
-         (static_cast<uint32_t>(M >> 4) << 24);
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// kind::f16 instruction descriptor: bf16 x bf16 (or fp16 x fp16: both operands have one type) -> fp32, A K-major,
+// B K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major, bool fp16 = false) {
+  return (1u << 4) | (fp16 ? 0u : (1u << 7) | (1u << 10)) | (b_mn_major ? (1u << 16) : 0u) |
+         (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 
 
@@ -398,11 +405,11 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_v)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_q)) : "memory");
     for (int i = 0; i < kSlots; ++i) {
-      mbar_init(B.full(i), FP8 ? kGroupThreads : 1);   // one TMA transaction, or every thread of the converter warps
+      mbar_init(B.full(i), FP8 ? 32 * kConvWarps : 1);   // one TMA transaction, or every thread of the converter warps
       mbar_init(B.empty(i), 1);
       if constexpr (FP8) {
         mbar_init(B.st_full(i), 1);
-        mbar_init(B.st_empty(i), kGroupThreads);
+        mbar_init(B.st_empty(i), 32 * kConvWarps);
       }
     }
     for (int i = 0; i < kSBufs; ++i) {
@@ -438,7 +445,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     // Entry n of the load sequence lives in slot n % kSlots with phase parity (n / kSlots) & 1.  Positions are kept
     // as running counters (no divisions on the threads that keep the tensor pipe fed).
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = instr_desc(kBlockM, kTileN, false);
+      constexpr uint32_t idesc_qk = instr_desc(kBlockM, kTileN, false, FP8);
       uint32_t ks = 0, kp = 0;       // slot / parity of the K tile of the next QK
       uint32_t gq = 0;               // steps issued so far (all items)
       uint32_t sb = 0, sph = 0;      // gq % 3 and (gq / 3) & 1
@@ -488,7 +495,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
   } else if (warp == kWarpPV) {
     // =========================================================================== PV issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, true);
+      constexpr uint32_t idesc_pv = instr_desc(kBlockM, D, true, FP8);
       uint32_t vs = 3, vp = 0;       // slot / parity of the V tile of the next PV: V(g) is entry 2g + 3
       uint32_t gp = 0;               // steps issued so far (all items)
       uint32_t sb = 0, sph = 0;      // gp % 3 and (gp / 3) & 1
@@ -563,7 +570,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         unsigned char* qdst = smem + S::kQ + r * 128;
 #pragma unroll
         for (int c = 0; c < 8 * S::kSlabs; ++c) {
-          const uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+          uint4 v = row_valid ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+          if constexpr (FP8) {     // the MMAs of this form take fp16 operands: every bf16 query of magnitude 2^-14 .. 65504 is one
+            v.x = pack_f16(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
+            v.y = pack_f16(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
+            v.z = pack_f16(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
+            v.w = pack_f16(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
+          }
           *reinterpret_cast<uint4*>(qdst + (c >> 3) * S::kSlabBytes + (((c & 7) ^ (r & 7)) << 4)) = v;
         }
         fence_proxy_async();
@@ -730,7 +743,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
               p1 = fast_exp2(b);
             }
             ls2[j & 1] = add2(ls2[j & 1], pack2(p0, p1));
-            pk[j] = pack_bf16(p0, p1);
+            pk[j] = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
           }
           tmem_st16(s_addr + c * 16, pk);
         };
@@ -912,28 +925,23 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
       }
     }
   } else if (FP8 && warp >= kWarpConvert) {
-    // =========================================================================== fp8 -> bf16 converter (warps 12-15)
+    // =========================================================================== fp8 -> fp16 converter (warps 11-14)
     // Thread r owns row r of every K / V tile: it reads the row's 128 codes from the staging slot (eight 16-byte chunks,
     // 128-byte swizzled as the copy laid them down), widens them, and writes the row's 256 bytes into the ring slot in
-    // the swizzled two-slab layout the MMAs read.  Every e4m3 number is a bf16 number, so this is exact: the code's
-    // exponent and mantissa bits are moved into place (which leaves the value 2^-120 times too small, subnormals
-    // included) and one bf16 multiplication by 2^120 restores it.  The scales are applied elsewhere.
+    // the swizzled two-slab layout the MMAs read.  Every e4m3 number is an fp16 number, subnormals included, so the
+    // hardware conversion (two codes per instruction) is exact.  The MMAs of this form therefore run fp16 x fp16 (an
+    // MMA takes one 16-bit type for both operands): the queries are converted as they are staged and P is written as
+    // fp16.  The scales are applied elsewhere.
     if constexpr (FP8) {
-      const int r = tid & (kBlockM - 1);
+      const int r0 = tid - 32 * kWarpConvert;
       uint32_t steps_total = 0;     // this CTA's steps over all its items
       for (int tp = tp_lo; tp < tp_hi; ++tp) {
         const WorkItem it = p.items[2 * tp + member];
         if (it.tile_end > it.tile_begin) steps_total += static_cast<uint32_t>(it.tile_end - it.tile_begin);
       }
-      const __nv_bfloat162 two120 = __halves2bfloat162(__ushort_as_bfloat16(0x7B80), __ushort_as_bfloat16(0x7B80));
-      auto widen = [&](uint32_t w, uint32_t& lo, uint32_t& hi) {
-        const uint32_t m = w & 0x7f7f7f7fu, sg = w & 0x80808080u;
-        uint32_t a = (__byte_perm(m, 0u, 0x4140) << 4) | __byte_perm(sg, 0u, 0x1404);   // codes 0 and 1 of the word
-        uint32_t b = (__byte_perm(m, 0u, 0x4342) << 4) | __byte_perm(sg, 0u, 0x3424);   // codes 2 and 3
-        __nv_bfloat162 x = __hmul2(*reinterpret_cast<__nv_bfloat162*>(&a), two120);
-        __nv_bfloat162 y = __hmul2(*reinterpret_cast<__nv_bfloat162*>(&b), two120);
-        lo = *reinterpret_cast<uint32_t*>(&x);
-        hi = *reinterpret_cast<uint32_t*>(&y);
+      auto widen = [](uint32_t w, uint32_t& lo, uint32_t& hi) {    // four codes -> four fp16 numbers
+        asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+            : "=r"(lo), "=r"(hi) : "r"(w));
       };
       // Entry n of the load sequence is K(n) for n < 3, V((n - 3) / 2) for odd n and K((n + 2) / 2) for even n after
       // that; the K entries of the last three steps do not exist (the producer skips them, the numbering keeps its gaps).
@@ -947,19 +955,24 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         if (!ok) break;
         ok = mbar_wait_warp(B.empty(slot), par ^ 1u, s_abort);    // the MMA that read the ring slot last has finished
         if (!ok) break;
-        const unsigned char* src = smem + S::kStage + slot * S::kCodeBytes + r * 128;
-        unsigned char* dst = smem + S::kRing + slot * S::kTileBytes + r * 128;
+#pragma unroll 1
+        for (int r = r0; r < kTileN; r += 32 * kConvWarps) {
+          const unsigned char* src = smem + S::kStage + slot * S::kCodeBytes + r * 128;
+          unsigned char* dst = smem + S::kRing + slot * S::kTileBytes + r * 128;
+          uint4 w[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {                              // codes 16c .. 16c + 15 of the row
-          const uint4 w = *reinterpret_cast<const uint4*>(src + ((c ^ (r & 7)) << 4));
-          uint4 u, v;
-          widen(w.x, u.x, u.y);
-          widen(w.y, u.z, u.w);
-          widen(w.z, v.x, v.y);
-          widen(w.w, v.z, v.w);
-          unsigned char* d = dst + (c >> 2) * S::kSlabBytes;       // 64 columns per slab: chunks 2c and 2c + 1 of the slab's row
-          *reinterpret_cast<uint4*>(d + ((((2 * c) & 7) ^ (r & 7)) << 4)) = u;
-          *reinterpret_cast<uint4*>(d + ((((2 * c + 1) & 7) ^ (r & 7)) << 4)) = v;
+          for (int c = 0; c < 8; ++c) w[c] = *reinterpret_cast<const uint4*>(src + ((c ^ (r & 7)) << 4));
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {                            // codes 16c .. 16c + 15 of the row
+            uint4 u, v;
+            widen(w[c].x, u.x, u.y);
+            widen(w[c].y, u.z, u.w);
+            widen(w[c].z, v.x, v.y);
+            widen(w[c].w, v.z, v.w);
+            unsigned char* d = dst + (c >> 2) * S::kSlabBytes;     // 64 columns per slab: chunks 2c and 2c + 1 of the slab's row
+            *reinterpret_cast<uint4*>(d + ((((2 * c) & 7) ^ (r & 7)) << 4)) = u;
+            *reinterpret_cast<uint4*>(d + ((((2 * c + 1) & 7) ^ (r & 7)) << 4)) = v;
+          }
         }
         fence_proxy_async();                                       // the MMAs read the slot through the async proxy
         mbar_arrive(B.full(slot));
@@ -1070,7 +1083,7 @@ cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t strea
     const long long bh = static_cast<long long>(p.B) * p.Hkv;
     if (!make_kv_map(&mk, p.k, p.D, p.S_cap, bh) || !make_kv_map(&mv, p.v, p.D, p.S_cap, bh)) return cudaErrorInvalidValue;
   }
-  p.q_tma = (kBlockM % p.G == 0) ? 1 : 0;
+  p.q_tma = (kBlockM % p.G == 0 && !fp8) ? 1 : 0;   // (the fp8 form converts the queries to fp16 as it stages them)
   if (p.q_tma) {
     if (!make_q_map(&mq, p.q, p.D, p.Hq, p.T_max, p.B, p.G)) return cudaErrorInvalidValue;
   } else {

@@ -1,6 +1,7 @@
 // Shared definitions of the tree-verification kernels (device-side plan records, workspace layout).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
