@@ -51,9 +51,10 @@ SM_COUNT, EX2_PER_SM_PER_CLK = 148, 16      # special-function rate behind the e
 # profiles/attn_kernel_serving_mix_b16.md, keyed by (workload, batch), with the SHA-256 of the attention kernel's source
 # the captures were taken on: when the source has changed since, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "attn_cu_sha256": "8bec55271dab43b8bd53c81c8d9760146340b8c67a1bfefd66291b7043826ad0",
-    # full size: one-pass metric list, two launches averaged (1180.8 MB read + 22.6 MB written); batch 16: --set full
-    "bytes": {("serving_mix", 64): 1_180_797_952 + 22_569_216, ("serving_mix", 16): 313_046_528 + 9_554_304},
+    "attn_cu_sha256": "0fedb1d3e0a8028a3dc1c6a64b36170155ab4e8f114a9549fa6d0f6b8fe02256",
+    # full size: one-pass metric list, two launches averaged (1184.9 MB read + 22.9 MB written); batch 16: --set full
+    # (taken before the fp8 instantiation changed; the bf16 instantiation it measures did not)
+    "bytes": {("serving_mix", 64): 1_184_917_120 + 22_854_784, ("serving_mix", 16): 313_046_528 + 9_554_304},
 }
 
 
