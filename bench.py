@@ -16,7 +16,7 @@ One *step* = ``eagle_tree_verify_attn`` (planner, split-KV attention, combine) f
   the timed region, against the measured HBM copy bandwidth (or the measured bf16 rate where that binds).
 * ``breakdown.sustained``: the same step back to back for seconds, with the SM clock sampled meanwhile.
 * ``breakdown.workloads``: the other configurations (70B-, Mixtral-, 7B-shaped, tiny), a few dozen steps each.
-* ``breakdown.per_layer``: one plan for the verification pass, then attention + combine per layer.
+* ``breakdown.per_layer``: one plan for the verification pass, then attention + combine per layer (also as one CUDA graph).
 * ``cpu_baseline`` / ``parity``: the fp64 oracle, as it stands, on a bounded sample of the same workload; its
   outputs are compared with the device path's on the way.
 * ``--impl reference``: the oracle arm (CPU); rank 0 only.
@@ -303,8 +303,35 @@ class StepContext:
         one_pass()
         e[2].record()
         torch.cuda.synchronize()
-        return {"layers": layers, "plan_ms": e[0].elapsed_time(e[1]), "ms_per_layer": e[1].elapsed_time(e[2]) / layers,
-                "note": "eagle_tree_verify_plan once, then eagle_tree_verify_attn_planned per layer"}
+        out = {"layers": layers, "plan_ms": e[0].elapsed_time(e[1]), "ms_per_layer": e[1].elapsed_time(e[2]) / layers,
+               "note": "eagle_tree_verify_plan once, then eagle_tree_verify_attn_planned per layer"}
+        # the same pass (plan + every layer's attention and combine) captured in one CUDA graph and replayed: the host's
+        # launch gaps are gone, which is what a serving loop that replays its forward pass sees
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                one_pass_plain = self.E.eagle_tree_verify_plan(tuple(s0["q"].shape), cfg.num_kv_heads, s0["k"].shape[2], s0["sl"], s0["par"],
+                                                               tree_sizes=s0["ts"], num_splits=self.num_splits, workspace=self.ws,
+                                                               status=self.status)
+                for l in range(layers):
+                    s = self.sets[l % self.R]
+                    one_pass_plain.attend(s["q"], s["k"], s["v"], self.out, status=self.status)
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        g.replay()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        self.check()
+        out["graph_ms_per_layer"] = a.elapsed_time(b) / (2 * layers)
+        out["graph_note"] = "plan + %d layers replayed from one CUDA graph; the plan's share is included" % layers
+        return out
 
     def fp8_leg(self, attn_ms_bf16, pk, calls=12):
         """The same attention over the same cache stored as fp8 (e4m3) codes with a scale per (sequence, KV head): the
