@@ -2,6 +2,8 @@
 
 Only the storage differs from the bf16 call: the codes are widened exactly, the scales are applied in fp32, so the same
 bounds hold against the oracle evaluated on the same codes and scales."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -68,6 +70,32 @@ def test_fp8_attention_matches_oracle(E, oracle, name):
         _check(out, ref, inp.tree_sizes)
     again, _ = _run(E, inp, f8, num_splits=3)
     assert torch.equal(out.view(torch.int16), again.view(torch.int16))
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("EAGLE_RANDOM_FP8", "8"))))
+def test_random_shapes_fp8(E, oracle, seed):
+    """Random head counts, group sizes (those that divide 128 and those that do not: the two ways a query tile is staged),
+    prefix ranges around the tile size and tree shapes, default split and a forced one, twice each (bit-identical)."""
+    rng = np.random.default_rng(7000 + seed)
+    Hkv = int(rng.choice([1, 2, 3, 5, 8]))
+    G = int(rng.choice([1, 2, 3, 4, 6, 8, 16]))
+    lo = int(rng.choice([0, 0, 1, 100, 127, 128, 129, 600]))
+    hi = lo + int(rng.choice([0, 1, 130, 700, 2500]))
+    t_lo = int(rng.integers(0, 40))
+    t_hi = int(rng.integers(max(t_lo, 1), 65))
+    depth = int(rng.choice([2, 5, 9, 64]))
+    shape = dict(max_depth=depth, child_cap=int(rng.choice([0, 2, 4])) if depth >= 9 else 0)
+    cfg = W.scaled(W.CONFIGS["7b_mha"], batch=int(rng.integers(1, 7)), num_q_heads=Hkv * G, num_kv_heads=Hkv, prefix=(lo, hi),
+                   tree=(t_lo, t_hi), **shape)
+    inp = W.make_attn_inputs(cfg, salt=seed, capacity_pad=int(rng.integers(0, 40)))
+    f8 = W.make_fp8_cache(inp)
+    ref = oracle.tree_verify_attn_fp8(inp.q, f8.k_codes, f8.v_codes, f8.k_scale, f8.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    for splits in (0, int(rng.choice([2, 3, 5]))):
+        out, status = _run(E, inp, f8, num_splits=splits)
+        assert status == 0, (cfg, splits)
+        _check(out, ref, inp.tree_sizes)
+        again, _ = _run(E, inp, f8, num_splits=splits)
+        assert torch.equal(out.view(torch.int16), again.view(torch.int16)), (cfg, splits)
 
 
 def test_every_code_is_widened_exactly(E, oracle):
