@@ -47,6 +47,8 @@ def _load():
         lib.oracle_tree_verify_attn_paged.restype = i32
         lib.oracle_tree_verify_attn_fp8.argtypes = [i32, i32, i32, i32, i32, i32, vp, dbl] + [vp] * 8
         lib.oracle_tree_verify_attn_fp8.restype = i32
+        lib.oracle_tree_verify_attn_fp8_paged.argtypes = [i32] * 8 + [vp, dbl] + [vp] * 9
+        lib.oracle_tree_verify_attn_fp8_paged.restype = i32
         lib.oracle_e4m3_table.argtypes = [vp]
         lib.oracle_e4m3_table.restype = None
         lib.oracle_tree_accept.argtypes = [i32, i32, i32, i32] + [vp] * 17
@@ -172,6 +174,29 @@ def tree_verify_attn_fp8(q, k_codes, v_codes, k_scale, v_scale, seq_lens, tree_p
                                              _ptr(ks), _ptr(vs), _ptr(sl), _ptr(par), _ptr(out))
     if rc != 0:
         raise ValueError(f"oracle_tree_verify_attn_fp8 failed: {rc}")
+    return out
+
+
+def tree_verify_attn_fp8_paged(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, tree_parent, tree_sizes=None,
+                              sm_scale: float = 0.0):
+    """fp64 tree-masked attention over a paged cache of e4m3 codes: k_pages, v_pages uint8 [num_pages, Hkv, page_size, D],
+    scales fp32 [B, Hkv], block_table int32 [B, max_pages_per_seq].  Returns float64 [B, T_max, Hq, D]."""
+    qa = _as(q, np.uint16)
+    ka, va = _as(k_pages, np.uint8), _as(v_pages, np.uint8)
+    B, T, Hq, D = qa.shape
+    P, Hkv, ps = ka.shape[0], ka.shape[1], ka.shape[2]
+    assert ka.shape == va.shape == (P, Hkv, ps, D)
+    ks, vs = _as(k_scale, np.float32), _as(v_scale, np.float32)
+    assert ks.shape == vs.shape == (B, Hkv)
+    bt = _as(block_table, np.int32)
+    assert bt.ndim == 2 and bt.shape[0] == B
+    sl, par, ts = _as(seq_lens, np.int32), _as(tree_parent, np.int32), _as(tree_sizes, np.int32)
+    assert par.shape == (B, T)
+    out = np.zeros((B, T, Hq, D), np.float64)
+    rc = _load().oracle_tree_verify_attn_fp8_paged(B, Hq, Hkv, D, T, P, ps, bt.shape[1], _ptr(ts), float(sm_scale), _ptr(qa),
+                                                   _ptr(ka), _ptr(va), _ptr(ks), _ptr(vs), _ptr(bt), _ptr(sl), _ptr(par), _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle_tree_verify_attn_fp8_paged failed: {rc}")
     return out
 
 

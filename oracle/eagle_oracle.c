@@ -14,6 +14,7 @@
  *                              prefix plus the node's ancestors and itself (plain definition).
  *   oracle_tree_verify_attn_paged - the same over a cache stored in pages addressed through a block table.
  *   oracle_tree_verify_attn_fp8 - the same over a cache stored as fp8 (e4m3) codes with one scale per (sequence, KV head).
+ *   oracle_tree_verify_attn_fp8_paged - the fp8 cache kept in pages behind a block table.
  *   oracle_tree_accept       - Algorithm 1 (multi-round speculative sampling, App. A.2) applied
  *                              recursively at every node from the root (Sec. 3.3); the greedy setting
  *                              (Preliminaries) is the same rule with a one-hot target distribution.
@@ -328,6 +329,60 @@ int oracle_tree_verify_attn_fp8(int batch, int num_q_heads, int num_kv_heads, in
     }
   }
   return failed ? ORACLE_ERR_NOMEM : ORACLE_OK;
+}
+
+/*
+ * The fp8 cache kept in pages: both storage choices at once (reading as for the two functions above; the scales
+ * stay per (sequence, KV head), pages belong to one sequence).
+ *
+ *   k_pages     e4m3 codes [num_pages, num_kv_heads, page_size, head_dim]   (v_pages alike)
+ *   block_table int32 [batch, max_pages_per_seq]: logical slot j of sequence b is row j % page_size of page
+ *               block_table[b, j / page_size]
+ *
+ * By definition: the slots a sequence can see (j < L_b + tree size) are copied out of their pages into a contiguous
+ * cache of codes of capacity max_pages_per_seq * page_size, and the contiguous fp8 definition is applied.
+ */
+int oracle_tree_verify_attn_fp8_paged(int batch, int num_q_heads, int num_kv_heads, int head_dim, int max_tree,
+                                      int num_pages, int page_size, int max_pages_per_seq, const int32_t* tree_sizes,
+                                      double sm_scale, const uint16_t* q, const uint8_t* k_pages, const uint8_t* v_pages,
+                                      const float* k_scale, const float* v_scale, const int32_t* block_table,
+                                      const int32_t* seq_lens, const int32_t* tree_parent, double* out) {
+  if (batch < 0 || num_kv_heads <= 0 || head_dim <= 0 || num_pages < 0 || page_size <= 0 || max_pages_per_seq < 0 ||
+      !block_table || !seq_lens)
+    return ORACLE_ERR_ARG;
+  const size_t cap = (size_t)max_pages_per_seq * page_size, D = (size_t)head_dim;
+  if (cap > 0x7fffffffu) return ORACLE_ERR_ARG;
+  const size_t elems = (size_t)batch * num_kv_heads * cap * D;
+  uint8_t* kc = (uint8_t*)calloc(elems ? elems : 1, 1);
+  uint8_t* vc = (uint8_t*)calloc(elems ? elems : 1, 1);
+  int rc = (kc && vc) ? ORACLE_OK : ORACLE_ERR_NOMEM;
+  for (int b = 0; b < batch && rc == ORACLE_OK; ++b) {
+    const int n = tree_size_of(tree_sizes, b, max_tree);
+    if (n < 0 || n > max_tree || seq_lens[b] < 0 || (size_t)seq_lens[b] + n > cap) {
+      rc = ORACLE_ERR_ARG;
+      break;
+    }
+    const int visible = n > 0 ? seq_lens[b] + n : 0;
+    for (int j = 0; j < visible && rc == ORACLE_OK; ++j) {
+      const int page = block_table[(size_t)b * max_pages_per_seq + j / page_size], row = j % page_size;
+      if (page < 0 || page >= num_pages) {
+        rc = ORACLE_ERR_ARG;
+        break;
+      }
+      for (int g = 0; g < num_kv_heads; ++g) {
+        const size_t src = (((size_t)page * num_kv_heads + g) * page_size + row) * D;
+        const size_t dst = (((size_t)b * num_kv_heads + g) * cap + j) * D;
+        memcpy(kc + dst, k_pages + src, D);
+        memcpy(vc + dst, v_pages + src, D);
+      }
+    }
+  }
+  if (rc == ORACLE_OK)
+    rc = oracle_tree_verify_attn_fp8(batch, num_q_heads, num_kv_heads, head_dim, max_tree, (int)cap, tree_sizes, sm_scale, q,
+                                     kc, vc, k_scale, v_scale, seq_lens, tree_parent, out);
+  free(kc);
+  free(vc);
+  return rc;
 }
 
 /*

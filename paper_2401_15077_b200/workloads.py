@@ -142,10 +142,11 @@ class PagedKV:
     page_size: int
 
 
-def make_paged_cache(inp: AttnInputs, page_size: int, salt: int = 0, spare_pages: int = 3, poison: bool = True) -> PagedKV:
+def make_paged_cache(inp: AttnInputs, page_size: int, salt: int = 0, spare_pages: int = 3, poison: bool = True, codes=None) -> PagedKV:
     """The same keys and values as ``inp`` stored in pages of ``page_size`` slots, scattered over the pool by a seeded
     permutation.  Only pages that hold a visible slot get a table entry; the other entries are -1, and rows of slots
-    that are not visible (as well as ``spare_pages`` unused pages) hold NaN when ``poison``."""
+    that are not visible (as well as ``spare_pages`` unused pages) hold NaN when ``poison``.  With ``codes`` (an
+    ``Fp8KV`` of the same cache) the pages hold its fp8 codes instead (uint8; the NaN code where not visible)."""
     cfg = inp.cfg
     B, Hkv, D = cfg.batch, cfg.num_kv_heads, cfg.head_dim
     vis = [int(inp.seq_lens[b] + inp.tree_sizes[b]) if int(inp.tree_sizes[b]) > 0 else 0 for b in range(B)]
@@ -153,9 +154,14 @@ def make_paged_cache(inp: AttnInputs, page_size: int, salt: int = 0, spare_pages
     max_pages = max(1, (inp.kv_capacity + page_size - 1) // page_size)
     total = sum(need) + spare_pages
     order = torch.randperm(total, generator=_gen(cfg.index, "pages", salt)).tolist()
-    fill = float("nan") if poison else 0.0
-    kp = torch.full((max(total, 1), Hkv, page_size, D), fill, dtype=torch.bfloat16)
-    vp = torch.full((max(total, 1), Hkv, page_size, D), fill, dtype=torch.bfloat16)
+    if codes is None:
+        src_k, src_v = inp.k_cache, inp.v_cache
+        fill, dtype = (float("nan") if poison else 0.0), torch.bfloat16
+    else:
+        src_k, src_v = codes.k_codes, codes.v_codes
+        fill, dtype = (0x7F if poison else 0), torch.uint8
+    kp = torch.full((max(total, 1), Hkv, page_size, D), fill, dtype=dtype)
+    vp = torch.full((max(total, 1), Hkv, page_size, D), fill, dtype=dtype)
     table = torch.full((B, max_pages), -1, dtype=torch.int32)
     nxt = 0
     for b in range(B):
@@ -164,8 +170,8 @@ def make_paged_cache(inp: AttnInputs, page_size: int, salt: int = 0, spare_pages
             nxt += 1
             table[b, i] = page
             rows = min(page_size, vis[b] - i * page_size)
-            kp[page, :, :rows] = inp.k_cache[b, :, i * page_size:i * page_size + rows]
-            vp[page, :, :rows] = inp.v_cache[b, :, i * page_size:i * page_size + rows]
+            kp[page, :, :rows] = src_k[b, :, i * page_size:i * page_size + rows]
+            vp[page, :, :rows] = src_v[b, :, i * page_size:i * page_size + rows]
     return PagedKV(kp, vp, table, page_size)
 
 

@@ -56,3 +56,62 @@ def test_scales(oracle):
     bad = f8.k_codes.clone()
     bad[0, 0, 0, 0] = 0x7F
     assert np.isnan(oracle.tree_verify_attn_fp8(inp.q, bad, f8.v_codes, f8.k_scale, f8.v_scale, *args)[0, 0, 0]).all()
+
+
+# ---- the fp8 cache kept in pages
+
+def _paged_case(salt, page_size):
+    inp = W.make_attn_inputs(CFG, salt=salt)
+    f8 = W.make_fp8_cache(inp)
+    return inp, f8, W.make_paged_cache(inp, page_size, salt=salt, codes=f8)
+
+
+def test_paged_fp8_matches_numpy_definition(oracle):
+    """An independent evaluation that reads the pages through the table itself and decodes with the library's conversion."""
+    page_size = 16
+    inp, f8, pk = _paged_case(4, page_size)
+    got = oracle.tree_verify_attn_fp8_paged(inp.q, pk.k_pages, pk.v_pages, f8.k_scale, f8.v_scale, pk.block_table, inp.seq_lens,
+                                            inp.tree_parent, inp.tree_sizes)
+    q = inp.q.to(torch.float64).numpy()
+    kp = pk.k_pages.view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    vp = pk.v_pages.view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    G = CFG.num_q_heads // CFG.num_kv_heads
+    for b in range(CFG.batch):
+        L, n = int(inp.seq_lens[b]), int(inp.tree_sizes[b])
+        for i in range(CFG.max_tree):
+            for h in range(CFG.num_q_heads):
+                if i >= n:
+                    assert np.all(got[b, i, h] == 0.0)
+                    continue
+                slots = list(range(L))
+                c = i
+                while c >= 0:
+                    slots.append(L + c)
+                    c = int(inp.tree_parent[b, c])
+                pages = [int(pk.block_table[b, j // page_size]) for j in slots]
+                rows = [j % page_size for j in slots]
+                K = kp[pages, h // G, rows] * float(f8.k_scale[b, h // G])
+                V = vp[pages, h // G, rows] * float(f8.v_scale[b, h // G])
+                s = K @ q[b, i, h] / np.sqrt(CFG.head_dim)
+                w = np.exp(s - s.max())
+                np.testing.assert_allclose(got[b, i, h], (w / w.sum()) @ V, rtol=1e-12, atol=1e-13)
+
+
+def test_paged_fp8_equals_contiguous_fp8_and_ignores_page_placement(oracle):
+    outs = []
+    for salt, page_size in ((5, 8), (5, 128), (6, 32)):
+        inp, f8, pk = _paged_case(5, page_size)
+        pk = W.make_paged_cache(inp, page_size, salt=salt, spare_pages=salt, codes=f8)
+        outs.append(oracle.tree_verify_attn_fp8_paged(inp.q, pk.k_pages, pk.v_pages, f8.k_scale, f8.v_scale, pk.block_table,
+                                                      inp.seq_lens, inp.tree_parent, inp.tree_sizes))
+    flat = oracle.tree_verify_attn_fp8(inp.q, f8.k_codes, f8.v_codes, f8.k_scale, f8.v_scale, inp.seq_lens, inp.tree_parent, inp.tree_sizes)
+    assert all(np.array_equal(o, flat) for o in outs)
+    # a visible slot without a page is an argument error
+    bad = pk.block_table.clone()
+    bad[1, 0] = pk.k_pages.shape[0]
+    try:
+        oracle.tree_verify_attn_fp8_paged(inp.q, pk.k_pages, pk.v_pages, f8.k_scale, f8.v_scale, bad, inp.seq_lens, inp.tree_parent,
+                                          inp.tree_sizes)
+        raise AssertionError("accepted a page outside the pool")
+    except ValueError:
+        pass
