@@ -138,7 +138,7 @@ size_t eagle_tree_verify_attn_static_capacity(void);
  * and values wherever a serving engine stores them).
  */
 typedef struct eagle_paged_kv {
-  const void* k_pages;          /* device bf16 [num_pages, Hkv, page_size, D], 16-byte aligned */
+  const void* k_pages;          /* device bf16 [num_pages, Hkv, page_size, D], 16-byte aligned (uint8 codes for the _fp8 calls) */
   const void* v_pages;          /* device bf16 [num_pages, Hkv, page_size, D], 16-byte aligned */
   const int32_t* block_table;   /* device int32 [B, max_pages_per_seq]: slot j of sequence b is row j % page_size of page
                                    block_table[b, j / page_size]; entries of pages that hold no slot below
@@ -196,7 +196,7 @@ int eagle_tree_verify_attn_planned_paged(const eagle_attn_desc* desc, const void
  * bf16 queries are converted to fp16 (exact for magnitudes from 2^-14 to 65504; smaller ones are rounded to multiples of
  * 2^-24, larger ones become infinite) and the probabilities are rounded to fp16 instead of bf16.  Everything else (fp32
  * scores / softmax / accumulation, bf16 output, planner, work split, errors) is as for eagle_tree_verify_attn.  What it
- * saves is half of the cache bytes held and read.  head_dim must be 128 and the cache contiguous (else EAGLE_ERR_SHAPE).
+ * saves is half of the cache bytes held and read.  head_dim must be 128 (else EAGLE_ERR_SHAPE).
  * Slots that are not visible may hold any code; one of the two NaN codes (0x7f, 0xff) in a VISIBLE slot makes the output
  * rows that see it NaN.
  * eagle_tree_verify_attn_planned_fp8 is the per-layer half over a plan made by eagle_tree_verify_plan (paged = NULL).
@@ -206,6 +206,22 @@ int eagle_tree_verify_attn_fp8(const eagle_attn_desc* desc, const void* q, const
                                void* out, eagle_stream_t stream);
 int eagle_tree_verify_attn_planned_fp8(const eagle_attn_desc* desc, const void* q, const void* k_codes, const void* v_codes,
                                        const float* k_scale, const float* v_scale, void* out, eagle_stream_t stream);
+
+/*
+ * The fp8 cache kept in pages: both storage choices of the same cache at once (Sec. 3.3 reads the same keys and values
+ * wherever and however a serving engine stores them).  kv->k_pages / kv->v_pages are device uint8
+ * [num_pages, Hkv, page_size, D] holding e4m3 codes, addressed through kv->block_table as for
+ * eagle_tree_verify_attn_paged; k_scale / v_scale are device fp32 [B, Hkv] as for eagle_tree_verify_attn_fp8 (a page
+ * belongs to one sequence, so the scales stay per (sequence, KV head)).  Arithmetic, errors and limits are those of the
+ * two calls it combines: head_dim 128 (else EAGLE_ERR_SHAPE), fp16 x fp16 products, EAGLE_ERR_SEQ / EAGLE_ERR_PAGE per
+ * sequence.  The planned form runs over a plan made by eagle_tree_verify_plan with the same `paged` description.
+ */
+int eagle_tree_verify_attn_paged_fp8(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* kv, const float* k_scale,
+                                     const float* v_scale, const int32_t* seq_lens, const int32_t* tree_parent, void* out,
+                                     eagle_stream_t stream);
+int eagle_tree_verify_attn_planned_paged_fp8(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* kv,
+                                             const float* k_scale, const float* v_scale, void* out, eagle_stream_t stream);
+
 
 /*
  * Where a plan keeps its tree masks (host function, no CUDA work): device uint64 [B, T_max] inside desc->workspace,

@@ -22,7 +22,8 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_commit_paged", "eagle_tree_verify_step_host_bytes", "eagle_tree_accept_cluster_width",
            "eagle_tree_verify_plan", "eagle_tree_verify_attn_planned", "eagle_tree_verify_attn_planned_paged",
            "eagle_tree_verify_plan_masks", "eagle_set_wait_limit_ns", "eagle_test_stall_kv_producer",
-           "eagle_tree_verify_attn_fp8", "eagle_tree_verify_attn_planned_fp8"]
+           "eagle_tree_verify_attn_fp8", "eagle_tree_verify_attn_planned_fp8", "eagle_tree_verify_attn_paged_fp8",
+           "eagle_tree_verify_attn_planned_paged_fp8"]
 _lib = None
 
 
@@ -89,6 +90,10 @@ def load():
         lib.eagle_tree_verify_attn_fp8.restype = ctypes.c_int
         lib.eagle_tree_verify_attn_planned_fp8.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 7
         lib.eagle_tree_verify_attn_planned_fp8.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_paged_fp8.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(PagedKV)] + [vp] * 6
+        lib.eagle_tree_verify_attn_paged_fp8.restype = ctypes.c_int
+        lib.eagle_tree_verify_attn_planned_paged_fp8.argtypes = [ctypes.POINTER(AttnDesc), vp, ctypes.POINTER(PagedKV)] + [vp] * 4
+        lib.eagle_tree_verify_attn_planned_paged_fp8.restype = ctypes.c_int
         lib.eagle_tree_verify_plan.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, ctypes.POINTER(PagedKV), vp]
         lib.eagle_tree_verify_plan.restype = ctypes.c_int
         lib.eagle_tree_verify_attn_planned.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp]
@@ -269,6 +274,35 @@ def eagle_tree_verify_attn_fp8(q, k_codes, v_codes, k_scale, v_scale, seq_lens, 
     return out
 
 
+def eagle_tree_verify_attn_paged_fp8(q, k_pages, v_pages, k_scale, v_scale, block_table, seq_lens, tree_parent, out=None, *,
+                                     tree_sizes=None, sm_scale=0.0, num_splits=0, workspace=None, status=None, events=None,
+                                     shared_tree=False):
+    """Tree-masked attention over a paged cache of fp8 e4m3 codes: k_pages / v_pages uint8 [num_pages,Hkv,page_size,D]
+    (D = 128), k_scale / v_scale fp32 [B,Hkv], block_table [B,max_pages_per_seq] int32."""
+    lib = load()
+    if q.dim() != 4 or k_pages.dim() != 4 or k_pages.shape != v_pages.shape or block_table.dim() != 2:
+        raise EagleError("bad tensor ranks / shapes")
+    B, T, Hq, D = q.shape
+    P, Hkv, ps = k_pages.shape[0], k_pages.shape[1], k_pages.shape[2]
+    if k_pages.shape[3] != D or block_table.shape[0] != B or tuple(seq_lens.shape) != (B,) or tuple(k_scale.shape) != (B, Hkv) or \
+            tuple(v_scale.shape) != (B, Hkv):
+        raise EagleError("inconsistent shapes")
+    _check_tree(tree_parent, tree_sizes, B, T, shared_tree)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = alloc_workspace(q, k_pages, num_splits)
+    d = _attn_desc(q, Hkv, 0, tree_sizes, sm_scale, num_splits, workspace, status, events, shared_tree)
+    pk = PagedKV(_dev(k_pages, torch.uint8, "k_pages"), _dev(v_pages, torch.uint8, "v_pages"),
+                 _dev(block_table, torch.int32, "block_table"), P, ps, block_table.shape[1])
+    rc = lib.eagle_tree_verify_attn_paged_fp8(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), ctypes.byref(pk),
+                                              _dev(k_scale, torch.float32, "k_scale"), _dev(v_scale, torch.float32, "v_scale"),
+                                              _dev(seq_lens, torch.int32, "seq_lens"), _dev(tree_parent, torch.int32, "tree_parent"),
+                                              _dev(out, torch.bfloat16, "out"), _stream())
+    _check(rc, "eagle_tree_verify_attn_paged_fp8")
+    return out
+
+
 class VerifyPlan:
     """The plan of one verification pass (tree masks + work split), made once by ``eagle_tree_verify_plan`` and used by
     every layer's ``attend`` / ``attend_paged``.  Holds the descriptor fields and the workspace; marshalling only."""
@@ -331,6 +365,21 @@ class VerifyPlan:
         rc = load().eagle_tree_verify_attn_planned_paged(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), ctypes.byref(pk),
                                                          _dev(out, torch.bfloat16, "out"), _stream())
         _check(rc, "eagle_tree_verify_attn_planned_paged")
+        return out
+
+    def attend_paged_fp8(self, q, k_pages, v_pages, k_scale, v_scale, block_table, out=None, *, sm_scale=0.0, status=None, events=None):
+        """One layer over a paged cache of fp8 codes, on a plan made with ``paged=``."""
+        if tuple(q.shape) != self.shape:
+            raise EagleError("tensors do not match the plan")
+        if out is None:
+            out = torch.empty_like(q)
+        d = self._desc(q.shape, sm_scale, status, events)
+        pk = PagedKV(_dev(k_pages, torch.uint8, "k_pages"), _dev(v_pages, torch.uint8, "v_pages"),
+                     _dev(block_table, torch.int32, "block_table"), k_pages.shape[0], k_pages.shape[2], block_table.shape[1])
+        rc = load().eagle_tree_verify_attn_planned_paged_fp8(ctypes.byref(d), _dev(q, torch.bfloat16, "q"), ctypes.byref(pk),
+                                                             _dev(k_scale, torch.float32, "k_scale"), _dev(v_scale, torch.float32, "v_scale"),
+                                                             _dev(out, torch.bfloat16, "out"), _stream())
+        _check(rc, "eagle_tree_verify_attn_planned_paged_fp8")
         return out
 
 

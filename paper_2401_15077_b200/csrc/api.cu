@@ -269,6 +269,31 @@ int eagle_tree_verify_attn_planned_fp8(const eagle_attn_desc* desc, const void* 
   return attention_with_workspace(desc, kAttendOnly, q, kv, nullptr, nullptr, out, stream_);
 }
 
+int eagle_tree_verify_attn_paged_fp8(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* pk, const float* k_scale,
+                                     const float* v_scale, const int32_t* seq_lens, const int32_t* tree_parent, void* out,
+                                     eagle_stream_t stream_) {
+  KvSource kv;
+  int rc = EAGLE_OK;
+  if (!paged_source(desc, pk, &kv, &rc)) return rc;
+  if (desc->head_dim != 128) return EAGLE_ERR_SHAPE;
+  if (desc->batch > 0 && desc->max_tree > 0 && (!k_scale || !v_scale)) return EAGLE_ERR_NULL;
+  kv.k_scale = k_scale;
+  kv.v_scale = v_scale;
+  return attention_with_workspace(desc, kPlanAndAttend, q, kv, seq_lens, tree_parent, out, stream_);
+}
+
+int eagle_tree_verify_attn_planned_paged_fp8(const eagle_attn_desc* desc, const void* q, const eagle_paged_kv* pk,
+                                             const float* k_scale, const float* v_scale, void* out, eagle_stream_t stream_) {
+  KvSource kv;
+  int rc = EAGLE_OK;
+  if (!paged_source(desc, pk, &kv, &rc)) return rc;
+  if (desc->head_dim != 128) return EAGLE_ERR_SHAPE;
+  if (desc->batch > 0 && desc->max_tree > 0 && (!k_scale || !v_scale)) return EAGLE_ERR_NULL;
+  kv.k_scale = k_scale;
+  kv.v_scale = v_scale;
+  return attention_with_workspace(desc, kAttendOnly, q, kv, nullptr, nullptr, out, stream_);
+}
+
 int eagle_tree_verify_plan(const eagle_attn_desc* desc, const int32_t* seq_lens, const int32_t* tree_parent,
                            const eagle_paged_kv* pk, eagle_stream_t stream_) {
   if (!desc) return EAGLE_ERR_NULL;

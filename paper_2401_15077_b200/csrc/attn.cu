@@ -19,7 +19,7 @@
 // rescaled only when the row maximum outgrows the shared reference by more than 2^8.  Every wait is bounded
 // (mbarrier try_wait + timer, or a bounded spin on a tagged word); on expiry the CTA raises EAGLE_ERR_TIMEOUT, all
 // roles leave their loops, TMEM is released and the kernel returns.
-// Instantiations: PAGED (the K/V producer gathers a tile page by page through a block table) and FP8 (the cache holds
+// Instantiations: PAGED (the K/V producer gathers a tile page by page through a block table), FP8, or both (the cache holds
 // e4m3 codes: tiles of codes land in a staging ring, four more warps widen them exactly into a ring of four fp16
 // slots and the MMAs run fp16 x fp16; the scales go into the softmax scale and the output).
 #include <cuda.h>
@@ -383,7 +383,7 @@ template <int D, bool PAGED, bool FP8>
 __global__ void __launch_bounds__(FP8 ? kThreadsFp8 : kThreads, 1)
 attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
             const __grid_constant__ CUtensorMap map_q) {
-  static_assert(!(FP8 && PAGED) && !(FP8 && D != 128), "the fp8 cache form is built for contiguous caches with 128-wide heads");
+  static_assert(!(FP8 && D != 128), "the fp8 cache form is built for 128-wide heads");
   using S = Smem<D, FP8>;
   constexpr int kSlots = S::kSlots;
   extern __shared__ __align__(1024) unsigned char smem[];
@@ -873,21 +873,33 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           // each; the boxes land one under the other, which is the tile's layout.  A box past the sequence's last page
           // fetches that last page again (its rows are masked), so the byte count of a tile never changes.  The page
           // number is read before the wait for the slot, so that its latency is not added to the slot's turnaround.
+          // (A page of fp8 codes: a row is one 128-byte line, so a box is the page's rows whole, and it lands in the staging slot.)
           const int rows = p.page_size < kTileN ? p.page_size : kTileN;
-          const int sl = lane % S::kSlabs;                      // lane = (box, 64-column slab): one TMA box per lane
-          const int r0 = (lane / S::kSlabs) * rows, key = c.tile * kTileN + r0;
+          constexpr int kBoxSlabs = FP8 ? 1 : S::kSlabs;
+          const int sl = lane % kBoxSlabs;                      // lane = (box, 64-column slab): one TMA box per lane
+          const int r0 = (lane / kBoxSlabs) * rows, key = c.tile * kTileN + r0;
           int page = 0;
           if (r0 < kTileN) {
             const int pi = key >> p.page_shift;
             page = __ldg(c.pages + (pi < c.last_page ? pi : c.last_page));
           }
-          ok = mbar_wait_warp(B.empty(slot), par, s_abort);
-          if (!ok) return;
-          if (lane == 0) mbar_expect_tx(B.full(slot), S::kTileBytes);
-          __syncwarp();
-          if (r0 < kTileN)
-            tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
-                        key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
+          if constexpr (FP8) {
+            ok = mbar_wait_warp(B.st_empty(slot), par, s_abort);
+            if (!ok) return;
+            if (lane == 0) mbar_expect_tx(B.st_full(slot), S::kCodeBytes);
+            __syncwarp();
+            if (r0 < kTileN)
+              tma_load_3d(sbase + S::kStage + slot * S::kCodeBytes + r0 * 128, is_v ? &map_v : &map_k, 0, key & (p.page_size - 1),
+                          page * p.Hkv + c.z, B.st_full(slot));
+          } else {
+            ok = mbar_wait_warp(B.empty(slot), par, s_abort);
+            if (!ok) return;
+            if (lane == 0) mbar_expect_tx(B.full(slot), S::kTileBytes);
+            __syncwarp();
+            if (r0 < kTileN)
+              tma_load_3d(sbase + S::kRing + slot * S::kTileBytes + sl * S::kSlabBytes + r0 * 128, is_v ? &map_v : &map_k, sl * 64,
+                          key & (p.page_size - 1), page * p.Hkv + c.z, B.full(slot));
+          }
         } else if constexpr (FP8) {
           // the tile of codes goes to the staging slot; the converter warps widen it into ring slot `slot`
           ok = mbar_wait(B.st_empty(slot), par, s_abort);
@@ -1022,12 +1034,12 @@ bool make_kv_map(CUtensorMap* map, const void* base, int D, int S_cap, long long
 }
 
 // A cache of fp8 codes [B*Hkv, S_cap, D] uint8: box = D x 128 rows x 1 (D = 128: one 128-byte swizzled row per slot).
-bool make_code_map(CUtensorMap* map, const void* base, int D, int S_cap, long long bh) {
+bool make_code_map(CUtensorMap* map, const void* base, int D, int S_cap, long long bh, int rows = kTileN) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S_cap), static_cast<cuuint64_t>(bh)};
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(D), static_cast<cuuint64_t>(S_cap) * D};
-  const cuuint32_t box[3] = {static_cast<cuuint32_t>(D), static_cast<cuuint32_t>(kTileN), 1};
+  const cuuint32_t box[3] = {static_cast<cuuint32_t>(D), static_cast<cuuint32_t>(rows), 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -1059,6 +1071,8 @@ cudaError_t attn_prepare(int head_dim) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(attn_kernel<128, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128, true>::kBytes);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(attn_kernel<128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128, true>::kBytes);
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(attn_kernel<128, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128, false>::kBytes);
   }
   e = cudaFuncSetAttribute(attn_kernel<64, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64, false>::kBytes);
@@ -1071,8 +1085,13 @@ cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t strea
   AttnParams p = p_in;
   CUtensorMap mk, mv, mq;
   const bool paged = p.page_size > 0, fp8 = p.k_scale != nullptr;
-  if (fp8) {
-    if (paged || p.D != 128) return cudaErrorInvalidValue;
+  if (fp8 && paged) {
+    if (p.D != 128) return cudaErrorInvalidValue;
+    const long long ph = static_cast<long long>(p.num_pages) * p.Hkv;
+    const int rows = p.page_size < kTileN ? p.page_size : kTileN;
+    if (!make_code_map(&mk, p.k, p.D, p.page_size, ph, rows) || !make_code_map(&mv, p.v, p.D, p.page_size, ph, rows)) return cudaErrorInvalidValue;
+  } else if (fp8) {
+    if (p.D != 128) return cudaErrorInvalidValue;
     const long long bh = static_cast<long long>(p.B) * p.Hkv;
     if (!make_code_map(&mk, p.k, p.D, p.S_cap, bh) || !make_code_map(&mv, p.v, p.D, p.S_cap, bh)) return cudaErrorInvalidValue;
   } else if (paged) {
@@ -1090,7 +1109,8 @@ cudaError_t launch_attn(const AttnParams& p_in, int num_ctas, cudaStream_t strea
     mq = mk;   // unused by the kernel
   }
   if (fp8) {
-    attn_kernel<128, false, true><<<num_ctas, kThreadsFp8, Smem<128, true>::kBytes, stream>>>(p, mk, mv, mq);
+    if (paged) attn_kernel<128, true, true><<<num_ctas, kThreadsFp8, Smem<128, true>::kBytes, stream>>>(p, mk, mv, mq);
+    else attn_kernel<128, false, true><<<num_ctas, kThreadsFp8, Smem<128, true>::kBytes, stream>>>(p, mk, mv, mq);
   } else if (p.D == 128) {
     if (paged) attn_kernel<128, true, false><<<num_ctas, kThreads, Smem<128, false>::kBytes, stream>>>(p, mk, mv, mq);
     else attn_kernel<128, false, false><<<num_ctas, kThreads, Smem<128, false>::kBytes, stream>>>(p, mk, mv, mq);

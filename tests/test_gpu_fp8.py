@@ -214,3 +214,66 @@ def test_fp8_wait_that_runs_out_is_reported(E, oracle):
     out, status = _run(E, inp, f8)
     assert status == 0
     _check(out, ref, inp.tree_sizes)
+
+
+# ---- the fp8 cache kept in pages
+
+def _run_paged(E, inp, f8, pk, num_splits=0):
+    d = torch.device("cuda:0")
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    out = torch.full(inp.q.shape, float("nan"), dtype=torch.bfloat16, device=d)
+    E.eagle_tree_verify_attn_paged_fp8(inp.q.to(d), pk.k_pages.to(d), pk.v_pages.to(d), f8.k_scale.to(d), f8.v_scale.to(d),
+                                       pk.block_table.to(d), inp.seq_lens.to(d), inp.tree_parent.to(d), out,
+                                       tree_sizes=inp.tree_sizes.to(d), num_splits=num_splits, status=status)
+    torch.cuda.synchronize()
+    return out.cpu(), int(status.item())
+
+
+@pytest.mark.parametrize("page_size", [16, 64, 128, 256])
+@pytest.mark.parametrize("name", ["serving_mix_small", "ragged_small_trees", "group3", "five_heads_three_tiles"])
+def test_paged_fp8_matches_oracle_and_the_contiguous_call(E, oracle, name, page_size):
+    """Pages of codes behind a block table (pages scattered over the pool, unused rows and spare pages hold the NaN code):
+    the oracle's paged fp8 form within the bounds, and the contiguous fp8 call bit for bit (same plan, same arithmetic)."""
+    cfg = CASES[name]
+    inp = W.make_attn_inputs(cfg, salt=11, capacity_pad=19)
+    f8 = W.make_fp8_cache(inp)
+    pk = W.make_paged_cache(inp, page_size, salt=page_size, codes=f8)
+    ref = oracle.tree_verify_attn_fp8_paged(inp.q, pk.k_pages, pk.v_pages, f8.k_scale, f8.v_scale, pk.block_table, inp.seq_lens,
+                                            inp.tree_parent, inp.tree_sizes)
+    for splits in (0, 3):
+        out, status = _run_paged(E, inp, f8, pk, num_splits=splits)
+        assert status == 0, (name, page_size, splits)
+        _check(out, ref, inp.tree_sizes)
+        flat, st = _run(E, inp, f8, num_splits=splits)
+        assert st == 0 and torch.equal(out.view(torch.int16), flat.view(torch.int16)), (name, page_size, splits)
+
+
+def test_paged_fp8_plan_once_attend_many_and_bad_page(E, oracle):
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=6, prefix=(30, 1500), tree=(0, 64), max_depth=64)
+    inp = W.make_attn_inputs(cfg, salt=6)
+    f8 = W.make_fp8_cache(inp)
+    pk = W.make_paged_cache(inp, 32, salt=2, codes=f8)
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    plan = E.eagle_tree_verify_plan(tuple(inp.q.shape), cfg.num_kv_heads, 0, inp.seq_lens.to(d), inp.tree_parent.to(d),
+                                    tree_sizes=inp.tree_sizes.to(d), status=status,
+                                    paged=(pk.block_table.to(d), pk.k_pages.shape[0], pk.page_size))
+    out = plan.attend_paged_fp8(inp.q.to(d), pk.k_pages.to(d), pk.v_pages.to(d), f8.k_scale.to(d), f8.v_scale.to(d),
+                                pk.block_table.to(d), status=status)
+    torch.cuda.synchronize()
+    whole, st = _run_paged(E, inp, f8, pk)
+    assert st == 0 and int(status.item()) == 0 and torch.equal(out.cpu().view(torch.int16), whole.view(torch.int16))
+    ref = oracle.tree_verify_attn_fp8_paged(inp.q, pk.k_pages, pk.v_pages, f8.k_scale, f8.v_scale, pk.block_table, inp.seq_lens,
+                                            inp.tree_parent, inp.tree_sizes)
+    _check(whole, ref, inp.tree_sizes)
+    # a visible slot whose page is outside the pool: that sequence is refused and zeroed, the others are untouched
+    b = int(torch.nonzero(inp.tree_sizes > 0)[0])
+    bad = W.PagedKV(pk.k_pages, pk.v_pages, pk.block_table.clone(), pk.page_size)
+    bad.block_table[b, 0] = pk.k_pages.shape[0]
+    got, st = _run_paged(E, inp, f8, bad)
+    assert st == -11          # EAGLE_ERR_PAGE
+    assert torch.all(got[b] == 0)
+    sizes = inp.tree_sizes.clone()       # (the work is split differently without that sequence: the others agree with
+    sizes[b] = 0                         # the oracle within the bounds, not with the first call bit for bit)
+    ref[b] = 0.0
+    _check(got, ref, sizes)
