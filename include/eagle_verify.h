@@ -427,6 +427,8 @@ typedef struct eagle_commit_desc {
  * exist yet).  A row that is not strictly increasing, leaves [0, T_max), or points at a slot >= S_cap (or L_b < 0)
  * sets *status to EAGLE_ERR_PATH: nothing of that sequence is moved, its length is unchanged and its feature rows are
  * zeros.  All pointers must be 16-byte aligned.  One launch, asynchronous on `stream`; no workspace.
+ * A cache of fp8 codes (uint8 [B, Hkv, S_cap, 128], see eagle_tree_verify_attn_fp8) is committed by the same call with
+ * head_dim = 64: a row of 128 codes is a row of 64 16-bit elements and rows are moved as bytes (the scales do not change).
  */
 int eagle_tree_commit(const eagle_commit_desc* desc, void* k_cache, void* v_cache, const int32_t* seq_lens,
                       const int32_t* accepted_path, const void* features_in, void* features_out,

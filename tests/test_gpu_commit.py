@@ -104,3 +104,53 @@ def test_invalid_paths_are_reported_and_left_alone(E, oracle):
     paths[4, :2] = torch.tensor([2, 9], dtype=torch.int32)      # slot 40 + 9 = 49 does not exist
     ref = _run_and_compare(E, oracle, k, v, lens, paths, T, feats, expect_status=-10)
     assert ref["valid"].tolist() == [0, 0, 1, 0, 0]
+
+
+@pytest.mark.parametrize("paged", [False, True])
+def test_commit_of_an_fp8_cache_moves_rows_of_codes(E, paged):
+    """A cache of fp8 codes [.., S, 128] uint8 is committed by the same call on its 16-bit view [.., S, 64]: rows are moved
+    as bytes.  The expected cache is built here from the codes, slot by slot."""
+    d = torch.device("cuda:0")
+    cfg = W.scaled(W.CONFIGS["serving_mix"], batch=5, prefix=(0, 300), tree=(0, 40))
+    inp = W.make_attn_inputs(cfg, salt=2, poison=False, capacity_pad=3)
+    f8 = W.make_fp8_cache(inp, poison=False)
+    for salt in range(8):     # a draw in which some accepted path moves rows (a path 0, 1, 2, ... moves nothing)
+        paths = W.make_accepted_paths(inp.tree_sizes, inp.tree_parent, cfg.max_tree, cfg.index, salt)
+        if any(int(paths[b, j]) > j for b in range(cfg.batch) for j in range(cfg.max_tree)):
+            break
+    want_k, want_v = f8.k_codes.clone(), f8.v_codes.clone()
+    want_len = inp.seq_lens.clone()
+    for b in range(cfg.batch):
+        L = int(inp.seq_lens[b])
+        path = [int(x) for x in paths[b] if int(x) >= 0]
+        for j, m in enumerate(path):
+            want_k[b, :, L + j] = f8.k_codes[b, :, L + m]
+            want_v[b, :, L + j] = f8.v_codes[b, :, L + m]
+        want_len[b] = L + len(path)
+    assert any(int(paths[b, j]) > j for b in range(cfg.batch) for j in range(cfg.max_tree))
+    status = torch.zeros(1, dtype=torch.int32, device=d)
+    if not paged:
+        kd, vd = f8.k_codes.to(d), f8.v_codes.to(d)
+        new_len, _ = E.eagle_tree_commit(kd.view(torch.bfloat16), vd.view(torch.bfloat16), inp.seq_lens.to(d), paths.to(d), cfg.max_tree,
+                                         status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(kd.cpu(), want_k) and torch.equal(vd.cpu(), want_v)
+    else:
+        pk = W.make_paged_cache(inp, 32, salt=4, poison=False, codes=f8)
+        kd, vd = pk.k_pages.to(d), pk.v_pages.to(d)
+        new_len, _ = E.eagle_tree_commit_paged(kd.view(torch.bfloat16), vd.view(torch.bfloat16), pk.block_table.to(d), inp.seq_lens.to(d),
+                                               paths.to(d), cfg.max_tree, status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        want = W.make_paged_cache(inp, 32, salt=4, poison=False, codes=W.Fp8KV(want_k, want_v, f8.k_scale, f8.v_scale))
+        # compare slot by slot through the table (rows of pages past the old visible range may differ: the committed
+        # prefix grew into them only up to the new length)
+        for b in range(cfg.batch):
+            if int(inp.tree_sizes[b]) == 0:
+                continue                     # (the generator gives a sequence without a tree no pages)
+            for j in range(int(want_len[b])):
+                page, row = int(pk.block_table[b, j // 32]), j % 32
+                assert torch.equal(kd[page, :, row].cpu(), want_k[b, :, j]) and torch.equal(vd[page, :, row].cpu(), want_v[b, :, j]), (b, j)
+        del want
+    assert torch.equal(new_len.cpu(), want_len)
