@@ -95,7 +95,7 @@ size_t eagle_tree_verify_attn_workspace(const eagle_attn_desc* desc);
  *                                                 rows of nodes i >= tree size are written as zeros
  *
  * Arithmetic: bf16 inputs, fp32 scores / softmax / accumulation, bf16 output (round to nearest even).
- * k_cache and v_cache must be 16-byte aligned.  Launches, in order on `stream`: the planner (tree masks +
+ * q, k_cache and v_cache must be 16-byte aligned, out 32-byte aligned (else EAGLE_ERR_SHAPE).  Launches, in order on `stream`: the planner (tree masks +
  * work list), the split-KV attention kernel, the combine kernel.  The workspace must not be shared by
  * calls that can overlap on the GPU.
  */

@@ -140,7 +140,7 @@ int attend_call(const eagle_attn_desc& d, const Workspace& w, int num_ctas, Devi
                 void* out, cudaStream_t stream) {
   if (!q || !kv.k || !kv.v || !out) return EAGLE_ERR_NULL;
   if ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
-      (reinterpret_cast<uintptr_t>(out) & 15))
+      (reinterpret_cast<uintptr_t>(out) & 31))
     return EAGLE_ERR_SHAPE;
   const int di = d.head_dim == 128 ? 1 : 0;
   if (!dev->attn_prepared[di]) {
@@ -204,7 +204,7 @@ int attention_with_workspace(const eagle_attn_desc* desc, int phase, const void*
   if (!d.workspace || (reinterpret_cast<uintptr_t>(d.workspace) & 255) || d.workspace_bytes < w.bytes) return EAGLE_ERR_WORKSPACE;
   if ((phase & kAttendOnly) &&
       ((reinterpret_cast<uintptr_t>(kv.k) & 15) || (reinterpret_cast<uintptr_t>(kv.v) & 15) || (reinterpret_cast<uintptr_t>(q) & 15) ||
-       (reinterpret_cast<uintptr_t>(out) & 15)))
+       (reinterpret_cast<uintptr_t>(out) & 31)))
     return EAGLE_ERR_SHAPE;
   int err = 0;
   DeviceInfo* dev = device_info(&err);

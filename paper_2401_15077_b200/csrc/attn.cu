@@ -256,6 +256,12 @@ __device__ __forceinline__ unsigned long long tag_wait(volatile uint32_t* slot, 
   return tag_wait_slow(slot, want, abort_flag);
 }
 
+// One 32-byte store (the address must be 32-byte aligned).
+__device__ __forceinline__ void st_global_v8(void* dst, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -787,34 +793,44 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             l_row = fmaf(*lfin, w, l_row);
           }
           const float inv = l_row > 0.f ? v_scale / l_row : 0.f;   // (v_scale is 1 unless the cache is fp8)
-          uint32_t o[32];
+          // The accumulator is read 32 columns at a time, the next chunk's load in flight while this one is scaled and
+          // stored.  These stores sit on the seam between two items (the group cannot take its next step, and the next
+          // item's first PV cannot start, before they are issued), and with a row per thread every lane of a store
+          // instruction is in a different line whatever its width: the output row leaves in 32-byte pieces (half as
+          // many instructions as with 16-byte ones), and the fp32 partial of a cut piece is laid out [4 columns][row],
+          // so that the 32 lanes of a store write 512 consecutive bytes.
+          uint32_t oa[32], ob[32];
+          auto store_chunk = [&](uint32_t (&o)[32], int c) {
+            if (!row_valid) return;
+            if (it.slot < 0) {
+              __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D;
 #pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            tmem_ld32(o_addr + c * 32, o);
-            tc_wait_ld();
-            if (row_valid) {
-              if (it.slot < 0) {
-                __nv_bfloat16* out_row = p.out + ((static_cast<size_t>(it.b) * p.T_max + node) * p.Hq + it.g * G + hh) * D;
+              for (int e = 0; e < 32; e += 16) {
+                uint32_t v[8];
 #pragma unroll
-                for (int e = 0; e < 32; e += 8) {
-                  uint4 v;
-                  v.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
-                  v.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-                  v.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-                  v.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-                  *reinterpret_cast<uint4*>(out_row + c * 32 + e) = v;
-                }
-              } else {
-                float* part_row = p.part_o + (static_cast<size_t>(it.slot) * kBlockM + r) * D;
-                if constexpr (FP8) {
-#pragma unroll
-                  for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * v_scale);
-                }
-#pragma unroll
-                for (int e = 0; e < 32; e += 4)
-                  *reinterpret_cast<uint4*>(part_row + c * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+                for (int k = 0; k < 8; ++k) v[k] = pack_bf16(__uint_as_float(o[e + 2 * k]) * inv, __uint_as_float(o[e + 2 * k + 1]) * inv);
+                st_global_v8(out_row + c * 32 + e, v);
               }
+            } else {
+              float* part = p.part_o + (static_cast<size_t>(it.slot) * (D / 4) + c * 8) * (kBlockM * 4) + r * 4;
+              if constexpr (FP8) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * v_scale);
+              }
+#pragma unroll
+              for (int e = 0; e < 32; e += 4)
+                *reinterpret_cast<uint4*>(part + (e / 4) * (kBlockM * 4)) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
             }
+          };
+          tmem_ld32(o_addr, oa);
+#pragma unroll
+          for (int c = 0; c < D / 32; c += 2) {
+            tc_wait_ld();
+            tmem_ld32(o_addr + (c + 1) * 32, ob);
+            store_chunk(oa, c);
+            tc_wait_ld();
+            if (c + 2 < D / 32) tmem_ld32(o_addr + (c + 2) * 32, oa);
+            store_chunk(ob, c + 1);
           }
           if (row_valid && it.slot >= 0) p.part_ml[static_cast<size_t>(it.slot) * kBlockM + r] = make_float2(m_ref, l_row);
           tc_fence_before();

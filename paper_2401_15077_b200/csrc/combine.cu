@@ -3,7 +3,7 @@
 // and the zero rows of padded tree nodes.
 // A fixed grid (a few blocks per SM) first writes zeros to the rows of nodes past the tree size (one contiguous range
 // of the output per sequence, eight work items each), then walks the planner's list of cut query tiles, sixteen work
-// items per tile (8 rows each, one row per warp).  Query tiles that stayed in one item were written by the
+// items per tile (8 rows each; a thread takes 4 columns of a row).  Query tiles that stayed in one item were written by the
 // attention kernel and do not appear in the list.
 #include "common.cuh"
 
@@ -12,15 +12,14 @@ namespace eagle {
 namespace {
 
 constexpr int kCombineThreads = 256;
-constexpr int kBlocksPerUnit = 16;                      // 8 rows per block: one per warp
+constexpr int kBlocksPerUnit = 16;                      // 8 rows per block
 constexpr int kRowsPerBlock = kBlockM / kBlocksPerUnit;
 constexpr int kZeroChunks = 8;                          // work items that share the zeroing of one sequence's padding rows
 constexpr int kPiecesAtOnce = 4;                        // pieces of a tile whose loads are in flight together
-static_assert(kRowsPerBlock * 32 == kCombineThreads, "one row per warp");
+static_assert(kRowsPerBlock == 8 && kCombineThreads == 256, "a warp reads four 8-row groups of 4 columns: 8 warps cover 128 columns");
 
 template <int D>
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) {
-  constexpr int E = D / 32;  // elements per lane
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int zero_items = p.B * kZeroChunks, total = zero_items + p.hdr->n_cut * kBlocksPerUnit;
   for (int work_all = blockIdx.x; work_all < total; work_all += gridDim.x) {
@@ -36,20 +35,22 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
     continue;
   }
   const int work = work_all - zero_items;
-  // work items of a query tile: (cut tile, 8-row chunk), one row per warp.  Everything a row needs hangs off the
-  // planner's record, so the loads of up to four pieces (item extent, (max, sum), partial row) are issued together.
+  // work items of a query tile: (cut tile, 8-row chunk).  A partial is stored [piece][4 columns][row] (the attention
+  // kernel writes a row per thread, so this is the order in which its stores are contiguous): a thread takes 4 columns
+  // of one row, the eight lanes of a row group read 128 consecutive bytes, a warp four such groups.  Everything a row
+  // needs hangs off the planner's record, so the loads of up to four pieces (item extent, (max, sum), partial values)
+  // are issued together.
   const CutTile ct = p.cut_tiles[work / kBlocksPerUnit];
-  const int r = (work % kBlocksPerUnit) * kRowsPerBlock + warp;
+  const int r = (work % kBlocksPerUnit) * kRowsPerBlock + (lane & 7);
+  const int c4 = warp * 4 + (lane >> 3);           // which 4 columns
   const int R = ct.mt * kBlockM + r;
-  if (R >= ct.m_valid) continue;
+  if (c4 >= D / 4 || R >= ct.m_valid) continue;
   const int i = R / p.G, h = ct.g * p.G + R % p.G;
-  float acc[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) acc[e] = 0.f;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
   float m_star = -INFINITY, l_star = 0.f;
   for (int s0 = 0; s0 < ct.count; s0 += kPiecesAtOnce) {
     float2 ml[kPiecesAtOnce];
-    float v[kPiecesAtOnce][E];
+    float4 v[kPiecesAtOnce];
     int t0[kPiecesAtOnce], t1[kPiecesAtOnce];
 #pragma unroll
     for (int u = 0; u < kPiecesAtOnce; ++u) {
@@ -57,16 +58,9 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
       const WorkItem* it = p.items + ct.item0 + ct.item_stride * s;
       t0[u] = it->tile_begin;
       t1[u] = it->tile_end;
-      const size_t row = static_cast<size_t>(ct.slot0 + s) * kBlockM + r;
-      ml[u] = p.part_ml[row];
-      const float* po = p.part_o + row * D + lane * E;
-      if constexpr (E == 4) {
-        const float4 x = *reinterpret_cast<const float4*>(po);
-        v[u][0] = x.x; v[u][1] = x.y; v[u][2] = x.z; v[u][3] = x.w;
-      } else {
-        const float2 x = *reinterpret_cast<const float2*>(po);
-        v[u][0] = x.x; v[u][1] = x.y;
-      }
+      const size_t slot = static_cast<size_t>(ct.slot0 + s);
+      ml[u] = p.part_ml[slot * kBlockM + r];
+      v[u] = *reinterpret_cast<const float4*>(p.part_o + (slot * (D / 4) + c4) * (kBlockM * 4) + r * 4);
     }
     // a piece counts when its item is not empty (an empty item never wrote its slot) and the row saw a key in it
     // (a row all of whose keys in the piece were masked keeps the reference -inf; its sum may hold rounding dust)
@@ -81,26 +75,24 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(AttnParams p) 
     const float keep = exp2f(m_star - m_new);     // 1 when the maximum did not move, 0 for the first pieces
     l_star *= keep;
 #pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] *= keep;
+    for (int e = 0; e < 4; ++e) acc[e] *= keep;
     m_star = m_new;
 #pragma unroll
     for (int u = 0; u < kPiecesAtOnce; ++u) {
       if (!use[u]) continue;
       const float w = exp2f(ml[u].x - m_star);
       l_star += ml[u].y * w;
-#pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] += v[u][e] * w;
+      acc[0] += v[u].x * w;
+      acc[1] += v[u].y * w;
+      acc[2] += v[u].z * w;
+      acc[3] += v[u].w * w;
     }
   }
   const float inv = l_star > 0.f ? 1.f / l_star : 0.f;
-  __nv_bfloat16* dst = p.out + ((static_cast<size_t>(ct.b) * p.T_max + i) * p.Hq + h) * D + lane * E;
+  __nv_bfloat16* dst = p.out + ((static_cast<size_t>(ct.b) * p.T_max + i) * p.Hq + h) * D + c4 * 4;
   __nv_bfloat162 lo = __floats2bfloat162_rn(acc[0] * inv, acc[1] * inv);
-  if constexpr (E == 4) {
-    __nv_bfloat162 hi = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
-    *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-  } else {
-    *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<uint32_t*>(&lo);
-  }
+  __nv_bfloat162 hi = __floats2bfloat162_rn(acc[2] * inv, acc[3] * inv);
+  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
   }
 }
 
