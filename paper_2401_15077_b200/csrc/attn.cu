@@ -617,10 +617,15 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
             else w = 0xffffffffu;
             if (rel <= -32) continue;                 // wholly in the prefix (uniform over the warp: the loads below are collective)
             uint32_t t[32];
-            tmem_ld32(s_addr + c * 32, t);
-            tc_wait_ld();
+            if (rel < n) {                            // (uniform too) some key of the chunk belongs to the tree
+              tmem_ld32(s_addr + c * 32, t);
+              tc_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) t[e] = (w >> e) & 1u ? t[e] : 0xff800000u;       // -inf
+              for (int e = 0; e < 32; ++e) t[e] = (w >> e) & 1u ? t[e] : 0xff800000u;       // -inf
+            } else {                                  // wholly past the tree: nothing to keep, nothing to fetch
+#pragma unroll
+              for (int e = 0; e < 32; ++e) t[e] = 0xff800000u;
+            }
             tmem_st32(s_addr + c * 32, t);
           }
           tc_wait_st();
