@@ -362,7 +362,7 @@ struct Smem {
   static constexpr int kTag = kStage + (FP8 ? kSlots * kCodeBytes : 0);   // uint32 [128 rows]: reference maximum | step number
   static constexpr int kLfin = kTag + kBlockM * 4;           // float [128 rows]: row sums on their way to the epilogue
   static constexpr int kBar = kLfin + kBlockM * 4;
-  static constexpr int kNumBars = 2 * kSlots + 3 * kSBufs + 3 + (FP8 ? 2 * kSlots : 0);
+  static constexpr int kNumBars = 2 * kSlots + 3 * kSBufs + 4 + (FP8 ? 2 * kSlots : 0);
   static constexpr int kMisc = kBar + 8 * kNumBars;           // tmem base, abort flag, wait limit (8 bytes)
   static constexpr int kBytes = kMisc + 16;
 };
@@ -380,9 +380,11 @@ struct Bars {
   __device__ __forceinline__ uint32_t q_full() const { return base + 8u * (2 * kSlots + 3 * kSBufs); }
   __device__ __forceinline__ uint32_t q_empty() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 1); }
   __device__ __forceinline__ uint32_t o_free() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 2); }
+  // the last PV MMA of an item has been issued
+  __device__ __forceinline__ uint32_t pv_last() const { return base + 8u * (2 * kSlots + 3 * kSBufs + 3); }
   // fp8 only: a staging slot holds a tile of codes / the converter warps are done with it
-  __device__ __forceinline__ uint32_t st_full(uint32_t i) const { return base + 8u * (2 * kSlots + 3 * kSBufs + 3 + i); }
-  __device__ __forceinline__ uint32_t st_empty(uint32_t i) const { return base + 8u * (3 * kSlots + 3 * kSBufs + 3 + i); }
+  __device__ __forceinline__ uint32_t st_full(uint32_t i) const { return base + 8u * (2 * kSlots + 3 * kSBufs + 4 + i); }
+  __device__ __forceinline__ uint32_t st_empty(uint32_t i) const { return base + 8u * (3 * kSlots + 3 * kSBufs + 4 + i); }
 };
 
 template <int D, bool PAGED, bool FP8>
@@ -426,6 +428,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
     mbar_init(B.q_full(), p.q_tma ? 1 : kGroupThreads);   // one TMA transaction, or every thread of the first softmax group
     mbar_init(B.q_empty(), 1);
     mbar_init(B.o_free(), kGroupThreads);
+    mbar_init(B.pv_last(), 1);
     *s_abort = 0;
     *reinterpret_cast<volatile unsigned long long*>(smem + S::kMisc + 8) = p.wait_limit_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -476,6 +479,13 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
         }
         ok = mbar_wait(B.q_full(), item_count & 1u, s_abort);
         if (!ok) break;
+        if (item_count > 0) {
+          // The tensor pipe runs the MMAs in the order they were issued: a score MMA of this item issued now would run
+          // before the last PV MMA of the item before, whose probabilities (the masked last tile) take longest, and the
+          // read-out of that item's accumulator, which everything behind the seam waits for, would start that much later.
+          ok = mbar_wait(B.pv_last(), (item_count - 1) & 1u, s_abort);
+          if (!ok) break;
+        }
         for (int s = 0; s < steps && ok; ++s, ++gq) {
           // the K tile arrives long before the score buffer frees up: look at it first, so that nothing but the
           // MMA issue follows the wait that matters
@@ -526,6 +536,7 @@ attn_kernel(AttnParams p, const __grid_constant__ CUtensorMap map_k, const __gri
           issue_pv_tile(tmem + kColO, tmem + kColS + sb * kTileN, ring_lo_v + vs * kTileStep, idesc_pv, s == 0 ? 0u : 1u);
           tc_commit(B.o_done(sb));
           tc_commit(B.empty(vs));
+          if (s == steps - 1) mbar_arrive(B.pv_last());
           vs += 2;
           if (vs >= kSlots) { vs -= kSlots; vp ^= 1u; }
           if (++sb == kSBufs) { sb = 0; sph ^= 1u; }
