@@ -51,10 +51,10 @@ SM_COUNT, EX2_PER_SM_PER_CLK = 148, 16      # special-function rate behind the e
 # profiles/attn_kernel_serving_mix_b16.md, keyed by (workload, batch), with the SHA-256 of the attention kernel's source
 # the captures were taken on: when the source has changed since, the figure is stale and `traffic` is reported as null.
 NCU_TRAFFIC = {
-    "attn_cu_sha256": "0d98cc137884a9807a7b451e9be9f0ec307e4cfbc29b940d31d06fe3ad6287d2",
-    # full size: one-pass metric list, two launches averaged (1177.1 MB read + 23.6 MB written); batch 16: --set full
+    "attn_cu_sha256": "45abb4aec25ea42f4cba9b9c12940521db7b31208c3f05b689e433d667c06e1e",
+    # full size: one-pass metric list, two launches averaged (1176.3 MB read + 22.8 MB written); batch 16: --set full
     # (taken before the epilogue's stores changed; the reads it measures did not)
-    "bytes": {("serving_mix", 64): 1_177_148_800 + 23_555_328, ("serving_mix", 16): 313_046_528 + 9_554_304},
+    "bytes": {("serving_mix", 64): 1_176_343_168 + 22_765_312, ("serving_mix", 16): 313_046_528 + 9_554_304},
 }
 
 
