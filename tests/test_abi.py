@@ -60,6 +60,10 @@ def test_host_checks_return_before_any_launch(lib):
     # non-null tensors but no workspace
     fake = ctypes.c_void_p(4096)
     assert lib.eagle_tree_verify_attn(ctypes.byref(d), fake, fake, fake, fake, fake, fake, None) == -3
+    # a workspace that would do, but an output that is not 32-byte aligned (or a query that is not 16-byte aligned)
+    dws = binding.AttnDesc(1, 8, 8, 64, 8, 300, None, 0.0, 0, 4096, 1 << 30, None, None, None)
+    assert lib.eagle_tree_verify_attn(ctypes.byref(dws), fake, fake, fake, fake, fake, ctypes.c_void_p(4096 + 16), None) == -2
+    assert lib.eagle_tree_verify_attn(ctypes.byref(dws), ctypes.c_void_p(4096 + 8), fake, fake, fake, fake, fake, None) == -2
     dbad = binding.AttnDesc(1, 8, 8, 80, 8, 300, None, 0.0, 0, None, 0, None, None, None)
     assert lib.eagle_tree_verify_attn(ctypes.byref(dbad), fake, fake, fake, fake, fake, fake, None) == -2
     a = binding.AcceptDesc(1, 65, 10, 8, None, None, None, None)
