@@ -301,6 +301,10 @@ int eagle_tree_accept(const eagle_accept_desc* desc, const float* target_probs, 
  * Negative EAGLE_ERR_* on a bad argument or when no sm_100 device is current.
  */
 int eagle_tree_accept_cluster_width(int32_t batch, int32_t vocab);
+/* The same for a call that passes draft_probs == NULL or uniforms == NULL, i.e. one whose sequences are all greedy (the
+ * setting of most of the paper's tables, temperature 0): its walk is argmax sweeps only, and where eight CTAs per tree
+ * would not fit the GPU at once it takes four. */
+int eagle_tree_accept_cluster_width_greedy(int32_t batch, int32_t vocab);
 
 /*
  * One whole verification step driven from HOST buffers (the two calls above, with the copies around them).

@@ -23,7 +23,7 @@ EXPORTS = ["eagle_tree_verify_attn_workspace", "eagle_tree_verify_attn", "eagle_
            "eagle_tree_verify_plan", "eagle_tree_verify_attn_planned", "eagle_tree_verify_attn_planned_paged",
            "eagle_tree_verify_plan_masks", "eagle_set_wait_limit_ns", "eagle_test_stall_kv_producer",
            "eagle_tree_verify_attn_fp8", "eagle_tree_verify_attn_planned_fp8", "eagle_tree_verify_attn_paged_fp8",
-           "eagle_tree_verify_attn_planned_paged_fp8"]
+           "eagle_tree_verify_attn_planned_paged_fp8", "eagle_tree_accept_cluster_width_greedy"]
 _lib = None
 
 
@@ -117,6 +117,8 @@ def load():
         lib.eagle_tree_accept.restype = ctypes.c_int
         lib.eagle_tree_accept_cluster_width.argtypes = [i32, i32]
         lib.eagle_tree_accept_cluster_width.restype = ctypes.c_int
+        lib.eagle_tree_accept_cluster_width_greedy.argtypes = [i32, i32]
+        lib.eagle_tree_accept_cluster_width_greedy.restype = ctypes.c_int
         lib.eagle_tree_accept_logits.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, vp]
         lib.eagle_tree_accept_logits.restype = ctypes.c_int
         lib.eagle_tree_expand.argtypes = [ctypes.POINTER(ExpandDesc), vp, vp, vp, vp, vp, vp]
@@ -470,9 +472,11 @@ def eagle_tree_accept(target_probs, draft_probs, draft_tokens, tree_parent, unif
     return accepted_path, bonus_token
 
 
-def eagle_tree_accept_cluster_width(batch: int, vocab: int) -> int:
-    """0 when a warp walks each tree, else the CTAs per cluster (1, 2, 4, 8) an acceptance call of this size uses here."""
-    rc = load().eagle_tree_accept_cluster_width(int(batch), int(vocab))
+def eagle_tree_accept_cluster_width(batch: int, vocab: int, all_greedy: bool = False) -> int:
+    """0 when a warp walks each tree, else the CTAs per cluster (1, 2, 4, 8) an acceptance call of this size uses here
+    (``all_greedy``: a call without draft rows or uniforms)."""
+    fn = load().eagle_tree_accept_cluster_width_greedy if all_greedy else load().eagle_tree_accept_cluster_width
+    rc = fn(int(batch), int(vocab))
     if rc < 0:
         _check(rc, "eagle_tree_accept_cluster_width")
     return rc

@@ -486,9 +486,12 @@ cudaError_t launch_cluster(const AcceptParams& p, cudaStream_t stream) {
 // wide as still fit the GPU with at most four CTAs per SM: the walk is a chain of dependent vocabulary sweeps, so a
 // tree finishes sooner the more SMs pull its rows.  (With 64 registers per thread only two CTAs of 512 threads are
 // resident per SM, so at batch 64 the clusters of eight run in two waves; measured, that is still faster than clusters
-// of four in one wave: 52 against 57 us on the 64-sequence mix.)
-int accept_cluster_width(int batch, int vocab, int sm_count) {
+// of four in one wave: 52 against 57 us on the 64-sequence mix.)  A call that passes no draft rows or no uniforms has
+// only greedy sequences (one argmax sweep per visited node, no rows to subtract): there clusters of four in one wave
+// are the faster ones (35 against 46 us at batch 64), so that case takes four where eight would need a second wave.
+int accept_cluster_width(int batch, int vocab, int sm_count, bool all_greedy) {
   if (vocab <= 4096) return 0;
+  if (all_greedy && 8ll * batch > 2ll * sm_count && 4ll * batch <= 2ll * sm_count) return 4;
   const long long resident = 4ll * sm_count;
   if (8ll * batch <= resident) return 8;
   if (4ll * batch <= resident) return 4;
@@ -499,7 +502,7 @@ int accept_cluster_width(int batch, int vocab, int sm_count) {
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream) {
   if (p.B == 0) return cudaSuccess;
   cudaError_t e;
-  switch (accept_cluster_width(p.B, p.V, sm_count)) {
+  switch (accept_cluster_width(p.B, p.V, sm_count, p.draft == nullptr || p.uniforms == nullptr)) {
     case 0: {
       const unsigned blocks = static_cast<unsigned>((p.B + kWarpTeamsPerCta - 1) / kWarpTeamsPerCta);
       if (p.logits) accept_kernel<32, 1, true><<<blocks, 32 * kWarpTeamsPerCta, 0, stream>>>(p);

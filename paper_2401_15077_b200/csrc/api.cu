@@ -391,6 +391,14 @@ int eagle_tree_accept_cluster_width(int32_t batch, int32_t vocab) {
   return accept_cluster_width(batch, vocab, dev->sm_count);
 }
 
+int eagle_tree_accept_cluster_width_greedy(int32_t batch, int32_t vocab) {
+  if (batch < 0 || vocab < 1) return EAGLE_ERR_SHAPE;
+  int err = 0;
+  DeviceInfo* dev = device_info(&err);
+  if (!dev) return err;
+  return accept_cluster_width(batch, vocab, dev->sm_count, true);
+}
+
 int eagle_tree_build_mask(const int32_t* tree_parent, const int32_t* tree_sizes, int32_t batch, int32_t max_tree,
                           uint64_t* anc_mask, uint8_t* depth, int32_t* status, eagle_stream_t stream_) {
   if (batch < 0 || max_tree < 0 || max_tree > kMaxTree) return EAGLE_ERR_SHAPE;

@@ -233,7 +233,7 @@ int attn_tile_keys();
 cudaError_t attn_prepare(int head_dim);
 cudaError_t launch_combine(const AttnParams& p, int unit_cap, int sm_count, cudaStream_t stream);
 cudaError_t launch_accept(const AcceptParams& p, int sm_count, cudaStream_t stream);
-int accept_cluster_width(int batch, int vocab, int sm_count);   // 0: a warp per tree; else CTAs per cluster
+int accept_cluster_width(int batch, int vocab, int sm_count, bool all_greedy = false);   // 0: a warp per tree; else CTAs per cluster
 
 cudaError_t launch_commit(const CommitParams& p, cudaStream_t stream);
 cudaError_t launch_expand(const ExpandParams& p, int sm_count, cudaStream_t stream);

@@ -107,6 +107,25 @@ def test_full_size_serving_mix_matches_oracle(E, oracle):
     assert int(ref["accept_len"].sum()) > cfg.batch
 
 
+def test_all_greedy_call_without_draft_rows_takes_clusters_of_four(E, oracle):
+    """Temperature 0 for the whole batch, no draft rows and no uniforms passed: at 64 trees clusters of eight would need a
+    second wave, so this kind of call takes four CTAs per tree; the tokens are the oracle's exactly."""
+    cfg = W.CONFIGS["serving_mix"]
+    inp = W.make_accept_inputs(cfg, salt=3, greedy="all")
+    assert inp.greedy.all()
+    assert E.eagle_tree_accept_cluster_width(cfg.batch, cfg.vocab, all_greedy=True) == 4
+    assert E.eagle_tree_accept_cluster_width(20, cfg.vocab, all_greedy=True) == 8
+    assert E.eagle_tree_accept_cluster_width(100, cfg.vocab, all_greedy=True) == 4      # (as for any call of that size)
+    ref = oracle.tree_accept(inp.target_probs, None, inp.draft_tokens, inp.tree_parent, None, tree_sizes=inp.tree_sizes, greedy=inp.greedy)
+    path, bonus, alen, status = _gpu_accept(E, inp, draft=False)
+    assert status == 0
+    assert _compare(inp, ref, path, bonus, alen) == 0
+    assert int(ref["accept_len"].sum()) > cfg.batch
+    # the same batch with the draft rows passed (clusters of eight): the same tokens
+    path8, bonus8, alen8, status = _gpu_accept(E, inp)
+    assert status == 0 and np.array_equal(path, path8) and np.array_equal(bonus, bonus8) and np.array_equal(alen, alen8)
+
+
 @pytest.mark.parametrize("name,cfg,kw,mode", CASES, ids=[c[0] for c in CASES])
 def test_accept_matches_oracle(E, oracle, name, cfg, kw, mode):
     tolerated_total, seqs = 0, 0
